@@ -1,0 +1,308 @@
+"""Pins of the CPU checker's verification step against things other than itself:
+library routines (torch, transformers' Llama), closed forms and brute force."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import verify as ov
+from paper_2407_12021_b200 import inputs as gen
+
+torch.set_num_threads(4)
+
+
+# ----------------------------------------------------------------------------- scalar blocks
+def test_round_bf16_matches_torch_cast():
+    g = torch.Generator().manual_seed(1)
+    x32 = torch.randn(200000, generator=g) * torch.exp(torch.randn(200000, generator=g) * 8)
+    edge = torch.tensor([0.0, -0.0, 1.0, 1.00390625, 1.005859375, 1.001953125, 3.3895e38, -3.3895e38,
+                         1e-40, 9.18e-41, -4.6e-41, 2.0 ** -133, 2.0 ** -134, 1.5 * 2.0 ** -133,
+                         65280.0, 65408.0, 0.1, 1 / 3], dtype=torch.float32)
+    x32 = torch.cat([x32, edge])
+    want = x32.to(torch.bfloat16).to(torch.float64).numpy()
+    got = ov.round_bf16(x32.to(torch.float64).numpy())
+    assert np.array_equal(got, want)
+
+
+def test_round_bf16_ties_and_single_rounding():
+    # exact ties go to the even neighbour
+    assert ov.round_bf16(np.array([1.0 + 2.0 ** -8]))[0] == 1.0
+    assert ov.round_bf16(np.array([1.0 + 3 * 2.0 ** -8]))[0] == 1.0 + 2.0 ** -6
+    # a float64 just above a tie must round up even though float32 would first land on the tie
+    x = 1.0 + 2.0 ** -8 + 2.0 ** -40
+    assert ov.round_bf16(np.array([x]))[0] == 1.0 + 2.0 ** -7
+    # idempotent
+    y = ov.round_bf16(np.linspace(-3, 3, 1001))
+    assert np.array_equal(ov.round_bf16(y), y)
+
+
+def test_rmsnorm_library_and_closed_form():
+    rng = np.random.default_rng(0)
+    h = rng.normal(size=(5, 48))
+    g = rng.normal(size=48)
+    want = torch.nn.functional.rms_norm(torch.from_numpy(h), (48,), torch.from_numpy(g), 1e-5).numpy()
+    assert np.allclose(ov.rmsnorm(h, g, 1e-5), want, rtol=1e-12, atol=1e-14)
+    # a constant row c normalises to sign(c) * gain (up to eps)
+    out = ov.rmsnorm(np.full((1, 16), -3.0), g[:16], 0.0)
+    assert np.allclose(out, -g[:16], rtol=1e-14)
+
+
+def test_rope_properties():
+    rng = np.random.default_rng(1)
+    x = rng.normal(size=(6, 3, 16))
+    pos = np.array([0, 1, 5, 17, 100, 1000])
+    y = ov.rope(x, pos, 10000.0)
+    assert np.allclose(y[0], x[0], atol=1e-15)                                    # position 0 is the identity
+    assert np.allclose(np.linalg.norm(y, axis=-1), np.linalg.norm(x, axis=-1))    # rotations keep lengths
+    # the score of a rotated query and key depends on the position difference only
+    q, k = rng.normal(size=(1, 1, 16)), rng.normal(size=(1, 1, 16))
+    def score(m, n):
+        return float(np.sum(ov.rope(q, np.array([m]), 1e4) * ov.rope(k, np.array([n]), 1e4)))
+    assert math.isclose(score(7, 3), score(104, 100), rel_tol=1e-10)
+    assert not math.isclose(score(7, 3), score(7, 4), rel_tol=1e-3)
+    # pair (0, hd/2) rotates by exactly `pos` radians (frequency index 0 has inverse frequency 1)
+    e = np.zeros((1, 1, 16)); e[0, 0, 0] = 1.0
+    r = ov.rope(e, np.array([2]), 1e4)[0, 0]
+    assert math.isclose(r[0], math.cos(2.0), rel_tol=1e-14) and math.isclose(r[8], math.sin(2.0), rel_tol=1e-14)
+    # the last pair turns at theta^(-(hd-2)/hd)
+    e = np.zeros((1, 1, 16)); e[0, 0, 7] = 1.0
+    r = ov.rope(e, np.array([3]), 1e4)[0, 0]
+    assert math.isclose(r[7], math.cos(3 * 1e4 ** (-14 / 16)), rel_tol=1e-13)
+
+
+def test_silu_softmax_library():
+    x = np.linspace(-20, 20, 401)
+    assert np.allclose(ov.silu(x), torch.nn.functional.silu(torch.from_numpy(x)).numpy(), rtol=1e-13, atol=1e-300)
+    s = np.random.default_rng(2).normal(size=(4, 9)) * 30
+    assert np.allclose(ov.softmax(s), torch.softmax(torch.from_numpy(s), -1).numpy(), rtol=1e-13)
+    assert np.allclose(ov.softmax(s).sum(-1), 1.0)
+
+
+def test_tree_bookkeeping_brute_force():
+    parents = [-1, 0, 1, 0, 3, 3, 2, 6]
+    paths, depth = ov.paths_and_depths(parents)
+    assert paths[7] == [0, 1, 2, 6, 7] and paths[5] == [0, 3, 5] and paths[0] == [0]
+    assert depth == [0, 1, 2, 1, 2, 2, 3, 4]
+    for bad in ([0], [-1, 1], [-1, -1], [-1, 0, 3, 1], []):
+        with pytest.raises(ValueError):
+            ov.check_tree(bad)
+
+
+def test_accept_walk_hand_cases():
+    #            0     1  2  3  4  5
+    parents = [-1,    0, 0, 1, 1, 3]
+    tokens = [9,      5, 6, 7, 8, 4]
+    # the model says: after root 5, after node 1 -> 7, after node 3 -> 4, after node 5 -> 2
+    best = [5, 7, 0, 4, 0, 2]
+    path, out = ov.accept_walk(tokens, parents, best)
+    assert path == [0, 1, 3, 5] and out == [5, 7, 4, 2]
+    # first mismatch stops the walk; the model's own token is still emitted (the bonus token)
+    best = [5, 1, 0, 4, 0, 2]
+    path, out = ov.accept_walk(tokens, parents, best)
+    assert path == [0, 1] and out == [5, 1]
+    best = [3, 7, 0, 4, 0, 2]
+    assert ov.accept_walk(tokens, parents, best) == ([0], [3])
+    # a lone root is plain autoregressive decoding: one token per pass
+    assert ov.accept_walk([9], [-1], [4]) == ([0], [4])
+
+
+# ----------------------------------------------------------------------------- whole forward vs a library Llama
+def _hf_model(shape, weights):
+    from transformers import LlamaConfig, LlamaForCausalLM
+    cfg = LlamaConfig(vocab_size=shape.vocab, hidden_size=shape.d_model, intermediate_size=shape.d_ffn,
+                      num_hidden_layers=shape.n_layers, num_attention_heads=shape.n_heads,
+                      num_key_value_heads=shape.n_heads, head_dim=shape.head_dim,
+                      max_position_embeddings=4096, rms_norm_eps=shape.rms_eps,
+                      rope_theta=shape.rope_theta, attention_bias=False, mlp_bias=False,
+                      tie_word_embeddings=False, attn_implementation="eager")
+    m = LlamaForCausalLM(cfg).double().eval()
+    d, f = shape.d_model, shape.d_ffn
+    sd = {"model.embed_tokens.weight": weights["embed"], "lm_head.weight": weights["lm_head"],
+          "model.norm.weight": weights["final_norm"]}
+    for l, p in enumerate(weights["layers"]):
+        pre = f"model.layers.{l}."
+        sd[pre + "self_attn.q_proj.weight"] = p["wqkv"][:d]
+        sd[pre + "self_attn.k_proj.weight"] = p["wqkv"][d:2 * d]
+        sd[pre + "self_attn.v_proj.weight"] = p["wqkv"][2 * d:]
+        sd[pre + "self_attn.o_proj.weight"] = p["wo"]
+        sd[pre + "mlp.gate_proj.weight"] = p["wgu"][:f]
+        sd[pre + "mlp.up_proj.weight"] = p["wgu"][f:]
+        sd[pre + "mlp.down_proj.weight"] = p["wd"]
+        sd[pre + "input_layernorm.weight"] = p["norm1"]
+        sd[pre + "post_attention_layernorm.weight"] = p["norm2"]
+    missing = m.load_state_dict({k: v.to(torch.float64) for k, v in sd.items()}, strict=False)
+    assert not [k for k in missing.missing_keys if "rotary" not in k], missing
+    return m
+
+
+SMALL = gen.ModelShape("pin", 2, 64, 4, 16, 96, 128, "f32")
+
+
+def _small_setup(seed=3, scale=6.0):
+    w = gen.model_weights(SMALL, seed)
+    # random gains and larger weights so that norms, attention and SwiGLU are far from linear
+    for p in w["layers"]:
+        for k in ("wqkv", "wo", "wgu", "wd"):
+            p[k] = p[k] * scale
+        p["norm1"] = 1 + 0.3 * gen.normal((SMALL.d_model,), 1.0, seed, 900)
+        p["norm2"] = 1 + 0.3 * gen.normal((SMALL.d_model,), 1.0, seed, 901)
+    w["final_norm"] = 1 + 0.3 * gen.normal((SMALL.d_model,), 1.0, seed, 902)
+    w["lm_head"] = w["lm_head"] * scale
+    return w
+
+
+def test_tree_forward_equals_each_path_as_causal_sequence_in_library_llama():
+    """Tree-masked attention with positions L + depth == running context + root-to-node path
+    through an ordinary causal Llama, for every node."""
+    w = _small_setup()
+    hf = _hf_model(SMALL, w)
+    arch = ov.arch_from_shape(SMALL)
+    ow = ov.Weights(w, keep=True)
+    ctx = gen.zipf_tokens(11, SMALL.vocab, 5, 1).tolist()
+    cache = ov.Cache(arch)
+    ov.append(arch, ow, cache, ctx, chunk=4)         # context goes in through chained chunks
+    assert cache.length == 11
+    tokens, parents = gen.make_tree(13, 4, 3, SMALL.vocab, 8)
+    logits, k_new, v_new = ov.forward_tree(arch, ow, cache, tokens, parents)
+    paths, depth = ov.paths_and_depths(parents)
+    assert max(depth) == 4
+    # the library keeps its rotary cos/sin tables in float32, so agreement is to ~1e-7, not 1e-15;
+    # any wrong convention (pairing, position, mask, slicing) is an O(1) error
+    tol = dict(rtol=1e-5, atol=2e-6)
+    for i in range(len(tokens)):
+        seq = ctx + [tokens[j] for j in paths[i]]
+        with torch.no_grad():
+            out = hf(torch.tensor([seq]), use_cache=True)
+        want = out.logits[0, -1].numpy()
+        assert np.allclose(logits[i], want, **tol), i
+        # the node's key/value equal the last position's cached key/value of the causal run
+        kv = out.past_key_values
+        for l in range(SMALL.n_layers):
+            lay = kv.layers[l] if hasattr(kv, "layers") else None
+            hk = (lay.keys if lay is not None else kv[l][0])[0, :, -1].numpy()
+            hv = (lay.values if lay is not None else kv[l][1])[0, :, -1].numpy()
+            assert np.allclose(k_new[l][:, i], hk, **tol)
+            assert np.allclose(v_new[l][:, i], hv, **tol)
+        # and the context part of the cache equals the causal run's first 11 positions
+        if i == 0:
+            for l in range(SMALL.n_layers):
+                lay = kv.layers[l] if hasattr(kv, "layers") else None
+                hk = (lay.keys if lay is not None else kv[l][0])[0, :, :11].numpy()
+                assert np.allclose(cache.k[l], hk, **tol)
+
+
+def test_greedy_acceptance_equals_autoregressive_decoding():
+    """verify() on a tree that contains the true continuation returns exactly the tokens that
+    plain greedy decoding (library generate, and the checker's own 1-node steps) produces."""
+    w = _small_setup(seed=4)
+    hf = _hf_model(SMALL, w)
+    arch = ov.arch_from_shape(SMALL)
+    ow = ov.Weights(w, keep=True)
+    ctx = gen.zipf_tokens(9, SMALL.vocab, 6, 1).tolist()
+    with torch.no_grad():
+        ar = hf.generate(torch.tensor([ctx]), max_new_tokens=6, do_sample=False,
+                         pad_token_id=0)[0, len(ctx):].tolist()
+
+    # (a) token-by-token with 1-node trees: accept_len is 1 every time
+    cache = ov.Cache(arch)
+    ov.append(arch, ow, cache, ctx[:-1])
+    cur, mine = ctx[-1], []
+    for _ in range(6):
+        res = ov.verify(arch, ow, cache, [cur], [-1])
+        assert res["accept_len"] == 1
+        cur = res["out_tokens"][0]
+        mine.append(cur)
+    assert mine == ar
+    cache_ar = cache
+
+    # (b) trees with p correct drafts planted on the full-depth chain: accept_len = p + 1
+    for p in range(0, 5):
+        cache = ov.Cache(arch)
+        ov.append(arch, ow, cache, ctx[:-1])
+        tokens, parents = gen.make_tree(12, 4, 3, SMALL.vocab, 20 + p, root_token=ctx[-1])
+        tokens = gen.plant_path(tokens, parents, ar[:p])
+        if p < 4:  # make sure the next draft on the chain is wrong
+            if tokens[p + 1] == ar[p]:
+                tokens[p + 1] = (ar[p] + 1) % SMALL.vocab
+            for s in range(len(tokens)):      # and that no sibling holds the right token by luck
+                if parents[s] == p and tokens[s] == ar[p]:
+                    tokens[s] = (ar[p] + 2) % SMALL.vocab
+        res = ov.verify(arch, ow, cache, tokens, parents)
+        assert res["out_tokens"] == ar[:p + 1], (p, res["out_tokens"], ar)
+        assert res["accept_len"] == p + 1
+        assert res["path"] == list(range(p + 1))
+        # cache after the step == cache of plain decoding over the same tokens
+        n = len(ctx) - 1 + p + 1
+        assert cache.length == n
+        for l in range(SMALL.n_layers):
+            assert np.allclose(cache.k[l], cache_ar.k[l][:, :n], rtol=1e-9, atol=1e-11)
+            assert np.allclose(cache.v[l], cache_ar.v[l][:, :n], rtol=1e-9, atol=1e-11)
+
+
+def test_sibling_order_does_not_change_output():
+    w = _small_setup(seed=5)
+    arch = ov.arch_from_shape(SMALL)
+    ow = ov.Weights(w, keep=True)
+    ctx = gen.zipf_tokens(6, SMALL.vocab, 7, 1).tolist()
+    cache = ov.Cache(arch)
+    ov.append(arch, ow, cache, ctx)
+    tokens = [3, 10, 11, 12, 13, 14]
+    parents = [-1, 0, 0, 1, 1, 2]
+    a, _, _ = ov.forward_tree(arch, ow, cache, tokens, parents)
+    # renumber: swap the two root children (and keep parents[i] < i)
+    tokens2 = [3, 11, 10, 14, 12, 13]
+    parents2 = [-1, 0, 0, 1, 2, 2]
+    b, _, _ = ov.forward_tree(arch, ow, cache, tokens2, parents2)
+    perm = [0, 2, 1, 4, 5, 3]   # node i of tree 1 is node perm[i] of tree 2
+    assert np.allclose(a, b[perm], rtol=1e-10, atol=1e-12)
+
+
+def test_bf16_mode_is_close_to_exact_and_lands_on_bf16_grid():
+    shape = gen.ModelShape("pin16", 2, 64, 4, 16, 96, 128, "bf16")
+    w = gen.model_weights(shape, 9)
+    for p in w["layers"]:
+        for k in ("wqkv", "wo", "wgu", "wd"):
+            p[k] = (p[k].float() * 4).to(torch.bfloat16)
+    arch16 = ov.arch_from_shape(shape)
+    arch64 = ov.Arch(**{**arch16.__dict__, "bf16": False})
+    ow = ov.Weights(w, keep=True)
+    ctx = gen.zipf_tokens(7, shape.vocab, 2, 1).tolist()
+    tokens, parents = gen.make_tree(10, 3, 3, shape.vocab, 4)
+    c16, c64 = ov.Cache(arch16), ov.Cache(arch64)
+    ov.append(arch16, ow, c16, ctx)
+    ov.append(arch64, ow, c64, ctx)
+    l16, k16, _ = ov.forward_tree(arch16, ow, c16, tokens, parents)
+    l64, _, _ = ov.forward_tree(arch64, ow, c64, tokens, parents)
+    rel = np.max(np.abs(l16 - l64)) / np.max(np.abs(l64))
+    assert 0 < rel < 3e-2
+    assert np.array_equal(ov.round_bf16(k16[0]), k16[0])     # cached keys are bf16 values
+    assert not np.array_equal(ov.round_bf16(l16), l16)       # logits are not rounded
+
+
+def test_cache_after_verify_holds_the_accepted_path_not_the_first_nodes():
+    """The accepted nodes are scattered in the tree numbering; what lands in the cache must be
+    their keys/values, in path order, equal to what plain decoding of the same tokens caches."""
+    w = _small_setup(seed=6)
+    arch = ov.arch_from_shape(SMALL)
+    ow = ov.Weights(w, keep=True)
+    ctx = gen.zipf_tokens(8, SMALL.vocab, 9, 1).tolist()
+    ar_cache = ov.Cache(arch)
+    ov.append(arch, ow, ar_cache, ctx[:-1])
+    cur, ar = ctx[-1], []
+    for _ in range(4):
+        cur = ov.verify(arch, ow, ar_cache, [cur], [-1])["out_tokens"][0]
+        ar.append(cur)
+    wrong = lambda t: (t + 17) % SMALL.vocab
+    #          0            1            2       3            4            5       6            7
+    parents = [-1,          0,           0,      1,           1,           2,      2,           5]
+    tokens = [ctx[-1], wrong(ar[0]), ar[0], wrong(ar[1]), wrong(ar[0]), ar[1], wrong(ar[1]), wrong(ar[2])]
+    cache = ov.Cache(arch)
+    ov.append(arch, ow, cache, ctx[:-1])
+    res = ov.verify(arch, ow, cache, tokens, parents)
+    assert res["path"] == [0, 2, 5] and res["out_tokens"] == ar[:3]
+    n = len(ctx) - 1 + 3
+    assert cache.length == n
+    for l in range(SMALL.n_layers):
+        assert np.allclose(cache.k[l], ar_cache.k[l][:, :n], rtol=1e-9, atol=1e-11)
+        assert np.allclose(cache.v[l], ar_cache.v[l][:, :n], rtol=1e-9, atol=1e-11)
