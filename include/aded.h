@@ -1,0 +1,203 @@
+/*
+ * aded.h -- C ABI of the B200 verification-step library for adaptive draft-verification
+ * decoding (ADED, "Adaptive Draft-Verification for Efficient Large Language Model Decoding").
+ *
+ * The library implements, for one GPU, the target-model side of the paper's loop
+ * (Methodology, Fig. 2): score a whole draft token tree in one forward pass with tree
+ * attention, approve drafts greedily, keep the approved path in the KV cache
+ * ("Draft Construction and Verification"); raise the tri-gram counts of freshly produced
+ * tokens (Algorithm 2); and list the most probable continuations of a two-token context
+ * (Eq. 1; "get potential words from tri-gram matrix", Algorithm 1).
+ *
+ * Conventions
+ *  - Every function returns an aded_status.  No exceptions, no global state.  A handle must
+ *    not be used from two threads at once; distinct handles are independent.
+ *  - Pointers named *_dev are DEVICE pointers on the device that was current when the handle
+ *    was created; pointers named *_host are HOST pointers.  The caller owns both and keeps
+ *    them alive until the work has finished on the stream.
+ *  - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).  Calls
+ *    taking device pointers only enqueue work and never synchronise.  Calls with a _host
+ *    suffix copy their arguments in and their results out and return after the stream has
+ *    drained.
+ *  - Errors the host can see (NULL handles, sizes out of range) are returned at once and
+ *    nothing is launched.  Errors only the device can see (malformed parent array, cache
+ *    capacity, hash table full, a bounded wait that ran out) are recorded in a device status
+ *    word: the offending call leaves the cache/table unchanged and reports accept length 0,
+ *    later calls on the handle do nothing until the handle's poll_status call has read and
+ *    cleared it.
+ */
+#ifndef ADED_H
+#define ADED_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum aded_status {
+    ADED_OK = 0,
+    ADED_ERR_INVALID_ARG = 1,
+    ADED_ERR_BAD_TREE = 2,     /* parents[0] != -1, or parents[i] not in [0, i) */
+    ADED_ERR_KV_CAPACITY = 3,  /* committed length + tree nodes exceeds the sequence's capacity */
+    ADED_ERR_TABLE_FULL = 4,   /* tri-gram store out of buckets */
+    ADED_ERR_OOM = 5,
+    ADED_ERR_CUDA = 6,
+    ADED_ERR_UNSUPPORTED = 7,
+    ADED_ERR_TIMEOUT = 8       /* a bounded device-side wait ran out */
+} aded_status;
+
+enum { ADED_F32 = 0, ADED_BF16 = 1 };
+
+/* Most nodes (root included) one sequence's draft tree may have. */
+#define ADED_MAX_NODES 128
+
+/* Llama-style decoder widths.  head_dim must be 64 or 128, d_model = n_heads * head_dim.
+ * dtype is the storage type of weights, activations and the KV cache; accumulation is fp32. */
+typedef struct aded_model_config {
+    int32_t n_layers, d_model, n_heads, head_dim, d_ffn, vocab;
+    int32_t dtype;          /* ADED_F32 or ADED_BF16 */
+    float rms_eps;          /* RMSNorm epsilon */
+    float rope_theta;       /* rotary base */
+    int32_t max_rows;       /* most tree nodes summed over the batch in one verify call (>= 1) */
+    int32_t max_batch;      /* most sequences in one verify call (>= 1) */
+} aded_model_config;
+
+/* Device pointers to row-major weights, output feature major ([out, in]); BORROWED: they must
+ * outlive the model.  wqkv [3d, d] holds the query rows, then key rows, then value rows, head h
+ * owning rows h*head_dim .. (h+1)*head_dim - 1 of each block; wgu [2F, d] holds the gate rows
+ * then the up rows; rotary pairs are (i, i + head_dim/2) within a head. */
+typedef struct aded_layer_weights {
+    const void *wqkv, *wo, *wgu, *wd, *norm1, *norm2;
+} aded_layer_weights;
+
+typedef struct aded_weights {
+    const void* embed;                 /* [vocab, d] */
+    const void* final_norm;            /* [d] */
+    const void* lm_head;               /* [vocab, d] */
+    const aded_layer_weights* layers;  /* HOST array of n_layers entries (copied) */
+} aded_weights;
+
+typedef struct aded_trigram_config {
+    int32_t vocab;            /* token ids are 0 .. vocab-1 */
+    int32_t log2_buckets;     /* 2^log2_buckets home buckets (one per two-token context), 4..28 */
+    int32_t overflow_buckets; /* extra buckets for contexts with more than 6 continuations */
+    uint32_t cap;             /* counts saturate here (Algorithm 2's maximum); 0 = 2^31 - 1 */
+    uint32_t min_count;       /* top-k skips entries below this count; 0 = off */
+} aded_trigram_config;
+
+typedef struct aded_model aded_model;     /* opaque, owned by the library */
+typedef struct aded_kv aded_kv;
+typedef struct aded_trigram aded_trigram;
+
+/* ---- lifetime ------------------------------------------------------------------------- */
+
+/* Validates the configuration, copies the weight pointer table and allocates the activation
+ * workspace for max_rows rows.  ADED_ERR_UNSUPPORTED for widths the kernels do not cover,
+ * ADED_ERR_OOM / ADED_ERR_CUDA if the device refuses. */
+aded_status aded_model_create(const aded_model_config* cfg, const aded_weights* weights, aded_model** out);
+aded_status aded_model_destroy(aded_model* m);
+
+/* KV cache for `batch` sequences (<= the model's max_batch); capacity_host[b] positions for
+ * sequence b.  Per sequence the cache is one block laid out
+ * [layer][K|V][head][position][head_dim] in the model dtype.  All committed lengths start at 0
+ * and live on the device. */
+aded_status aded_kv_create(const aded_model* m, int32_t batch, const int32_t* capacity_host, aded_kv** out);
+aded_status aded_kv_destroy(aded_kv* kv);
+/* Committed length of sequence `seq`; synchronises `stream`. */
+aded_status aded_kv_len(const aded_kv* kv, int32_t seq, int32_t* out_len_host, void* stream);
+/* Overwrite positions [0, n_pos) of layer `layer` of sequence `seq` with given keys/values
+ * (device pointers, [head][n_pos][head_dim], model dtype) and set the committed length to
+ * n_pos.  For workloads that start from a pre-filled cache. */
+aded_status aded_kv_load(aded_kv* kv, int32_t seq, int32_t layer, const void* k_dev, const void* v_dev,
+                         int32_t n_pos, void* stream);
+/* Copy out positions [pos0, pos0 + n_pos) of one layer: k_dev / v_dev receive
+ * [head][n_pos][head_dim].  For tests. */
+aded_status aded_kv_read(const aded_kv* kv, int32_t seq, int32_t layer, int32_t pos0, int32_t n_pos,
+                         void* k_dev, void* v_dev, void* stream);
+
+/* Put n committed tokens (1 <= n <= min(max_rows, 128)) into the cache of sequence `seq`:
+ * the verification pipeline on a chain whose every node is accepted, without the LM head. */
+aded_status aded_append(aded_model* m, aded_kv* kv, int32_t seq, const int32_t* tokens_dev, int32_t n,
+                        void* stream);
+
+/* ---- the verification step ("Draft Construction and Verification") ---------------------- */
+
+/* Verify one draft tree against the model for the single sequence of `kv` (batch 1).
+ *   tree_tokens_dev[n_nodes]  token of each node; node 0 is the last committed token, whose
+ *                             K/V are not cached yet (last prompt token or previous bonus token)
+ *   tree_parents_dev[n_nodes] parent index, -1 for node 0, otherwise in [0, i)
+ *   out_tokens_dev[n_nodes]   receives the emitted tokens: the model's greedy token after the
+ *                             root, then after each approved draft; entries past accept_len
+ *                             are left alone
+ *   out_accept_len_dev[1]     approved drafts + 1 (the model's own token always counts);
+ *                             0 if the call failed on the device
+ * Each node attends to all committed positions and to its ancestors and itself; rotary
+ * position = committed length + depth.  Greedy choice = largest fp32 logit, lowest id among
+ * equals.  Approval walks from the root to the child whose token equals the parent's greedy
+ * token until none matches.  Afterwards the K/V of the approved nodes sit at positions
+ * L .. L+accept_len-1 and the committed length is L + accept_len. */
+aded_status aded_verify(aded_model* m, aded_kv* kv, const int32_t* tree_tokens_dev,
+                        const int32_t* tree_parents_dev, int32_t n_nodes, int32_t* out_tokens_dev,
+                        int32_t* out_accept_len_dev, void* stream);
+
+/* Same for every sequence of `kv` at once.  tree_offsets_host[batch + 1] gives each sequence's
+ * slice of the concatenated token/parent arrays (parents are local to the slice; each slice has
+ * 1..ADED_MAX_NODES nodes; the total is at most max_rows).  Sequence b's emitted tokens go to
+ * out_tokens_dev[b * out_stride ...] (out_stride >= its node count). */
+aded_status aded_verify_batch(aded_model* m, aded_kv* kv, const int32_t* tree_offsets_host,
+                              const int32_t* tree_tokens_dev, const int32_t* tree_parents_dev,
+                              int32_t* out_tokens_dev, int32_t out_stride, int32_t* out_accept_len_dev,
+                              void* stream);
+
+/* aded_verify with HOST arrays: copies the tree in, runs, copies the results out, waits. */
+aded_status aded_verify_host(aded_model* m, aded_kv* kv, const int32_t* tree_tokens_host,
+                             const int32_t* tree_parents_host, int32_t n_nodes, int32_t* out_tokens_host,
+                             int32_t* out_accept_len_host, void* stream);
+
+/* Ask the next verify call to also write every node's logits ([rows][vocab] fp32, may be NULL)
+ * and greedy token ([rows] int32, may be NULL) to the given device buffers.  Parity checks only. */
+aded_status aded_debug_capture(aded_model* m, float* logits_dev, int32_t* best_dev);
+
+/* Read and clear the model's device status word; synchronises `stream`. */
+aded_status aded_model_poll_status(aded_model* m, aded_status* out_host, void* stream);
+
+/* ---- tri-gram store (Eq. 1, Algorithm 2) ---------------------------------------------- */
+
+aded_status aded_trigram_create(const aded_trigram_config* cfg, aded_trigram** out);
+aded_status aded_trigram_destroy(aded_trigram* t);
+
+/* Algorithm 2 over a token span: every window (tok[i-2], tok[i-1], tok[i]), i = 2 .. n-1, has
+ * its count raised by one (saturating at cap), absent tri-grams are inserted with count 1.
+ * n < 3 does nothing.  The caller chooses the span; to count a stream piecewise pass each piece
+ * with the two tokens that precede it.  A token outside [0, vocab) sets ADED_ERR_INVALID_ARG in
+ * the status word and its windows are skipped. */
+aded_status aded_trigram_update(aded_trigram* t, const int32_t* tokens_dev, int32_t n, void* stream);
+aded_status aded_trigram_update_host(aded_trigram* t, const int32_t* tokens_host, int32_t n, void* stream);
+
+/* For each of q contexts (ctx[2*i], ctx[2*i+1]) the k (1..32) continuations with the largest
+ * counts -- equivalently the largest Eq. 1 probabilities -- count descending, token id ascending
+ * among equals, padded with token -1 / count 0.  out_total (may be NULL) receives the sum of the
+ * context's counts, the denominator of Eq. 1. */
+aded_status aded_trigram_topk(const aded_trigram* t, const int32_t* ctx_dev, int32_t q, int32_t k,
+                              int32_t* out_tokens_dev, uint32_t* out_counts_dev, uint32_t* out_total_dev,
+                              void* stream);
+aded_status aded_trigram_topk_host(const aded_trigram* t, const int32_t* ctx_host, int32_t q, int32_t k,
+                                   int32_t* out_tokens_host, uint32_t* out_counts_host,
+                                   uint32_t* out_total_host, void* stream);
+
+/* Count of one tri-gram (0 if absent); synchronises `stream`.  For tests. */
+aded_status aded_trigram_get(const aded_trigram* t, int32_t a, int32_t b, int32_t c,
+                             uint32_t* out_count_host, void* stream);
+/* Number of stored tri-grams and of buckets in use; synchronises `stream`. */
+aded_status aded_trigram_stats(const aded_trigram* t, uint64_t* out_entries_host, uint64_t* out_buckets_host,
+                               void* stream);
+/* Read and clear the store's device status word; synchronises `stream`. */
+aded_status aded_trigram_poll_status(aded_trigram* t, aded_status* out_host, void* stream);
+
+const char* aded_status_string(aded_status s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ADED_H */

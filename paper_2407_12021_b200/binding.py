@@ -1,0 +1,309 @@
+"""ctypes binding of libaded.so: one Python function per C entry point, same names.
+
+Argument marshalling only: tensors are passed as raw pointers, every computation happens in the
+library's CUDA kernels.  There is no CPU fallback: importing this module without the built
+library raises, and a non-OK status raises AdedError.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from ctypes import POINTER, Structure, c_char_p, c_float, c_int32, c_uint32, c_uint64, c_void_p
+from typing import Dict, List, Optional, Sequence
+
+import torch
+
+_LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libaded.so")
+
+ADED_OK = 0
+ADED_F32, ADED_BF16 = 0, 1
+ADED_MAX_NODES = 128
+STATUS_NAMES = {0: "ADED_OK", 1: "ADED_ERR_INVALID_ARG", 2: "ADED_ERR_BAD_TREE", 3: "ADED_ERR_KV_CAPACITY",
+                4: "ADED_ERR_TABLE_FULL", 5: "ADED_ERR_OOM", 6: "ADED_ERR_CUDA", 7: "ADED_ERR_UNSUPPORTED",
+                8: "ADED_ERR_TIMEOUT"}
+
+EXPORTS = [
+    "aded_model_create", "aded_model_destroy", "aded_kv_create", "aded_kv_destroy", "aded_kv_len",
+    "aded_kv_load", "aded_kv_read", "aded_append", "aded_verify", "aded_verify_batch", "aded_verify_host",
+    "aded_debug_capture", "aded_model_poll_status", "aded_trigram_create", "aded_trigram_destroy",
+    "aded_trigram_update", "aded_trigram_update_host", "aded_trigram_topk", "aded_trigram_topk_host",
+    "aded_trigram_get", "aded_trigram_stats", "aded_trigram_poll_status", "aded_status_string",
+]
+
+
+class AdedError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {STATUS_NAMES.get(status, status)}")
+
+
+class ModelConfig(Structure):
+    _fields_ = [("n_layers", c_int32), ("d_model", c_int32), ("n_heads", c_int32), ("head_dim", c_int32),
+                ("d_ffn", c_int32), ("vocab", c_int32), ("dtype", c_int32), ("rms_eps", c_float),
+                ("rope_theta", c_float), ("max_rows", c_int32), ("max_batch", c_int32)]
+
+
+class LayerWeights(Structure):
+    _fields_ = [(n, c_void_p) for n in ("wqkv", "wo", "wgu", "wd", "norm1", "norm2")]
+
+
+class Weights(Structure):
+    _fields_ = [("embed", c_void_p), ("final_norm", c_void_p), ("lm_head", c_void_p),
+                ("layers", POINTER(LayerWeights))]
+
+
+class TrigramConfig(Structure):
+    _fields_ = [("vocab", c_int32), ("log2_buckets", c_int32), ("overflow_buckets", c_int32),
+                ("cap", c_uint32), ("min_count", c_uint32)]
+
+
+def load_library(path: str = _LIB_PATH) -> ctypes.CDLL:
+    if not os.path.exists(path):
+        raise ImportError(f"{path} is missing: build it with `python -m paper_2407_12021_b200.build` "
+                          "(there is no fallback implementation)")
+    lib = ctypes.CDLL(path)
+    for name in EXPORTS:
+        fn = getattr(lib, name)          # AttributeError if the symbol is not exported
+        fn.restype = c_char_p if name == "aded_status_string" else c_int32
+    return lib
+
+
+_lib = load_library()
+
+
+def _check(status: int, where: str) -> None:
+    if status != ADED_OK:
+        raise AdedError(status, where)
+
+
+def _ptr(t: Optional[torch.Tensor]) -> c_void_p:
+    return c_void_p(0 if t is None else t.data_ptr())
+
+
+def _stream() -> c_void_p:
+    return c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _dev_i32(t: torch.Tensor, what: str) -> torch.Tensor:
+    if not (t.is_cuda and t.dtype == torch.int32 and t.is_contiguous()):
+        raise TypeError(f"{what} must be a contiguous int32 CUDA tensor")
+    return t
+
+
+def _host_i32(t: torch.Tensor, what: str) -> torch.Tensor:
+    if t.is_cuda or t.dtype != torch.int32 or not t.is_contiguous():
+        raise TypeError(f"{what} must be a contiguous int32 host tensor")
+    return t
+
+
+class Model:
+    """Owns an aded_model* and keeps the weight tensors alive."""
+
+    def __init__(self, handle: c_void_p, keep, cfg: ModelConfig):
+        self.handle, self._keep, self.cfg = handle, keep, cfg
+
+    def __del__(self):
+        if getattr(self, "handle", None):
+            _lib.aded_model_destroy(self.handle)
+            self.handle = None
+
+
+class KV:
+    def __init__(self, handle: c_void_p, model: Model, batch: int):
+        self.handle, self.model, self.batch = handle, model, batch
+
+    def __del__(self):
+        if getattr(self, "handle", None):
+            _lib.aded_kv_destroy(self.handle)
+            self.handle = None
+
+
+class Trigram:
+    def __init__(self, handle: c_void_p, cfg: TrigramConfig):
+        self.handle, self.cfg = handle, cfg
+
+    def __del__(self):
+        if getattr(self, "handle", None):
+            _lib.aded_trigram_destroy(self.handle)
+            self.handle = None
+
+
+# ---- model / cache -----------------------------------------------------------------------
+def aded_model_create(shape, weights: Dict[str, object], max_rows: int = 128, max_batch: int = 1) -> Model:
+    """shape: any object with n_layers, d_model, n_heads, head_dim, d_ffn, vocab, dtype ("f32"/"bf16"),
+    rms_eps, rope_theta.  weights: dict laid out as inputs.model_weights, CUDA tensors."""
+    dt = {"f32": (ADED_F32, torch.float32), "bf16": (ADED_BF16, torch.bfloat16)}[shape.dtype]
+    cfg = ModelConfig(shape.n_layers, shape.d_model, shape.n_heads, shape.head_dim, shape.d_ffn, shape.vocab,
+                      dt[0], shape.rms_eps, shape.rope_theta, max_rows, max_batch)
+    keep = []
+
+    def dev(t: torch.Tensor, dims) -> int:
+        if not (t.is_cuda and t.dtype == dt[1] and t.is_contiguous() and tuple(t.shape) == tuple(dims)):
+            raise TypeError(f"weight tensor must be contiguous CUDA {dt[1]} of shape {tuple(dims)}, got "
+                            f"{t.dtype} {tuple(t.shape)} on {t.device}")
+        keep.append(t)
+        return t.data_ptr()
+
+    d, f, v = shape.d_model, shape.d_ffn, shape.vocab
+    layers = (LayerWeights * shape.n_layers)()
+    for l, p in enumerate(weights["layers"]):
+        layers[l] = LayerWeights(dev(p["wqkv"], (3 * d, d)), dev(p["wo"], (d, d)), dev(p["wgu"], (2 * f, d)),
+                                 dev(p["wd"], (d, f)), dev(p["norm1"], (d,)), dev(p["norm2"], (d,)))
+    w = Weights(dev(weights["embed"], (v, d)), dev(weights["final_norm"], (d,)), dev(weights["lm_head"], (v, d)),
+                layers)
+    out = c_void_p()
+    _check(_lib.aded_model_create(ctypes.byref(cfg), ctypes.byref(w), ctypes.byref(out)), "aded_model_create")
+    return Model(out, keep, cfg)
+
+
+def aded_kv_create(model: Model, capacities: Sequence[int]) -> KV:
+    caps = (c_int32 * len(capacities))(*capacities)
+    out = c_void_p()
+    _check(_lib.aded_kv_create(model.handle, c_int32(len(capacities)), caps, ctypes.byref(out)), "aded_kv_create")
+    return KV(out, model, len(capacities))
+
+
+def aded_kv_len(kv: KV, seq: int = 0) -> int:
+    out = c_int32()
+    _check(_lib.aded_kv_len(kv.handle, c_int32(seq), ctypes.byref(out), _stream()), "aded_kv_len")
+    return out.value
+
+
+def aded_kv_load(kv: KV, seq: int, layer: int, k: torch.Tensor, v: torch.Tensor) -> None:
+    assert k.is_cuda and v.is_cuda and k.is_contiguous() and v.is_contiguous() and k.shape == v.shape
+    _check(_lib.aded_kv_load(kv.handle, c_int32(seq), c_int32(layer), _ptr(k), _ptr(v), c_int32(k.shape[1]),
+                             _stream()), "aded_kv_load")
+
+
+def aded_kv_read(kv: KV, seq: int, layer: int, pos0: int, n_pos: int):
+    cfg = kv.model.cfg
+    dt = torch.bfloat16 if cfg.dtype == ADED_BF16 else torch.float32
+    k = torch.empty((cfg.n_heads, n_pos, cfg.head_dim), dtype=dt, device="cuda")
+    v = torch.empty_like(k)
+    _check(_lib.aded_kv_read(kv.handle, c_int32(seq), c_int32(layer), c_int32(pos0), c_int32(n_pos), _ptr(k),
+                             _ptr(v), _stream()), "aded_kv_read")
+    return k, v
+
+
+def aded_append(model: Model, kv: KV, tokens_dev: torch.Tensor, seq: int = 0) -> None:
+    _dev_i32(tokens_dev, "tokens")
+    _check(_lib.aded_append(model.handle, kv.handle, c_int32(seq), _ptr(tokens_dev), c_int32(tokens_dev.numel()),
+                            _stream()), "aded_append")
+
+
+# ---- verification -----------------------------------------------------------------------
+def aded_verify(model: Model, kv: KV, tree_tokens: torch.Tensor, tree_parents: torch.Tensor,
+                out_tokens: torch.Tensor, out_accept_len: torch.Tensor) -> None:
+    """All four are int32 CUDA tensors; out_tokens has at least as many entries as the tree."""
+    n = _dev_i32(tree_tokens, "tree_tokens").numel()
+    _dev_i32(tree_parents, "tree_parents"), _dev_i32(out_tokens, "out_tokens"), _dev_i32(out_accept_len, "out_accept_len")
+    if tree_parents.numel() != n or out_tokens.numel() < n or out_accept_len.numel() < 1:
+        raise ValueError("tree_parents / out_tokens / out_accept_len are too short for the tree")
+    _check(_lib.aded_verify(model.handle, kv.handle, _ptr(tree_tokens), _ptr(tree_parents), c_int32(n),
+                            _ptr(out_tokens), _ptr(out_accept_len), _stream()), "aded_verify")
+
+
+def aded_verify_batch(model: Model, kv: KV, tree_offsets: Sequence[int], tree_tokens: torch.Tensor,
+                      tree_parents: torch.Tensor, out_tokens: torch.Tensor, out_accept_len: torch.Tensor) -> None:
+    """tree_offsets: host list of batch+1 ints; out_tokens [batch, stride] int32 CUDA."""
+    _dev_i32(tree_tokens, "tree_tokens"), _dev_i32(tree_parents, "tree_parents")
+    _dev_i32(out_tokens, "out_tokens"), _dev_i32(out_accept_len, "out_accept_len")
+    if len(tree_offsets) != kv.batch + 1 or out_tokens.dim() != 2 or out_tokens.shape[0] != kv.batch:
+        raise ValueError("tree_offsets needs batch+1 entries and out_tokens one row per sequence")
+    if tree_tokens.numel() < tree_offsets[-1] or tree_parents.numel() < tree_offsets[-1] or out_accept_len.numel() < kv.batch:
+        raise ValueError("token / parent / accept-length arrays are too short")
+    offs = (c_int32 * len(tree_offsets))(*tree_offsets)
+    _check(_lib.aded_verify_batch(model.handle, kv.handle, offs, _ptr(tree_tokens), _ptr(tree_parents),
+                                  _ptr(out_tokens), c_int32(out_tokens.shape[1]), _ptr(out_accept_len), _stream()),
+           "aded_verify_batch")
+
+
+def aded_verify_host(model: Model, kv: KV, tree_tokens: torch.Tensor, tree_parents: torch.Tensor,
+                     out_tokens: torch.Tensor, out_accept_len: torch.Tensor) -> None:
+    """Same with int32 HOST tensors (pinned memory makes the copies asynchronous); blocks until done."""
+    n = _host_i32(tree_tokens, "tree_tokens").numel()
+    _host_i32(tree_parents, "tree_parents"), _host_i32(out_tokens, "out_tokens"), _host_i32(out_accept_len, "out_accept_len")
+    if tree_parents.numel() != n or out_tokens.numel() < n or out_accept_len.numel() < 1:
+        raise ValueError("tree_parents / out_tokens / out_accept_len are too short for the tree")
+    _check(_lib.aded_verify_host(model.handle, kv.handle, _ptr(tree_tokens), _ptr(tree_parents), c_int32(n),
+                                 _ptr(out_tokens), _ptr(out_accept_len), _stream()), "aded_verify_host")
+
+
+def aded_debug_capture(model: Model, logits: Optional[torch.Tensor], best: Optional[torch.Tensor]) -> None:
+    if logits is not None:
+        assert logits.is_cuda and logits.dtype == torch.float32 and logits.is_contiguous()
+    if best is not None:
+        _dev_i32(best, "best")
+    _check(_lib.aded_debug_capture(model.handle, _ptr(logits), _ptr(best)), "aded_debug_capture")
+
+
+def aded_model_poll_status(model: Model) -> int:
+    out = c_int32()
+    _check(_lib.aded_model_poll_status(model.handle, ctypes.byref(out), _stream()), "aded_model_poll_status")
+    return out.value
+
+
+# ---- tri-gram store ------------------------------------------------------------------------
+def aded_trigram_create(vocab: int, log2_buckets: int = 20, overflow_buckets: int = 1 << 18, cap: int = 0,
+                        min_count: int = 0) -> Trigram:
+    cfg = TrigramConfig(vocab, log2_buckets, overflow_buckets, cap, min_count)
+    out = c_void_p()
+    _check(_lib.aded_trigram_create(ctypes.byref(cfg), ctypes.byref(out)), "aded_trigram_create")
+    return Trigram(out, cfg)
+
+
+def aded_trigram_update(t: Trigram, tokens_dev: torch.Tensor) -> None:
+    _dev_i32(tokens_dev, "tokens")
+    _check(_lib.aded_trigram_update(t.handle, _ptr(tokens_dev), c_int32(tokens_dev.numel()), _stream()),
+           "aded_trigram_update")
+
+
+def aded_trigram_update_host(t: Trigram, tokens_host: torch.Tensor) -> None:
+    _host_i32(tokens_host, "tokens")
+    _check(_lib.aded_trigram_update_host(t.handle, _ptr(tokens_host), c_int32(tokens_host.numel()), _stream()),
+           "aded_trigram_update_host")
+
+
+def aded_trigram_topk(t: Trigram, ctx_dev: torch.Tensor, k: int, out_tokens: torch.Tensor, out_counts: torch.Tensor,
+                      out_total: Optional[torch.Tensor] = None) -> None:
+    """ctx_dev [q, 2] int32 CUDA; out_tokens [q, k] int32, out_counts [q, k] int32 (bit pattern of uint32),
+    out_total [q] int32 or None."""
+    _dev_i32(ctx_dev, "ctx"), _dev_i32(out_tokens, "out_tokens"), _dev_i32(out_counts, "out_counts")
+    q = ctx_dev.numel() // 2
+    if out_tokens.numel() < q * k or out_counts.numel() < q * k or (out_total is not None and out_total.numel() < q):
+        raise ValueError("output arrays are too short")
+    _check(_lib.aded_trigram_topk(t.handle, _ptr(ctx_dev), c_int32(q), c_int32(k), _ptr(out_tokens), _ptr(out_counts),
+                                  _ptr(out_total), _stream()), "aded_trigram_topk")
+
+
+def aded_trigram_topk_host(t: Trigram, ctx_host: torch.Tensor, k: int, out_tokens: torch.Tensor,
+                           out_counts: torch.Tensor, out_total: Optional[torch.Tensor] = None) -> None:
+    _host_i32(ctx_host, "ctx"), _host_i32(out_tokens, "out_tokens"), _host_i32(out_counts, "out_counts")
+    q = ctx_host.numel() // 2
+    if out_tokens.numel() < q * k or out_counts.numel() < q * k or (out_total is not None and out_total.numel() < q):
+        raise ValueError("output arrays are too short")
+    _check(_lib.aded_trigram_topk_host(t.handle, _ptr(ctx_host), c_int32(q), c_int32(k), _ptr(out_tokens),
+                                       _ptr(out_counts), _ptr(out_total), _stream()), "aded_trigram_topk_host")
+
+
+def aded_trigram_get(t: Trigram, a: int, b: int, c: int) -> int:
+    out = c_uint32()
+    _check(_lib.aded_trigram_get(t.handle, c_int32(a), c_int32(b), c_int32(c), ctypes.byref(out), _stream()),
+           "aded_trigram_get")
+    return out.value
+
+
+def aded_trigram_stats(t: Trigram):
+    e, b = c_uint64(), c_uint64()
+    _check(_lib.aded_trigram_stats(t.handle, ctypes.byref(e), ctypes.byref(b), _stream()), "aded_trigram_stats")
+    return e.value, b.value
+
+
+def aded_trigram_poll_status(t: Trigram) -> int:
+    out = c_int32()
+    _check(_lib.aded_trigram_poll_status(t.handle, ctypes.byref(out), _stream()), "aded_trigram_poll_status")
+    return out.value
+
+
+def aded_status_string(status: int) -> str:
+    return _lib.aded_status_string(c_int32(status)).decode()

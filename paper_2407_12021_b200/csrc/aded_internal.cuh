@@ -1,0 +1,116 @@
+// Internal declarations shared by the library's translation units (not part of the ABI).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <vector>
+
+#include "aded.h"
+
+#define ADED_CUDA_TRY(expr)                      \
+    do {                                         \
+        cudaError_t _e = (expr);                 \
+        if (_e != cudaSuccess) {                 \
+            aded::note_cuda_error(_e, #expr);    \
+            return ADED_ERR_CUDA;                \
+        }                                        \
+    } while (0)
+
+namespace aded {
+
+void note_cuda_error(cudaError_t e, const char* what);
+
+// ---- element types ---------------------------------------------------------------------
+typedef __nv_bfloat16 bf16;
+
+__device__ __forceinline__ float to_f32(float v) { return v; }
+__device__ __forceinline__ float to_f32(bf16 v) { return __bfloat162float(v); }
+template <typename T> __device__ __forceinline__ T from_f32(float v);
+template <> __device__ __forceinline__ float from_f32<float>(float v) { return v; }
+template <> __device__ __forceinline__ bf16 from_f32<bf16>(float v) { return __float2bfloat16_rn(v); }
+
+// ---- per-call row bookkeeping (device arrays sized for max_rows / max_batch) --------------
+struct RowMeta {
+    int32_t* seq;      // [R] sequence of the row
+    int32_t* local;    // [R] node index inside its tree
+    int32_t* depth;    // [R] edges from the root
+    int32_t* pos;      // [R] rotary position = committed length + depth
+    uint64_t* anc;     // [R][2] bit j set <=> local node j is an ancestor of the row's node, or itself
+};
+
+struct SeqMeta {
+    int32_t* row_off;  // [B+1] first row of each sequence
+    int32_t* path;     // [B][ADED_MAX_NODES] accepted path (local node indices), root first
+    int32_t* new_len;  // [B] committed length after this call
+};
+
+}  // namespace aded
+
+struct aded_kv {
+    const aded_model* model;
+    int device;
+    int batch;
+    size_t elem;                  // bytes per element
+    std::vector<int32_t> cap;     // host copy of capacities
+    std::vector<char*> base;      // host copy of the per-sequence block pointers (device memory)
+    char** base_dev;              // [B] device array of the same pointers
+    int32_t* cap_dev;             // [B]
+    int32_t* len_dev;             // [B] committed lengths
+};
+
+struct aded_model {
+    aded_model_config cfg;
+    int device;
+    aded_weights top;
+    std::vector<aded_layer_weights> layers;
+    size_t elem;
+
+    // activations, all [max_rows, *]
+    void* h;        // residual stream            [R, d]   model dtype
+    void* x;        // normalised input of a GEMM [R, d]
+    void* q;        // rotated queries            [R, d]
+    void* attn;     // attention output           [R, d]
+    void* act;      // SwiGLU product             [R, F]
+    float* y32;     // fp32 GEMM output, widest of 3d / 2F / d columns
+    float* logits;  // [R, V] fp32
+    float* rope_cos;  // [R, hd/2]
+    float* rope_sin;
+    int32_t* best;    // [R] greedy token per row
+    int32_t* tokens;  // [R] staging for the _host entry points
+    int32_t* parents;
+    int32_t* out_tokens;   // [R]
+    int32_t* out_len;      // [max_batch]
+    int32_t* status;  // device status word
+    aded::RowMeta rows;
+    aded::SeqMeta seqs;
+    std::vector<void*> owned;   // everything cudaMalloc'ed for this handle
+
+    float* dbg_logits;
+    int32_t* dbg_best;
+};
+
+namespace aded {
+
+// ---- launchers (each enqueues on `st`; shapes are validated by the callers) ---------------
+// tree.cu
+void launch_tree_prologue(aded_model* m, aded_kv* kv, const int32_t* tokens, const int32_t* parents,
+                          int batch, int chain_mode, cudaStream_t st);
+void launch_accept(aded_model* m, aded_kv* kv, const int32_t* tokens, const int32_t* parents, int batch,
+                   int32_t* out_tokens, int out_stride, int32_t* out_len, cudaStream_t st);
+void launch_compact_commit(aded_model* m, aded_kv* kv, int batch, int chain_mode, cudaStream_t st);
+
+// dense.cu
+void launch_embed(aded_model* m, const int32_t* tokens, int rows, cudaStream_t st);
+void launch_rope_table(aded_model* m, int rows, cudaStream_t st);
+void launch_add_rmsnorm(aded_model* m, const float* y, const void* gain, int rows, cudaStream_t st);
+void launch_gemm(aded_model* m, const void* x, const void* w, float* y, int rows, int n, int k, cudaStream_t st);
+void launch_rope_kv(aded_model* m, aded_kv* kv, int layer, int rows, cudaStream_t st);
+void launch_swiglu(aded_model* m, int rows, cudaStream_t st);
+void launch_argmax(aded_model* m, int rows, cudaStream_t st);
+
+// tree_attention.cu
+void launch_tree_attention(aded_model* m, aded_kv* kv, int layer, int batch, int rows, cudaStream_t st);
+
+}  // namespace aded

@@ -1,0 +1,360 @@
+// Host side of the verification step: handles, argument checks and the launch sequence of one
+// forward pass over a draft tree (see include/aded.h for the contract of every entry point).
+#include <cstdio>
+#include <cstring>
+#include <new>
+
+#include "aded_internal.cuh"
+
+namespace aded {
+
+static thread_local char g_last_cuda_error[256];
+
+void note_cuda_error(cudaError_t e, const char* what) {
+    snprintf(g_last_cuda_error, sizeof g_last_cuda_error, "%s: %s", what, cudaGetErrorString(e));
+    if (getenv("ADED_VERBOSE")) fprintf(stderr, "[aded] CUDA error: %s\n", g_last_cuda_error);
+    cudaGetLastError();
+}
+
+template <typename T>
+static aded_status dev_alloc(aded_model* m, T** p, size_t count) {
+    void* v = nullptr;
+    cudaError_t e = cudaMalloc(&v, count * sizeof(T) > 0 ? count * sizeof(T) : 1);
+    if (e != cudaSuccess) {
+        cudaGetLastError();
+        return e == cudaErrorMemoryAllocation ? ADED_ERR_OOM : ADED_ERR_CUDA;
+    }
+    m->owned.push_back(v);
+    *p = static_cast<T*>(v);
+    return ADED_OK;
+}
+
+#define TRY(expr) do { aded_status _s = (expr); if (_s != ADED_OK) return _s; } while (0)
+
+static aded_status alloc_model(aded_model* m) {
+    const aded_model_config& c = m->cfg;
+    const size_t R = c.max_rows, d = c.d_model, F = c.d_ffn, V = c.vocab, B = c.max_batch;
+    size_t wide = 3 * d;
+    if (2 * F > wide) wide = 2 * F;
+    char* p;
+    TRY(dev_alloc(m, &p, R * d * m->elem)); m->h = p;
+    TRY(dev_alloc(m, &p, R * d * m->elem)); m->x = p;
+    TRY(dev_alloc(m, &p, R * d * m->elem)); m->q = p;
+    TRY(dev_alloc(m, &p, R * d * m->elem)); m->attn = p;
+    TRY(dev_alloc(m, &p, R * F * m->elem)); m->act = p;
+    TRY(dev_alloc(m, &m->y32, R * wide));
+    TRY(dev_alloc(m, &m->logits, R * V));
+    TRY(dev_alloc(m, &m->rope_cos, R * (c.head_dim / 2)));
+    TRY(dev_alloc(m, &m->rope_sin, R * (c.head_dim / 2)));
+    TRY(dev_alloc(m, &m->best, R));
+    TRY(dev_alloc(m, &m->tokens, R));
+    TRY(dev_alloc(m, &m->parents, R));
+    TRY(dev_alloc(m, &m->out_tokens, R));
+    TRY(dev_alloc(m, &m->out_len, B));
+    TRY(dev_alloc(m, &m->status, 1));
+    TRY(dev_alloc(m, &m->rows.seq, R));
+    TRY(dev_alloc(m, &m->rows.local, R));
+    TRY(dev_alloc(m, &m->rows.depth, R));
+    TRY(dev_alloc(m, &m->rows.pos, R));
+    TRY(dev_alloc(m, &m->rows.anc, 2 * R));
+    TRY(dev_alloc(m, &m->seqs.row_off, B + 1));
+    TRY(dev_alloc(m, &m->seqs.path, B * ADED_MAX_NODES));
+    TRY(dev_alloc(m, &m->seqs.new_len, B));
+    ADED_CUDA_TRY(cudaMemset(m->status, 0, sizeof(int32_t)));
+    ADED_CUDA_TRY(cudaMemset(m->h, 0, R * d * m->elem));
+    ADED_CUDA_TRY(cudaMemset(m->x, 0, R * d * m->elem));
+    ADED_CUDA_TRY(cudaMemset(m->attn, 0, R * d * m->elem));
+    ADED_CUDA_TRY(cudaMemset(m->act, 0, R * F * m->elem));
+    return ADED_OK;
+}
+
+// The launch sequence of one pass.  chain_mode: the rows form a chain per sequence, every row is
+// accepted and no logits are needed (prefill).
+static aded_status forward(aded_model* m, aded_kv* kv, const int32_t* tokens, const int32_t* parents,
+                           const int32_t* offsets_host, int batch, int chain_mode, int32_t* out_tokens,
+                           int out_stride, int32_t* out_len, cudaStream_t st) {
+    const aded_model_config& c = m->cfg;
+    const int rows = offsets_host[batch];
+    const int d = c.d_model, F = c.d_ffn;
+    ADED_CUDA_TRY(cudaMemcpyAsync(m->seqs.row_off, offsets_host, (batch + 1) * sizeof(int32_t),
+                                  cudaMemcpyHostToDevice, st));
+    launch_tree_prologue(m, kv, tokens, parents, batch, chain_mode, st);
+    launch_embed(m, tokens, rows, st);
+    launch_rope_table(m, rows, st);
+    launch_add_rmsnorm(m, nullptr, m->layers[0].norm1, rows, st);
+    for (int l = 0; l < c.n_layers; ++l) {
+        const aded_layer_weights& w = m->layers[l];
+        launch_gemm(m, m->x, w.wqkv, m->y32, rows, 3 * d, d, st);
+        launch_rope_kv(m, kv, l, rows, st);
+        launch_tree_attention(m, kv, l, batch, rows, st);
+        launch_gemm(m, m->attn, w.wo, m->y32, rows, d, d, st);
+        launch_add_rmsnorm(m, m->y32, w.norm2, rows, st);
+        launch_gemm(m, m->x, w.wgu, m->y32, rows, 2 * F, d, st);
+        launch_swiglu(m, rows, st);
+        launch_gemm(m, m->act, w.wd, m->y32, rows, d, F, st);
+        const void* next_gain = l + 1 < c.n_layers ? m->layers[l + 1].norm1 : m->top.final_norm;
+        launch_add_rmsnorm(m, m->y32, next_gain, rows, st);
+    }
+    if (!chain_mode) {
+        launch_gemm(m, m->x, m->top.lm_head, m->logits, rows, c.vocab, d, st);
+        launch_argmax(m, rows, st);
+        if (m->dbg_logits)
+            ADED_CUDA_TRY(cudaMemcpyAsync(m->dbg_logits, m->logits, (size_t)rows * c.vocab * sizeof(float),
+                                          cudaMemcpyDeviceToDevice, st));
+        if (m->dbg_best)
+            ADED_CUDA_TRY(cudaMemcpyAsync(m->dbg_best, m->best, (size_t)rows * sizeof(int32_t),
+                                          cudaMemcpyDeviceToDevice, st));
+        m->dbg_logits = nullptr;
+        m->dbg_best = nullptr;
+        launch_accept(m, kv, tokens, parents, batch, out_tokens, out_stride, out_len, st);
+    }
+    launch_compact_commit(m, kv, batch, chain_mode, st);
+    ADED_CUDA_TRY(cudaGetLastError());
+    return ADED_OK;
+}
+
+}  // namespace aded
+
+using namespace aded;
+
+extern "C" {
+
+aded_status aded_model_create(const aded_model_config* cfg, const aded_weights* weights, aded_model** out) {
+    if (!cfg || !weights || !out || !weights->layers) return ADED_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (cfg->n_layers < 1 || cfg->d_model < 1 || cfg->n_heads < 1 || cfg->d_ffn < 1 || cfg->vocab < 1 ||
+        cfg->max_rows < 1 || cfg->max_batch < 1 || cfg->max_batch > cfg->max_rows)
+        return ADED_ERR_INVALID_ARG;
+    if (cfg->dtype != ADED_F32 && cfg->dtype != ADED_BF16) return ADED_ERR_INVALID_ARG;
+    if (cfg->head_dim != 64 && cfg->head_dim != 128) return ADED_ERR_UNSUPPORTED;
+    if (cfg->d_model != cfg->n_heads * cfg->head_dim) return ADED_ERR_INVALID_ARG;
+    if (cfg->d_model % 16 || cfg->d_ffn % 16) return ADED_ERR_UNSUPPORTED;
+    if (!weights->embed || !weights->final_norm || !weights->lm_head) return ADED_ERR_INVALID_ARG;
+    for (int l = 0; l < cfg->n_layers; ++l) {
+        const aded_layer_weights& w = weights->layers[l];
+        if (!w.wqkv || !w.wo || !w.wgu || !w.wd || !w.norm1 || !w.norm2) return ADED_ERR_INVALID_ARG;
+    }
+    aded_model* m = new (std::nothrow) aded_model();
+    if (!m) return ADED_ERR_OOM;
+    m->cfg = *cfg;
+    m->top = *weights;
+    m->layers.assign(weights->layers, weights->layers + cfg->n_layers);
+    m->top.layers = m->layers.data();
+    m->elem = cfg->dtype == ADED_BF16 ? 2 : 4;
+    m->dbg_logits = nullptr;
+    m->dbg_best = nullptr;
+    if (cudaGetDevice(&m->device) != cudaSuccess) {
+        delete m;
+        return ADED_ERR_CUDA;
+    }
+    aded_status s = alloc_model(m);
+    if (s != ADED_OK) {
+        aded_model_destroy(m);
+        return s;
+    }
+    *out = m;
+    return ADED_OK;
+}
+
+aded_status aded_model_destroy(aded_model* m) {
+    if (!m) return ADED_ERR_INVALID_ARG;
+    for (void* p : m->owned) cudaFree(p);
+    delete m;
+    return ADED_OK;
+}
+
+aded_status aded_kv_create(const aded_model* m, int32_t batch, const int32_t* capacity_host, aded_kv** out) {
+    if (!m || !capacity_host || !out || batch < 1 || batch > m->cfg.max_batch) return ADED_ERR_INVALID_ARG;
+    *out = nullptr;
+    for (int b = 0; b < batch; ++b)
+        if (capacity_host[b] < 1) return ADED_ERR_INVALID_ARG;
+    aded_kv* kv = new (std::nothrow) aded_kv();
+    if (!kv) return ADED_ERR_OOM;
+    kv->model = m;
+    kv->device = m->device;
+    kv->batch = batch;
+    kv->elem = m->elem;
+    kv->cap.assign(capacity_host, capacity_host + batch);
+    kv->base_dev = nullptr;
+    kv->cap_dev = nullptr;
+    kv->len_dev = nullptr;
+    const aded_model_config& c = m->cfg;
+    aded_status s = ADED_OK;
+    for (int b = 0; b < batch && s == ADED_OK; ++b) {
+        const size_t bytes = (size_t)c.n_layers * 2 * c.d_model * kv->cap[b] * kv->elem;
+        void* p = nullptr;
+        cudaError_t e = cudaMalloc(&p, bytes);
+        if (e != cudaSuccess) {
+            cudaGetLastError();
+            s = e == cudaErrorMemoryAllocation ? ADED_ERR_OOM : ADED_ERR_CUDA;
+            break;
+        }
+        kv->base.push_back(static_cast<char*>(p));
+    }
+    if (s == ADED_OK && (cudaMalloc((void**)&kv->base_dev, batch * sizeof(char*)) != cudaSuccess ||
+                         cudaMalloc((void**)&kv->cap_dev, batch * sizeof(int32_t)) != cudaSuccess ||
+                         cudaMalloc((void**)&kv->len_dev, batch * sizeof(int32_t)) != cudaSuccess))
+        s = ADED_ERR_OOM;
+    if (s == ADED_OK && (cudaMemcpy(kv->base_dev, kv->base.data(), batch * sizeof(char*), cudaMemcpyHostToDevice) != cudaSuccess ||
+                         cudaMemcpy(kv->cap_dev, kv->cap.data(), batch * sizeof(int32_t), cudaMemcpyHostToDevice) != cudaSuccess ||
+                         cudaMemset(kv->len_dev, 0, batch * sizeof(int32_t)) != cudaSuccess))
+        s = ADED_ERR_CUDA;
+    if (s != ADED_OK) {
+        cudaGetLastError();
+        aded_kv_destroy(kv);
+        return s;
+    }
+    *out = kv;
+    return ADED_OK;
+}
+
+aded_status aded_kv_destroy(aded_kv* kv) {
+    if (!kv) return ADED_ERR_INVALID_ARG;
+    for (char* p : kv->base) cudaFree(p);
+    if (kv->base_dev) cudaFree(kv->base_dev);
+    if (kv->cap_dev) cudaFree(kv->cap_dev);
+    if (kv->len_dev) cudaFree(kv->len_dev);
+    delete kv;
+    return ADED_OK;
+}
+
+aded_status aded_kv_len(const aded_kv* kv, int32_t seq, int32_t* out_len_host, void* stream) {
+    if (!kv || !out_len_host || seq < 0 || seq >= kv->batch) return ADED_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    ADED_CUDA_TRY(cudaMemcpyAsync(out_len_host, kv->len_dev + seq, sizeof(int32_t), cudaMemcpyDeviceToHost, st));
+    ADED_CUDA_TRY(cudaStreamSynchronize(st));
+    return ADED_OK;
+}
+
+// Copies between the caller's [head][n_pos][hd] arrays and one layer's K and V planes.
+static aded_status kv_copy(const aded_kv* kv, int seq, int layer, int pos0, int n_pos, void* k, void* v,
+                           bool into_cache, cudaStream_t st) {
+    const aded_model_config& c = kv->model->cfg;
+    const size_t row = (size_t)c.head_dim * kv->elem;
+    const size_t cap = kv->cap[seq];
+    for (int which = 0; which < 2; ++which) {
+        char* user = static_cast<char*>(which ? v : k);
+        char* plane = kv->base[seq] + (((size_t)layer * 2 + which) * c.n_heads * cap + pos0) * row;
+        // n_heads strided blocks of n_pos rows each
+        if (into_cache)
+            ADED_CUDA_TRY(cudaMemcpy2DAsync(plane, cap * row, user, (size_t)n_pos * row, (size_t)n_pos * row,
+                                            c.n_heads, cudaMemcpyDeviceToDevice, st));
+        else
+            ADED_CUDA_TRY(cudaMemcpy2DAsync(user, (size_t)n_pos * row, plane, cap * row, (size_t)n_pos * row,
+                                            c.n_heads, cudaMemcpyDeviceToDevice, st));
+    }
+    return ADED_OK;
+}
+
+aded_status aded_kv_load(aded_kv* kv, int32_t seq, int32_t layer, const void* k_dev, const void* v_dev,
+                         int32_t n_pos, void* stream) {
+    if (!kv || !k_dev || !v_dev || seq < 0 || seq >= kv->batch) return ADED_ERR_INVALID_ARG;
+    if (layer < 0 || layer >= kv->model->cfg.n_layers || n_pos < 1) return ADED_ERR_INVALID_ARG;
+    if (n_pos > kv->cap[seq]) return ADED_ERR_KV_CAPACITY;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    aded_status s = kv_copy(kv, seq, layer, 0, n_pos, const_cast<void*>(k_dev), const_cast<void*>(v_dev), true, st);
+    if (s != ADED_OK) return s;
+    ADED_CUDA_TRY(cudaMemcpyAsync(kv->len_dev + seq, &n_pos, sizeof(int32_t), cudaMemcpyHostToDevice, st));
+    ADED_CUDA_TRY(cudaStreamSynchronize(st));   // n_pos is a stack variable
+    return ADED_OK;
+}
+
+aded_status aded_kv_read(const aded_kv* kv, int32_t seq, int32_t layer, int32_t pos0, int32_t n_pos,
+                         void* k_dev, void* v_dev, void* stream) {
+    if (!kv || !k_dev || !v_dev || seq < 0 || seq >= kv->batch) return ADED_ERR_INVALID_ARG;
+    if (layer < 0 || layer >= kv->model->cfg.n_layers || pos0 < 0 || n_pos < 1) return ADED_ERR_INVALID_ARG;
+    if ((int64_t)pos0 + n_pos > kv->cap[seq]) return ADED_ERR_KV_CAPACITY;
+    return kv_copy(kv, seq, layer, pos0, n_pos, k_dev, v_dev, false, static_cast<cudaStream_t>(stream));
+}
+
+aded_status aded_append(aded_model* m, aded_kv* kv, int32_t seq, const int32_t* tokens_dev, int32_t n, void* stream) {
+    if (!m || !kv || !tokens_dev || kv->model != m) return ADED_ERR_INVALID_ARG;
+    if (kv->batch != 1 || seq != 0) return ADED_ERR_UNSUPPORTED;
+    if (n < 1 || n > ADED_MAX_NODES || n > m->cfg.max_rows) return ADED_ERR_INVALID_ARG;
+    const int32_t off[2] = {0, n};
+    return forward(m, kv, tokens_dev, nullptr, off, 1, 1, nullptr, 0, nullptr, static_cast<cudaStream_t>(stream));
+}
+
+aded_status aded_verify_batch(aded_model* m, aded_kv* kv, const int32_t* tree_offsets_host,
+                              const int32_t* tree_tokens_dev, const int32_t* tree_parents_dev,
+                              int32_t* out_tokens_dev, int32_t out_stride, int32_t* out_accept_len_dev,
+                              void* stream) {
+    if (!m || !kv || !tree_offsets_host || !tree_tokens_dev || !tree_parents_dev || !out_tokens_dev ||
+        !out_accept_len_dev || kv->model != m)
+        return ADED_ERR_INVALID_ARG;
+    const int batch = kv->batch;
+    if (tree_offsets_host[0] != 0) return ADED_ERR_INVALID_ARG;
+    for (int b = 0; b < batch; ++b) {
+        const int t = tree_offsets_host[b + 1] - tree_offsets_host[b];
+        if (t < 1 || t > ADED_MAX_NODES || t > out_stride) return ADED_ERR_INVALID_ARG;
+    }
+    if (tree_offsets_host[batch] > m->cfg.max_rows) return ADED_ERR_INVALID_ARG;
+    return forward(m, kv, tree_tokens_dev, tree_parents_dev, tree_offsets_host, batch, 0, out_tokens_dev,
+                   out_stride, out_accept_len_dev, static_cast<cudaStream_t>(stream));
+}
+
+aded_status aded_verify(aded_model* m, aded_kv* kv, const int32_t* tree_tokens_dev,
+                        const int32_t* tree_parents_dev, int32_t n_nodes, int32_t* out_tokens_dev,
+                        int32_t* out_accept_len_dev, void* stream) {
+    if (!kv || kv->batch != 1) return ADED_ERR_INVALID_ARG;
+    if (n_nodes < 1 || n_nodes > ADED_MAX_NODES) return ADED_ERR_INVALID_ARG;
+    const int32_t off[2] = {0, n_nodes};
+    return aded_verify_batch(m, kv, off, tree_tokens_dev, tree_parents_dev, out_tokens_dev, n_nodes,
+                             out_accept_len_dev, stream);
+}
+
+aded_status aded_verify_host(aded_model* m, aded_kv* kv, const int32_t* tree_tokens_host,
+                             const int32_t* tree_parents_host, int32_t n_nodes, int32_t* out_tokens_host,
+                             int32_t* out_accept_len_host, void* stream) {
+    if (!m || !kv || !tree_tokens_host || !tree_parents_host || !out_tokens_host || !out_accept_len_host)
+        return ADED_ERR_INVALID_ARG;
+    if (n_nodes < 1 || n_nodes > ADED_MAX_NODES || n_nodes > m->cfg.max_rows) return ADED_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const size_t bytes = (size_t)n_nodes * sizeof(int32_t);
+    ADED_CUDA_TRY(cudaMemcpyAsync(m->tokens, tree_tokens_host, bytes, cudaMemcpyHostToDevice, st));
+    ADED_CUDA_TRY(cudaMemcpyAsync(m->parents, tree_parents_host, bytes, cudaMemcpyHostToDevice, st));
+    aded_status s = aded_verify(m, kv, m->tokens, m->parents, n_nodes, m->out_tokens, m->out_len, stream);
+    if (s != ADED_OK) return s;
+    ADED_CUDA_TRY(cudaMemcpyAsync(out_tokens_host, m->out_tokens, bytes, cudaMemcpyDeviceToHost, st));
+    ADED_CUDA_TRY(cudaMemcpyAsync(out_accept_len_host, m->out_len, sizeof(int32_t), cudaMemcpyDeviceToHost, st));
+    ADED_CUDA_TRY(cudaStreamSynchronize(st));
+    return ADED_OK;
+}
+
+aded_status aded_debug_capture(aded_model* m, float* logits_dev, int32_t* best_dev) {
+    if (!m) return ADED_ERR_INVALID_ARG;
+    m->dbg_logits = logits_dev;
+    m->dbg_best = best_dev;
+    return ADED_OK;
+}
+
+aded_status aded_model_poll_status(aded_model* m, aded_status* out_host, void* stream) {
+    if (!m || !out_host) return ADED_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    int32_t v = 0;
+    ADED_CUDA_TRY(cudaMemcpyAsync(&v, m->status, sizeof v, cudaMemcpyDeviceToHost, st));
+    ADED_CUDA_TRY(cudaStreamSynchronize(st));
+    if (v != 0) {
+        ADED_CUDA_TRY(cudaMemsetAsync(m->status, 0, sizeof v, st));
+        ADED_CUDA_TRY(cudaStreamSynchronize(st));
+    }
+    *out_host = static_cast<aded_status>(v);
+    return ADED_OK;
+}
+
+const char* aded_status_string(aded_status s) {
+    switch (s) {
+        case ADED_OK: return "ok";
+        case ADED_ERR_INVALID_ARG: return "invalid argument";
+        case ADED_ERR_BAD_TREE: return "malformed draft tree";
+        case ADED_ERR_KV_CAPACITY: return "KV cache capacity exceeded";
+        case ADED_ERR_TABLE_FULL: return "tri-gram store full";
+        case ADED_ERR_OOM: return "out of device memory";
+        case ADED_ERR_CUDA: return "CUDA runtime error";
+        case ADED_ERR_UNSUPPORTED: return "unsupported configuration";
+        case ADED_ERR_TIMEOUT: return "device-side wait ran out";
+    }
+    return "unknown status";
+}
+
+}  // extern "C"

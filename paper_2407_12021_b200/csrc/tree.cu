@@ -1,0 +1,153 @@
+// Draft-tree bookkeeping around the forward pass ("Draft Construction and Verification"):
+// validation + depths + ancestor masks before it, draft approval and cache compaction after it.
+#include "aded_internal.cuh"
+
+namespace aded {
+
+// One block per sequence, one thread per node.  Checks that node 0 is the only root and every
+// other node points at an earlier node, that tokens are in the vocabulary and that the cache has
+// room; then each thread climbs from its node to the root, collecting the ancestor bit set and
+// the depth.  The climb is bounded by the node count (parents decrease strictly).
+__global__ void k_tree_prologue(const int32_t* __restrict__ tokens, const int32_t* __restrict__ parents,
+                                const int32_t* __restrict__ row_off, const int32_t* __restrict__ len,
+                                const int32_t* __restrict__ cap, int vocab, int chain_mode,
+                                RowMeta rows, int32_t* status) {
+    const int b = blockIdx.x;
+    const int off = row_off[b];
+    const int T = row_off[b + 1] - off;
+    const int i = threadIdx.x;
+    __shared__ int s_bad;
+    if (i == 0) s_bad = 0;
+    __syncthreads();
+    if (*status != 0) return;   // an earlier error is still pending: do nothing
+    int p = -1;
+    if (i < T) {
+        p = chain_mode ? i - 1 : parents[off + i];
+        const int t = tokens[off + i];
+        if (t < 0 || t >= vocab) atomicMax(&s_bad, (int)ADED_ERR_INVALID_ARG);
+        if (i == 0 ? (p != -1) : (p < 0 || p >= i)) atomicMax(&s_bad, (int)ADED_ERR_BAD_TREE);
+    }
+    if (i == 0 && len[b] + T > cap[b]) atomicMax(&s_bad, (int)ADED_ERR_KV_CAPACITY);
+    __syncthreads();
+    if (s_bad != 0) {
+        if (i == 0) atomicCAS(status, 0, s_bad);
+        return;
+    }
+    if (i < T) {
+        uint64_t lo = 0, hi = 0;
+        int depth = 0, cur = i;
+        for (int step = 0; step < T; ++step) {
+            if (cur < 64) lo |= 1ull << cur; else hi |= 1ull << (cur - 64);
+            const int up = chain_mode ? cur - 1 : parents[off + cur];
+            if (up < 0) break;
+            cur = up;
+            ++depth;
+        }
+        const int r = off + i;
+        rows.seq[r] = b;
+        rows.local[r] = i;
+        rows.depth[r] = depth;
+        rows.pos[r] = len[b] + depth;
+        rows.anc[2 * r] = lo;
+        rows.anc[2 * r + 1] = hi;
+    }
+}
+
+// Draft approval, one thread per sequence (a tree has at most 128 nodes).  A node is approved when
+// its parent is approved and its token equals the model's greedy token at the parent; the deepest
+// approved node (lowest index among equals) ends the accepted path.  Emits the greedy token of
+// every path node: the approved drafts' successors, ending with the model's own next token.
+__global__ void k_accept(const int32_t* __restrict__ tokens, const int32_t* __restrict__ parents,
+                         const int32_t* __restrict__ row_off, const int32_t* __restrict__ best,
+                         const int32_t* __restrict__ depth, const int32_t* __restrict__ len,
+                         int32_t* __restrict__ path, int32_t* __restrict__ new_len,
+                         int32_t* __restrict__ out_tokens, int out_stride, int32_t* __restrict__ out_len,
+                         const int32_t* status, int batch) {
+    const int b = blockIdx.x * blockDim.x + threadIdx.x;
+    if (b >= batch) return;
+    if (*status != 0) {
+        out_len[b] = 0;
+        new_len[b] = len[b];
+        return;
+    }
+    const int off = row_off[b];
+    const int T = row_off[b + 1] - off;
+    uint64_t ok_lo = 1ull, ok_hi = 0ull;   // approved set; the root always is
+    int deepest = 0, deepest_depth = 0;
+    for (int i = 1; i < T; ++i) {
+        const int p = parents[off + i];
+        const bool p_ok = p < 64 ? (ok_lo >> p) & 1 : (ok_hi >> (p - 64)) & 1;
+        if (p_ok && tokens[off + i] == best[off + p]) {
+            if (i < 64) ok_lo |= 1ull << i; else ok_hi |= 1ull << (i - 64);
+            const int d = depth[off + i];
+            if (d > deepest_depth) { deepest_depth = d; deepest = i; }
+        }
+    }
+    // path[j] for j = depth .. 0 by climbing; the node at depth j is path element j
+    int cur = deepest;
+    for (int j = deepest_depth; j >= 0; --j) {
+        path[b * ADED_MAX_NODES + j] = cur;
+        out_tokens[(size_t)b * out_stride + j] = best[off + cur];
+        cur = parents[off + cur];
+    }
+    out_len[b] = deepest_depth + 1;
+    new_len[b] = len[b] + deepest_depth + 1;
+}
+
+// Compaction: the tree's K/V were written at slots L + node index; the accepted path p_0 = 0 <
+// p_1 < ... moves to slots L + 0, L + 1, ...  Because p_j >= j and the p_j increase, the source of a
+// later move is never the destination of an earlier one, and a thread that owns one element
+// column and walks j upwards reads every slot before it overwrites it.
+template <typename T>
+__global__ void k_compact(char* const* __restrict__ base, const int32_t* __restrict__ cap,
+                          const int32_t* __restrict__ len, const int32_t* __restrict__ new_len,
+                          const int32_t* __restrict__ path, int hd, const int32_t* status) {
+    if (*status != 0) return;
+    const int b = blockIdx.y;
+    const int n_acc = new_len[b] - len[b];
+    if (n_acc <= 1) return;
+    const size_t plane = (size_t)blockIdx.x;   // (layer * 2 + k|v) * H + head
+    T* p = reinterpret_cast<T*>(base[b]) + (plane * cap[b] + len[b]) * hd;
+    for (int e = threadIdx.x; e < hd; e += blockDim.x) {
+        for (int j = 1; j < n_acc; ++j) {
+            const int src = path[b * ADED_MAX_NODES + j];
+            if (src != j) p[(size_t)j * hd + e] = p[(size_t)src * hd + e];
+        }
+    }
+}
+
+__global__ void k_commit(int32_t* len, const int32_t* __restrict__ new_len, const int32_t* __restrict__ row_off,
+                         int chain_mode, const int32_t* status, int batch) {
+    const int b = blockIdx.x * blockDim.x + threadIdx.x;
+    if (b >= batch || *status != 0) return;
+    len[b] = chain_mode ? len[b] + (row_off[b + 1] - row_off[b]) : new_len[b];
+}
+
+void launch_tree_prologue(aded_model* m, aded_kv* kv, const int32_t* tokens, const int32_t* parents,
+                          int batch, int chain_mode, cudaStream_t st) {
+    k_tree_prologue<<<batch, ADED_MAX_NODES, 0, st>>>(tokens, parents, m->seqs.row_off, kv->len_dev, kv->cap_dev,
+                                                      m->cfg.vocab, chain_mode, m->rows, m->status);
+}
+
+void launch_accept(aded_model* m, aded_kv* kv, const int32_t* tokens, const int32_t* parents, int batch,
+                   int32_t* out_tokens, int out_stride, int32_t* out_len, cudaStream_t st) {
+    k_accept<<<(batch + 31) / 32, 32, 0, st>>>(tokens, parents, m->seqs.row_off, m->best, m->rows.depth,
+                                               kv->len_dev, m->seqs.path, m->seqs.new_len, out_tokens,
+                                               out_stride, out_len, m->status, batch);
+}
+
+void launch_compact_commit(aded_model* m, aded_kv* kv, int batch, int chain_mode, cudaStream_t st) {
+    if (!chain_mode) {
+        dim3 grid(m->cfg.n_layers * 2 * m->cfg.n_heads, batch);
+        if (m->cfg.dtype == ADED_BF16)
+            k_compact<bf16><<<grid, 128, 0, st>>>(kv->base_dev, kv->cap_dev, kv->len_dev, m->seqs.new_len,
+                                                  m->seqs.path, m->cfg.head_dim, m->status);
+        else
+            k_compact<float><<<grid, 128, 0, st>>>(kv->base_dev, kv->cap_dev, kv->len_dev, m->seqs.new_len,
+                                                   m->seqs.path, m->cfg.head_dim, m->status);
+    }
+    k_commit<<<(batch + 31) / 32, 32, 0, st>>>(kv->len_dev, m->seqs.new_len, m->seqs.row_off, chain_mode,
+                                               m->status, batch);
+}
+
+}  // namespace aded

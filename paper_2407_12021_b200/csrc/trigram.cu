@@ -1,0 +1,367 @@
+// Tri-gram store on the GPU (Eq. 1 counts, Algorithm 2 update, top-k continuation lookup).
+//
+// Layout: an array of 64-byte buckets.  The first 2^log2_buckets are "home" buckets, found by
+// hashing the two-token context (a, b) and probing linearly; a context owns its home bucket and,
+// when it has more than six continuations, a chain of overflow buckets taken from a bump
+// allocator.  A bucket holds the context key, the index of the next bucket of the chain (0 = none)
+// and six (token, count) entries that fill front to back and are never removed.  All contexts'
+// continuations are therefore reachable from one hash probe, which is what top-k needs, and an
+// update is one probe plus one atomic add.
+#include <cstdio>
+#include <new>
+
+#include "aded_internal.cuh"
+
+namespace aded {
+
+struct TgSlot { int32_t tok; uint32_t cnt; };
+struct __align__(64) Bucket {
+    unsigned long long key;
+    uint32_t next;
+    uint32_t pad;
+    TgSlot e[6];
+};
+static_assert(sizeof(Bucket) == 64, "bucket must be 64 bytes");
+
+constexpr unsigned long long TG_EMPTY = ~0ull;
+constexpr int TG_MAX_PROBE = 4096;
+
+struct TgView {
+    Bucket* buckets;
+    uint32_t n_home_mask;
+    uint32_t n_home;
+    uint32_t n_over;
+    uint32_t* over_used;
+    int32_t* status;
+    int32_t vocab;
+    uint32_t cap;
+    uint32_t min_count;
+};
+
+__device__ __forceinline__ uint32_t tg_hash(unsigned long long k) {
+    k ^= k >> 30; k *= 0xBF58476D1CE4E5B9ull;
+    k ^= k >> 27; k *= 0x94D049BB133111EBull;
+    k ^= k >> 31;
+    return (uint32_t)k;
+}
+
+__device__ __forceinline__ unsigned long long tg_key(int a, int b) {
+    return ((unsigned long long)(uint32_t)a << 32) | (uint32_t)b;
+}
+
+// Home bucket of a context; claims an empty one when `insert`.  Returns -1 if absent / no room.
+__device__ __forceinline__ int64_t tg_find_home(const TgView& t, unsigned long long key, bool insert) {
+    const uint32_t h = tg_hash(key);
+    const int limit = t.n_home < (uint32_t)TG_MAX_PROBE ? (int)t.n_home : TG_MAX_PROBE;
+    for (int probe = 0; probe < limit; ++probe) {
+        const uint32_t idx = (h + probe) & t.n_home_mask;
+        unsigned long long k = *reinterpret_cast<volatile unsigned long long*>(&t.buckets[idx].key);
+        if (k == key) return idx;
+        if (k == TG_EMPTY) {
+            if (!insert) return -1;
+            k = atomicCAS(&t.buckets[idx].key, TG_EMPTY, key);
+            if (k == TG_EMPTY || k == key) return idx;
+        }
+    }
+    return -1;
+}
+
+__global__ void k_tg_init(Bucket* b, size_t n) {
+    for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
+        Bucket z;
+        z.key = TG_EMPTY;
+        z.next = 0;
+        z.pad = 0;
+        for (int e = 0; e < 6; ++e) { z.e[e].tok = -1; z.e[e].cnt = 0; }
+        b[i] = z;
+    }
+}
+
+// Algorithm 2, one thread per window.  Duplicate windows inside one call are independent atomic
+// adds, so the result is min(count + multiplicity, cap) whatever the thread order.
+__global__ void k_tg_update(TgView t, const int32_t* __restrict__ tok, int n) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x + 2;
+    if (i >= n || *t.status != 0) return;
+    const int a = tok[i - 2], b = tok[i - 1], c = tok[i];
+    if (a < 0 || b < 0 || c < 0 || a >= t.vocab || b >= t.vocab || c >= t.vocab) {
+        atomicCAS(t.status, 0, (int)ADED_ERR_INVALID_ARG);
+        return;
+    }
+    const unsigned long long key = tg_key(a, b);
+    int64_t cur = tg_find_home(t, key, true);
+    if (cur < 0) { atomicCAS(t.status, 0, (int)ADED_ERR_TABLE_FULL); return; }
+    // a chain can never be longer than every overflow bucket plus the home bucket
+    for (uint32_t hop = 0; hop <= t.n_over; ++hop) {
+        Bucket* bk = t.buckets + cur;
+        for (int e = 0; e < 6; ++e) {
+            int32_t have = *reinterpret_cast<volatile int32_t*>(&bk->e[e].tok);
+            if (have == -1) have = atomicCAS(&bk->e[e].tok, -1, c) == -1 ? c : *reinterpret_cast<volatile int32_t*>(&bk->e[e].tok);
+            if (have == c) {
+                const uint32_t old = atomicAdd(&bk->e[e].cnt, 1u);
+                if (old >= t.cap) atomicMin(&bk->e[e].cnt, t.cap);
+                return;
+            }
+        }
+        uint32_t nxt = *reinterpret_cast<volatile uint32_t*>(&bk->next);
+        if (nxt == 0) {
+            const uint32_t fresh = atomicAdd(t.over_used, 1u);
+            if (fresh >= t.n_over) {
+                atomicCAS(t.status, 0, (int)ADED_ERR_TABLE_FULL);
+                return;
+            }
+            const uint32_t idx = t.n_home + fresh;
+            t.buckets[idx].key = key;
+            __threadfence();
+            const uint32_t prev = atomicCAS(&bk->next, 0u, idx);
+            nxt = prev == 0 ? idx : prev;   // lost the race: follow the winner (our bucket stays unused)
+        }
+        cur = nxt;
+    }
+    atomicCAS(t.status, 0, (int)ADED_ERR_TIMEOUT);
+}
+
+// One warp per query.  k selection rounds over the context's chain; a round picks the largest
+// packed (count, ~token) strictly below the previous pick, which yields count descending, token
+// ascending among equals, without storing the list.
+__global__ void k_tg_topk(TgView t, const int32_t* __restrict__ ctx, int q, int k, int32_t* __restrict__ out_tok,
+                          uint32_t* __restrict__ out_cnt, uint32_t* __restrict__ out_total) {
+    const int w = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int lane = threadIdx.x & 31;
+    if (w >= q) return;
+    const int a = ctx[2 * w], b = ctx[2 * w + 1];
+    int64_t home = -1;
+    if (a >= 0 && b >= 0 && a < t.vocab && b < t.vocab) home = tg_find_home(t, tg_key(a, b), false);
+    unsigned long long prev = ~0ull;
+    for (int round = 0; round < k; ++round) {
+        unsigned long long best = 0;
+        uint32_t total = 0;
+        int64_t cur = home;
+        for (uint32_t hop = 0; cur >= 0 && hop <= t.n_over; ++hop) {
+            const Bucket* bk = t.buckets + cur;
+            if (lane < 6) {
+                const int32_t tk = bk->e[lane].tok;
+                const uint32_t cn = bk->e[lane].cnt;
+                if (tk >= 0) {
+                    total += cn;
+                    const unsigned long long key = ((unsigned long long)cn << 32) | (0xFFFFFFFFu - (uint32_t)tk);
+                    if (cn >= t.min_count && cn > 0 && key < prev && key > best) best = key;
+                }
+            }
+            const uint32_t nxt = bk->next;
+            cur = nxt == 0 ? -1 : (int64_t)nxt;
+        }
+        for (int o = 16; o > 0; o >>= 1) {
+            const unsigned long long ob = __shfl_xor_sync(0xffffffffu, best, o);
+            if (ob > best) best = ob;
+            total += __shfl_xor_sync(0xffffffffu, total, o);
+        }
+        if (lane == 0) {
+            out_tok[(size_t)w * k + round] = best ? (int32_t)(0xFFFFFFFFu - (uint32_t)best) : -1;
+            out_cnt[(size_t)w * k + round] = (uint32_t)(best >> 32);
+            if (round == 0 && out_total) out_total[w] = total;
+        }
+        prev = best ? best : 0;   // nothing left: later rounds find nothing either
+    }
+}
+
+__global__ void k_tg_get(TgView t, int a, int b, int c, uint32_t* out) {
+    *out = 0;
+    if (a < 0 || b < 0 || c < 0 || a >= t.vocab || b >= t.vocab || c >= t.vocab) return;
+    int64_t cur = tg_find_home(t, tg_key(a, b), false);
+    for (uint32_t hop = 0; cur >= 0 && hop <= t.n_over; ++hop) {
+        const Bucket* bk = t.buckets + cur;
+        for (int e = 0; e < 6; ++e)
+            if (bk->e[e].tok == c) { *out = bk->e[e].cnt; return; }
+        cur = bk->next == 0 ? -1 : (int64_t)bk->next;
+    }
+}
+
+__global__ void k_tg_stats(TgView t, unsigned long long* out) {
+    unsigned long long entries = 0, used = 0;
+    const size_t n = (size_t)t.n_home + t.n_over;
+    for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
+        const Bucket* bk = t.buckets + i;
+        int here = 0;
+        for (int e = 0; e < 6; ++e) here += bk->e[e].tok >= 0;
+        entries += here;
+        used += bk->key != TG_EMPTY;
+    }
+    atomicAdd(out, entries);
+    atomicAdd(out + 1, used);
+}
+
+}  // namespace aded
+
+struct aded_trigram {
+    aded_trigram_config cfg;
+    int device;
+    aded::TgView view;
+    int32_t* stage_i;    // staging for the _host entry points
+    uint32_t* stage_u;
+    size_t stage_n;
+    unsigned long long* stats_dev;
+};
+
+using namespace aded;
+
+static constexpr size_t TG_STAGE = 1 << 16;
+
+extern "C" {
+
+aded_status aded_trigram_create(const aded_trigram_config* cfg, aded_trigram** out) {
+    if (!cfg || !out) return ADED_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (cfg->vocab < 1 || cfg->log2_buckets < 4 || cfg->log2_buckets > 28 || cfg->overflow_buckets < 0)
+        return ADED_ERR_INVALID_ARG;
+    aded_trigram* t = new (std::nothrow) aded_trigram();
+    if (!t) return ADED_ERR_OOM;
+    t->cfg = *cfg;
+    t->stage_i = nullptr;
+    t->stage_u = nullptr;
+    t->stats_dev = nullptr;
+    t->view = TgView();
+    const size_t n_home = (size_t)1 << cfg->log2_buckets, n = n_home + (size_t)cfg->overflow_buckets;
+    bool ok = cudaGetDevice(&t->device) == cudaSuccess;
+    cudaError_t e = cudaSuccess;
+    if (ok) { e = cudaMalloc((void**)&t->view.buckets, n * sizeof(Bucket)); ok = e == cudaSuccess; }
+    if (ok) ok = cudaMalloc((void**)&t->view.over_used, sizeof(uint32_t)) == cudaSuccess;
+    if (ok) ok = cudaMalloc((void**)&t->view.status, sizeof(int32_t)) == cudaSuccess;
+    if (ok) ok = cudaMalloc((void**)&t->stage_i, TG_STAGE * sizeof(int32_t)) == cudaSuccess;
+    if (ok) ok = cudaMalloc((void**)&t->stage_u, TG_STAGE * sizeof(uint32_t)) == cudaSuccess;
+    if (ok) ok = cudaMalloc((void**)&t->stats_dev, 2 * sizeof(unsigned long long)) == cudaSuccess;
+    if (!ok) {
+        cudaGetLastError();
+        aded_trigram_destroy(t);
+        return e == cudaErrorMemoryAllocation ? ADED_ERR_OOM : ADED_ERR_CUDA;
+    }
+    t->view.n_home = (uint32_t)n_home;
+    t->view.n_home_mask = (uint32_t)n_home - 1;
+    t->view.n_over = (uint32_t)cfg->overflow_buckets;
+    t->view.vocab = cfg->vocab;
+    t->view.cap = cfg->cap == 0 ? 0x7fffffffu : cfg->cap;
+    t->view.min_count = cfg->min_count;
+    k_tg_init<<<1024, 256>>>(t->view.buckets, n);
+    ok = cudaMemset(t->view.over_used, 0, sizeof(uint32_t)) == cudaSuccess &&
+         cudaMemset(t->view.status, 0, sizeof(int32_t)) == cudaSuccess && cudaDeviceSynchronize() == cudaSuccess;
+    if (!ok) {
+        cudaGetLastError();
+        aded_trigram_destroy(t);
+        return ADED_ERR_CUDA;
+    }
+    *out = t;
+    return ADED_OK;
+}
+
+aded_status aded_trigram_destroy(aded_trigram* t) {
+    if (!t) return ADED_ERR_INVALID_ARG;
+    if (t->view.buckets) cudaFree(t->view.buckets);
+    if (t->view.over_used) cudaFree(t->view.over_used);
+    if (t->view.status) cudaFree(t->view.status);
+    if (t->stage_i) cudaFree(t->stage_i);
+    if (t->stage_u) cudaFree(t->stage_u);
+    if (t->stats_dev) cudaFree(t->stats_dev);
+    delete t;
+    return ADED_OK;
+}
+
+aded_status aded_trigram_update(aded_trigram* t, const int32_t* tokens_dev, int32_t n, void* stream) {
+    if (!t || n < 0 || (n > 0 && !tokens_dev)) return ADED_ERR_INVALID_ARG;
+    if (n < 3) return ADED_OK;
+    const int windows = n - 2;
+    k_tg_update<<<(windows + 255) / 256, 256, 0, static_cast<cudaStream_t>(stream)>>>(t->view, tokens_dev, n);
+    ADED_CUDA_TRY(cudaGetLastError());
+    return ADED_OK;
+}
+
+aded_status aded_trigram_update_host(aded_trigram* t, const int32_t* tokens_host, int32_t n, void* stream) {
+    if (!t || n < 0 || (n > 0 && !tokens_host)) return ADED_ERR_INVALID_ARG;
+    if (n < 3) return ADED_OK;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    // long spans go through the staging buffer in pieces that overlap by two tokens
+    for (int64_t lo = 0; lo + 2 < n; lo += (int64_t)TG_STAGE - 2) {
+        const int64_t m = n - lo < (int64_t)TG_STAGE ? n - lo : (int64_t)TG_STAGE;
+        ADED_CUDA_TRY(cudaMemcpyAsync(t->stage_i, tokens_host + lo, m * sizeof(int32_t), cudaMemcpyHostToDevice, st));
+        aded_status s = aded_trigram_update(t, t->stage_i, (int32_t)m, stream);
+        if (s != ADED_OK) return s;
+        ADED_CUDA_TRY(cudaStreamSynchronize(st));
+    }
+    return ADED_OK;
+}
+
+aded_status aded_trigram_topk(const aded_trigram* t, const int32_t* ctx_dev, int32_t q, int32_t k,
+                              int32_t* out_tokens_dev, uint32_t* out_counts_dev, uint32_t* out_total_dev,
+                              void* stream) {
+    if (!t || q < 0 || k < 1 || k > 32) return ADED_ERR_INVALID_ARG;
+    if (q == 0) return ADED_OK;
+    if (!ctx_dev || !out_tokens_dev || !out_counts_dev) return ADED_ERR_INVALID_ARG;
+    const int warps_per_block = 4;
+    k_tg_topk<<<(q + warps_per_block - 1) / warps_per_block, warps_per_block * 32, 0, static_cast<cudaStream_t>(stream)>>>(
+        t->view, ctx_dev, q, k, out_tokens_dev, out_counts_dev, out_total_dev);
+    ADED_CUDA_TRY(cudaGetLastError());
+    return ADED_OK;
+}
+
+aded_status aded_trigram_topk_host(const aded_trigram* t, const int32_t* ctx_host, int32_t q, int32_t k,
+                                   int32_t* out_tokens_host, uint32_t* out_counts_host, uint32_t* out_total_host,
+                                   void* stream) {
+    if (!t || q < 0 || k < 1 || k > 32) return ADED_ERR_INVALID_ARG;
+    if (q == 0) return ADED_OK;
+    if (!ctx_host || !out_tokens_host || !out_counts_host) return ADED_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    // staging: [ctx 2*qq | tokens qq*k] in stage_i, [counts qq*k | totals qq] in stage_u
+    const int per = (int)(TG_STAGE / (size_t)(k + 2));
+    for (int lo = 0; lo < q; lo += per) {
+        const int qq = q - lo < per ? q - lo : per;
+        int32_t* ctx_d = t->stage_i;
+        int32_t* tok_d = t->stage_i + 2 * qq;
+        uint32_t* cnt_d = t->stage_u;
+        uint32_t* tot_d = t->stage_u + (size_t)qq * k;
+        ADED_CUDA_TRY(cudaMemcpyAsync(ctx_d, ctx_host + 2 * (size_t)lo, 2 * (size_t)qq * sizeof(int32_t), cudaMemcpyHostToDevice, st));
+        aded_status s = aded_trigram_topk(t, ctx_d, qq, k, tok_d, cnt_d, tot_d, stream);
+        if (s != ADED_OK) return s;
+        ADED_CUDA_TRY(cudaMemcpyAsync(out_tokens_host + (size_t)lo * k, tok_d, (size_t)qq * k * sizeof(int32_t), cudaMemcpyDeviceToHost, st));
+        ADED_CUDA_TRY(cudaMemcpyAsync(out_counts_host + (size_t)lo * k, cnt_d, (size_t)qq * k * sizeof(uint32_t), cudaMemcpyDeviceToHost, st));
+        if (out_total_host)
+            ADED_CUDA_TRY(cudaMemcpyAsync(out_total_host + lo, tot_d, (size_t)qq * sizeof(uint32_t), cudaMemcpyDeviceToHost, st));
+        ADED_CUDA_TRY(cudaStreamSynchronize(st));
+    }
+    return ADED_OK;
+}
+
+aded_status aded_trigram_get(const aded_trigram* t, int32_t a, int32_t b, int32_t c, uint32_t* out_count_host, void* stream) {
+    if (!t || !out_count_host) return ADED_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    k_tg_get<<<1, 1, 0, st>>>(t->view, a, b, c, t->stage_u);
+    ADED_CUDA_TRY(cudaMemcpyAsync(out_count_host, t->stage_u, sizeof(uint32_t), cudaMemcpyDeviceToHost, st));
+    ADED_CUDA_TRY(cudaStreamSynchronize(st));
+    return ADED_OK;
+}
+
+aded_status aded_trigram_stats(const aded_trigram* t, uint64_t* out_entries_host, uint64_t* out_buckets_host, void* stream) {
+    if (!t || !out_entries_host || !out_buckets_host) return ADED_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    unsigned long long res[2] = {0, 0};
+    ADED_CUDA_TRY(cudaMemsetAsync(t->stats_dev, 0, sizeof res, st));
+    k_tg_stats<<<1024, 256, 0, st>>>(t->view, t->stats_dev);
+    ADED_CUDA_TRY(cudaMemcpyAsync(res, t->stats_dev, sizeof res, cudaMemcpyDeviceToHost, st));
+    ADED_CUDA_TRY(cudaStreamSynchronize(st));
+    *out_entries_host = res[0];
+    *out_buckets_host = res[1];
+    return ADED_OK;
+}
+
+aded_status aded_trigram_poll_status(aded_trigram* t, aded_status* out_host, void* stream) {
+    if (!t || !out_host) return ADED_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    int32_t v = 0;
+    ADED_CUDA_TRY(cudaMemcpyAsync(&v, t->view.status, sizeof v, cudaMemcpyDeviceToHost, st));
+    ADED_CUDA_TRY(cudaStreamSynchronize(st));
+    if (v != 0) {
+        ADED_CUDA_TRY(cudaMemsetAsync(t->view.status, 0, sizeof v, st));
+        ADED_CUDA_TRY(cudaStreamSynchronize(st));
+    }
+    *out_host = static_cast<aded_status>(v);
+    return ADED_OK;
+}
+
+}  // extern "C"
