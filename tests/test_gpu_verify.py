@@ -1,0 +1,193 @@
+"""GPU parity of the verification step against the CPU checker, through the C ABI."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import verify as ov
+from paper_2407_12021_b200 import inputs as gen
+from tests import helpers as H
+
+pytestmark = pytest.mark.gpu
+
+
+def _c1_setup(cuda_device, seed=11):
+    shape = gen.TINY
+    w = gen.model_weights(shape, seed)
+    sess = H.GpuSession(shape, H.weights_to(w, cuda_device), capacity=256)
+    arch = ov.arch_from_shape(shape)
+    ow = ov.Weights(w, keep=True)
+    prompt = gen.zipf_tokens(64, shape.vocab, seed, 50).tolist()
+    cache = ov.Cache(arch)
+    ov.append(arch, ow, cache, prompt[:-1])
+    sess.append(prompt[:-1])
+    assert sess.length() == 63
+    return shape, arch, ow, cache, sess, prompt
+
+
+def test_c1_tiny_fp32_tree(cuda_device):
+    """Workload 1: 2-layer fp32 decoder, 64-token Zipf prompt, 16-node depth-4 tree."""
+    shape, arch, ow, cache, sess, prompt = _c1_setup(cuda_device)
+    H.compare_cache(shape, sess, cache, 0, 63, range(shape.n_layers), "prefill")
+    tokens, parents = gen.make_tree(16, 4, 4, shape.vocab, 3, root_token=prompt[-1])
+    cpu = ov.verify(arch, ow, cache, tokens, parents)
+    gpu = sess.verify(tokens, parents)
+    assert gpu["status"] == 0
+    worst = H.compare_step(shape, gpu, cpu, tokens, parents, "c1")
+    assert worst["flipped"] == 0
+    assert sess.length() == cache.length
+    H.compare_cache(shape, sess, cache, 63, cpu["accept_len"], range(shape.n_layers), "after verify")
+
+
+def test_c1_planted_paths_and_multi_step(cuda_device):
+    """Accept lengths 1..5: plant the checker's own greedy continuation on the deep chain, then keep
+    decoding from the resulting cache so that compaction errors would surface in the next step."""
+    shape, arch, ow, cache, sess, prompt = _c1_setup(cuda_device, seed=12)
+    # the checker's autoregressive continuation
+    probe = cache.clone()
+    cur, ar = prompt[-1], []
+    for _ in range(24):
+        cur = ov.verify(arch, ow, probe, [cur], [-1])["out_tokens"][0]
+        ar.append(cur)
+    done = 0
+    root = prompt[-1]
+    seen = set()
+    for step, p in enumerate([2, 0, 4, 1, 3, 4]):
+        tokens, parents = gen.make_tree(16, 4, 4, shape.vocab, 100 + step, root_token=root)
+        tokens = gen.plant_path(tokens, parents, ar[done:done + p])
+        cpu = ov.verify(arch, ow, cache, tokens, parents)
+        gpu = sess.verify(tokens, parents)
+        assert gpu["status"] == 0
+        worst = H.compare_step(shape, gpu, cpu, tokens, parents, f"step {step}")
+        assert worst["flipped"] == 0
+        assert cpu["accept_len"] >= p + 1
+        seen.add(cpu["accept_len"])
+        assert gpu["out_tokens"] == ar[done:done + cpu["accept_len"]]
+        done += cpu["accept_len"]
+        root = gpu["out_tokens"][-1]
+        assert sess.length() == cache.length == 63 + done
+        H.compare_cache(shape, sess, cache, 63, done, range(shape.n_layers), f"cache after step {step}")
+    assert {1, 2, 3, 5} <= seen
+
+
+def test_scattered_accept_path_is_compacted(cuda_device):
+    shape, arch, ow, cache, sess, prompt = _c1_setup(cuda_device, seed=13)
+    probe = cache.clone()
+    cur, ar = prompt[-1], []
+    for _ in range(4):
+        cur = ov.verify(arch, ow, probe, [cur], [-1])["out_tokens"][0]
+        ar.append(cur)
+    wrong = lambda t: (t + 17) % shape.vocab
+    parents = [-1, 0, 0, 1, 1, 2, 2, 5, 5, 8]
+    tokens = [prompt[-1], wrong(ar[0]), ar[0], wrong(ar[1]), wrong(ar[0]), ar[1], wrong(ar[1]), wrong(ar[2]),
+              ar[2], wrong(ar[3])]
+    cpu = ov.verify(arch, ow, cache, tokens, parents)
+    assert cpu["path"] == [0, 2, 5, 8]
+    gpu = sess.verify(tokens, parents)
+    H.compare_step(shape, gpu, cpu, tokens, parents, "scattered")
+    assert gpu["out_tokens"] == ar[:4]
+    H.compare_cache(shape, sess, cache, 63, 4, range(shape.n_layers), "scattered path")
+    # the next step reads the compacted rows
+    tokens2, parents2 = gen.make_tree(9, 3, 3, shape.vocab, 5, root_token=ar[3])
+    cpu2 = ov.verify(arch, ow, cache, tokens2, parents2)
+    gpu2 = sess.verify(tokens2, parents2)
+    H.compare_step(shape, gpu2, cpu2, tokens2, parents2, "after compaction")
+
+
+def test_single_node_tree_is_autoregressive_decoding(cuda_device):
+    shape, arch, ow, cache, sess, prompt = _c1_setup(cuda_device, seed=14)
+    cur = prompt[-1]
+    for step in range(5):
+        cpu = ov.verify(arch, ow, cache, [cur], [-1])
+        gpu = sess.verify([cur], [-1])
+        H.compare_step(shape, gpu, cpu, [cur], [-1], f"ar {step}")
+        assert gpu["accept_len"] == 1
+        cur = gpu["out_tokens"][0]
+
+
+def test_chain_tree_equals_append(cuda_device):
+    """A chain verified as a tree leaves the same K/V rows as appending the same tokens."""
+    shape, arch, ow, cache, sess, prompt = _c1_setup(cuda_device, seed=15)
+    more = gen.zipf_tokens(7, shape.vocab, 15, 77).tolist()
+    sess.append(more)
+    k_app, v_app = sess.read_kv(1, 63, 7)
+    # a second session verifies the chain; whatever is accepted, slots 63.. hold the chain rows before compaction
+    w = gen.model_weights(shape, 15)
+    sess2 = H.GpuSession(shape, H.weights_to(w, cuda_device), capacity=256)
+    sess2.append(prompt[:-1])
+    gpu = sess2.verify(more, [-1] + list(range(6)))
+    n = gpu["accept_len"]
+    k2, v2 = sess2.read_kv(1, 63, n)
+    assert np.array_equal(k2, k_app[:, :n]) and np.array_equal(v2, v_app[:, :n])
+
+
+def test_device_detected_errors_leave_cache_unchanged(cuda_device):
+    shape, arch, ow, cache, sess, prompt = _c1_setup(cuda_device, seed=16)
+    before = sess.read_kv(0, 0, 63)
+    for tokens, parents, code in (([1, 2, 3], [-1, 2, 0], 2), ([1, 2, 3], [0, 0, 1], 2), ([1, 2, 3], [-1, -1, 0], 2),
+                                  ([1, shape.vocab, 3], [-1, 0, 0], 1)):
+        gpu = sess.verify(tokens, parents, capture=False)
+        assert gpu["status"] == code and gpu["accept_len"] == 0
+        assert gpu["out_raw"] == [-7] * len(tokens)
+        assert sess.length() == 63
+    after = sess.read_kv(0, 0, 63)
+    assert np.array_equal(before[0], after[0]) and np.array_equal(before[1], after[1])
+    # capacity: 63 cached + 200 > 256 is caught on the device ...
+    small = H.GpuSession(shape, H.weights_to(gen.model_weights(shape, 16), cuda_device), capacity=70)
+    small.append(prompt[:-1])
+    tokens, parents = gen.make_tree(16, 4, 4, shape.vocab, 3)
+    gpu = small.verify(tokens, parents, capture=False)
+    assert gpu["status"] == 3 and gpu["accept_len"] == 0 and small.length() == 63
+    # ... and the handle works again after the status was read
+    gpu = small.verify(tokens[:5], [-1, 0, 1, 2, 3], capture=False)
+    assert gpu["status"] == 0 and gpu["accept_len"] >= 1
+    # host-detected: too many nodes
+    from paper_2407_12021_b200.binding import AdedError
+    with pytest.raises(AdedError):
+        sess.verify(list(range(129)), [-1] + list(range(128)), capture=False)
+
+
+def test_verify_host_entry_point(cuda_device):
+    shape, arch, ow, cache, sess, prompt = _c1_setup(cuda_device, seed=17)
+    tokens, parents = gen.make_tree(16, 4, 4, shape.vocab, 9, root_token=prompt[-1])
+    cpu = ov.verify(arch, ow, cache, tokens, parents)
+    B = sess.B
+    t = torch.tensor(tokens, dtype=torch.int32).pin_memory()
+    p = torch.tensor(parents, dtype=torch.int32).pin_memory()
+    out = torch.zeros(16, dtype=torch.int32).pin_memory()
+    n = torch.zeros(1, dtype=torch.int32).pin_memory()
+    B.aded_verify_host(sess.model, sess.kv, t, p, out, n)
+    assert int(n[0]) == cpu["accept_len"] and out[:int(n[0])].tolist() == cpu["out_tokens"]
+
+
+def test_c2_one_7b_layer_bf16(cuda_device):
+    """Workload 2: one Llama-2-7B-shaped layer + LM head in bf16, cache pre-filled with 1024 N(0,1)
+    positions, 64-node depth-6 tree with branching <= 4."""
+    shape = gen.LLAMA7B_1L
+    w = gen.model_weights(shape, 21, device=cuda_device)
+    sess = H.GpuSession(shape, w, capacity=1024 + 128)
+    k, v = gen.kv_normal(shape, 1024, 21, 0, device=cuda_device)
+    sess.B.aded_kv_load(sess.kv, 0, 0, k, v)
+    assert sess.length() == 1024
+    arch = ov.arch_from_shape(shape)
+    ow = ov.Weights(w, keep=True)
+    cache = ov.Cache(arch)
+    cache.load(0, k, v)
+    tokens, parents = gen.make_tree(64, 6, 4, shape.vocab, 22)
+    cpu = ov.verify(arch, ow, cache, tokens, parents)
+    gpu = sess.verify(tokens, parents)
+    assert gpu["status"] == 0
+    worst = H.compare_step(shape, gpu, cpu, tokens, parents, "c2")
+    print("c2 worst", worst)
+    if worst["flipped"] == 0:
+        H.compare_cache(shape, sess, cache, 1024, cpu["accept_len"], [0], "c2 cache")
+    # planted: the checker's greedy tokens along the deep chain are accepted
+    cache2 = ov.Cache(arch)
+    cache2.load(0, k, v)
+    sess.B.aded_kv_load(sess.kv, 0, 0, k, v)
+    planted = list(tokens)
+    paths, _ = ov.paths_and_depths(parents)
+    planted[1] = int(cpu["best"][0])
+    cpu2 = ov.verify(arch, ow, cache2, planted, parents)
+    gpu2 = sess.verify(planted, parents)
+    H.compare_step(shape, gpu2, cpu2, planted, parents, "c2 planted")
+    assert cpu2["accept_len"] >= 2
