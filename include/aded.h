@@ -111,6 +111,10 @@ aded_status aded_kv_len(const aded_kv* kv, int32_t seq, int32_t* out_len_host, v
  * n_pos.  For workloads that start from a pre-filled cache. */
 aded_status aded_kv_load(aded_kv* kv, int32_t seq, int32_t layer, const void* k_dev, const void* v_dev,
                          int32_t n_pos, void* stream);
+/* Set the committed length of sequence `seq` to new_len (0 <= new_len <= capacity): roll a
+ * sequence back to an earlier point, e.g. to the end of its prompt.  Rows past new_len stay in
+ * memory and are overwritten by later calls. */
+aded_status aded_kv_set_len(aded_kv* kv, int32_t seq, int32_t new_len, void* stream);
 /* Copy out positions [pos0, pos0 + n_pos) of one layer: k_dev / v_dev receive
  * [head][n_pos][head_dim].  For tests. */
 aded_status aded_kv_read(const aded_kv* kv, int32_t seq, int32_t layer, int32_t pos0, int32_t n_pos,
@@ -158,6 +162,15 @@ aded_status aded_verify_host(aded_model* m, aded_kv* kv, const int32_t* tree_tok
 /* Ask the next verify call to also write every node's logits ([rows][vocab] fp32, may be NULL)
  * and greedy token ([rows] int32, may be NULL) to the given device buffers.  Parity checks only. */
 aded_status aded_debug_capture(aded_model* m, float* logits_dev, int32_t* best_dev);
+
+/* Per-kernel timing for roofline reports (not part of the paper's method).  Between begin and end
+ * every launch of the model's kernels is bracketed by CUDA events on its stream, grouped as
+ * 0 = projection/FFN/LM-head GEMMs, 1 = tree attention, 2 = everything else.  end() synchronises
+ * the stream and writes the summed milliseconds and launch counts of each group (arrays of 3). */
+aded_status aded_profile_begin(aded_model* m);
+aded_status aded_profile_end(aded_model* m, float* out_ms_host, int32_t* out_launches_host, void* stream);
+/* Kernels launched by this library in this process so far (all handles). */
+uint64_t aded_launch_count(void);
 
 /* Read and clear the model's device status word; synchronises `stream`. */
 aded_status aded_model_poll_status(aded_model* m, aded_status* out_host, void* stream);

@@ -24,8 +24,8 @@ STATUS_NAMES = {0: "ADED_OK", 1: "ADED_ERR_INVALID_ARG", 2: "ADED_ERR_BAD_TREE",
 
 EXPORTS = [
     "aded_model_create", "aded_model_destroy", "aded_kv_create", "aded_kv_destroy", "aded_kv_len",
-    "aded_kv_load", "aded_kv_read", "aded_append", "aded_verify", "aded_verify_batch", "aded_verify_host",
-    "aded_debug_capture", "aded_model_poll_status", "aded_trigram_create", "aded_trigram_destroy",
+    "aded_kv_load", "aded_kv_set_len", "aded_kv_read", "aded_append", "aded_verify", "aded_verify_batch", "aded_verify_host",
+    "aded_debug_capture", "aded_profile_begin", "aded_profile_end", "aded_launch_count", "aded_model_poll_status", "aded_trigram_create", "aded_trigram_destroy",
     "aded_trigram_update", "aded_trigram_update_host", "aded_trigram_topk", "aded_trigram_topk_host",
     "aded_trigram_get", "aded_trigram_stats", "aded_trigram_poll_status", "aded_status_string",
 ]
@@ -64,7 +64,7 @@ def load_library(path: str = _LIB_PATH) -> ctypes.CDLL:
     lib = ctypes.CDLL(path)
     for name in EXPORTS:
         fn = getattr(lib, name)          # AttributeError if the symbol is not exported
-        fn.restype = c_char_p if name == "aded_status_string" else c_int32
+        fn.restype = {"aded_status_string": c_char_p, "aded_launch_count": c_uint64}.get(name, c_int32)
     return lib
 
 
@@ -175,6 +175,10 @@ def aded_kv_load(kv: KV, seq: int, layer: int, k: torch.Tensor, v: torch.Tensor)
                              _stream()), "aded_kv_load")
 
 
+def aded_kv_set_len(kv: KV, seq: int, new_len: int) -> None:
+    _check(_lib.aded_kv_set_len(kv.handle, c_int32(seq), c_int32(new_len), _stream()), "aded_kv_set_len")
+
+
 def aded_kv_read(kv: KV, seq: int, layer: int, pos0: int, n_pos: int):
     cfg = kv.model.cfg
     dt = torch.bfloat16 if cfg.dtype == ADED_BF16 else torch.float32
@@ -235,6 +239,23 @@ def aded_debug_capture(model: Model, logits: Optional[torch.Tensor], best: Optio
     if best is not None:
         _dev_i32(best, "best")
     _check(_lib.aded_debug_capture(model.handle, _ptr(logits), _ptr(best)), "aded_debug_capture")
+
+
+def aded_profile_begin(model: Model) -> None:
+    _check(_lib.aded_profile_begin(model.handle), "aded_profile_begin")
+
+
+def aded_profile_end(model: Model):
+    """-> ({"gemm": ms, "attention": ms, "other": ms}, {"gemm": launches, ...})"""
+    ms = (c_float * 3)()
+    n = (c_int32 * 3)()
+    _check(_lib.aded_profile_end(model.handle, ms, n, _stream()), "aded_profile_end")
+    names = ("gemm", "attention", "other")
+    return dict(zip(names, [float(v) for v in ms])), dict(zip(names, [int(v) for v in n]))
+
+
+def aded_launch_count() -> int:
+    return int(_lib.aded_launch_count())
 
 
 def aded_model_poll_status(model: Model) -> int:

@@ -21,6 +21,10 @@
 namespace aded {
 
 void note_cuda_error(cudaError_t e, const char* what);
+void note_launch(int n = 1);   // bumps the process-wide launch counter
+
+enum { PROF_GEMM = 0, PROF_ATTN = 1, PROF_OTHER = 2, PROF_GROUPS = 3 };
+struct ProfSpan { int group; int launches; cudaEvent_t a, b; };
 
 // ---- element types ---------------------------------------------------------------------
 typedef __nv_bfloat16 bf16;
@@ -89,6 +93,10 @@ struct aded_model {
 
     float* dbg_logits;
     int32_t* dbg_best;
+
+    bool prof_on;
+    std::vector<aded::ProfSpan> prof_spans;   // spans recorded since aded_profile_begin
+    std::vector<cudaEvent_t> prof_pool;       // events kept for reuse
 };
 
 namespace aded {

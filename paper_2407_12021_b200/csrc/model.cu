@@ -1,6 +1,8 @@
 // Host side of the verification step: handles, argument checks and the launch sequence of one
 // forward pass over a draft tree (see include/aded.h for the contract of every entry point).
+#include <atomic>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <new>
 
@@ -15,6 +17,33 @@ void note_cuda_error(cudaError_t e, const char* what) {
     if (getenv("ADED_VERBOSE")) fprintf(stderr, "[aded] CUDA error: %s\n", g_last_cuda_error);
     cudaGetLastError();
 }
+
+static std::atomic<uint64_t> g_launches{0};
+void note_launch(int n) { g_launches.fetch_add((uint64_t)n, std::memory_order_relaxed); }
+
+// Brackets a group of launches with events while profiling is on; otherwise only counts them.
+struct Span {
+    aded_model* m;
+    cudaStream_t st;
+    ProfSpan rec;
+    bool on;
+    Span(aded_model* m_, int group, int launches, cudaStream_t st_) : m(m_), st(st_), on(m_->prof_on) {
+        note_launch(launches);
+        if (!on) return;
+        rec.group = group;
+        rec.launches = launches;
+        for (cudaEvent_t* e : {&rec.a, &rec.b}) {
+            if (!m->prof_pool.empty()) { *e = m->prof_pool.back(); m->prof_pool.pop_back(); }
+            else if (cudaEventCreate(e) != cudaSuccess) { on = false; cudaGetLastError(); return; }
+        }
+        cudaEventRecord(rec.a, st);
+    }
+    ~Span() {
+        if (!on) return;
+        cudaEventRecord(rec.b, st);
+        m->prof_spans.push_back(rec);
+    }
+};
 
 template <typename T>
 static aded_status dev_alloc(aded_model* m, T** p, size_t count) {
@@ -78,25 +107,29 @@ static aded_status forward(aded_model* m, aded_kv* kv, const int32_t* tokens, co
     const int d = c.d_model, F = c.d_ffn;
     ADED_CUDA_TRY(cudaMemcpyAsync(m->seqs.row_off, offsets_host, (batch + 1) * sizeof(int32_t),
                                   cudaMemcpyHostToDevice, st));
-    launch_tree_prologue(m, kv, tokens, parents, batch, chain_mode, st);
-    launch_embed(m, tokens, rows, st);
-    launch_rope_table(m, rows, st);
-    launch_add_rmsnorm(m, nullptr, m->layers[0].norm1, rows, st);
+    {
+        Span sp(m, PROF_OTHER, 4, st);
+        launch_tree_prologue(m, kv, tokens, parents, batch, chain_mode, st);
+        launch_embed(m, tokens, rows, st);
+        launch_rope_table(m, rows, st);
+        launch_add_rmsnorm(m, nullptr, m->layers[0].norm1, rows, st);
+    }
     for (int l = 0; l < c.n_layers; ++l) {
         const aded_layer_weights& w = m->layers[l];
-        launch_gemm(m, m->x, w.wqkv, m->y32, rows, 3 * d, d, st);
-        launch_rope_kv(m, kv, l, rows, st);
-        launch_tree_attention(m, kv, l, batch, rows, st);
-        launch_gemm(m, m->attn, w.wo, m->y32, rows, d, d, st);
-        launch_add_rmsnorm(m, m->y32, w.norm2, rows, st);
-        launch_gemm(m, m->x, w.wgu, m->y32, rows, 2 * F, d, st);
-        launch_swiglu(m, rows, st);
-        launch_gemm(m, m->act, w.wd, m->y32, rows, d, F, st);
+        { Span sp(m, PROF_GEMM, 1, st); launch_gemm(m, m->x, w.wqkv, m->y32, rows, 3 * d, d, st); }
+        { Span sp(m, PROF_OTHER, 1, st); launch_rope_kv(m, kv, l, rows, st); }
+        { Span sp(m, PROF_ATTN, 1, st); launch_tree_attention(m, kv, l, batch, rows, st); }
+        { Span sp(m, PROF_GEMM, 1, st); launch_gemm(m, m->attn, w.wo, m->y32, rows, d, d, st); }
+        { Span sp(m, PROF_OTHER, 1, st); launch_add_rmsnorm(m, m->y32, w.norm2, rows, st); }
+        { Span sp(m, PROF_GEMM, 1, st); launch_gemm(m, m->x, w.wgu, m->y32, rows, 2 * F, d, st); }
+        { Span sp(m, PROF_OTHER, 1, st); launch_swiglu(m, rows, st); }
+        { Span sp(m, PROF_GEMM, 1, st); launch_gemm(m, m->act, w.wd, m->y32, rows, d, F, st); }
         const void* next_gain = l + 1 < c.n_layers ? m->layers[l + 1].norm1 : m->top.final_norm;
-        launch_add_rmsnorm(m, m->y32, next_gain, rows, st);
+        { Span sp(m, PROF_OTHER, 1, st); launch_add_rmsnorm(m, m->y32, next_gain, rows, st); }
     }
     if (!chain_mode) {
-        launch_gemm(m, m->x, m->top.lm_head, m->logits, rows, c.vocab, d, st);
+        { Span sp(m, PROF_GEMM, 1, st); launch_gemm(m, m->x, m->top.lm_head, m->logits, rows, c.vocab, d, st); }
+        Span sp(m, PROF_OTHER, 2, st);
         launch_argmax(m, rows, st);
         if (m->dbg_logits)
             ADED_CUDA_TRY(cudaMemcpyAsync(m->dbg_logits, m->logits, (size_t)rows * c.vocab * sizeof(float),
@@ -108,7 +141,10 @@ static aded_status forward(aded_model* m, aded_kv* kv, const int32_t* tokens, co
         m->dbg_best = nullptr;
         launch_accept(m, kv, tokens, parents, batch, out_tokens, out_stride, out_len, st);
     }
-    launch_compact_commit(m, kv, batch, chain_mode, st);
+    {
+        Span sp(m, PROF_OTHER, chain_mode ? 1 : 2, st);
+        launch_compact_commit(m, kv, batch, chain_mode, st);
+    }
     ADED_CUDA_TRY(cudaGetLastError());
     return ADED_OK;
 }
@@ -143,6 +179,7 @@ aded_status aded_model_create(const aded_model_config* cfg, const aded_weights* 
     m->elem = cfg->dtype == ADED_BF16 ? 2 : 4;
     m->dbg_logits = nullptr;
     m->dbg_best = nullptr;
+    m->prof_on = false;
     if (cudaGetDevice(&m->device) != cudaSuccess) {
         delete m;
         return ADED_ERR_CUDA;
@@ -159,6 +196,8 @@ aded_status aded_model_create(const aded_model_config* cfg, const aded_weights* 
 aded_status aded_model_destroy(aded_model* m) {
     if (!m) return ADED_ERR_INVALID_ARG;
     for (void* p : m->owned) cudaFree(p);
+    for (ProfSpan& sp : m->prof_spans) { cudaEventDestroy(sp.a); cudaEventDestroy(sp.b); }
+    for (cudaEvent_t e : m->prof_pool) cudaEventDestroy(e);
     delete m;
     return ADED_OK;
 }
@@ -259,6 +298,15 @@ aded_status aded_kv_load(aded_kv* kv, int32_t seq, int32_t layer, const void* k_
     return ADED_OK;
 }
 
+aded_status aded_kv_set_len(aded_kv* kv, int32_t seq, int32_t new_len, void* stream) {
+    if (!kv || seq < 0 || seq >= kv->batch || new_len < 0) return ADED_ERR_INVALID_ARG;
+    if (new_len > kv->cap[seq]) return ADED_ERR_KV_CAPACITY;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    ADED_CUDA_TRY(cudaMemcpyAsync(kv->len_dev + seq, &new_len, sizeof(int32_t), cudaMemcpyHostToDevice, st));
+    ADED_CUDA_TRY(cudaStreamSynchronize(st));   // new_len is a stack variable
+    return ADED_OK;
+}
+
 aded_status aded_kv_read(const aded_kv* kv, int32_t seq, int32_t layer, int32_t pos0, int32_t n_pos,
                          void* k_dev, void* v_dev, void* stream) {
     if (!kv || !k_dev || !v_dev || seq < 0 || seq >= kv->batch) return ADED_ERR_INVALID_ARG;
@@ -327,6 +375,33 @@ aded_status aded_debug_capture(aded_model* m, float* logits_dev, int32_t* best_d
     m->dbg_best = best_dev;
     return ADED_OK;
 }
+
+aded_status aded_profile_begin(aded_model* m) {
+    if (!m) return ADED_ERR_INVALID_ARG;
+    for (ProfSpan& sp : m->prof_spans) { m->prof_pool.push_back(sp.a); m->prof_pool.push_back(sp.b); }
+    m->prof_spans.clear();
+    m->prof_on = true;
+    return ADED_OK;
+}
+
+aded_status aded_profile_end(aded_model* m, float* out_ms_host, int32_t* out_launches_host, void* stream) {
+    if (!m || !out_ms_host || !out_launches_host) return ADED_ERR_INVALID_ARG;
+    m->prof_on = false;
+    ADED_CUDA_TRY(cudaStreamSynchronize(static_cast<cudaStream_t>(stream)));
+    for (int g = 0; g < PROF_GROUPS; ++g) { out_ms_host[g] = 0.f; out_launches_host[g] = 0; }
+    for (ProfSpan& sp : m->prof_spans) {
+        float ms = 0.f;
+        ADED_CUDA_TRY(cudaEventElapsedTime(&ms, sp.a, sp.b));
+        out_ms_host[sp.group] += ms;
+        out_launches_host[sp.group] += sp.launches;
+        m->prof_pool.push_back(sp.a);
+        m->prof_pool.push_back(sp.b);
+    }
+    m->prof_spans.clear();
+    return ADED_OK;
+}
+
+uint64_t aded_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 
 aded_status aded_model_poll_status(aded_model* m, aded_status* out_host, void* stream) {
     if (!m || !out_host) return ADED_ERR_INVALID_ARG;

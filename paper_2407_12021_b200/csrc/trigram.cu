@@ -25,6 +25,8 @@ static_assert(sizeof(Bucket) == 64, "bucket must be 64 bytes");
 
 constexpr unsigned long long TG_EMPTY = ~0ull;
 constexpr int TG_MAX_PROBE = 4096;
+constexpr uint32_t TG_LOCKED = 0xFFFFFFFFu;   // `next` while its chain is being extended
+constexpr int TG_MAX_SPIN = 1 << 20;
 
 struct TgView {
     Bucket* buckets;
@@ -102,19 +104,33 @@ __global__ void k_tg_update(TgView t, const int32_t* __restrict__ tok, int n) {
                 return;
             }
         }
+        // Extend the chain under a one-word lock so that concurrent inserts into a hot context do
+        // not each take a bucket: the thread that swings `next` from 0 to TG_LOCKED allocates and
+        // publishes the index; the others wait for it, for a bounded number of polls.
         uint32_t nxt = *reinterpret_cast<volatile uint32_t*>(&bk->next);
         if (nxt == 0) {
-            const uint32_t fresh = atomicAdd(t.over_used, 1u);
-            if (fresh >= t.n_over) {
-                atomicCAS(t.status, 0, (int)ADED_ERR_TABLE_FULL);
-                return;
+            const uint32_t prev = atomicCAS(&bk->next, 0u, TG_LOCKED);
+            if (prev == 0) {
+                const uint32_t fresh = atomicAdd(t.over_used, 1u);
+                if (fresh >= t.n_over) {
+                    atomicExch(&bk->next, 0u);
+                    atomicCAS(t.status, 0, (int)ADED_ERR_TABLE_FULL);
+                    return;
+                }
+                nxt = t.n_home + fresh;
+                t.buckets[nxt].key = key;
+                __threadfence();
+                atomicExch(&bk->next, nxt);
+            } else {
+                nxt = prev;
             }
-            const uint32_t idx = t.n_home + fresh;
-            t.buckets[idx].key = key;
-            __threadfence();
-            const uint32_t prev = atomicCAS(&bk->next, 0u, idx);
-            nxt = prev == 0 ? idx : prev;   // lost the race: follow the winner (our bucket stays unused)
         }
+        for (int spin = 0; nxt == TG_LOCKED && spin < TG_MAX_SPIN; ++spin) {
+            __nanosleep(64);
+            nxt = *reinterpret_cast<volatile uint32_t*>(&bk->next);
+        }
+        if (nxt == TG_LOCKED) { atomicCAS(t.status, 0, (int)ADED_ERR_TIMEOUT); return; }
+        if (nxt == 0) return;   // the allocating thread ran out of buckets and has reported it
         cur = nxt;
     }
     atomicCAS(t.status, 0, (int)ADED_ERR_TIMEOUT);
@@ -268,6 +284,7 @@ aded_status aded_trigram_update(aded_trigram* t, const int32_t* tokens_dev, int3
     if (!t || n < 0 || (n > 0 && !tokens_dev)) return ADED_ERR_INVALID_ARG;
     if (n < 3) return ADED_OK;
     const int windows = n - 2;
+    note_launch();
     k_tg_update<<<(windows + 255) / 256, 256, 0, static_cast<cudaStream_t>(stream)>>>(t->view, tokens_dev, n);
     ADED_CUDA_TRY(cudaGetLastError());
     return ADED_OK;
@@ -295,6 +312,7 @@ aded_status aded_trigram_topk(const aded_trigram* t, const int32_t* ctx_dev, int
     if (q == 0) return ADED_OK;
     if (!ctx_dev || !out_tokens_dev || !out_counts_dev) return ADED_ERR_INVALID_ARG;
     const int warps_per_block = 4;
+    note_launch();
     k_tg_topk<<<(q + warps_per_block - 1) / warps_per_block, warps_per_block * 32, 0, static_cast<cudaStream_t>(stream)>>>(
         t->view, ctx_dev, q, k, out_tokens_dev, out_counts_dev, out_total_dev);
     ADED_CUDA_TRY(cudaGetLastError());

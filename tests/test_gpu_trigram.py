@@ -57,7 +57,7 @@ def test_incremental_updates_match_stepwise(cuda_device):
     from paper_2407_12021_b200 import binding as B
     stream = gen.zipf_tokens(3000, 50, 32, 1).tolist()     # tiny vocabulary: long chains, many duplicates
     st = TrigramStore()
-    t = B.aded_trigram_create(50, log2_buckets=8, overflow_buckets=2048)
+    t = B.aded_trigram_create(50, log2_buckets=12, overflow_buckets=2048)
     pos = 2
     lens = gen.randint(2000, 9, 32, 2)
     i = 0
