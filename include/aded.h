@@ -163,6 +163,13 @@ aded_status aded_verify_host(aded_model* m, aded_kv* kv, const int32_t* tree_tok
  * and greedy token ([rows] int32, may be NULL) to the given device buffers.  Parity checks only. */
 aded_status aded_debug_capture(aded_model* m, float* logits_dev, int32_t* best_dev);
 
+/* Run one of the model's projections alone, through the same kernel the verification step uses:
+ * y[rows, N] (fp32) = x[rows, K] (model dtype) * W^T, with W = layer `layer`'s wqkv (which = 0),
+ * wo (1), wgu (2), wd (3), or the LM head (4; layer ignored).  rows <= max_rows.  Parity checks of
+ * the dense contraction ("forward pass through the model", Introduction) only. */
+aded_status aded_debug_gemm(aded_model* m, int32_t layer, int32_t which, const void* x_dev, int32_t rows,
+                            float* y_dev, void* stream);
+
 /* Per-kernel timing for roofline reports (not part of the paper's method).  Between begin and end
  * every launch of the model's kernels is bracketed by CUDA events on its stream, grouped as
  * 0 = projection/FFN/LM-head GEMMs, 1 = tree attention, 2 = everything else.  end() synchronises

@@ -25,7 +25,7 @@ STATUS_NAMES = {0: "ADED_OK", 1: "ADED_ERR_INVALID_ARG", 2: "ADED_ERR_BAD_TREE",
 EXPORTS = [
     "aded_model_create", "aded_model_destroy", "aded_kv_create", "aded_kv_destroy", "aded_kv_len",
     "aded_kv_load", "aded_kv_set_len", "aded_kv_read", "aded_append", "aded_verify", "aded_verify_batch", "aded_verify_host",
-    "aded_debug_capture", "aded_profile_begin", "aded_profile_end", "aded_launch_count", "aded_model_poll_status", "aded_trigram_create", "aded_trigram_destroy",
+    "aded_debug_capture", "aded_debug_gemm", "aded_profile_begin", "aded_profile_end", "aded_launch_count", "aded_model_poll_status", "aded_trigram_create", "aded_trigram_destroy",
     "aded_trigram_update", "aded_trigram_update_host", "aded_trigram_topk", "aded_trigram_topk_host",
     "aded_trigram_get", "aded_trigram_stats", "aded_trigram_poll_status", "aded_status_string",
 ]
@@ -239,6 +239,21 @@ def aded_debug_capture(model: Model, logits: Optional[torch.Tensor], best: Optio
     if best is not None:
         _dev_i32(best, "best")
     _check(_lib.aded_debug_capture(model.handle, _ptr(logits), _ptr(best)), "aded_debug_capture")
+
+
+def aded_debug_gemm(model: Model, layer: int, which: int, x: torch.Tensor) -> torch.Tensor:
+    """y = x @ W^T in fp32 through the library's GEMM kernel; which: 0 wqkv, 1 wo, 2 wgu, 3 wd, 4 LM head."""
+    cfg = model.cfg
+    d, f = cfg.d_model, cfg.d_ffn
+    n = {0: 3 * d, 1: d, 2: 2 * f, 3: d, 4: cfg.vocab}[which]
+    k = f if which == 3 else d
+    dt = torch.bfloat16 if cfg.dtype == ADED_BF16 else torch.float32
+    if not (x.is_cuda and x.dtype == dt and x.is_contiguous() and x.dim() == 2 and x.shape[1] == k):
+        raise TypeError(f"x must be a contiguous CUDA {dt} tensor [rows, {k}]")
+    y = torch.empty((x.shape[0], n), dtype=torch.float32, device=x.device)
+    _check(_lib.aded_debug_gemm(model.handle, c_int32(layer), c_int32(which), _ptr(x), c_int32(x.shape[0]), _ptr(y),
+                                _stream()), "aded_debug_gemm")
+    return y
 
 
 def aded_profile_begin(model: Model) -> None:

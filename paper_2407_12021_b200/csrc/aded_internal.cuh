@@ -1,6 +1,7 @@
 // Internal declarations shared by the library's translation units (not part of the ABI).
 #pragma once
 
+#include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -94,6 +95,12 @@ struct aded_model {
     float* dbg_logits;
     int32_t* dbg_best;
 
+    // tensor-core GEMM path (bf16 models): TMA descriptors and split-tile scratch
+    bool ws_ready;
+    std::vector<CUtensorMap> ws_maps;   // per layer: wqkv, wo, wgu, wd; then lm_head; then x, attn, act
+    float* ws_slots;                    // partial tiles of CTAs that share a W tile
+    int32_t* ws_tile_count;             // arrival counters, zero between launches
+
     bool prof_on;
     std::vector<aded::ProfSpan> prof_spans;   // spans recorded since aded_profile_begin
     std::vector<cudaEvent_t> prof_pool;       // events kept for reuse
@@ -113,10 +120,21 @@ void launch_compact_commit(aded_model* m, aded_kv* kv, int batch, int chain_mode
 void launch_embed(aded_model* m, const int32_t* tokens, int rows, cudaStream_t st);
 void launch_rope_table(aded_model* m, int rows, cudaStream_t st);
 void launch_add_rmsnorm(aded_model* m, const float* y, const void* gain, int rows, cudaStream_t st);
-void launch_gemm(aded_model* m, const void* x, const void* w, float* y, int rows, int n, int k, cudaStream_t st);
+// w_map / x_map: indices into m->ws_maps of the operands' TMA descriptors (-1: none, plain kernel)
+void launch_gemm(aded_model* m, int w_map, int x_map, const void* x, const void* w, float* y, int rows, int n, int k,
+                 cudaStream_t st);
 void launch_rope_kv(aded_model* m, aded_kv* kv, int layer, int rows, cudaStream_t st);
 void launch_swiglu(aded_model* m, int rows, cudaStream_t st);
 void launch_argmax(aded_model* m, int rows, cudaStream_t st);
+
+// gemm_ws.cu
+bool ws_make_map(CUtensorMap* map, const void* ptr, uint64_t rows, uint64_t cols, uint32_t box_rows);
+bool ws_supported(int n, int k);
+int ws_grid_limit(int device);
+size_t ws_slot_floats(int device);
+cudaError_t ws_launch(const CUtensorMap& map_w, const CUtensorMap& map_x, float* y, int rows, int row0, int n, int k,
+                      float* slots, int32_t* tile_count, int32_t* status, int device, cudaStream_t st);
+enum { WS_MAP_QKV = 0, WS_MAP_O = 1, WS_MAP_GU = 2, WS_MAP_D = 3 };   // per-layer map order
 
 // tree_attention.cu
 void launch_tree_attention(aded_model* m, aded_kv* kv, int layer, int batch, int rows, cudaStream_t st);

@@ -214,7 +214,17 @@ static void launch_gemm_plain(aded_model* m, const void* x, const void* w, float
              (k_gemm_plain<float><<<grid, 256, 0, st>>>((const float*)x, (const float*)w, y, rows, n, k, m->status)));
 }
 
-void launch_gemm(aded_model* m, const void* x, const void* w, float* y, int rows, int n, int k, cudaStream_t st) {
+void launch_gemm(aded_model* m, int w_map, int x_map, const void* x, const void* w, float* y, int rows, int n, int k,
+                 cudaStream_t st) {
+    if (m->ws_ready && w_map >= 0 && x_map >= 0 && ws_supported(n, k)) {
+        // tensor-core path, 128 rows of x per pass over the weights
+        for (int row0 = 0; row0 < rows; row0 += 128) {
+            const int part = rows - row0 < 128 ? rows - row0 : 128;
+            ws_launch(m->ws_maps[w_map], m->ws_maps[x_map], y, part, row0, n, k, m->ws_slots, m->ws_tile_count,
+                      m->status, m->device, st);
+        }
+        return;
+    }
     launch_gemm_plain(m, x, w, y, rows, n, k, st);
 }
 

@@ -1,0 +1,394 @@
+// Weight-streaming bf16 GEMM for the decoder's projections, FFN and LM head on the 5th-generation
+// tensor cores (tcgen05, accumulators in TMEM, operands staged by TMA).
+//
+//   y[r, n] = sum_k x[r, k] * w[n, k]        r < rows <= 128,  w row-major [N, K], x row-major [R, K]
+//
+// A verification step multiplies at most 128 tree nodes with every weight matrix, so the kernel is
+// bound by reading W once from HBM.  Mapping:
+//   * the 128 rows of a W tile are the M dimension of the MMA (all 128 TMEM lanes busy), the tree
+//     nodes are its N dimension (rows padded to a multiple of 16), K advances 64 elements (one
+//     128-byte swizzled line) per pipeline stage;
+//   * work = (W tile, k block) units, split evenly over all resident CTAs (two per SM), so every CTA
+//     streams the same number of bytes whatever N and K are; a CTA's range covers the tail of one
+//     tile, whole tiles, and the head of another;
+//   * a tile shared by several CTAs is finished by whichever of them arrives last: each writes its
+//     fp32 partial to a private slot, bumps the tile's counter, and the last one adds the slots in
+//     CTA order -- a fixed order, so results do not depend on timing.  Nobody waits for anybody.
+//   * warp 0 issues TMA loads, warp 1 issues MMAs, warps 2..5 drain TMEM and run the epilogue; two
+//     TMEM accumulators let the MMAs of the next segment run under the epilogue of the last.
+// Every mbarrier wait is bounded; a wait that runs out raises ADED_ERR_TIMEOUT in the status word
+// and the CTA unwinds (drains its own copies, frees TMEM).
+#include <cuda.h>
+
+#include <cstdio>
+
+#include "aded_internal.cuh"
+
+namespace aded {
+
+constexpr int WS_BM = 128;           // W rows per tile (MMA M)
+constexpr int WS_BK = 64;            // k elements per stage (128 bytes of bf16)
+constexpr int WS_THREADS = 192;
+constexpr long long WS_WAIT_CYCLES = 4000000000ll;   // about two seconds of SM clock
+
+struct WsParams {
+    int rows;            // valid rows of x
+    int rb;              // rows padded to a multiple of 16 = MMA N
+    int row0;            // first row of x / y handled by this launch
+    int n, k;            // W is [n, k]
+    int n_tiles, kb;     // tiles of 128 W rows, k blocks per tile
+    int stages;
+    int tmem_cols;       // power of two >= 2 * rb
+    float* y;            // [R, n] fp32
+    float* slots;        // [gridDim.x][2][rb][128] fp32 partial tiles
+    int32_t* tile_count; // [n_tiles] arrival counters, zero between launches
+    int32_t* status;
+};
+
+// ---- PTX wrappers -------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+// Bounded wait for the phase with the given parity; false when the limit ran out.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
+    const uint32_t addr = smem_u32(bar);
+    const long long t0 = clock64();
+    for (uint32_t spin = 0;; ++spin) {
+        uint32_t done;
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(done) : "r"(addr), "r"(parity) : "memory");
+        if (done) return true;
+        if ((spin & 1023) == 1023 && clock64() - t0 > WS_WAIT_CYCLES) return false;
+    }
+}
+__device__ __forceinline__ void tma_load_2d(const CUtensorMap* map, uint64_t* bar, void* dst, int c0, int c1) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+        ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1) : "memory");
+}
+__device__ __forceinline__ void tma_load_2d_hint(const CUtensorMap* map, uint64_t* bar, void* dst, int c0, int c1,
+                                                 uint64_t policy) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%3, %4}], [%2], %5;"
+        ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "l"(policy) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint64_t* bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void tc_mma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// 16 consecutive fp32 columns of this warp's 32 TMEM lanes: register j = column col + j.
+__device__ __forceinline__ void tc_ld16(uint32_t taddr, float* v) {
+    uint32_t r[16];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr) : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int j = 0; j < 16; ++j) v[j] = __uint_as_float(r[j]);
+}
+
+// Shared-memory operand descriptor: K-major tile, 128-byte rows, 128B swizzle, 8-row groups 1024 B apart.
+__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr) {
+    uint64_t d = 0;
+    d |= (uint64_t)((addr & 0x3FFFF) >> 4);          // start address, 16-byte units
+    d |= (uint64_t)1 << 16;                          // leading byte offset (unused with swizzle)
+    d |= (uint64_t)(1024 >> 4) << 32;                // stride between 8-row groups
+    d |= (uint64_t)1 << 46;                          // descriptor version
+    d |= (uint64_t)2 << 61;                          // 128-byte swizzle
+    return d;
+}
+
+// First unit of CTA c when `units` units are split over `g` CTAs.
+__device__ __host__ __forceinline__ long long ws_start(long long c, long long units, long long g) { return c * units / g; }
+// CTA that owns unit u.
+__device__ __forceinline__ int ws_owner(long long u, long long units, long long g) {
+    long long c = ((u + 1) * g - 1) / units;
+    if (c >= g) c = g - 1;
+    while (c > 0 && ws_start(c, units, g) > u) --c;
+    while (c + 1 < g && ws_start(c + 1, units, g) <= u) ++c;
+    return (int)c;
+}
+
+__global__ void __launch_bounds__(WS_THREADS, 2)
+k_gemm_ws(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_x, WsParams p) {
+    extern __shared__ __align__(1024) uint8_t smem_raw[];
+    // carve: stages x (W tile 16 KB | x tile rb*128 B), then barriers
+    uint8_t* base = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    const uint32_t a_bytes = WS_BM * 128, b_bytes = (uint32_t)p.rb * 128, stage_bytes = a_bytes + b_bytes;
+    uint64_t* bars = (uint64_t*)(base + (size_t)p.stages * stage_bytes);
+    uint64_t* full = bars;
+    uint64_t* empty = bars + p.stages;
+    uint64_t* acc_full = bars + 2 * p.stages;
+    uint64_t* acc_empty = acc_full + 2;
+    uint32_t* s_tmem = (uint32_t*)(acc_empty + 2);
+    volatile int* s_flag = (volatile int*)(s_tmem + 1);   // [0] abort, [1] "this CTA finishes the tile", [2] live
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const long long units = (long long)p.n_tiles * p.kb;
+    const long long G = gridDim.x;
+    const long long u0 = ws_start(blockIdx.x, units, G), u1 = ws_start(blockIdx.x + 1, units, G);
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < p.stages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
+        for (int a = 0; a < 2; ++a) { mbar_init(&acc_full[a], 1); mbar_init(&acc_empty[a], 4); }
+        s_flag[0] = 0;
+        s_flag[1] = 0;
+        s_flag[2] = *p.status == 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(s_tmem)), "r"((uint32_t)p.tmem_cols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *s_tmem;
+    const bool live = s_flag[2] != 0 && u1 > u0;
+
+    if (warp == 0) {
+        // ---------------- TMA producer ----------------
+        if (lane == 0 && live) {
+            asm volatile("prefetch.tensormap [%0];" ::"l"(&map_w) : "memory");
+            asm volatile("prefetch.tensormap [%0];" ::"l"(&map_x) : "memory");
+            uint64_t pol_stream;
+            asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol_stream));
+            int s = 0;
+            uint32_t ph = 0;
+            for (long long u = u0; u < u1 && !s_flag[0]; ++u) {
+                const int tile = (int)(u / p.kb), kb = (int)(u % p.kb);
+                if (!mbar_wait(&empty[s], ph ^ 1)) { s_flag[0] = 1; atomicCAS(p.status, 0, (int)ADED_ERR_TIMEOUT); break; }
+                uint8_t* sa = base + (size_t)s * stage_bytes;
+                uint8_t* sb = sa + a_bytes;
+                mbar_expect_tx(&full[s], stage_bytes);
+                tma_load_2d_hint(&map_w, &full[s], sa, kb * WS_BK, tile * WS_BM, pol_stream);
+                for (int r = 0; r < p.rb; r += 16) tma_load_2d(&map_x, &full[s], sb + r * 128, kb * WS_BK, p.row0 + r);
+                if (++s == p.stages) { s = 0; ph ^= 1; }
+            }
+        }
+    } else if (warp == 1) {
+        // ---------------- MMA issuer ----------------
+        if (lane == 0 && live) {
+            const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(p.rb >> 3) << 17) | ((uint32_t)(WS_BM >> 4) << 24);
+            int s = 0;
+            uint32_t ph = 0;
+            int seg = 0;
+            long long u = u0;
+            while (u < u1 && !s_flag[0]) {
+                const int kb0 = (int)(u % p.kb);
+                long long ue = u + (p.kb - kb0);
+                if (ue > u1) ue = u1;
+                const int a = seg & 1;
+                const uint32_t aph = (uint32_t)(seg >> 1) & 1;
+                if (!mbar_wait(&acc_empty[a], aph ^ 1)) { s_flag[0] = 1; atomicCAS(p.status, 0, (int)ADED_ERR_TIMEOUT); break; }
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + (uint32_t)(a * p.rb);
+                bool first = true;
+                for (; u < ue; ++u) {
+                    if (!mbar_wait(&full[s], ph)) { s_flag[0] = 1; atomicCAS(p.status, 0, (int)ADED_ERR_TIMEOUT); break; }
+                    tc_fence_after();
+                    const uint32_t sa = smem_u32(base + (size_t)s * stage_bytes);
+                    const uint64_t da = smem_desc_sw128(sa), db = smem_desc_sw128(sa + a_bytes);
+#pragma unroll
+                    for (int kk = 0; kk < WS_BK / 16; ++kk) {
+                        tc_mma_bf16(d_tmem, da + (uint64_t)(kk * 2), db + (uint64_t)(kk * 2), idesc, first && kk == 0 ? 0u : 1u);
+                    }
+                    first = false;
+                    tc_commit(&empty[s]);      // stage reusable once these MMAs have read it
+                    if (++s == p.stages) { s = 0; ph ^= 1; }
+                }
+                if (s_flag[0]) break;
+                tc_commit(&acc_full[a]);       // accumulator complete
+                ++seg;
+            }
+        }
+    } else {
+        // ---------------- epilogue: warps 2..5, TMEM lane quarter = warp % 4 ----------------
+        const int quarter = warp & 3;
+        const int row_in_tile = quarter * 32 + lane;           // W row inside the tile = TMEM lane
+        const int ep_tid = threadIdx.x - 64;                   // 0..127
+        float* my_slots = p.slots + (size_t)blockIdx.x * 2 * p.rb * WS_BM;
+        int seg = 0;
+        long long u = u0;
+        // (the abort flag is not polled here: a stalled pipeline shows up as a timed-out wait below,
+        //  the same for all four warps, so they leave the loop together and never split at bar.sync)
+        while (live && u < u1) {
+            const int tile = (int)(u / p.kb), kb0 = (int)(u % p.kb);
+            long long ue = u + (p.kb - kb0);
+            if (ue > u1) ue = u1;
+            const bool whole = kb0 == 0 && ue - u == p.kb;
+            const int a = seg & 1;
+            const uint32_t aph = (uint32_t)(seg >> 1) & 1;
+            if (!mbar_wait(&acc_full[a], aph)) { s_flag[0] = 1; atomicCAS(p.status, 0, (int)ADED_ERR_TIMEOUT); break; }
+            tc_fence_after();
+            const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(a * p.rb);
+            const int n_glob = tile * WS_BM + row_in_tile;
+            float* slot = my_slots + (size_t)(kb0 == 0 ? 1 : 0) * p.rb * WS_BM;   // head of a tile -> slot 1, tail -> slot 0
+            for (int c0 = 0; c0 < p.rb; c0 += 16) {
+                float v[16];
+                tc_ld16(taddr + (uint32_t)c0, v);
+                if (whole) {
+                    if (n_glob < p.n) {
+#pragma unroll
+                        for (int j = 0; j < 16; ++j)
+                            if (c0 + j < p.rows) p.y[(size_t)(p.row0 + c0 + j) * p.n + n_glob] = v[j];
+                    }
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) slot[(size_t)(c0 + j) * WS_BM + row_in_tile] = v[j];
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&acc_empty[a]);
+            if (!whole) {
+                // publish the partial, learn whether this CTA is the last contributor of the tile
+                __threadfence();
+                asm volatile("bar.sync 1, 128;" ::: "memory");
+                const int c_first = ws_owner((long long)tile * p.kb, units, G);
+                const int c_last = ws_owner((long long)(tile + 1) * p.kb - 1, units, G);
+                if (ep_tid == 0) {
+                    const int prev = atomicAdd(&p.tile_count[tile], 1);
+                    const int last = prev == c_last - c_first;
+                    if (last) p.tile_count[tile] = 0;          // everyone has arrived: reset for the next launch
+                    s_flag[1] = last;
+                }
+                asm volatile("bar.sync 1, 128;" ::: "memory");
+                if (s_flag[1]) {
+                    __threadfence();
+                    if (n_glob < p.n) {
+                        for (int c = 0; c < p.rows; ++c) {
+                            float sum = 0.f;
+                            for (int cc = c_first; cc <= c_last; ++cc) {
+                                // contributor cc holds the tile's head in slot 1 if it started the tile, else its tail in slot 0
+                                const int which = cc == c_first ? 1 : 0;
+                                const float* src = p.slots + ((size_t)cc * 2 + which) * p.rb * WS_BM;
+                                sum += __ldcg(src + (size_t)c * WS_BM + row_in_tile);
+                            }
+                            p.y[(size_t)(p.row0 + c) * p.n + n_glob] = sum;
+                        }
+                    }
+                }
+                asm volatile("bar.sync 1, 128;" ::: "memory");   // s_flag[1] may be rewritten next segment
+            }
+            u = ue;
+            ++seg;
+        }
+    }
+
+    // ---------------- teardown ----------------
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0 && lane == 0 && s_flag[0]) {
+        // unwinding after a timeout: give copies that are still in flight time to land (bounded)
+        for (int i = 0; i < 1000; ++i) __nanosleep(1000);
+    }
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)p.tmem_cols) : "memory");
+    }
+}
+
+// ---- host side --------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    return fn;
+}
+
+// 2-D bf16 tensor [rows, cols] row-major, box = box_rows x 64 columns, 128-byte swizzle.
+bool ws_make_map(CUtensorMap* map, const void* ptr, uint64_t rows, uint64_t cols, uint32_t box_rows) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[2] = {cols, rows};
+    const cuuint64_t strides[1] = {cols * 2};
+    const cuuint32_t box[2] = {WS_BK, box_rows};
+    const cuuint32_t elem[2] = {1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, elem,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+int ws_grid_limit(int device) {
+    static int cached_dev = -1, cached = 0;
+    if (cached_dev != device) {
+        int sms = 0;
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device);
+        cached = 2 * sms;
+        cached_dev = device;
+    }
+    return cached;
+}
+
+size_t ws_slot_floats(int device) { return (size_t)ws_grid_limit(device) * 2 * 128 * WS_BM; }
+
+// Shapes the tensor-core path takes.
+bool ws_supported(int n, int k) { return n % WS_BM == 0 && k % WS_BK == 0 && k >= WS_BK; }
+
+cudaError_t ws_launch(const CUtensorMap& map_w, const CUtensorMap& map_x, float* y, int rows, int row0, int n, int k,
+                      float* slots, int32_t* tile_count, int32_t* status, int device, cudaStream_t st) {
+    WsParams p;
+    p.rows = rows;
+    p.rb = (rows + 15) / 16 * 16;
+    p.row0 = row0;
+    p.n = n;
+    p.k = k;
+    p.n_tiles = n / WS_BM;
+    p.kb = k / WS_BK;
+    const uint32_t stage_bytes = WS_BM * 128 + p.rb * 128;
+    p.stages = (int)((100 * 1024) / stage_bytes);
+    if (p.stages > 8) p.stages = 8;
+    p.tmem_cols = 32;
+    while (p.tmem_cols < 2 * p.rb) p.tmem_cols *= 2;
+    p.y = y;
+    p.slots = slots;
+    p.tile_count = tile_count;
+    p.status = status;
+    const size_t smem = (size_t)p.stages * stage_bytes + 1024 + 256;
+    static bool attr_set = false;
+    if (!attr_set) {
+        cudaError_t e = cudaFuncSetAttribute(k_gemm_ws, cudaFuncAttributeMaxDynamicSharedMemorySize, 112 * 1024);
+        if (e != cudaSuccess) return e;
+        attr_set = true;
+    }
+    long long units = (long long)p.n_tiles * p.kb;
+    int grid = ws_grid_limit(device);
+    if (grid > units) grid = (int)units;
+    k_gemm_ws<<<grid, WS_THREADS, smem, st>>>(map_w, map_x, p);
+    return cudaGetLastError();
+}
+
+}  // namespace aded

@@ -62,7 +62,7 @@ static aded_status dev_alloc(aded_model* m, T** p, size_t count) {
 
 static aded_status alloc_model(aded_model* m) {
     const aded_model_config& c = m->cfg;
-    const size_t R = c.max_rows, d = c.d_model, F = c.d_ffn, V = c.vocab, B = c.max_batch;
+    const size_t R = ((size_t)c.max_rows + 15) / 16 * 16, d = c.d_model, F = c.d_ffn, V = c.vocab, B = c.max_batch;
     size_t wide = 3 * d;
     if (2 * F > wide) wide = 2 * F;
     char* p;
@@ -94,6 +94,35 @@ static aded_status alloc_model(aded_model* m) {
     ADED_CUDA_TRY(cudaMemset(m->x, 0, R * d * m->elem));
     ADED_CUDA_TRY(cudaMemset(m->attn, 0, R * d * m->elem));
     ADED_CUDA_TRY(cudaMemset(m->act, 0, R * F * m->elem));
+
+    // tensor-core GEMM path: bf16 models whose every matrix tiles into 128-row x 64-column blocks
+    m->ws_ready = false;
+    if (c.dtype == ADED_BF16 && !getenv("ADED_PLAIN_GEMM") && ws_supported(3 * (int)d, (int)d) && ws_supported((int)d, (int)d) &&
+        ws_supported(2 * (int)F, (int)d) && ws_supported((int)d, (int)F) && ws_supported((int)V, (int)d)) {
+        const int L = c.n_layers;
+        m->ws_maps.resize(4 * L + 4);
+        bool ok = true;
+        for (int l = 0; l < L && ok; ++l) {
+            const aded_layer_weights& w = m->layers[l];
+            ok = ws_make_map(&m->ws_maps[4 * l + WS_MAP_QKV], w.wqkv, 3 * d, d, 128) &&
+                 ws_make_map(&m->ws_maps[4 * l + WS_MAP_O], w.wo, d, d, 128) &&
+                 ws_make_map(&m->ws_maps[4 * l + WS_MAP_GU], w.wgu, 2 * F, d, 128) &&
+                 ws_make_map(&m->ws_maps[4 * l + WS_MAP_D], w.wd, d, F, 128);
+        }
+        ok = ok && ws_make_map(&m->ws_maps[4 * L], m->top.lm_head, V, d, 128) &&
+             ws_make_map(&m->ws_maps[4 * L + 1], m->x, R, d, 16) && ws_make_map(&m->ws_maps[4 * L + 2], m->attn, R, d, 16) &&
+             ws_make_map(&m->ws_maps[4 * L + 3], m->act, R, F, 16);
+        if (ok) {
+            size_t tiles = 3 * d;
+            if (2 * F > tiles) tiles = 2 * F;
+            if (V > tiles) tiles = V;
+            tiles = tiles / 128 + 1;
+            TRY(dev_alloc(m, &m->ws_slots, ws_slot_floats(m->device)));
+            TRY(dev_alloc(m, &m->ws_tile_count, tiles));
+            ADED_CUDA_TRY(cudaMemset(m->ws_tile_count, 0, tiles * sizeof(int32_t)));
+            m->ws_ready = true;
+        }
+    }
     return ADED_OK;
 }
 
@@ -105,6 +134,7 @@ static aded_status forward(aded_model* m, aded_kv* kv, const int32_t* tokens, co
     const aded_model_config& c = m->cfg;
     const int rows = offsets_host[batch];
     const int d = c.d_model, F = c.d_ffn;
+    const int xm = 4 * c.n_layers + 1;   // TMA descriptor indices of x, attn, act
     ADED_CUDA_TRY(cudaMemcpyAsync(m->seqs.row_off, offsets_host, (batch + 1) * sizeof(int32_t),
                                   cudaMemcpyHostToDevice, st));
     {
@@ -116,19 +146,19 @@ static aded_status forward(aded_model* m, aded_kv* kv, const int32_t* tokens, co
     }
     for (int l = 0; l < c.n_layers; ++l) {
         const aded_layer_weights& w = m->layers[l];
-        { Span sp(m, PROF_GEMM, 1, st); launch_gemm(m, m->x, w.wqkv, m->y32, rows, 3 * d, d, st); }
+        { Span sp(m, PROF_GEMM, 1, st); launch_gemm(m, 4 * l + WS_MAP_QKV, xm, m->x, w.wqkv, m->y32, rows, 3 * d, d, st); }
         { Span sp(m, PROF_OTHER, 1, st); launch_rope_kv(m, kv, l, rows, st); }
         { Span sp(m, PROF_ATTN, 1, st); launch_tree_attention(m, kv, l, batch, rows, st); }
-        { Span sp(m, PROF_GEMM, 1, st); launch_gemm(m, m->attn, w.wo, m->y32, rows, d, d, st); }
+        { Span sp(m, PROF_GEMM, 1, st); launch_gemm(m, 4 * l + WS_MAP_O, xm + 1, m->attn, w.wo, m->y32, rows, d, d, st); }
         { Span sp(m, PROF_OTHER, 1, st); launch_add_rmsnorm(m, m->y32, w.norm2, rows, st); }
-        { Span sp(m, PROF_GEMM, 1, st); launch_gemm(m, m->x, w.wgu, m->y32, rows, 2 * F, d, st); }
+        { Span sp(m, PROF_GEMM, 1, st); launch_gemm(m, 4 * l + WS_MAP_GU, xm, m->x, w.wgu, m->y32, rows, 2 * F, d, st); }
         { Span sp(m, PROF_OTHER, 1, st); launch_swiglu(m, rows, st); }
-        { Span sp(m, PROF_GEMM, 1, st); launch_gemm(m, m->act, w.wd, m->y32, rows, d, F, st); }
+        { Span sp(m, PROF_GEMM, 1, st); launch_gemm(m, 4 * l + WS_MAP_D, xm + 2, m->act, w.wd, m->y32, rows, d, F, st); }
         const void* next_gain = l + 1 < c.n_layers ? m->layers[l + 1].norm1 : m->top.final_norm;
         { Span sp(m, PROF_OTHER, 1, st); launch_add_rmsnorm(m, m->y32, next_gain, rows, st); }
     }
     if (!chain_mode) {
-        { Span sp(m, PROF_GEMM, 1, st); launch_gemm(m, m->x, m->top.lm_head, m->logits, rows, c.vocab, d, st); }
+        { Span sp(m, PROF_GEMM, 1, st); launch_gemm(m, 4 * c.n_layers, xm, m->x, m->top.lm_head, m->logits, rows, c.vocab, d, st); }
         Span sp(m, PROF_OTHER, 2, st);
         launch_argmax(m, rows, st);
         if (m->dbg_logits)
@@ -180,6 +210,9 @@ aded_status aded_model_create(const aded_model_config* cfg, const aded_weights* 
     m->dbg_logits = nullptr;
     m->dbg_best = nullptr;
     m->prof_on = false;
+    m->ws_ready = false;
+    m->ws_slots = nullptr;
+    m->ws_tile_count = nullptr;
     if (cudaGetDevice(&m->device) != cudaSuccess) {
         delete m;
         return ADED_ERR_CUDA;
@@ -366,6 +399,32 @@ aded_status aded_verify_host(aded_model* m, aded_kv* kv, const int32_t* tree_tok
     ADED_CUDA_TRY(cudaMemcpyAsync(out_tokens_host, m->out_tokens, bytes, cudaMemcpyDeviceToHost, st));
     ADED_CUDA_TRY(cudaMemcpyAsync(out_accept_len_host, m->out_len, sizeof(int32_t), cudaMemcpyDeviceToHost, st));
     ADED_CUDA_TRY(cudaStreamSynchronize(st));
+    return ADED_OK;
+}
+
+aded_status aded_debug_gemm(aded_model* m, int32_t layer, int32_t which, const void* x_dev, int32_t rows,
+                            float* y_dev, void* stream) {
+    if (!m || !x_dev || !y_dev || which < 0 || which > 4 || rows < 1 || rows > m->cfg.max_rows)
+        return ADED_ERR_INVALID_ARG;
+    if (which < 4 && (layer < 0 || layer >= m->cfg.n_layers)) return ADED_ERR_INVALID_ARG;
+    const aded_model_config& c = m->cfg;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const int d = c.d_model, F = c.d_ffn, xm = 4 * c.n_layers + 1;
+    const int n = which == 0 ? 3 * d : which == 2 ? 2 * F : which == 4 ? c.vocab : d;
+    const int k = which == 3 ? F : d;
+    void* xbuf = which == 1 ? m->attn : which == 3 ? m->act : m->x;
+    const int x_map = which == 1 ? xm + 1 : which == 3 ? xm + 2 : xm;
+    const void* w = which == 4 ? m->top.lm_head
+                               : which == 0 ? m->layers[layer].wqkv
+                                            : which == 1 ? m->layers[layer].wo
+                                                         : which == 2 ? m->layers[layer].wgu : m->layers[layer].wd;
+    const int w_map = which == 4 ? 4 * c.n_layers : 4 * layer + which;
+    float* ybuf = which == 4 ? m->logits : m->y32;
+    ADED_CUDA_TRY(cudaMemcpyAsync(xbuf, x_dev, (size_t)rows * k * m->elem, cudaMemcpyDeviceToDevice, st));
+    note_launch();
+    launch_gemm(m, w_map, x_map, xbuf, w, ybuf, rows, n, k, st);
+    ADED_CUDA_TRY(cudaMemcpyAsync(y_dev, ybuf, (size_t)rows * n * sizeof(float), cudaMemcpyDeviceToDevice, st));
+    ADED_CUDA_TRY(cudaGetLastError());
     return ADED_OK;
 }
 
