@@ -9,6 +9,7 @@
 #include <vector>
 
 #include "aded.h"
+#include "gemm_out.cuh"
 
 #define ADED_CUDA_TRY(expr)                      \
     do {                                         \
@@ -98,8 +99,7 @@ struct aded_model {
     // tensor-core GEMM path (bf16 models): TMA descriptors and split-tile scratch
     bool ws_ready;
     std::vector<CUtensorMap> ws_maps;   // per layer: wqkv, wo, wgu, wd; then lm_head; then x, attn, act
-    float* ws_slots;                    // partial tiles of CTAs that share a W tile
-    int32_t* ws_tile_count;             // arrival counters, zero between launches
+    float* ws_slots;                    // partial result tiles (see gemm_out.cuh)
 
     bool prof_on;
     std::vector<aded::ProfSpan> prof_spans;   // spans recorded since aded_profile_begin
@@ -119,21 +119,26 @@ void launch_compact_commit(aded_model* m, aded_kv* kv, int batch, int chain_mode
 // dense.cu
 void launch_embed(aded_model* m, const int32_t* tokens, int rows, cudaStream_t st);
 void launch_rope_table(aded_model* m, int rows, cudaStream_t st);
-void launch_add_rmsnorm(aded_model* m, const float* y, const void* gain, int rows, cudaStream_t st);
-// w_map / x_map: indices into m->ws_maps of the operands' TMA descriptors (-1: none, plain kernel)
-void launch_gemm(aded_model* m, int w_map, int x_map, const void* x, const void* w, float* y, int rows, int n, int k,
-                 cudaStream_t st);
-void launch_rope_kv(aded_model* m, aded_kv* kv, int layer, int rows, cudaStream_t st);
-void launch_swiglu(aded_model* m, int rows, cudaStream_t st);
-void launch_argmax(aded_model* m, int rows, cudaStream_t st);
+// `y` (may be NULL): projection result added to the residual stream before the norm
+void launch_add_rmsnorm(aded_model* m, const GemmOut* y, const void* gain, int rows, cudaStream_t st);
+// w_map / x_map: indices into m->ws_maps of the operands' TMA descriptors (-1: none, plain kernel).
+// `y` is the fp32 buffer the plain kernel writes; the returned descriptor says where the result is.
+GemmOut launch_gemm(aded_model* m, int w_map, int x_map, const void* x, const void* w, float* y, int rows, int n, int k,
+                    cudaStream_t st);
+void launch_rope_kv(aded_model* m, aded_kv* kv, const GemmOut& qkv, int layer, int rows, cudaStream_t st);
+void launch_swiglu(aded_model* m, const GemmOut& gu, int rows, cudaStream_t st);
+void launch_argmax(aded_model* m, const GemmOut& logits, int rows, cudaStream_t st);
+// Writes a projection result as a plain [rows, n] fp32 matrix (debug paths).
+void launch_materialize(aded_model* m, const GemmOut& src, float* dst, int rows, cudaStream_t st);
 
 // gemm_ws.cu
 bool ws_make_map(CUtensorMap* map, const void* ptr, uint64_t rows, uint64_t cols, uint32_t box_rows);
 bool ws_supported(int n, int k);
 int ws_grid_limit(int device);
-size_t ws_slot_floats(int device);
-cudaError_t ws_launch(const CUtensorMap& map_w, const CUtensorMap& map_x, float* y, int rows, int row0, int n, int k,
-                      float* slots, int32_t* tile_count, int32_t* status, int device, cudaStream_t st);
+int ws_grid(int device, int n, int k);
+size_t ws_slot_floats(int device, int max_n, int max_rows);
+cudaError_t ws_launch(const CUtensorMap& map_w, const CUtensorMap& map_x, int rows, int row0, int n, int k,
+                      float* slots, int32_t* status, int device, cudaStream_t st);
 enum { WS_MAP_QKV = 0, WS_MAP_O = 1, WS_MAP_GU = 2, WS_MAP_D = 3 };   // per-layer map order
 
 // tree_attention.cu

@@ -51,17 +51,23 @@ __global__ void k_rope_table(const int32_t* __restrict__ pos, float* __restrict_
 
 // x = round(h * rsqrt(mean(h^2) + eps) * gain); when `y` is given, first h = round(h + y).
 template <typename T>
-__global__ void k_add_rmsnorm(T* __restrict__ h, const float* __restrict__ y, const T* __restrict__ gain,
+__global__ void k_add_rmsnorm(T* __restrict__ h, GemmOut y, int has_y, const T* __restrict__ gain,
                               T* __restrict__ x, int d, float eps, const int32_t* status) {
     if (*status != 0) return;
     __shared__ float red[32];
+    __shared__ TileRef tiles[64];          // contributors of each 128-column tile of y (d <= 8192)
     const int r = blockIdx.x;
+    if (has_y && y.mode == 1) {
+        for (int t = threadIdx.x; t < y.n_tiles; t += blockDim.x) tiles[t] = gemm_tile_ref(y, t);
+        __syncthreads();
+    }
     T* hr = h + (size_t)r * d;
     float ss = 0.f;
     for (int c = threadIdx.x; c < d; c += blockDim.x) {
         float v = to_f32(hr[c]);
-        if (y != nullptr) {
-            const T nv = from_f32<T>(v + y[(size_t)r * d + c]);
+        if (has_y) {
+            const float add = y.mode == 0 ? y.y[(size_t)r * d + c] : gemm_out_at(y, tiles[c >> 7], r, c & 127);
+            const T nv = from_f32<T>(v + add);
             hr[c] = nv;
             v = to_f32(nv);
         }
@@ -117,7 +123,7 @@ __global__ void __launch_bounds__(256) k_gemm_plain(const T* __restrict__ x, con
 // Rotary embedding of q and k (pairs (i, i + hd/2), angle from the table), then q -> q buffer and
 // k, v -> the cache at slot committed length + local node index.  Block = (row, head).
 template <typename T>
-__global__ void k_rope_kv(const float* __restrict__ qkv, const float* __restrict__ cs, const float* __restrict__ sn,
+__global__ void k_rope_kv(GemmOut qkv, const float* __restrict__ cs, const float* __restrict__ sn,
                           T* __restrict__ q, char* const* __restrict__ base, const int32_t* __restrict__ cap,
                           const int32_t* __restrict__ len, const int32_t* __restrict__ row_seq,
                           const int32_t* __restrict__ row_local, int layer, int H, int hd, const int32_t* status) {
@@ -128,42 +134,52 @@ __global__ void k_rope_kv(const float* __restrict__ qkv, const float* __restrict
     const size_t cp = cap[b];
     T* kdst = reinterpret_cast<T*>(base[b]) + ((((size_t)layer * 2 + 0) * H + hh) * cp + slot) * hd;
     T* vdst = reinterpret_cast<T*>(base[b]) + ((((size_t)layer * 2 + 1) * H + hh) * cp + slot) * hd;
-    const float* row = qkv + (size_t)r * 3 * d;
+    // the head's q, k and v columns each lie inside one 128-column tile of the projection result
+    const int cq = hh * hd, ck = d + hh * hd, cv = 2 * d + hh * hd;
+    TileRef tq = {0, 0}, tk = {0, 0}, tv = {0, 0};
+    if (qkv.mode == 1) { tq = gemm_tile_ref(qkv, cq >> 7); tk = gemm_tile_ref(qkv, ck >> 7); tv = gemm_tile_ref(qkv, cv >> 7); }
+    auto at = [&](const TileRef& t, int col) {
+        return qkv.mode == 0 ? qkv.y[(size_t)r * 3 * d + col] : gemm_out_at(qkv, t, r, col & 127);
+    };
     for (int i = threadIdx.x; i < half; i += blockDim.x) {
         const float c = cs[r * half + i], s = sn[r * half + i];
-        const float q0 = row[hh * hd + i], q1 = row[hh * hd + i + half];
-        const float k0 = row[d + hh * hd + i], k1 = row[d + hh * hd + i + half];
+        const float q0 = at(tq, cq + i), q1 = at(tq, cq + i + half);
+        const float k0 = at(tk, ck + i), k1 = at(tk, ck + i + half);
         q[(size_t)r * d + hh * hd + i] = from_f32<T>(q0 * c - q1 * s);
         q[(size_t)r * d + hh * hd + i + half] = from_f32<T>(q1 * c + q0 * s);
         kdst[i] = from_f32<T>(k0 * c - k1 * s);
         kdst[i + half] = from_f32<T>(k1 * c + k0 * s);
-        vdst[i] = from_f32<T>(row[2 * d + hh * hd + i]);
-        vdst[i + half] = from_f32<T>(row[2 * d + hh * hd + i + half]);
+        vdst[i] = from_f32<T>(at(tv, cv + i));
+        vdst[i + half] = from_f32<T>(at(tv, cv + i + half));
     }
 }
 
 // act = round(silu(gate) * up), gate = gu[:, :F], up = gu[:, F:].
 template <typename T>
-__global__ void k_swiglu(const float* __restrict__ gu, T* __restrict__ act, int F, const int32_t* status) {
+__global__ void k_swiglu(GemmOut gu, T* __restrict__ act, int F, const int32_t* status) {
     if (*status != 0) return;
     const int r = blockIdx.y;
     const int c = blockIdx.x * blockDim.x + threadIdx.x;
     if (c >= F) return;
-    const float g = gu[(size_t)r * 2 * F + c], u = gu[(size_t)r * 2 * F + F + c];
+    const float g = gemm_out_load(gu, r, c), u = gemm_out_load(gu, r, F + c);
     act[(size_t)r * F + c] = from_f32<T>(g / (1.f + expf(-g)) * u);
 }
 
 // Greedy choice per row: largest fp32 logit, lowest index among equals.
-__global__ void k_argmax(const float* __restrict__ logits, int32_t* __restrict__ best, int V, const int32_t* status) {
+__global__ void k_argmax(GemmOut logits, int32_t* __restrict__ best, int V, const int32_t* status) {
     if (*status != 0) return;
     __shared__ float sv[32];
     __shared__ int si[32];
+    extern __shared__ TileRef tiles[];     // contributors of each 128-column tile (tensor-core path)
     const int r = blockIdx.x;
-    const float* row = logits + (size_t)r * V;
+    if (logits.mode == 1) {
+        for (int t = threadIdx.x; t < logits.n_tiles; t += blockDim.x) tiles[t] = gemm_tile_ref(logits, t);
+        __syncthreads();
+    }
     float bv = -INFINITY;
     int bi = 0x7fffffff;
     for (int c = threadIdx.x; c < V; c += blockDim.x) {
-        const float v = row[c];
+        const float v = logits.mode == 0 ? logits.y[(size_t)r * V + c] : gemm_out_at(logits, tiles[c >> 7], r, c & 127);
         if (v > bv) { bv = v; bi = c; }   // c ascends per thread: first maximum kept
     }
     for (int o = 16; o > 0; o >>= 1) {
@@ -187,6 +203,13 @@ __global__ void k_argmax(const float* __restrict__ logits, int32_t* __restrict__
     }
 }
 
+__global__ void k_materialize(GemmOut src, float* __restrict__ dst, int n, const int32_t* status) {
+    if (*status != 0) return;
+    const int r = blockIdx.y;
+    const int c = blockIdx.x * blockDim.x + threadIdx.x;
+    if (c < n) dst[(size_t)r * n + c] = gemm_out_load(src, r, c);
+}
+
 // ---- launchers --------------------------------------------------------------------------
 #define BY_DTYPE(m, CALL_BF16, CALL_F32) \
     do { if ((m)->cfg.dtype == ADED_BF16) { CALL_BF16; } else { CALL_F32; } } while (0)
@@ -202,10 +225,13 @@ void launch_rope_table(aded_model* m, int rows, cudaStream_t st) {
                                       (double)m->cfg.rope_theta, m->status);
 }
 
-void launch_add_rmsnorm(aded_model* m, const float* y, const void* gain, int rows, cudaStream_t st) {
+void launch_add_rmsnorm(aded_model* m, const GemmOut* y, const void* gain, int rows, cudaStream_t st) {
     const int d = m->cfg.d_model;
-    BY_DTYPE(m, (k_add_rmsnorm<bf16><<<rows, 256, 0, st>>>((bf16*)m->h, y, (const bf16*)gain, (bf16*)m->x, d, m->cfg.rms_eps, m->status)),
-             (k_add_rmsnorm<float><<<rows, 256, 0, st>>>((float*)m->h, y, (const float*)gain, (float*)m->x, d, m->cfg.rms_eps, m->status)));
+    GemmOut none = {};
+    const GemmOut& yy = y ? *y : none;
+    const int has = y != nullptr;
+    BY_DTYPE(m, (k_add_rmsnorm<bf16><<<rows, 256, 0, st>>>((bf16*)m->h, yy, has, (const bf16*)gain, (bf16*)m->x, d, m->cfg.rms_eps, m->status)),
+             (k_add_rmsnorm<float><<<rows, 256, 0, st>>>((float*)m->h, yy, has, (const float*)gain, (float*)m->x, d, m->cfg.rms_eps, m->status)));
 }
 
 static void launch_gemm_plain(aded_model* m, const void* x, const void* w, float* y, int rows, int n, int k, cudaStream_t st) {
@@ -214,36 +240,52 @@ static void launch_gemm_plain(aded_model* m, const void* x, const void* w, float
              (k_gemm_plain<float><<<grid, 256, 0, st>>>((const float*)x, (const float*)w, y, rows, n, k, m->status)));
 }
 
-void launch_gemm(aded_model* m, int w_map, int x_map, const void* x, const void* w, float* y, int rows, int n, int k,
-                 cudaStream_t st) {
+GemmOut launch_gemm(aded_model* m, int w_map, int x_map, const void* x, const void* w, float* y, int rows, int n, int k,
+                    cudaStream_t st) {
+    GemmOut out = {};
+    out.n = n;
+    out.rows = rows;
     if (m->ws_ready && w_map >= 0 && x_map >= 0 && ws_supported(n, k)) {
-        // tensor-core path, 128 rows of x per pass over the weights
+        // tensor-core path, 128 rows of x per pass over the weights; the result stays in slots
         for (int row0 = 0; row0 < rows; row0 += 128) {
             const int part = rows - row0 < 128 ? rows - row0 : 128;
-            ws_launch(m->ws_maps[w_map], m->ws_maps[x_map], y, part, row0, n, k, m->ws_slots, m->ws_tile_count,
-                      m->status, m->device, st);
+            ws_launch(m->ws_maps[w_map], m->ws_maps[x_map], part, row0, n, k, m->ws_slots, m->status, m->device, st);
         }
-        return;
+        out.mode = 1;
+        out.slots = m->ws_slots;
+        out.n_tiles = n / 128;
+        out.kb = k / 64;
+        out.g = ws_grid(m->device, n, k);
+        return out;
     }
     launch_gemm_plain(m, x, w, y, rows, n, k, st);
+    out.mode = 0;
+    out.y = y;
+    return out;
 }
 
-void launch_rope_kv(aded_model* m, aded_kv* kv, int layer, int rows, cudaStream_t st) {
+void launch_materialize(aded_model* m, const GemmOut& src, float* dst, int rows, cudaStream_t st) {
+    dim3 grid((src.n + 255) / 256, rows);
+    k_materialize<<<grid, 256, 0, st>>>(src, dst, src.n, m->status);
+}
+
+void launch_rope_kv(aded_model* m, aded_kv* kv, const GemmOut& qkv, int layer, int rows, cudaStream_t st) {
     dim3 grid(rows, m->cfg.n_heads);
     const int H = m->cfg.n_heads, hd = m->cfg.head_dim;
-    BY_DTYPE(m, (k_rope_kv<bf16><<<grid, 64, 0, st>>>(m->y32, m->rope_cos, m->rope_sin, (bf16*)m->q, kv->base_dev, kv->cap_dev, kv->len_dev, m->rows.seq, m->rows.local, layer, H, hd, m->status)),
-             (k_rope_kv<float><<<grid, 64, 0, st>>>(m->y32, m->rope_cos, m->rope_sin, (float*)m->q, kv->base_dev, kv->cap_dev, kv->len_dev, m->rows.seq, m->rows.local, layer, H, hd, m->status)));
+    BY_DTYPE(m, (k_rope_kv<bf16><<<grid, 64, 0, st>>>(qkv, m->rope_cos, m->rope_sin, (bf16*)m->q, kv->base_dev, kv->cap_dev, kv->len_dev, m->rows.seq, m->rows.local, layer, H, hd, m->status)),
+             (k_rope_kv<float><<<grid, 64, 0, st>>>(qkv, m->rope_cos, m->rope_sin, (float*)m->q, kv->base_dev, kv->cap_dev, kv->len_dev, m->rows.seq, m->rows.local, layer, H, hd, m->status)));
 }
 
-void launch_swiglu(aded_model* m, int rows, cudaStream_t st) {
+void launch_swiglu(aded_model* m, const GemmOut& gu, int rows, cudaStream_t st) {
     const int F = m->cfg.d_ffn;
     dim3 grid((F + 255) / 256, rows);
-    BY_DTYPE(m, (k_swiglu<bf16><<<grid, 256, 0, st>>>(m->y32, (bf16*)m->act, F, m->status)),
-             (k_swiglu<float><<<grid, 256, 0, st>>>(m->y32, (float*)m->act, F, m->status)));
+    BY_DTYPE(m, (k_swiglu<bf16><<<grid, 256, 0, st>>>(gu, (bf16*)m->act, F, m->status)),
+             (k_swiglu<float><<<grid, 256, 0, st>>>(gu, (float*)m->act, F, m->status)));
 }
 
-void launch_argmax(aded_model* m, int rows, cudaStream_t st) {
-    k_argmax<<<rows, 256, 0, st>>>(m->logits, m->best, m->cfg.vocab, m->status);
+void launch_argmax(aded_model* m, const GemmOut& logits, int rows, cudaStream_t st) {
+    const size_t smem = logits.mode == 1 ? (size_t)logits.n_tiles * sizeof(TileRef) : 0;
+    k_argmax<<<rows, 256, smem, st>>>(logits, m->best, m->cfg.vocab, m->status);
 }
 
 }  // namespace aded

@@ -1,0 +1,84 @@
+// Where a projection's fp32 result lives, and how its consumers read it.
+//
+// The plain GEMM writes y[r, n] directly.  The tensor-core weight-streaming GEMM splits its
+// (W tile, k block) work units evenly over its CTAs, so a 128-column tile of the result is
+// generally the sum of several CTAs' partial tiles.  Rather than reducing inside the GEMM (which
+// would put counters, fences and a dependent read at the end of a kernel that runs for a few
+// microseconds), every CTA stores its partial tile to a slot and the consumer of the result
+// (rotary/K-V write, residual add + RMSNorm, SwiGLU, greedy choice) adds the slots while it
+// reads, always in ascending CTA order, so the sum is the same on every run.
+//
+// Slot numbering: the segment of tile t computed by CTA c goes to slot t + c.  Walking the units
+// in order, (t, c) never decreases and one of them grows at every segment boundary, so the sums
+// are distinct.  A slot holds [rb][128] floats (rb = rows of the pass padded to 16).  Passes over
+// more than 128 rows use one slot region per 128-row block.
+#pragma once
+
+#include <stdint.h>
+
+namespace aded {
+
+struct GemmOut {
+    const float* y;       // mode 0: [rows, n] row-major
+    const float* slots;   // mode 1: partial tiles
+    int mode;
+    int n;                // result columns
+    int n_tiles, kb, g;   // mode 1: 128-column tiles, k blocks per tile, CTAs of the GEMM launch
+    int rows;             // rows of the whole result (all row blocks)
+};
+
+// First work unit of CTA c when `units` units are split over `g` CTAs.
+__host__ __device__ __forceinline__ long long ws_start(long long c, long long units, long long g) {
+    return c * units / g;
+}
+// CTA that owns unit u.
+__host__ __device__ __forceinline__ int ws_owner(long long u, long long units, long long g) {
+    long long c = ((u + 1) * g - 1) / units;
+    if (c >= g) c = g - 1;
+    while (c > 0 && ws_start(c, units, g) > u) --c;
+    while (c + 1 < g && ws_start(c + 1, units, g) <= u) ++c;
+    return (int)c;
+}
+
+// The contributors of one tile: first slot and how many consecutive slots to add.
+struct TileRef {
+    int first_slot;
+    int count;
+};
+
+__device__ __forceinline__ TileRef gemm_tile_ref(const GemmOut& o, int tile) {
+    const long long units = (long long)o.n_tiles * o.kb;
+    const int c_first = ws_owner((long long)tile * o.kb, units, o.g);
+    const int c_last = ws_owner((long long)(tile + 1) * o.kb - 1, units, o.g);
+    TileRef t;
+    t.first_slot = tile + c_first;
+    t.count = c_last - c_first + 1;
+    return t;
+}
+
+// Rows padded to 16 of the 128-row block that holds row r.
+__device__ __forceinline__ int gemm_block_rb(const GemmOut& o, int r) {
+    const int left = o.rows - (r & ~127);
+    const int in_blk = left < 128 ? left : 128;
+    return (in_blk + 15) & ~15;
+}
+
+// Value of result element (r, tile * 128 + col) given the tile's contributors.
+__device__ __forceinline__ float gemm_out_at(const GemmOut& o, const TileRef& t, int r, int col) {
+    const int rb = gemm_block_rb(o, r);
+    const size_t region = (size_t)(r >> 7) * (size_t)(o.n_tiles + o.g) * 128 * 128;
+    const float* p = o.slots + region + ((size_t)t.first_slot * rb + (r & 127)) * 128 + col;
+    const size_t stride = (size_t)rb * 128;
+    float sum = 0.f;
+    for (int i = 0; i < t.count; ++i) sum += __ldcg(p + (size_t)i * stride);
+    return sum;
+}
+
+// Any element, any mode (computes the tile's contributors on the spot).
+__device__ __forceinline__ float gemm_out_load(const GemmOut& o, int r, int c) {
+    if (o.mode == 0) return o.y[(size_t)r * o.n + c];
+    const TileRef t = gemm_tile_ref(o, c >> 7);
+    return gemm_out_at(o, t, r, c & 127);
+}
+
+}  // namespace aded

@@ -11,9 +11,9 @@
 //   * work = (W tile, k block) units, split evenly over all resident CTAs (two per SM), so every CTA
 //     streams the same number of bytes whatever N and K are; a CTA's range covers the tail of one
 //     tile, whole tiles, and the head of another;
-//   * a tile shared by several CTAs is finished by whichever of them arrives last: each writes its
-//     fp32 partial to a private slot, bumps the tile's counter, and the last one adds the slots in
-//     CTA order -- a fixed order, so results do not depend on timing.  Nobody waits for anybody.
+//   * a CTA stores the fp32 partial tile of each of its segments to a slot; the kernel that consumes
+//     the result adds a tile's slots in CTA order -- a fixed order, so results do not depend on
+//     timing, and the GEMM itself ends without counters, fences or dependent reads;
 //   * warp 0 issues TMA loads, warp 1 issues MMAs, warps 2..5 drain TMEM and run the epilogue; two
 //     TMEM accumulators let the MMAs of the next segment run under the epilogue of the last.
 // Every mbarrier wait is bounded; a wait that runs out raises ADED_ERR_TIMEOUT in the status word
@@ -23,6 +23,7 @@
 #include <cstdio>
 
 #include "aded_internal.cuh"
+#include "gemm_out.cuh"
 
 namespace aded {
 
@@ -39,9 +40,7 @@ struct WsParams {
     int n_tiles, kb;     // tiles of 128 W rows, k blocks per tile
     int stages;
     int tmem_cols;       // power of two >= 2 * rb
-    float* y;            // [R, n] fp32
-    float* slots;        // [gridDim.x][2][rb][128] fp32 partial tiles
-    int32_t* tile_count; // [n_tiles] arrival counters, zero between launches
+    float* slots;        // this row block's slot region: [n_tiles + gridDim.x][rb][128] fp32
     int32_t* status;
 };
 
@@ -119,17 +118,6 @@ __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr) {
     return d;
 }
 
-// First unit of CTA c when `units` units are split over `g` CTAs.
-__device__ __host__ __forceinline__ long long ws_start(long long c, long long units, long long g) { return c * units / g; }
-// CTA that owns unit u.
-__device__ __forceinline__ int ws_owner(long long u, long long units, long long g) {
-    long long c = ((u + 1) * g - 1) / units;
-    if (c >= g) c = g - 1;
-    while (c > 0 && ws_start(c, units, g) > u) --c;
-    while (c + 1 < g && ws_start(c + 1, units, g) <= u) ++c;
-    return (int)c;
-}
-
 __global__ void __launch_bounds__(WS_THREADS, 2)
 k_gemm_ws(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_x, WsParams p) {
     extern __shared__ __align__(1024) uint8_t smem_raw[];
@@ -142,7 +130,7 @@ k_gemm_ws(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUt
     uint64_t* acc_full = bars + 2 * p.stages;
     uint64_t* acc_empty = acc_full + 2;
     uint32_t* s_tmem = (uint32_t*)(acc_empty + 2);
-    volatile int* s_flag = (volatile int*)(s_tmem + 1);   // [0] abort, [1] "this CTA finishes the tile", [2] live
+    volatile int* s_flag = (volatile int*)(s_tmem + 1);   // [0] abort, [2] live
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const long long units = (long long)p.n_tiles * p.kb;
@@ -226,73 +214,31 @@ k_gemm_ws(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUt
         }
     } else {
         // ---------------- epilogue: warps 2..5, TMEM lane quarter = warp % 4 ----------------
+        // Every segment's partial tile goes to slot (tile + CTA); the consumer of the result adds a
+        // tile's slots in CTA order (see gemm_out.cuh).
         const int quarter = warp & 3;
         const int row_in_tile = quarter * 32 + lane;           // W row inside the tile = TMEM lane
-        const int ep_tid = threadIdx.x - 64;                   // 0..127
-        float* my_slots = p.slots + (size_t)blockIdx.x * 2 * p.rb * WS_BM;
         int seg = 0;
         long long u = u0;
-        // (the abort flag is not polled here: a stalled pipeline shows up as a timed-out wait below,
-        //  the same for all four warps, so they leave the loop together and never split at bar.sync)
         while (live && u < u1) {
             const int tile = (int)(u / p.kb), kb0 = (int)(u % p.kb);
             long long ue = u + (p.kb - kb0);
             if (ue > u1) ue = u1;
-            const bool whole = kb0 == 0 && ue - u == p.kb;
             const int a = seg & 1;
             const uint32_t aph = (uint32_t)(seg >> 1) & 1;
             if (!mbar_wait(&acc_full[a], aph)) { s_flag[0] = 1; atomicCAS(p.status, 0, (int)ADED_ERR_TIMEOUT); break; }
             tc_fence_after();
             const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(a * p.rb);
-            const int n_glob = tile * WS_BM + row_in_tile;
-            float* slot = my_slots + (size_t)(kb0 == 0 ? 1 : 0) * p.rb * WS_BM;   // head of a tile -> slot 1, tail -> slot 0
+            float* slot = p.slots + (size_t)(tile + (int)blockIdx.x) * p.rb * WS_BM + row_in_tile;
             for (int c0 = 0; c0 < p.rb; c0 += 16) {
                 float v[16];
                 tc_ld16(taddr + (uint32_t)c0, v);
-                if (whole) {
-                    if (n_glob < p.n) {
 #pragma unroll
-                        for (int j = 0; j < 16; ++j)
-                            if (c0 + j < p.rows) p.y[(size_t)(p.row0 + c0 + j) * p.n + n_glob] = v[j];
-                    }
-                } else {
-#pragma unroll
-                    for (int j = 0; j < 16; ++j) slot[(size_t)(c0 + j) * WS_BM + row_in_tile] = v[j];
-                }
+                for (int j = 0; j < 16; ++j) __stcg(slot + (size_t)(c0 + j) * WS_BM, v[j]);
             }
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(&acc_empty[a]);
-            if (!whole) {
-                // publish the partial, learn whether this CTA is the last contributor of the tile
-                __threadfence();
-                asm volatile("bar.sync 1, 128;" ::: "memory");
-                const int c_first = ws_owner((long long)tile * p.kb, units, G);
-                const int c_last = ws_owner((long long)(tile + 1) * p.kb - 1, units, G);
-                if (ep_tid == 0) {
-                    const int prev = atomicAdd(&p.tile_count[tile], 1);
-                    const int last = prev == c_last - c_first;
-                    if (last) p.tile_count[tile] = 0;          // everyone has arrived: reset for the next launch
-                    s_flag[1] = last;
-                }
-                asm volatile("bar.sync 1, 128;" ::: "memory");
-                if (s_flag[1]) {
-                    __threadfence();
-                    if (n_glob < p.n) {
-                        for (int c = 0; c < p.rows; ++c) {
-                            float sum = 0.f;
-                            for (int cc = c_first; cc <= c_last; ++cc) {
-                                // contributor cc holds the tile's head in slot 1 if it started the tile, else its tail in slot 0
-                                const int which = cc == c_first ? 1 : 0;
-                                const float* src = p.slots + ((size_t)cc * 2 + which) * p.rb * WS_BM;
-                                sum += __ldcg(src + (size_t)c * WS_BM + row_in_tile);
-                            }
-                            p.y[(size_t)(p.row0 + c) * p.n + n_glob] = sum;
-                        }
-                    }
-                }
-                asm volatile("bar.sync 1, 128;" ::: "memory");   // s_flag[1] may be rewritten next segment
-            }
             u = ue;
             ++seg;
         }
@@ -353,13 +299,26 @@ int ws_grid_limit(int device) {
     return cached;
 }
 
-size_t ws_slot_floats(int device) { return (size_t)ws_grid_limit(device) * 2 * 128 * WS_BM; }
+// CTAs a launch over n_tiles x kb units uses.
+int ws_grid(int device, int n, int k) {
+    const long long units = (long long)(n / WS_BM) * (k / WS_BK);
+    const int g = ws_grid_limit(device);
+    return units < g ? (int)units : g;
+}
+
+// Floats of slot storage for results of up to max_n columns and max_rows rows.
+size_t ws_slot_floats(int device, int max_n, int max_rows) {
+    const size_t blocks = ((size_t)max_rows + 127) / 128;
+    return blocks * ((size_t)max_n / WS_BM + ws_grid_limit(device)) * 128 * WS_BM;
+}
 
 // Shapes the tensor-core path takes.
 bool ws_supported(int n, int k) { return n % WS_BM == 0 && k % WS_BK == 0 && k >= WS_BK; }
 
-cudaError_t ws_launch(const CUtensorMap& map_w, const CUtensorMap& map_x, float* y, int rows, int row0, int n, int k,
-                      float* slots, int32_t* tile_count, int32_t* status, int device, cudaStream_t st) {
+// One pass: rows [row0, row0 + rows) of x (rows <= 128) against all of W.  Partial tiles go to the
+// slot region of row block row0 / 128.
+cudaError_t ws_launch(const CUtensorMap& map_w, const CUtensorMap& map_x, int rows, int row0, int n, int k,
+                      float* slots, int32_t* status, int device, cudaStream_t st) {
     WsParams p;
     p.rows = rows;
     p.rb = (rows + 15) / 16 * 16;
@@ -373,9 +332,8 @@ cudaError_t ws_launch(const CUtensorMap& map_w, const CUtensorMap& map_x, float*
     if (p.stages > 8) p.stages = 8;
     p.tmem_cols = 32;
     while (p.tmem_cols < 2 * p.rb) p.tmem_cols *= 2;
-    p.y = y;
-    p.slots = slots;
-    p.tile_count = tile_count;
+    const int grid = ws_grid(device, n, k);
+    p.slots = slots + (size_t)(row0 / 128) * (size_t)(p.n_tiles + grid) * 128 * WS_BM;
     p.status = status;
     const size_t smem = (size_t)p.stages * stage_bytes + 1024 + 256;
     static bool attr_set = false;
@@ -384,9 +342,6 @@ cudaError_t ws_launch(const CUtensorMap& map_w, const CUtensorMap& map_x, float*
         if (e != cudaSuccess) return e;
         attr_set = true;
     }
-    long long units = (long long)p.n_tiles * p.kb;
-    int grid = ws_grid_limit(device);
-    if (grid > units) grid = (int)units;
     k_gemm_ws<<<grid, WS_THREADS, smem, st>>>(map_w, map_x, p);
     return cudaGetLastError();
 }

@@ -113,13 +113,10 @@ static aded_status alloc_model(aded_model* m) {
              ws_make_map(&m->ws_maps[4 * L + 1], m->x, R, d, 16) && ws_make_map(&m->ws_maps[4 * L + 2], m->attn, R, d, 16) &&
              ws_make_map(&m->ws_maps[4 * L + 3], m->act, R, F, 16);
         if (ok) {
-            size_t tiles = 3 * d;
-            if (2 * F > tiles) tiles = 2 * F;
-            if (V > tiles) tiles = V;
-            tiles = tiles / 128 + 1;
-            TRY(dev_alloc(m, &m->ws_slots, ws_slot_floats(m->device)));
-            TRY(dev_alloc(m, &m->ws_tile_count, tiles));
-            ADED_CUDA_TRY(cudaMemset(m->ws_tile_count, 0, tiles * sizeof(int32_t)));
+            size_t widest = 3 * d;
+            if (2 * F > widest) widest = 2 * F;
+            if (V > widest) widest = V;
+            TRY(dev_alloc(m, &m->ws_slots, ws_slot_floats(m->device, (int)widest, (int)R)));
             m->ws_ready = true;
         }
     }
@@ -142,28 +139,28 @@ static aded_status forward(aded_model* m, aded_kv* kv, const int32_t* tokens, co
         launch_tree_prologue(m, kv, tokens, parents, batch, chain_mode, st);
         launch_embed(m, tokens, rows, st);
         launch_rope_table(m, rows, st);
-        launch_add_rmsnorm(m, nullptr, m->layers[0].norm1, rows, st);
+        launch_add_rmsnorm(m, (const GemmOut*)nullptr, m->layers[0].norm1, rows, st);
     }
     for (int l = 0; l < c.n_layers; ++l) {
         const aded_layer_weights& w = m->layers[l];
-        { Span sp(m, PROF_GEMM, 1, st); launch_gemm(m, 4 * l + WS_MAP_QKV, xm, m->x, w.wqkv, m->y32, rows, 3 * d, d, st); }
-        { Span sp(m, PROF_OTHER, 1, st); launch_rope_kv(m, kv, l, rows, st); }
+        GemmOut o;
+        { Span sp(m, PROF_GEMM, 1, st); o = launch_gemm(m, 4 * l + WS_MAP_QKV, xm, m->x, w.wqkv, m->y32, rows, 3 * d, d, st); }
+        { Span sp(m, PROF_OTHER, 1, st); launch_rope_kv(m, kv, o, l, rows, st); }
         { Span sp(m, PROF_ATTN, 1, st); launch_tree_attention(m, kv, l, batch, rows, st); }
-        { Span sp(m, PROF_GEMM, 1, st); launch_gemm(m, 4 * l + WS_MAP_O, xm + 1, m->attn, w.wo, m->y32, rows, d, d, st); }
-        { Span sp(m, PROF_OTHER, 1, st); launch_add_rmsnorm(m, m->y32, w.norm2, rows, st); }
-        { Span sp(m, PROF_GEMM, 1, st); launch_gemm(m, 4 * l + WS_MAP_GU, xm, m->x, w.wgu, m->y32, rows, 2 * F, d, st); }
-        { Span sp(m, PROF_OTHER, 1, st); launch_swiglu(m, rows, st); }
-        { Span sp(m, PROF_GEMM, 1, st); launch_gemm(m, 4 * l + WS_MAP_D, xm + 2, m->act, w.wd, m->y32, rows, d, F, st); }
+        { Span sp(m, PROF_GEMM, 1, st); o = launch_gemm(m, 4 * l + WS_MAP_O, xm + 1, m->attn, w.wo, m->y32, rows, d, d, st); }
+        { Span sp(m, PROF_OTHER, 1, st); launch_add_rmsnorm(m, &o, w.norm2, rows, st); }
+        { Span sp(m, PROF_GEMM, 1, st); o = launch_gemm(m, 4 * l + WS_MAP_GU, xm, m->x, w.wgu, m->y32, rows, 2 * F, d, st); }
+        { Span sp(m, PROF_OTHER, 1, st); launch_swiglu(m, o, rows, st); }
+        { Span sp(m, PROF_GEMM, 1, st); o = launch_gemm(m, 4 * l + WS_MAP_D, xm + 2, m->act, w.wd, m->y32, rows, d, F, st); }
         const void* next_gain = l + 1 < c.n_layers ? m->layers[l + 1].norm1 : m->top.final_norm;
-        { Span sp(m, PROF_OTHER, 1, st); launch_add_rmsnorm(m, m->y32, next_gain, rows, st); }
+        { Span sp(m, PROF_OTHER, 1, st); launch_add_rmsnorm(m, &o, next_gain, rows, st); }
     }
     if (!chain_mode) {
-        { Span sp(m, PROF_GEMM, 1, st); launch_gemm(m, 4 * c.n_layers, xm, m->x, m->top.lm_head, m->logits, rows, c.vocab, d, st); }
+        GemmOut lg;
+        { Span sp(m, PROF_GEMM, 1, st); lg = launch_gemm(m, 4 * c.n_layers, xm, m->x, m->top.lm_head, m->logits, rows, c.vocab, d, st); }
         Span sp(m, PROF_OTHER, 2, st);
-        launch_argmax(m, rows, st);
-        if (m->dbg_logits)
-            ADED_CUDA_TRY(cudaMemcpyAsync(m->dbg_logits, m->logits, (size_t)rows * c.vocab * sizeof(float),
-                                          cudaMemcpyDeviceToDevice, st));
+        launch_argmax(m, lg, rows, st);
+        if (m->dbg_logits) launch_materialize(m, lg, m->dbg_logits, rows, st);
         if (m->dbg_best)
             ADED_CUDA_TRY(cudaMemcpyAsync(m->dbg_best, m->best, (size_t)rows * sizeof(int32_t),
                                           cudaMemcpyDeviceToDevice, st));
@@ -212,7 +209,6 @@ aded_status aded_model_create(const aded_model_config* cfg, const aded_weights* 
     m->prof_on = false;
     m->ws_ready = false;
     m->ws_slots = nullptr;
-    m->ws_tile_count = nullptr;
     if (cudaGetDevice(&m->device) != cudaSuccess) {
         delete m;
         return ADED_ERR_CUDA;
@@ -422,8 +418,8 @@ aded_status aded_debug_gemm(aded_model* m, int32_t layer, int32_t which, const v
     float* ybuf = which == 4 ? m->logits : m->y32;
     ADED_CUDA_TRY(cudaMemcpyAsync(xbuf, x_dev, (size_t)rows * k * m->elem, cudaMemcpyDeviceToDevice, st));
     note_launch();
-    launch_gemm(m, w_map, x_map, xbuf, w, ybuf, rows, n, k, st);
-    ADED_CUDA_TRY(cudaMemcpyAsync(y_dev, ybuf, (size_t)rows * n * sizeof(float), cudaMemcpyDeviceToDevice, st));
+    const GemmOut o = launch_gemm(m, w_map, x_map, xbuf, w, ybuf, rows, n, k, st);
+    launch_materialize(m, o, y_dev, rows, st);
     ADED_CUDA_TRY(cudaGetLastError());
     return ADED_OK;
 }
