@@ -96,6 +96,11 @@ struct aded_model {
     float* dbg_logits;
     int32_t* dbg_best;
 
+    // split-KV attention partials (bf16 models)
+    float* att_o;       // [splits][R][H][hd] unnormalised outputs
+    float* att_ml;      // [splits][R][H][2]  running max (log2 domain) and sum
+    int32_t att_splits_max;
+
     // tensor-core GEMM path (bf16 models): TMA descriptors and split-tile scratch
     bool ws_ready;
     std::vector<CUtensorMap> ws_maps;   // per layer: wqkv, wo, wgu, wd; then lm_head; then x, attn, act
@@ -142,6 +147,7 @@ cudaError_t ws_launch(const CUtensorMap& map_w, const CUtensorMap& map_x, int ro
 enum { WS_MAP_QKV = 0, WS_MAP_O = 1, WS_MAP_GU = 2, WS_MAP_D = 3 };   // per-layer map order
 
 // tree_attention.cu
-void launch_tree_attention(aded_model* m, aded_kv* kv, int layer, int batch, int rows, cudaStream_t st);
+// max_tree: most nodes any sequence's tree has in this call
+void launch_tree_attention(aded_model* m, aded_kv* kv, int layer, int batch, int rows, int max_tree, cudaStream_t st);
 
 }  // namespace aded

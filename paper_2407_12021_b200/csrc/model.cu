@@ -95,6 +95,15 @@ static aded_status alloc_model(aded_model* m) {
     ADED_CUDA_TRY(cudaMemset(m->attn, 0, R * d * m->elem));
     ADED_CUDA_TRY(cudaMemset(m->act, 0, R * F * m->elem));
 
+    m->att_o = nullptr;
+    m->att_ml = nullptr;
+    m->att_splits_max = 1;
+    if (c.dtype == ADED_BF16 && !getenv("ADED_PLAIN_ATTN")) {
+        m->att_splits_max = R <= 128 ? 16 : (int)(16 * 128 / R > 0 ? 16 * 128 / R : 1);
+        TRY(dev_alloc(m, &m->att_o, (size_t)m->att_splits_max * R * d));
+        TRY(dev_alloc(m, &m->att_ml, (size_t)m->att_splits_max * R * c.n_heads * 2));
+    }
+
     // tensor-core GEMM path: bf16 models whose every matrix tiles into 128-row x 64-column blocks
     m->ws_ready = false;
     if (c.dtype == ADED_BF16 && !getenv("ADED_PLAIN_GEMM") && ws_supported(3 * (int)d, (int)d) && ws_supported((int)d, (int)d) &&
@@ -132,6 +141,9 @@ static aded_status forward(aded_model* m, aded_kv* kv, const int32_t* tokens, co
     const int rows = offsets_host[batch];
     const int d = c.d_model, F = c.d_ffn;
     const int xm = 4 * c.n_layers + 1;   // TMA descriptor indices of x, attn, act
+    int max_tree = 1;
+    for (int b = 0; b < batch; ++b)
+        if (offsets_host[b + 1] - offsets_host[b] > max_tree) max_tree = offsets_host[b + 1] - offsets_host[b];
     ADED_CUDA_TRY(cudaMemcpyAsync(m->seqs.row_off, offsets_host, (batch + 1) * sizeof(int32_t),
                                   cudaMemcpyHostToDevice, st));
     {
@@ -146,7 +158,7 @@ static aded_status forward(aded_model* m, aded_kv* kv, const int32_t* tokens, co
         GemmOut o;
         { Span sp(m, PROF_GEMM, 1, st); o = launch_gemm(m, 4 * l + WS_MAP_QKV, xm, m->x, w.wqkv, m->y32, rows, 3 * d, d, st); }
         { Span sp(m, PROF_OTHER, 1, st); launch_rope_kv(m, kv, o, l, rows, st); }
-        { Span sp(m, PROF_ATTN, 1, st); launch_tree_attention(m, kv, l, batch, rows, st); }
+        { Span sp(m, PROF_ATTN, 1, st); launch_tree_attention(m, kv, l, batch, rows, max_tree, st); }
         { Span sp(m, PROF_GEMM, 1, st); o = launch_gemm(m, 4 * l + WS_MAP_O, xm + 1, m->attn, w.wo, m->y32, rows, d, d, st); }
         { Span sp(m, PROF_OTHER, 1, st); launch_add_rmsnorm(m, &o, w.norm2, rows, st); }
         { Span sp(m, PROF_GEMM, 1, st); o = launch_gemm(m, 4 * l + WS_MAP_GU, xm, m->x, w.wgu, m->y32, rows, 2 * F, d, st); }

@@ -3,13 +3,23 @@
 //
 // The tree's own keys/values already sit in the cache at slots L + node index (written by the
 // rotary/K-V kernel), so the key set of node i is cache[0, L) plus { L + j : bit j of anc[i] }.
+//
+// bf16 models: split-KV kernel on tensor cores.  A CTA owns (sequence, head, key split); each of
+// its warps owns 16 tree nodes (query rows) and walks the split's keys in blocks of 64 that all
+// warps share through shared memory (double-buffered cp.async).  Scores S = Q K^T and O += P V
+// are m16n8k16 bf16 MMAs with fp32 accumulators; the online softmax keeps a running maximum and
+// sum per row in registers (quad shuffles).  Only the blocks that reach past L apply the ancestor
+// bit mask.  Each split writes an unnormalised partial (O, max, sum); a merge kernel combines the
+// splits and rounds to bf16.  The key range is derived on the device from the committed length.
+//
+// fp32 models use the plain one-warp-per-(row, head) kernel below.
 #include "aded_internal.cuh"
 
 namespace aded {
 
-// Plain version: one warp per (row, head).  The lanes split head_dim; each key costs a warp
-// reduction for the score and one online-softmax update (running max m, running sum l, and
-// hd/32 output elements per lane).  Scores and probabilities are fp32 throughout.
+// ------------------------------------------------------------------------------------------
+// plain kernel (fp32 models; also a readable statement of the computation)
+// ------------------------------------------------------------------------------------------
 template <typename T, int HD>
 __global__ void __launch_bounds__(128) k_tree_attn_plain(
         const T* __restrict__ q, T* __restrict__ out, char* const* __restrict__ base,
@@ -61,9 +71,306 @@ __global__ void __launch_bounds__(128) k_tree_attn_plain(
     for (int e = 0; e < PER; ++e) out[((size_t)r * H + hh) * HD + lane * PER + e] = from_f32<T>(acc[e] * inv);
 }
 
-void launch_tree_attention(aded_model* m, aded_kv* kv, int layer, int batch, int rows, cudaStream_t st) {
-    (void)batch;
+// ------------------------------------------------------------------------------------------
+// tensor-core split-KV kernel (bf16)
+// ------------------------------------------------------------------------------------------
+constexpr int TA_BLK = 64;   // keys per shared-memory block
+
+__device__ __forceinline__ void cp_async16(void* smem, const void* gmem) {
+    const uint32_t s = (uint32_t)__cvta_generic_to_shared(smem);
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(s), "l"(gmem) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
+__device__ __forceinline__ void ldmatrix_x4(uint32_t* r, const void* smem) {
+    const uint32_t s = (uint32_t)__cvta_generic_to_shared(smem);
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(s));
+}
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t* r, const void* smem) {
+    const uint32_t s = (uint32_t)__cvta_generic_to_shared(smem);
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(s));
+}
+__device__ __forceinline__ void mma_bf16_16816(float* c, const uint32_t* a, uint32_t b0, uint32_t b1) {
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
+                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t*>(&v);
+}
+
+// Address of the 16-byte chunk `chunk` of row `row` in a [rows][HD] bf16 tile whose chunks are
+// XOR-swizzled inside each group of eight (conflict-free ldmatrix over eight rows).
+template <int HD>
+__device__ __forceinline__ bf16* tile_chunk(bf16* tile, int row, int chunk) {
+    return tile + (size_t)row * HD + (((chunk & ~7) | ((chunk ^ row) & 7)) << 3);
+}
+
+struct AttnArgs {
+    const bf16* q;                 // [R][H][HD]
+    float* part_o;                 // [S][R][H][HD]
+    float* part_ml;                // [S][R][H][2]  (running max in the log2 domain, sum)
+    char* const* base;
+    const int32_t* cap;
+    const int32_t* len;
+    const int32_t* row_off;
+    const uint64_t* anc;
+    int layer, H, n_splits, rows_total;
+    float scale_log2;              // softmax scale * log2(e)
+    const int32_t* status;
+};
+
+template <int HD, int NW>
+__global__ void __launch_bounds__(NW * 32) k_tree_attn_mma(AttnArgs a) {
+    if (*a.status != 0) return;
+    constexpr int KSTEPS = HD / 16;        // k steps of Q K^T
+    constexpr int ONT = HD / 8;            // n tiles of the output
+    constexpr int CHUNKS = HD / 8;         // 16-byte chunks per row
+    extern __shared__ __align__(128) uint8_t smem_raw[];
+    bf16* sk = reinterpret_cast<bf16*>(smem_raw);                 // [2][TA_BLK][HD]
+    bf16* sv = sk + 2 * TA_BLK * HD;                              // [2][TA_BLK][HD]
+
+    const int hh = blockIdx.x, split = blockIdx.y, b = blockIdx.z;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, tig = lane & 3;
+    const int off = a.row_off[b];
+    const int T = a.row_off[b + 1] - off;
+    const int L = a.len[b];
+    const size_t cp = a.cap[b];
+    const int n_keys = L + T;
+    const int nb = (n_keys + TA_BLK - 1) / TA_BLK;
+    const int bps = (nb + a.n_splits - 1) / a.n_splits;
+    const int blk0 = split * bps;
+    const int blk1 = min(nb, blk0 + bps);
+
+    // this thread's two query rows (local node indices) and their global rows
+    const int i0 = warp * 16 + g, i1 = i0 + 8;
+    const bool v0 = i0 < T, v1 = i1 < T;
+    const size_t pstride = (size_t)a.rows_total * a.H;            // (row, head) pairs per split
+    if (blk0 >= blk1) {                                           // nothing in this split
+        if (tig == 0) {
+            if (v0) { float* ml = a.part_ml + ((size_t)split * pstride + (size_t)(off + i0) * a.H + hh) * 2; ml[0] = -INFINITY; ml[1] = 0.f; }
+            if (v1) { float* ml = a.part_ml + ((size_t)split * pstride + (size_t)(off + i1) * a.H + hh) * 2; ml[0] = -INFINITY; ml[1] = 0.f; }
+        }
+        return;
+    }
+    const bf16* kg = reinterpret_cast<const bf16*>(a.base[b]) + (((size_t)a.layer * 2 + 0) * a.H + hh) * cp * HD;
+    const bf16* vg = reinterpret_cast<const bf16*>(a.base[b]) + (((size_t)a.layer * 2 + 1) * a.H + hh) * cp * HD;
+
+    // Q fragments straight from global memory in the MMA A layout
+    uint32_t qf[KSTEPS][4];
+    {
+        const bf16* q0 = a.q + ((size_t)(off + (v0 ? i0 : 0)) * a.H + hh) * HD;
+        const bf16* q1 = a.q + ((size_t)(off + (v1 ? i1 : 0)) * a.H + hh) * HD;
+#pragma unroll
+        for (int ks = 0; ks < KSTEPS; ++ks) {
+            const int c = ks * 16 + 2 * tig;
+            qf[ks][0] = v0 ? *reinterpret_cast<const uint32_t*>(q0 + c) : 0u;
+            qf[ks][1] = v1 ? *reinterpret_cast<const uint32_t*>(q1 + c) : 0u;
+            qf[ks][2] = v0 ? *reinterpret_cast<const uint32_t*>(q0 + c + 8) : 0u;
+            qf[ks][3] = v1 ? *reinterpret_cast<const uint32_t*>(q1 + c + 8) : 0u;
+        }
+    }
+    uint64_t m0lo = 0, m0hi = 0, m1lo = 0, m1hi = 0;             // ancestor bit sets of the two rows
+    if (v0) { m0lo = a.anc[2 * (off + i0)]; m0hi = a.anc[2 * (off + i0) + 1]; }
+    if (v1) { m1lo = a.anc[2 * (off + i1)]; m1hi = a.anc[2 * (off + i1) + 1]; }
+
+    float oacc[ONT][4];
+#pragma unroll
+    for (int n = 0; n < ONT; ++n) { oacc[n][0] = oacc[n][1] = oacc[n][2] = oacc[n][3] = 0.f; }
+    float mrow0 = -INFINITY, mrow1 = -INFINITY, lrow0 = 0.f, lrow1 = 0.f;
+
+    auto load_block = [&](int blk, int buf) {
+        // positions past the last key are clamped to it (they are masked below); the clamp keeps
+        // every address inside the rows this call may touch
+        const int p0 = blk * TA_BLK;
+        bf16* dk = sk + (size_t)buf * TA_BLK * HD;
+        bf16* dv = sv + (size_t)buf * TA_BLK * HD;
+        for (int e = threadIdx.x; e < TA_BLK * CHUNKS; e += NW * 32) {
+            const int row = e / CHUNKS, chunk = e % CHUNKS;
+            const int pos = min(p0 + row, n_keys - 1);
+            cp_async16(tile_chunk<HD>(dk, row, chunk), kg + (size_t)pos * HD + chunk * 8);
+            cp_async16(tile_chunk<HD>(dv, row, chunk), vg + (size_t)pos * HD + chunk * 8);
+        }
+        cp_async_commit();
+    };
+
+    load_block(blk0, 0);
+    for (int blk = blk0; blk < blk1; ++blk) {
+        const int buf = (blk - blk0) & 1;
+        if (blk + 1 < blk1) { load_block(blk + 1, buf ^ 1); cp_async_wait<1>(); } else { cp_async_wait<0>(); }
+        __syncthreads();
+        bf16* tk = sk + (size_t)buf * TA_BLK * HD;
+        bf16* tv = sv + (size_t)buf * TA_BLK * HD;
+
+        // ---- S = Q K^T for 64 keys: 8 n tiles x KSTEPS k steps ----
+        float sacc[TA_BLK / 8][4];
+#pragma unroll
+        for (int n = 0; n < TA_BLK / 8; ++n) { sacc[n][0] = sacc[n][1] = sacc[n][2] = sacc[n][3] = 0.f; }
+#pragma unroll
+        for (int ks = 0; ks < KSTEPS; ++ks) {
+#pragma unroll
+            for (int np = 0; np < TA_BLK / 16; ++np) {
+                uint32_t kb[4];
+                const int row = np * 16 + (lane & 7) + ((lane >> 4) << 3);
+                const int chunk = ks * 2 + ((lane >> 3) & 1);
+                ldmatrix_x4(kb, tile_chunk<HD>(tk, row, chunk));
+                mma_bf16_16816(sacc[2 * np], qf[ks], kb[0], kb[1]);
+                mma_bf16_16816(sacc[2 * np + 1], qf[ks], kb[2], kb[3]);
+            }
+        }
+        // ---- scale, mask, online softmax ----
+        const int p0 = blk * TA_BLK;
+        const bool need_mask = p0 + TA_BLK > L;
+        float bm0 = -INFINITY, bm1 = -INFINITY;
+#pragma unroll
+        for (int n = 0; n < TA_BLK / 8; ++n) {
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                float s = sacc[n][e] * a.scale_log2;
+                if (need_mask) {
+                    const int pos = p0 + n * 8 + 2 * tig + (e & 1);
+                    const int j = pos - L;
+                    bool ok = j < 0;
+                    if (!ok && j < T) {
+                        const uint64_t lo = e < 2 ? m0lo : m1lo, hi = e < 2 ? m0hi : m1hi;
+                        ok = j < 64 ? (lo >> j) & 1 : (hi >> (j - 64)) & 1;
+                    }
+                    if (!ok) s = -INFINITY;
+                }
+                sacc[n][e] = s;
+                if (e < 2) bm0 = fmaxf(bm0, s); else bm1 = fmaxf(bm1, s);
+            }
+        }
+        bm0 = fmaxf(bm0, __shfl_xor_sync(0xffffffffu, bm0, 1));
+        bm0 = fmaxf(bm0, __shfl_xor_sync(0xffffffffu, bm0, 2));
+        bm1 = fmaxf(bm1, __shfl_xor_sync(0xffffffffu, bm1, 1));
+        bm1 = fmaxf(bm1, __shfl_xor_sync(0xffffffffu, bm1, 2));
+        const float nm0 = fmaxf(mrow0, bm0), nm1 = fmaxf(mrow1, bm1);
+        const float use0 = nm0 == -INFINITY ? 0.f : nm0, use1 = nm1 == -INFINITY ? 0.f : nm1;
+        const float corr0 = exp2f(mrow0 - use0), corr1 = exp2f(mrow1 - use1);
+        mrow0 = nm0;
+        mrow1 = nm1;
+        float ps0 = 0.f, ps1 = 0.f;
+        uint32_t pf[TA_BLK / 16][4];
+#pragma unroll
+        for (int n = 0; n < TA_BLK / 8; ++n) {
+            const float e0 = exp2f(sacc[n][0] - use0), e1 = exp2f(sacc[n][1] - use0);
+            const float e2 = exp2f(sacc[n][2] - use1), e3 = exp2f(sacc[n][3] - use1);
+            ps0 += e0 + e1;
+            ps1 += e2 + e3;
+            pf[n >> 1][(n & 1) * 2 + 0] = pack_bf16(e0, e1);
+            pf[n >> 1][(n & 1) * 2 + 1] = pack_bf16(e2, e3);
+        }
+        lrow0 = lrow0 * corr0 + ps0;
+        lrow1 = lrow1 * corr1 + ps1;
+#pragma unroll
+        for (int n = 0; n < ONT; ++n) {
+            oacc[n][0] *= corr0; oacc[n][1] *= corr0;
+            oacc[n][2] *= corr1; oacc[n][3] *= corr1;
+        }
+        // ---- O += P V ----
+#pragma unroll
+        for (int kk = 0; kk < TA_BLK / 16; ++kk) {
+#pragma unroll
+            for (int np = 0; np < ONT / 2; ++np) {
+                uint32_t vb[4];
+                const int row = kk * 16 + (lane & 7) + (((lane >> 3) & 1) << 3);
+                const int chunk = np * 2 + (lane >> 4);
+                ldmatrix_x4_trans(vb, tile_chunk<HD>(tv, row, chunk));
+                mma_bf16_16816(oacc[2 * np], pf[kk], vb[0], vb[1]);
+                mma_bf16_16816(oacc[2 * np + 1], pf[kk], vb[2], vb[3]);
+            }
+        }
+        __syncthreads();   // the buffer is refilled two iterations later by load_block(blk + 2, buf)
+    }
+    // ---- write the split's partial result ----
+    lrow0 += __shfl_xor_sync(0xffffffffu, lrow0, 1);
+    lrow0 += __shfl_xor_sync(0xffffffffu, lrow0, 2);
+    lrow1 += __shfl_xor_sync(0xffffffffu, lrow1, 1);
+    lrow1 += __shfl_xor_sync(0xffffffffu, lrow1, 2);
+    if (v0) {
+        const size_t idx = (size_t)split * pstride + (size_t)(off + i0) * a.H + hh;
+        float* po = a.part_o + idx * HD;
+#pragma unroll
+        for (int n = 0; n < ONT; ++n) *reinterpret_cast<float2*>(po + n * 8 + 2 * tig) = make_float2(oacc[n][0], oacc[n][1]);
+        if (tig == 0) { a.part_ml[idx * 2] = mrow0; a.part_ml[idx * 2 + 1] = lrow0; }
+    }
+    if (v1) {
+        const size_t idx = (size_t)split * pstride + (size_t)(off + i1) * a.H + hh;
+        float* po = a.part_o + idx * HD;
+#pragma unroll
+        for (int n = 0; n < ONT; ++n) *reinterpret_cast<float2*>(po + n * 8 + 2 * tig) = make_float2(oacc[n][2], oacc[n][3]);
+        if (tig == 0) { a.part_ml[idx * 2] = mrow1; a.part_ml[idx * 2 + 1] = lrow1; }
+    }
+}
+
+// Combines the splits of one (row, head): out = sum_s O_s 2^(m_s - M) / sum_s l_s 2^(m_s - M).
+template <int HD>
+__global__ void __launch_bounds__(HD) k_tree_attn_merge(const float* __restrict__ part_o, const float* __restrict__ part_ml,
+                                                       bf16* __restrict__ out, int n_splits, int rows, int H,
+                                                       const int32_t* status) {
+    if (*status != 0) return;
+    const int r = blockIdx.x, hh = blockIdx.y, e = threadIdx.x;
+    const size_t pstride = (size_t)rows * H, idx = (size_t)r * H + hh;
+    float M = -INFINITY;
+    for (int s = 0; s < n_splits; ++s) M = fmaxf(M, part_ml[((size_t)s * pstride + idx) * 2]);
+    float num = 0.f, den = 0.f;
+    for (int s = 0; s < n_splits; ++s) {
+        const float m = part_ml[((size_t)s * pstride + idx) * 2];
+        if (m == -INFINITY) continue;
+        const float w = exp2f(m - M);
+        den += part_ml[((size_t)s * pstride + idx) * 2 + 1] * w;
+        num += part_o[((size_t)s * pstride + idx) * HD + e] * w;
+    }
+    out[idx * HD + e] = __float2bfloat16_rn(num / den);
+}
+
+template <int HD>
+static void launch_mma(aded_model* m, aded_kv* kv, int layer, int batch, int rows, int max_tree, cudaStream_t st) {
+    AttnArgs a;
+    a.q = (const bf16*)m->q;
+    a.part_o = m->att_o;
+    a.part_ml = m->att_ml;
+    a.base = kv->base_dev;
+    a.cap = kv->cap_dev;
+    a.len = kv->len_dev;
+    a.row_off = m->seqs.row_off;
+    a.anc = m->rows.anc;
+    a.layer = layer;
+    a.H = m->cfg.n_heads;
+    // enough (head, split) CTAs for about two per SM, within what the partial buffers hold
+    int splits = (ws_grid_limit(m->device) + m->cfg.n_heads * batch - 1) / (m->cfg.n_heads * batch);
+    if (splits > m->att_splits_max) splits = m->att_splits_max;
+    if (splits < 1) splits = 1;
+    a.n_splits = splits;
+    a.rows_total = rows;
+    a.scale_log2 = 1.4426950408889634f / sqrtf((float)HD);
+    a.status = m->status;
+    dim3 grid(m->cfg.n_heads, splits, batch);
+    const size_t smem = (size_t)4 * TA_BLK * HD * sizeof(bf16);
+    static bool attr_done = false;
+    if (!attr_done) {
+        cudaFuncSetAttribute(k_tree_attn_mma<HD, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        cudaFuncSetAttribute(k_tree_attn_mma<HD, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        attr_done = true;
+    }
+    if (max_tree <= 64) k_tree_attn_mma<HD, 4><<<grid, 128, smem, st>>>(a);
+    else k_tree_attn_mma<HD, 8><<<grid, 256, smem, st>>>(a);
+    dim3 mgrid(rows, m->cfg.n_heads);
+    k_tree_attn_merge<HD><<<mgrid, HD, 0, st>>>(m->att_o, m->att_ml, (bf16*)m->attn, splits, rows, m->cfg.n_heads, m->status);
+}
+
+void launch_tree_attention(aded_model* m, aded_kv* kv, int layer, int batch, int rows, int max_tree, cudaStream_t st) {
     const int H = m->cfg.n_heads, hd = m->cfg.head_dim;
+    if (m->cfg.dtype == ADED_BF16 && m->att_o != nullptr) {
+        if (hd == 128) launch_mma<128>(m, kv, layer, batch, rows, max_tree, st);
+        else launch_mma<64>(m, kv, layer, batch, rows, max_tree, st);
+        return;
+    }
     const float scale = 1.f / sqrtf((float)hd);
     const int warps = rows * H;
     const int blocks = (warps + 3) / 4;
