@@ -218,8 +218,6 @@ def run_ours(args, rank, world):
     assert B.aded_trigram_poll_status(tg) == 0 and B.aded_model_poll_status(model) == 0
 
     # ---------------- pass 2: the same decode from device-resident inputs ---------------------------------
-    B.aded_kv_set_len(kv, 0, base_len)
-    tg = fresh_table()
     d_tok = torch.tensor([r["tokens"] for r in rec], dtype=torch.int32, device=dev)
     d_par = torch.tensor([r["parents"] for r in rec], dtype=torch.int32, device=dev)
     d_out = torch.zeros((total, n), dtype=torch.int32, device=dev)
@@ -229,37 +227,48 @@ def run_ours(args, rank, world):
     qmax = max(len(r["ctxs"]) for r in rec)
     d_tk = torch.empty((qmax, wl.topk), dtype=torch.int32, device=dev)
     d_cn = torch.empty((qmax, wl.topk), dtype=torch.int32, device=dev)
-    torch.cuda.synchronize()
-    launches0 = 0
-    step_ev = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
+
+    def replay(profile):
+        """Rolls cache and table back to the end of the prompt and runs all steps from device memory.
+        profile=False is the timed run; profile=True repeats it with per-kernel event timing."""
+        B.aded_kv_set_len(kv, 0, base_len)
+        table = fresh_table()
+        d_out.zero_()
+        d_len.zero_()
+        torch.cuda.synchronize()
+        step_ev = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
+        launches0 = 0
+        for step in range(total):
+            if step == warm:
+                if world > 1:
+                    torch.distributed.barrier()
+                torch.cuda.synchronize()
+                launches0 = B.aded_launch_count()
+                if profile:
+                    B.aded_profile_begin(model)
+                step_ev[0].record()
+            B.aded_trigram_topk(table, d_ctx[step], wl.topk, d_tk, d_cn)
+            B.aded_verify(model, kv, d_tok[step], d_par[step], d_out[step], d_len[step])
+            B.aded_trigram_update(table, d_span[step])
+            if step >= warm:
+                step_ev[step - warm + 1].record()
+        torch.cuda.synchronize()
+        if world > 1:
+            torch.distributed.barrier()
+        prof = B.aded_profile_end(model) if profile else None
+        launches = B.aded_launch_count() - launches0
+        lens = d_len[:, 0].tolist()
+        for step in range(total):   # the replay must reproduce the recorded decode
+            assert d_out[step, :lens[step]].tolist() == rec[step]["out"], f"replay diverged at step {step}"
+        per_step = [step_ev[i].elapsed_time(step_ev[i + 1]) for i in range(steps)]
+        return step_ev[0].elapsed_time(step_ev[-1]), per_step, launches, sum(lens[warm:]), prof
+
     sampler.start()
-    for step in range(total):
-        if step == warm:
-            if world > 1:
-                torch.distributed.barrier()
-            torch.cuda.synchronize()
-            launches0 = B.aded_launch_count()
-            B.aded_profile_begin(model)
-            step_ev[0].record()
-        B.aded_trigram_topk(tg, d_ctx[step], wl.topk, d_tk, d_cn)
-        B.aded_verify(model, kv, d_tok[step], d_par[step], d_out[step], d_len[step])
-        B.aded_trigram_update(tg, d_span[step])
-        if step >= warm:
-            step_ev[step - warm + 1].record()
-    torch.cuda.synchronize()
-    if world > 1:
-        torch.distributed.barrier()
+    dev_ms, per_step, launches, accepted, _ = replay(profile=False)
     clocks = sampler.stop()
-    prof_ms, prof_n = B.aded_profile_end(model)
-    launches = B.aded_launch_count() - launches0
-    dev_ms = step_ev[0].elapsed_time(step_ev[-1])
-    per_step = [step_ev[i].elapsed_time(step_ev[i + 1]) for i in range(steps)]
-    lens = d_len[:, 0].tolist()
-    for step in range(total):   # the replay must reproduce the recorded decode
-        assert d_out[step, :lens[step]].tolist() == rec[step]["out"], f"replay diverged at step {step}"
-    accepted = sum(lens[warm:])
     assert accepted == accepted_e2e
     final_len = B.aded_kv_len(kv, 0)
+    _, _, _, _, (prof_ms, prof_n) = replay(profile=True)
 
     # ---------------- roofline of the dominant kernel (the weight-streaming GEMMs) ------------------------
     pk = peaks()

@@ -25,6 +25,7 @@ namespace aded {
 void note_cuda_error(cudaError_t e, const char* what);
 void note_launch(int n = 1);   // bumps the process-wide launch counter
 
+enum { ARGMAX_CHUNKS = 16 };
 enum { PROF_GEMM = 0, PROF_ATTN = 1, PROF_OTHER = 2, PROF_GROUPS = 3 };
 struct ProfSpan { int group; int launches; cudaEvent_t a, b; };
 
@@ -44,6 +45,17 @@ struct RowMeta {
     int32_t* depth;    // [R] edges from the root
     int32_t* pos;      // [R] rotary position = committed length + depth
     uint64_t* anc;     // [R][2] bit j set <=> local node j is an ancestor of the row's node, or itself
+};
+
+// The caller's arrays of one verify/append call.  Kernels read them through this record, which
+// lives at a fixed device address and is rewritten before every call, so that a captured launch
+// sequence can be replayed with other arrays.
+struct CallPtrs {
+    const int32_t* tokens;
+    const int32_t* parents;
+    int32_t* out_tokens;
+    int32_t* out_len;
+    int32_t out_stride;
 };
 
 struct SeqMeta {
@@ -91,6 +103,7 @@ struct aded_model {
     int32_t* status;  // device status word
     aded::RowMeta rows;
     aded::SeqMeta seqs;
+    aded::CallPtrs* call_dev;   // device copy of the current call's array pointers
     std::vector<void*> owned;   // everything cudaMalloc'ed for this handle
 
     float* dbg_logits;
@@ -105,9 +118,31 @@ struct aded_model {
     bool ws_ready;
     std::vector<CUtensorMap> ws_maps;   // per layer: wqkv, wo, wgu, wd; then lm_head; then x, attn, act
     float* ws_slots;                    // partial result tiles (see gemm_out.cuh)
+    aded::TileRef* ws_tiles[5];         // contributor tables of the wqkv, wo, wgu, wd and LM-head results
+
+    float* norm_ssq;        // [R][32] per-chunk sums of squares of the RMSNorm kernel
+    int32_t* norm_count;    // [R] chunk arrival counters, zero between launches
+    float* argmax_val;      // [R][ARGMAX_CHUNKS] best logit of each column chunk
+    int32_t* argmax_idx;
+
+    // captured launch sequences, one per call shape (see model.cu)
+    struct GraphEntry {
+        std::vector<int64_t> key;
+        cudaGraphExec_t exec;
+        int32_t* offsets_pin;     // pinned copy of the row offsets the graph uploads
+        uint64_t last_use;
+        std::vector<aded::ProfSpan> spans;   // event pairs recorded by the graph (profiling variant only)
+    };
+    std::vector<GraphEntry> graphs;
+    uint64_t graph_clock;
+    bool graphs_on;
 
     bool prof_on;
-    std::vector<aded::ProfSpan> prof_spans;   // spans recorded since aded_profile_begin
+    std::vector<aded::ProfSpan>* capture_spans;   // while a profiling graph is being captured: where its spans go
+    int prof_pending;                             // index of the graph whose last replay's events are unread, or -1
+    float prof_ms[aded::PROF_GROUPS];             // harvested so far
+    int32_t prof_n[aded::PROF_GROUPS];
+    std::vector<aded::ProfSpan> prof_spans;   // spans recorded by direct launches since aded_profile_begin
     std::vector<cudaEvent_t> prof_pool;       // events kept for reuse
 };
 
@@ -115,14 +150,12 @@ namespace aded {
 
 // ---- launchers (each enqueues on `st`; shapes are validated by the callers) ---------------
 // tree.cu
-void launch_tree_prologue(aded_model* m, aded_kv* kv, const int32_t* tokens, const int32_t* parents,
-                          int batch, int chain_mode, cudaStream_t st);
-void launch_accept(aded_model* m, aded_kv* kv, const int32_t* tokens, const int32_t* parents, int batch,
-                   int32_t* out_tokens, int out_stride, int32_t* out_len, cudaStream_t st);
+void launch_tree_prologue(aded_model* m, aded_kv* kv, int batch, int chain_mode, cudaStream_t st);
+void launch_accept(aded_model* m, aded_kv* kv, int batch, cudaStream_t st);
 void launch_compact_commit(aded_model* m, aded_kv* kv, int batch, int chain_mode, cudaStream_t st);
 
 // dense.cu
-void launch_embed(aded_model* m, const int32_t* tokens, int rows, cudaStream_t st);
+void launch_embed(aded_model* m, int rows, cudaStream_t st);
 void launch_rope_table(aded_model* m, int rows, cudaStream_t st);
 // `y` (may be NULL): projection result added to the residual stream before the norm
 void launch_add_rmsnorm(aded_model* m, const GemmOut* y, const void* gain, int rows, cudaStream_t st);
@@ -139,6 +172,8 @@ void launch_materialize(aded_model* m, const GemmOut& src, float* dst, int rows,
 // gemm_ws.cu
 bool ws_make_map(CUtensorMap* map, const void* ptr, uint64_t rows, uint64_t cols, uint32_t box_rows);
 bool ws_supported(int n, int k);
+bool ws_prepare();
+bool attn_prepare();
 int ws_grid_limit(int device);
 int ws_grid(int device, int n, int k);
 size_t ws_slot_floats(int device, int max_n, int max_rows);

@@ -1,9 +1,10 @@
-// Row-wise pieces of the Llama-style decoder around the projections: embedding gather, RMSNorm,
-// residual add, rotary embedding + K/V write, SwiGLU, per-row greedy choice, and a plain
+// Row-wise pieces of the Llama-style decoder around the projections: embedding gather, residual
+// add + RMSNorm, rotary embedding + K/V write, SwiGLU, per-row greedy choice, and a plain
 // shared-memory GEMM used for fp32 models and for shapes the tensor-core path does not take.
 //
 // Rounding: activations are stored in the model dtype (bf16 models round to nearest even at
-// every store below); all sums are fp32.
+// every store below); all sums are fp32.  Kernels that consume a projection read it through
+// GemmOut (gemm_out.cuh): either a plain fp32 matrix or per-CTA partial tiles added in CTA order.
 #include "aded_internal.cuh"
 
 namespace aded {
@@ -26,9 +27,10 @@ __device__ __forceinline__ float block_sum(float v, float* red) {
 }
 
 template <typename T>
-__global__ void k_embed(const T* __restrict__ table, const int32_t* __restrict__ tokens, T* __restrict__ h,
+__global__ void k_embed(const T* __restrict__ table, const CallPtrs* __restrict__ call, T* __restrict__ h,
                         int d, const int32_t* status) {
     if (*status != 0) return;
+    const int32_t* __restrict__ tokens = call->tokens;
     const int r = blockIdx.x;
     const T* src = table + (size_t)tokens[r] * d;
     for (int c = threadIdx.x; c < d; c += blockDim.x) h[(size_t)r * d + c] = src[c];
@@ -49,34 +51,62 @@ __global__ void k_rope_table(const int32_t* __restrict__ pos, float* __restrict_
     }
 }
 
-// x = round(h * rsqrt(mean(h^2) + eps) * gain); when `y` is given, first h = round(h + y).
+// Residual add + RMSNorm:  h = round(h + y) (when y is given), x = round(h * rsqrt(mean(h^2) + eps) * gain).
+// Grid (column chunks of 256, rows): each thread owns one column of one row, so the partial tiles of
+// y are gathered with full parallelism.  A chunk leaves its sum of squares in `ssq`; the chunk that
+// finishes a row last (per-row counter) adds the row's chunk sums in chunk order and writes x for
+// the whole row.  The order of every sum is fixed, so the result does not depend on timing.
 template <typename T>
-__global__ void k_add_rmsnorm(T* __restrict__ h, GemmOut y, int has_y, const T* __restrict__ gain,
-                              T* __restrict__ x, int d, float eps, const int32_t* status) {
+__global__ void __launch_bounds__(256) k_add_rmsnorm(T* __restrict__ h, GemmOut y, int has_y, const T* __restrict__ gain,
+                                                     T* __restrict__ x, int d, float eps, float* __restrict__ ssq,
+                                                     int32_t* __restrict__ row_count, const int32_t* status) {
     if (*status != 0) return;
     __shared__ float red[32];
-    __shared__ TileRef tiles[64];          // contributors of each 128-column tile of y (d <= 8192)
-    const int r = blockIdx.x;
-    if (has_y && y.mode == 1) {
-        for (int t = threadIdx.x; t < y.n_tiles; t += blockDim.x) tiles[t] = gemm_tile_ref(y, t);
-        __syncthreads();
-    }
-    T* hr = h + (size_t)r * d;
-    float ss = 0.f;
-    for (int c = threadIdx.x; c < d; c += blockDim.x) {
-        float v = to_f32(hr[c]);
+    __shared__ int s_last;
+    const int r = blockIdx.y, c = blockIdx.x * 256 + threadIdx.x;
+    float sq = 0.f;
+    if (c < d) {
+        float v = to_f32(h[(size_t)r * d + c]);
         if (has_y) {
-            const float add = y.mode == 0 ? y.y[(size_t)r * d + c] : gemm_out_at(y, tiles[c >> 7], r, c & 127);
+            const float add = y.mode == 0 ? y.y[(size_t)r * d + c] : gemm_out_at(y, y.tiles[c >> 7], r, c & 127);
             const T nv = from_f32<T>(v + add);
-            hr[c] = nv;
+            h[(size_t)r * d + c] = nv;
             v = to_f32(nv);
         }
-        ss += v * v;
+        sq = v * v;
     }
-    ss = block_sum(ss, red);
-    const float inv = rsqrtf(ss / (float)d + eps);
-    for (int c = threadIdx.x; c < d; c += blockDim.x)
-        x[(size_t)r * d + c] = from_f32<T>(to_f32(hr[c]) * inv * to_f32(gain[c]));
+    sq = block_sum(sq, red);
+    if (threadIdx.x == 0) {
+        ssq[r * 32 + blockIdx.x] = sq;
+        __threadfence();
+        const int prev = atomicAdd(&row_count[r], 1);
+        s_last = prev == (int)gridDim.x - 1;
+        if (s_last) row_count[r] = 0;
+    }
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();
+    float total = 0.f;
+    for (int i = 0; i < (int)gridDim.x; ++i) total += __ldcg(ssq + r * 32 + i);
+    const float inv = rsqrtf(total / (float)d + eps);
+    if (sizeof(T) == 2) {
+        // two columns per access
+        const uint32_t* hr = reinterpret_cast<const uint32_t*>(h + (size_t)r * d);
+        const uint32_t* gr = reinterpret_cast<const uint32_t*>(gain);
+        uint32_t* xr = reinterpret_cast<uint32_t*>(x + (size_t)r * d);
+        for (int cc = threadIdx.x; cc < d / 2; cc += 256) {
+            const uint32_t hv = __ldcg(hr + cc), gv = gr[cc];
+            const __nv_bfloat162 hb = *reinterpret_cast<const __nv_bfloat162*>(&hv);
+            const __nv_bfloat162 gb = *reinterpret_cast<const __nv_bfloat162*>(&gv);
+            const __nv_bfloat162 o = __floats2bfloat162_rn(__low2float(hb) * inv * __low2float(gb),
+                                                           __high2float(hb) * inv * __high2float(gb));
+            xr[cc] = *reinterpret_cast<const uint32_t*>(&o);
+        }
+    } else {
+        const float* hr = reinterpret_cast<const float*>(h) + (size_t)r * d;
+        for (int cc = threadIdx.x; cc < d; cc += 256)
+            x[(size_t)r * d + cc] = from_f32<T>(__ldcg(hr + cc) * inv * to_f32(gain[cc]));
+    }
 }
 
 // y[r, n] = sum_k x[r, k] * w[n, k]; 64 x 64 output tile per block, 16-wide k slabs in shared
@@ -137,7 +167,7 @@ __global__ void k_rope_kv(GemmOut qkv, const float* __restrict__ cs, const float
     // the head's q, k and v columns each lie inside one 128-column tile of the projection result
     const int cq = hh * hd, ck = d + hh * hd, cv = 2 * d + hh * hd;
     TileRef tq = {0, 0}, tk = {0, 0}, tv = {0, 0};
-    if (qkv.mode == 1) { tq = gemm_tile_ref(qkv, cq >> 7); tk = gemm_tile_ref(qkv, ck >> 7); tv = gemm_tile_ref(qkv, cv >> 7); }
+    if (qkv.mode == 1) { tq = qkv.tiles[cq >> 7]; tk = qkv.tiles[ck >> 7]; tv = qkv.tiles[cv >> 7]; }
     auto at = [&](const TileRef& t, int col) {
         return qkv.mode == 0 ? qkv.y[(size_t)r * 3 * d + col] : gemm_out_at(qkv, t, r, col & 127);
     };
@@ -165,21 +195,20 @@ __global__ void k_swiglu(GemmOut gu, T* __restrict__ act, int F, const int32_t* 
     act[(size_t)r * F + c] = from_f32<T>(g / (1.f + expf(-g)) * u);
 }
 
-// Greedy choice per row: largest fp32 logit, lowest index among equals.
-__global__ void k_argmax(GemmOut logits, int32_t* __restrict__ best, int V, const int32_t* status) {
+// Greedy choice per row: largest fp32 logit, lowest index among equals.  Stage 1: grid (chunks, rows),
+// every block scans `chunk` columns of one row and leaves (value, index) of its best; stage 2 (one
+// thread per row) takes the best of the chunks in ascending column order.
+__global__ void __launch_bounds__(256) k_argmax_chunks(GemmOut logits, float* __restrict__ pv, int32_t* __restrict__ pi,
+                                                       int V, int chunk, const int32_t* status) {
     if (*status != 0) return;
-    __shared__ float sv[32];
-    __shared__ int si[32];
-    extern __shared__ TileRef tiles[];     // contributors of each 128-column tile (tensor-core path)
-    const int r = blockIdx.x;
-    if (logits.mode == 1) {
-        for (int t = threadIdx.x; t < logits.n_tiles; t += blockDim.x) tiles[t] = gemm_tile_ref(logits, t);
-        __syncthreads();
-    }
+    __shared__ float sv[8];
+    __shared__ int si[8];
+    const int r = blockIdx.y;
+    const int c0 = blockIdx.x * chunk, c1 = min(V, c0 + chunk);
     float bv = -INFINITY;
     int bi = 0x7fffffff;
-    for (int c = threadIdx.x; c < V; c += blockDim.x) {
-        const float v = logits.mode == 0 ? logits.y[(size_t)r * V + c] : gemm_out_at(logits, tiles[c >> 7], r, c & 127);
+    for (int c = c0 + threadIdx.x; c < c1; c += 256) {
+        const float v = gemm_out_load(logits, r, c);
         if (v > bv) { bv = v; bi = c; }   // c ascends per thread: first maximum kept
     }
     for (int o = 16; o > 0; o >>= 1) {
@@ -190,17 +219,27 @@ __global__ void k_argmax(GemmOut logits, int32_t* __restrict__ best, int V, cons
     const int w = threadIdx.x >> 5, l = threadIdx.x & 31;
     if (l == 0) { sv[w] = bv; si[w] = bi; }
     __syncthreads();
-    if (w == 0) {
-        const int nw = blockDim.x >> 5;
-        bv = l < nw ? sv[l] : -INFINITY;
-        bi = l < nw ? si[l] : 0x7fffffff;
-        for (int o = 16; o > 0; o >>= 1) {
-            const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
-            const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
-            if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
-        }
-        if (l == 0) best[r] = bi == 0x7fffffff ? 0 : bi;
+    if (threadIdx.x == 0) {
+        for (int i = 1; i < 8; ++i)
+            if (sv[i] > bv || (sv[i] == bv && si[i] < bi)) { bv = sv[i]; bi = si[i]; }
+        pv[r * gridDim.x + blockIdx.x] = bv;
+        pi[r * gridDim.x + blockIdx.x] = bi;
     }
+}
+
+__global__ void k_argmax_final(const float* __restrict__ pv, const int32_t* __restrict__ pi, int32_t* __restrict__ best,
+                               int chunks, int rows, const int32_t* status) {
+    if (*status != 0) return;
+    const int r = blockIdx.x * blockDim.x + threadIdx.x;
+    if (r >= rows) return;
+    float bv = -INFINITY;
+    int bi = 0x7fffffff;
+    for (int i = 0; i < chunks; ++i) {
+        const float v = pv[r * chunks + i];
+        const int idx = pi[r * chunks + i];
+        if (v > bv || (v == bv && idx < bi)) { bv = v; bi = idx; }
+    }
+    best[r] = bi == 0x7fffffff ? 0 : bi;
 }
 
 __global__ void k_materialize(GemmOut src, float* __restrict__ dst, int n, const int32_t* status) {
@@ -214,10 +253,10 @@ __global__ void k_materialize(GemmOut src, float* __restrict__ dst, int n, const
 #define BY_DTYPE(m, CALL_BF16, CALL_F32) \
     do { if ((m)->cfg.dtype == ADED_BF16) { CALL_BF16; } else { CALL_F32; } } while (0)
 
-void launch_embed(aded_model* m, const int32_t* tokens, int rows, cudaStream_t st) {
+void launch_embed(aded_model* m, int rows, cudaStream_t st) {
     const int d = m->cfg.d_model;
-    BY_DTYPE(m, (k_embed<bf16><<<rows, 256, 0, st>>>((const bf16*)m->top.embed, tokens, (bf16*)m->h, d, m->status)),
-             (k_embed<float><<<rows, 256, 0, st>>>((const float*)m->top.embed, tokens, (float*)m->h, d, m->status)));
+    BY_DTYPE(m, (k_embed<bf16><<<rows, 256, 0, st>>>((const bf16*)m->top.embed, m->call_dev, (bf16*)m->h, d, m->status)),
+             (k_embed<float><<<rows, 256, 0, st>>>((const float*)m->top.embed, m->call_dev, (float*)m->h, d, m->status)));
 }
 
 void launch_rope_table(aded_model* m, int rows, cudaStream_t st) {
@@ -230,8 +269,9 @@ void launch_add_rmsnorm(aded_model* m, const GemmOut* y, const void* gain, int r
     GemmOut none = {};
     const GemmOut& yy = y ? *y : none;
     const int has = y != nullptr;
-    BY_DTYPE(m, (k_add_rmsnorm<bf16><<<rows, 256, 0, st>>>((bf16*)m->h, yy, has, (const bf16*)gain, (bf16*)m->x, d, m->cfg.rms_eps, m->status)),
-             (k_add_rmsnorm<float><<<rows, 256, 0, st>>>((float*)m->h, yy, has, (const float*)gain, (float*)m->x, d, m->cfg.rms_eps, m->status)));
+    dim3 grid((d + 255) / 256, rows);
+    BY_DTYPE(m, (k_add_rmsnorm<bf16><<<grid, 256, 0, st>>>((bf16*)m->h, yy, has, (const bf16*)gain, (bf16*)m->x, d, m->cfg.rms_eps, m->norm_ssq, m->norm_count, m->status)),
+             (k_add_rmsnorm<float><<<grid, 256, 0, st>>>((float*)m->h, yy, has, (const float*)gain, (float*)m->x, d, m->cfg.rms_eps, m->norm_ssq, m->norm_count, m->status)));
 }
 
 static void launch_gemm_plain(aded_model* m, const void* x, const void* w, float* y, int rows, int n, int k, cudaStream_t st) {
@@ -256,6 +296,7 @@ GemmOut launch_gemm(aded_model* m, int w_map, int x_map, const void* x, const vo
         out.n_tiles = n / 128;
         out.kb = k / 64;
         out.g = ws_grid(m->device, n, k);
+        out.tiles = m->ws_tiles[w_map < 4 * m->cfg.n_layers ? w_map % 4 : 4];
         return out;
     }
     launch_gemm_plain(m, x, w, y, rows, n, k, st);
@@ -284,8 +325,12 @@ void launch_swiglu(aded_model* m, const GemmOut& gu, int rows, cudaStream_t st) 
 }
 
 void launch_argmax(aded_model* m, const GemmOut& logits, int rows, cudaStream_t st) {
-    const size_t smem = logits.mode == 1 ? (size_t)logits.n_tiles * sizeof(TileRef) : 0;
-    k_argmax<<<rows, 256, smem, st>>>(logits, m->best, m->cfg.vocab, m->status);
+    const int V = m->cfg.vocab;
+    const int chunks = ARGMAX_CHUNKS;
+    const int chunk = ((V + chunks - 1) / chunks + 127) / 128 * 128;   // whole 128-column tiles per block
+    dim3 grid(chunks, rows);
+    k_argmax_chunks<<<grid, 256, 0, st>>>(logits, m->argmax_val, m->argmax_idx, V, chunk, m->status);
+    k_argmax_final<<<(rows + 127) / 128, 128, 0, st>>>(m->argmax_val, m->argmax_idx, m->best, chunks, rows, m->status);
 }
 
 }  // namespace aded

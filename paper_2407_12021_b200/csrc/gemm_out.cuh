@@ -18,9 +18,16 @@
 
 namespace aded {
 
+// The contributors of one tile: first slot and how many consecutive slots to add.
+struct TileRef {
+    int first_slot;
+    int count;
+};
+
 struct GemmOut {
     const float* y;       // mode 0: [rows, n] row-major
     const float* slots;   // mode 1: partial tiles
+    const TileRef* tiles; // mode 1: contributors of every tile (device table, one per GEMM shape)
     int mode;
     int n;                // result columns
     int n_tiles, kb, g;   // mode 1: 128-column tiles, k blocks per tile, CTAs of the GEMM launch
@@ -40,16 +47,11 @@ __host__ __device__ __forceinline__ int ws_owner(long long u, long long units, l
     return (int)c;
 }
 
-// The contributors of one tile: first slot and how many consecutive slots to add.
-struct TileRef {
-    int first_slot;
-    int count;
-};
-
-__device__ __forceinline__ TileRef gemm_tile_ref(const GemmOut& o, int tile) {
-    const long long units = (long long)o.n_tiles * o.kb;
-    const int c_first = ws_owner((long long)tile * o.kb, units, o.g);
-    const int c_last = ws_owner((long long)(tile + 1) * o.kb - 1, units, o.g);
+// Contributors of tile `tile` when n_tiles x kb units are split over g CTAs (host: fills the tables).
+__host__ __device__ __forceinline__ TileRef gemm_tile_ref(int n_tiles, int kb, int g, int tile) {
+    const long long units = (long long)n_tiles * kb;
+    const int c_first = ws_owner((long long)tile * kb, units, g);
+    const int c_last = ws_owner((long long)(tile + 1) * kb - 1, units, g);
     TileRef t;
     t.first_slot = tile + c_first;
     t.count = c_last - c_first + 1;
@@ -70,15 +72,15 @@ __device__ __forceinline__ float gemm_out_at(const GemmOut& o, const TileRef& t,
     const float* p = o.slots + region + ((size_t)t.first_slot * rb + (r & 127)) * 128 + col;
     const size_t stride = (size_t)rb * 128;
     float sum = 0.f;
+#pragma unroll 4
     for (int i = 0; i < t.count; ++i) sum += __ldcg(p + (size_t)i * stride);
     return sum;
 }
 
-// Any element, any mode (computes the tile's contributors on the spot).
+// Any element, any mode.
 __device__ __forceinline__ float gemm_out_load(const GemmOut& o, int r, int c) {
     if (o.mode == 0) return o.y[(size_t)r * o.n + c];
-    const TileRef t = gemm_tile_ref(o, c >> 7);
-    return gemm_out_at(o, t, r, c & 127);
+    return gemm_out_at(o, o.tiles[c >> 7], r, c & 127);
 }
 
 }  // namespace aded

@@ -312,6 +312,11 @@ size_t ws_slot_floats(int device, int max_n, int max_rows) {
     return blocks * ((size_t)max_n / WS_BM + ws_grid_limit(device)) * 128 * WS_BM;
 }
 
+// Raises the kernel's dynamic shared-memory limit; once per process, before any launch or capture.
+bool ws_prepare() {
+    return cudaFuncSetAttribute(k_gemm_ws, cudaFuncAttributeMaxDynamicSharedMemorySize, 112 * 1024) == cudaSuccess;
+}
+
 // Shapes the tensor-core path takes.
 bool ws_supported(int n, int k) { return n % WS_BM == 0 && k % WS_BK == 0 && k >= WS_BK; }
 
@@ -336,12 +341,6 @@ cudaError_t ws_launch(const CUtensorMap& map_w, const CUtensorMap& map_x, int ro
     p.slots = slots + (size_t)(row0 / 128) * (size_t)(p.n_tiles + grid) * 128 * WS_BM;
     p.status = status;
     const size_t smem = (size_t)p.stages * stage_bytes + 1024 + 256;
-    static bool attr_set = false;
-    if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(k_gemm_ws, cudaFuncAttributeMaxDynamicSharedMemorySize, 112 * 1024);
-        if (e != cudaSuccess) return e;
-        attr_set = true;
-    }
     k_gemm_ws<<<grid, WS_THREADS, smem, st>>>(map_w, map_x, p);
     return cudaGetLastError();
 }

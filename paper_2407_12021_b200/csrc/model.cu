@@ -36,12 +36,13 @@ struct Span {
             if (!m->prof_pool.empty()) { *e = m->prof_pool.back(); m->prof_pool.pop_back(); }
             else if (cudaEventCreate(e) != cudaSuccess) { on = false; cudaGetLastError(); return; }
         }
-        cudaEventRecord(rec.a, st);
+        // inside a capture the record becomes a node of the graph and is timed on every replay
+        cudaEventRecordWithFlags(rec.a, st, m->capture_spans ? cudaEventRecordExternal : cudaEventRecordDefault);
     }
     ~Span() {
         if (!on) return;
-        cudaEventRecord(rec.b, st);
-        m->prof_spans.push_back(rec);
+        cudaEventRecordWithFlags(rec.b, st, m->capture_spans ? cudaEventRecordExternal : cudaEventRecordDefault);
+        (m->capture_spans ? *m->capture_spans : m->prof_spans).push_back(rec);
     }
 };
 
@@ -89,6 +90,13 @@ static aded_status alloc_model(aded_model* m) {
     TRY(dev_alloc(m, &m->seqs.row_off, B + 1));
     TRY(dev_alloc(m, &m->seqs.path, B * ADED_MAX_NODES));
     TRY(dev_alloc(m, &m->seqs.new_len, B));
+    TRY(dev_alloc(m, &m->call_dev, 1));
+    TRY(dev_alloc(m, &m->norm_ssq, R * 32));
+    TRY(dev_alloc(m, &m->norm_count, R));
+    TRY(dev_alloc(m, &m->argmax_val, R * ARGMAX_CHUNKS));
+    TRY(dev_alloc(m, &m->argmax_idx, R * ARGMAX_CHUNKS));
+    ADED_CUDA_TRY(cudaMemset(m->norm_count, 0, R * sizeof(int32_t)));
+    if (d > 32 * 256) return ADED_ERR_UNSUPPORTED;   // the norm kernel keeps at most 32 column chunks per row
     ADED_CUDA_TRY(cudaMemset(m->status, 0, sizeof(int32_t)));
     ADED_CUDA_TRY(cudaMemset(m->h, 0, R * d * m->elem));
     ADED_CUDA_TRY(cudaMemset(m->x, 0, R * d * m->elem));
@@ -98,7 +106,7 @@ static aded_status alloc_model(aded_model* m) {
     m->att_o = nullptr;
     m->att_ml = nullptr;
     m->att_splits_max = 1;
-    if (c.dtype == ADED_BF16 && !getenv("ADED_PLAIN_ATTN")) {
+    if (c.dtype == ADED_BF16 && !getenv("ADED_PLAIN_ATTN") && attn_prepare()) {
         m->att_splits_max = R <= 128 ? 16 : (int)(16 * 128 / R > 0 ? 16 * 128 / R : 1);
         TRY(dev_alloc(m, &m->att_o, (size_t)m->att_splits_max * R * d));
         TRY(dev_alloc(m, &m->att_ml, (size_t)m->att_splits_max * R * c.n_heads * 2));
@@ -110,7 +118,7 @@ static aded_status alloc_model(aded_model* m) {
         ws_supported(2 * (int)F, (int)d) && ws_supported((int)d, (int)F) && ws_supported((int)V, (int)d)) {
         const int L = c.n_layers;
         m->ws_maps.resize(4 * L + 4);
-        bool ok = true;
+        bool ok = ws_prepare();
         for (int l = 0; l < L && ok; ++l) {
             const aded_layer_weights& w = m->layers[l];
             ok = ws_make_map(&m->ws_maps[4 * l + WS_MAP_QKV], w.wqkv, 3 * d, d, 128) &&
@@ -126,30 +134,45 @@ static aded_status alloc_model(aded_model* m) {
             if (2 * F > widest) widest = 2 * F;
             if (V > widest) widest = V;
             TRY(dev_alloc(m, &m->ws_slots, ws_slot_floats(m->device, (int)widest, (int)R)));
+            // which slots make up each 128-column tile of each projection's result
+            const int shapes[5][2] = {{3 * (int)d, (int)d}, {(int)d, (int)d}, {2 * (int)F, (int)d}, {(int)d, (int)F}, {(int)V, (int)d}};
+            for (int i = 0; i < 5; ++i) {
+                const int nt = shapes[i][0] / 128, kb = shapes[i][1] / 64, g = ws_grid(m->device, shapes[i][0], shapes[i][1]);
+                std::vector<TileRef> table(nt);
+                for (int t = 0; t < nt; ++t) table[t] = gemm_tile_ref(nt, kb, g, t);
+                TRY(dev_alloc(m, &m->ws_tiles[i], (size_t)nt));
+                ADED_CUDA_TRY(cudaMemcpy(m->ws_tiles[i], table.data(), nt * sizeof(TileRef), cudaMemcpyHostToDevice));
+            }
             m->ws_ready = true;
         }
     }
     return ADED_OK;
 }
 
-// The launch sequence of one pass.  chain_mode: the rows form a chain per sequence, every row is
-// accepted and no logits are needed (prefill).
-static aded_status forward(aded_model* m, aded_kv* kv, const int32_t* tokens, const int32_t* parents,
-                           const int32_t* offsets_host, int batch, int chain_mode, int32_t* out_tokens,
-                           int out_stride, int32_t* out_len, cudaStream_t st) {
+// Kernels one pass launches (what enqueue_pass enqueues), for the launch counter of graph replays.
+static int pass_launches(const aded_model* m, int rows, int chain_mode) {
+    const int gemm_passes = (rows + 127) / 128;   // the tensor-core GEMM runs once per 128 rows
+    const int per_gemm = m->ws_ready ? gemm_passes : 1;
+    int n = 4 + m->cfg.n_layers * (4 * per_gemm + 3 + (m->att_o ? 2 : 1));
+    n += chain_mode ? 1 : per_gemm + 5;
+    return n;
+}
+
+// The launch sequence of one pass over `rows` rows.  Everything it touches is owned by the handles
+// (the caller's arrays are reached through m->call_dev), so the sequence can be captured once per
+// call shape and replayed.  chain_mode: the rows form a chain per sequence, every row is accepted
+// and no logits are needed (prefill).
+static aded_status enqueue_pass(aded_model* m, aded_kv* kv, const int32_t* offsets_src, int batch, int rows,
+                                int max_tree, int chain_mode, cudaStream_t st) {
     const aded_model_config& c = m->cfg;
-    const int rows = offsets_host[batch];
     const int d = c.d_model, F = c.d_ffn;
     const int xm = 4 * c.n_layers + 1;   // TMA descriptor indices of x, attn, act
-    int max_tree = 1;
-    for (int b = 0; b < batch; ++b)
-        if (offsets_host[b + 1] - offsets_host[b] > max_tree) max_tree = offsets_host[b + 1] - offsets_host[b];
-    ADED_CUDA_TRY(cudaMemcpyAsync(m->seqs.row_off, offsets_host, (batch + 1) * sizeof(int32_t),
+    ADED_CUDA_TRY(cudaMemcpyAsync(m->seqs.row_off, offsets_src, (batch + 1) * sizeof(int32_t),
                                   cudaMemcpyHostToDevice, st));
     {
         Span sp(m, PROF_OTHER, 4, st);
-        launch_tree_prologue(m, kv, tokens, parents, batch, chain_mode, st);
-        launch_embed(m, tokens, rows, st);
+        launch_tree_prologue(m, kv, batch, chain_mode, st);
+        launch_embed(m, rows, st);
         launch_rope_table(m, rows, st);
         launch_add_rmsnorm(m, (const GemmOut*)nullptr, m->layers[0].norm1, rows, st);
     }
@@ -158,7 +181,7 @@ static aded_status forward(aded_model* m, aded_kv* kv, const int32_t* tokens, co
         GemmOut o;
         { Span sp(m, PROF_GEMM, 1, st); o = launch_gemm(m, 4 * l + WS_MAP_QKV, xm, m->x, w.wqkv, m->y32, rows, 3 * d, d, st); }
         { Span sp(m, PROF_OTHER, 1, st); launch_rope_kv(m, kv, o, l, rows, st); }
-        { Span sp(m, PROF_ATTN, 1, st); launch_tree_attention(m, kv, l, batch, rows, max_tree, st); }
+        { Span sp(m, PROF_ATTN, 2, st); launch_tree_attention(m, kv, l, batch, rows, max_tree, st); }
         { Span sp(m, PROF_GEMM, 1, st); o = launch_gemm(m, 4 * l + WS_MAP_O, xm + 1, m->attn, w.wo, m->y32, rows, d, d, st); }
         { Span sp(m, PROF_OTHER, 1, st); launch_add_rmsnorm(m, &o, w.norm2, rows, st); }
         { Span sp(m, PROF_GEMM, 1, st); o = launch_gemm(m, 4 * l + WS_MAP_GU, xm, m->x, w.wgu, m->y32, rows, 2 * F, d, st); }
@@ -170,15 +193,13 @@ static aded_status forward(aded_model* m, aded_kv* kv, const int32_t* tokens, co
     if (!chain_mode) {
         GemmOut lg;
         { Span sp(m, PROF_GEMM, 1, st); lg = launch_gemm(m, 4 * c.n_layers, xm, m->x, m->top.lm_head, m->logits, rows, c.vocab, d, st); }
-        Span sp(m, PROF_OTHER, 2, st);
+        Span sp(m, PROF_OTHER, 3, st);
         launch_argmax(m, lg, rows, st);
         if (m->dbg_logits) launch_materialize(m, lg, m->dbg_logits, rows, st);
         if (m->dbg_best)
             ADED_CUDA_TRY(cudaMemcpyAsync(m->dbg_best, m->best, (size_t)rows * sizeof(int32_t),
                                           cudaMemcpyDeviceToDevice, st));
-        m->dbg_logits = nullptr;
-        m->dbg_best = nullptr;
-        launch_accept(m, kv, tokens, parents, batch, out_tokens, out_stride, out_len, st);
+        launch_accept(m, kv, batch, st);
     }
     {
         Span sp(m, PROF_OTHER, chain_mode ? 1 : 2, st);
@@ -188,9 +209,118 @@ static aded_status forward(aded_model* m, aded_kv* kv, const int32_t* tokens, co
     return ADED_OK;
 }
 
+// Adds the event times of the last replay of a profiling graph to the totals (synchronises).
+static void harvest_profile(aded_model* m, cudaStream_t st) {
+    if (m->prof_pending < 0) return;
+    cudaStreamSynchronize(st);
+    for (ProfSpan& sp : m->graphs[m->prof_pending].spans) {
+        float ms = 0.f;
+        if (cudaEventElapsedTime(&ms, sp.a, sp.b) == cudaSuccess) {
+            m->prof_ms[sp.group] += ms;
+            m->prof_n[sp.group] += sp.launches;
+        } else {
+            cudaGetLastError();
+        }
+    }
+    m->prof_pending = -1;
+}
+
+static void drop_graph(aded_model::GraphEntry& e) {
+    for (ProfSpan& sp : e.spans) { cudaEventDestroy(sp.a); cudaEventDestroy(sp.b); }
+    e.spans.clear();
+    if (e.exec) cudaGraphExecDestroy(e.exec);
+    if (e.offsets_pin) cudaFreeHost(e.offsets_pin);
+    e.exec = nullptr;
+    e.offsets_pin = nullptr;
+}
+
+// One verify / append call: publish the caller's array pointers, then run the pass -- replayed from a
+// CUDA graph captured per call shape (mode, cache handle, row offsets), launched directly while a
+// debug capture or the profiler is armed, or when graphs are switched off (ADED_NO_GRAPH).
+static aded_status forward(aded_model* m, aded_kv* kv, const int32_t* tokens, const int32_t* parents,
+                           const int32_t* offsets_host, int batch, int chain_mode, int32_t* out_tokens,
+                           int out_stride, int32_t* out_len, cudaStream_t st) {
+    const int rows = offsets_host[batch];
+    int max_tree = 1;
+    for (int b = 0; b < batch; ++b)
+        if (offsets_host[b + 1] - offsets_host[b] > max_tree) max_tree = offsets_host[b + 1] - offsets_host[b];
+    CallPtrs cp;
+    cp.tokens = tokens;
+    cp.parents = parents;
+    cp.out_tokens = out_tokens;
+    cp.out_len = out_len;
+    cp.out_stride = out_stride;
+    // pageable source: the runtime stages the bytes before returning, so the stack object may go
+    ADED_CUDA_TRY(cudaMemcpyAsync(m->call_dev, &cp, sizeof cp, cudaMemcpyHostToDevice, st));
+
+    cudaStreamCaptureStatus cap_state = cudaStreamCaptureStatusNone;
+    cudaStreamIsCapturing(st, &cap_state);
+    const bool direct = !m->graphs_on || m->dbg_logits || m->dbg_best || cap_state != cudaStreamCaptureStatusNone;
+    if (direct) {
+        aded_status s = enqueue_pass(m, kv, offsets_host, batch, rows, max_tree, chain_mode, st);
+        m->dbg_logits = nullptr;
+        m->dbg_best = nullptr;
+        return s;
+    }
+    std::vector<int64_t> key;
+    key.push_back(chain_mode + (m->prof_on ? 2 : 0));   // the profiling variant carries event nodes
+    key.push_back((int64_t)(uintptr_t)kv);
+    if (m->prof_on) harvest_profile(m, st);
+    for (int b = 0; b <= batch; ++b) key.push_back(offsets_host[b]);
+    aded_model::GraphEntry* hit = nullptr;
+    for (auto& e : m->graphs)
+        if (e.key == key) { hit = &e; break; }
+    if (!hit) {
+        if (m->graphs.size() >= 24) {          // forget the least recently used shape
+            size_t old = 0;
+            for (size_t i = 1; i < m->graphs.size(); ++i)
+                if (m->graphs[i].last_use < m->graphs[old].last_use) old = i;
+            harvest_profile(m, st);
+            drop_graph(m->graphs[old]);
+            m->graphs.erase(m->graphs.begin() + old);
+        }
+        aded_model::GraphEntry e;
+        e.key = key;
+        e.exec = nullptr;
+        e.offsets_pin = nullptr;
+        e.last_use = 0;
+        if (cudaMallocHost((void**)&e.offsets_pin, (batch + 1) * sizeof(int32_t)) != cudaSuccess) {
+            cudaGetLastError();
+            return enqueue_pass(m, kv, offsets_host, batch, rows, max_tree, chain_mode, st);
+        }
+        memcpy(e.offsets_pin, offsets_host, (batch + 1) * sizeof(int32_t));
+        cudaGraph_t graph = nullptr;
+        bool ok = cudaStreamBeginCapture(st, cudaStreamCaptureModeThreadLocal) == cudaSuccess;
+        if (ok) {
+            const uint64_t before = aded_launch_count();
+            m->capture_spans = &e.spans;
+            const aded_status s = enqueue_pass(m, kv, e.offsets_pin, batch, rows, max_tree, chain_mode, st);
+            m->capture_spans = nullptr;
+            note_launch(-(int)(aded_launch_count() - before));   // captured, not launched
+            ok = cudaStreamEndCapture(st, &graph) == cudaSuccess && s == ADED_OK && graph != nullptr;
+        }
+        if (ok) ok = cudaGraphInstantiate(&e.exec, graph, 0) == cudaSuccess;
+        if (graph) cudaGraphDestroy(graph);
+        if (!ok) {
+            cudaGetLastError();
+            drop_graph(e);
+            return enqueue_pass(m, kv, offsets_host, batch, rows, max_tree, chain_mode, st);
+        }
+        m->graphs.push_back(e);
+        hit = &m->graphs.back();
+    }
+    hit->last_use = ++m->graph_clock;
+    ADED_CUDA_TRY(cudaGraphLaunch(hit->exec, st));
+    if (m->prof_on) m->prof_pending = (int)(hit - m->graphs.data());
+    note_launch(pass_launches(m, rows, chain_mode));
+    return ADED_OK;
+}
+
 }  // namespace aded
 
 using namespace aded;
+
+extern "C" uint64_t aded_launch_count(void);
 
 extern "C" {
 
@@ -219,6 +349,11 @@ aded_status aded_model_create(const aded_model_config* cfg, const aded_weights* 
     m->dbg_logits = nullptr;
     m->dbg_best = nullptr;
     m->prof_on = false;
+    m->capture_spans = nullptr;
+    m->prof_pending = -1;
+    m->graphs_on = getenv("ADED_NO_GRAPH") == nullptr;
+    m->graph_clock = 0;
+    m->call_dev = nullptr;
     m->ws_ready = false;
     m->ws_slots = nullptr;
     if (cudaGetDevice(&m->device) != cudaSuccess) {
@@ -237,6 +372,7 @@ aded_status aded_model_create(const aded_model_config* cfg, const aded_weights* 
 aded_status aded_model_destroy(aded_model* m) {
     if (!m) return ADED_ERR_INVALID_ARG;
     for (void* p : m->owned) cudaFree(p);
+    for (auto& e : m->graphs) drop_graph(e);
     for (ProfSpan& sp : m->prof_spans) { cudaEventDestroy(sp.a); cudaEventDestroy(sp.b); }
     for (cudaEvent_t e : m->prof_pool) cudaEventDestroy(e);
     delete m;
@@ -447,24 +583,28 @@ aded_status aded_profile_begin(aded_model* m) {
     if (!m) return ADED_ERR_INVALID_ARG;
     for (ProfSpan& sp : m->prof_spans) { m->prof_pool.push_back(sp.a); m->prof_pool.push_back(sp.b); }
     m->prof_spans.clear();
+    m->prof_pending = -1;
+    for (int g = 0; g < PROF_GROUPS; ++g) { m->prof_ms[g] = 0.f; m->prof_n[g] = 0; }
     m->prof_on = true;
     return ADED_OK;
 }
 
 aded_status aded_profile_end(aded_model* m, float* out_ms_host, int32_t* out_launches_host, void* stream) {
     if (!m || !out_ms_host || !out_launches_host) return ADED_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
     m->prof_on = false;
-    ADED_CUDA_TRY(cudaStreamSynchronize(static_cast<cudaStream_t>(stream)));
-    for (int g = 0; g < PROF_GROUPS; ++g) { out_ms_host[g] = 0.f; out_launches_host[g] = 0; }
+    harvest_profile(m, st);
+    ADED_CUDA_TRY(cudaStreamSynchronize(st));
     for (ProfSpan& sp : m->prof_spans) {
         float ms = 0.f;
         ADED_CUDA_TRY(cudaEventElapsedTime(&ms, sp.a, sp.b));
-        out_ms_host[sp.group] += ms;
-        out_launches_host[sp.group] += sp.launches;
+        m->prof_ms[sp.group] += ms;
+        m->prof_n[sp.group] += sp.launches;
         m->prof_pool.push_back(sp.a);
         m->prof_pool.push_back(sp.b);
     }
     m->prof_spans.clear();
+    for (int g = 0; g < PROF_GROUPS; ++g) { out_ms_host[g] = m->prof_ms[g]; out_launches_host[g] = m->prof_n[g]; }
     return ADED_OK;
 }
 

@@ -8,10 +8,12 @@ namespace aded {
 // other node points at an earlier node, that tokens are in the vocabulary and that the cache has
 // room; then each thread climbs from its node to the root, collecting the ancestor bit set and
 // the depth.  The climb is bounded by the node count (parents decrease strictly).
-__global__ void k_tree_prologue(const int32_t* __restrict__ tokens, const int32_t* __restrict__ parents,
+__global__ void k_tree_prologue(const CallPtrs* __restrict__ call,
                                 const int32_t* __restrict__ row_off, const int32_t* __restrict__ len,
                                 const int32_t* __restrict__ cap, int vocab, int chain_mode,
                                 RowMeta rows, int32_t* status) {
+    const int32_t* __restrict__ tokens = call->tokens;
+    const int32_t* __restrict__ parents = call->parents;
     const int b = blockIdx.x;
     const int off = row_off[b];
     const int T = row_off[b + 1] - off;
@@ -57,12 +59,16 @@ __global__ void k_tree_prologue(const int32_t* __restrict__ tokens, const int32_
 // its parent is approved and its token equals the model's greedy token at the parent; the deepest
 // approved node (lowest index among equals) ends the accepted path.  Emits the greedy token of
 // every path node: the approved drafts' successors, ending with the model's own next token.
-__global__ void k_accept(const int32_t* __restrict__ tokens, const int32_t* __restrict__ parents,
+__global__ void k_accept(const CallPtrs* __restrict__ call,
                          const int32_t* __restrict__ row_off, const int32_t* __restrict__ best,
                          const int32_t* __restrict__ depth, const int32_t* __restrict__ len,
                          int32_t* __restrict__ path, int32_t* __restrict__ new_len,
-                         int32_t* __restrict__ out_tokens, int out_stride, int32_t* __restrict__ out_len,
                          const int32_t* status, int batch) {
+    const int32_t* __restrict__ tokens = call->tokens;
+    const int32_t* __restrict__ parents = call->parents;
+    int32_t* __restrict__ out_tokens = call->out_tokens;
+    int32_t* __restrict__ out_len = call->out_len;
+    const int out_stride = call->out_stride;
     const int b = blockIdx.x * blockDim.x + threadIdx.x;
     if (b >= batch) return;
     if (*status != 0) {
@@ -123,17 +129,14 @@ __global__ void k_commit(int32_t* len, const int32_t* __restrict__ new_len, cons
     len[b] = chain_mode ? len[b] + (row_off[b + 1] - row_off[b]) : new_len[b];
 }
 
-void launch_tree_prologue(aded_model* m, aded_kv* kv, const int32_t* tokens, const int32_t* parents,
-                          int batch, int chain_mode, cudaStream_t st) {
-    k_tree_prologue<<<batch, ADED_MAX_NODES, 0, st>>>(tokens, parents, m->seqs.row_off, kv->len_dev, kv->cap_dev,
+void launch_tree_prologue(aded_model* m, aded_kv* kv, int batch, int chain_mode, cudaStream_t st) {
+    k_tree_prologue<<<batch, ADED_MAX_NODES, 0, st>>>(m->call_dev, m->seqs.row_off, kv->len_dev, kv->cap_dev,
                                                       m->cfg.vocab, chain_mode, m->rows, m->status);
 }
 
-void launch_accept(aded_model* m, aded_kv* kv, const int32_t* tokens, const int32_t* parents, int batch,
-                   int32_t* out_tokens, int out_stride, int32_t* out_len, cudaStream_t st) {
-    k_accept<<<(batch + 31) / 32, 32, 0, st>>>(tokens, parents, m->seqs.row_off, m->best, m->rows.depth,
-                                               kv->len_dev, m->seqs.path, m->seqs.new_len, out_tokens,
-                                               out_stride, out_len, m->status, batch);
+void launch_accept(aded_model* m, aded_kv* kv, int batch, cudaStream_t st) {
+    k_accept<<<(batch + 31) / 32, 32, 0, st>>>(m->call_dev, m->seqs.row_off, m->best, m->rows.depth,
+                                               kv->len_dev, m->seqs.path, m->seqs.new_len, m->status, batch);
 }
 
 void launch_compact_commit(aded_model* m, aded_kv* kv, int batch, int chain_mode, cudaStream_t st) {

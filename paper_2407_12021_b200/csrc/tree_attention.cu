@@ -352,16 +352,20 @@ static void launch_mma(aded_model* m, aded_kv* kv, int layer, int batch, int row
     a.status = m->status;
     dim3 grid(m->cfg.n_heads, splits, batch);
     const size_t smem = (size_t)4 * TA_BLK * HD * sizeof(bf16);
-    static bool attr_done = false;
-    if (!attr_done) {
-        cudaFuncSetAttribute(k_tree_attn_mma<HD, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        cudaFuncSetAttribute(k_tree_attn_mma<HD, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        attr_done = true;
-    }
     if (max_tree <= 64) k_tree_attn_mma<HD, 4><<<grid, 128, smem, st>>>(a);
     else k_tree_attn_mma<HD, 8><<<grid, 256, smem, st>>>(a);
     dim3 mgrid(rows, m->cfg.n_heads);
     k_tree_attn_merge<HD><<<mgrid, HD, 0, st>>>(m->att_o, m->att_ml, (bf16*)m->attn, splits, rows, m->cfg.n_heads, m->status);
+}
+
+// Raises the split-KV kernels' dynamic shared-memory limit; once per process, before any launch.
+bool attn_prepare() {
+    bool ok = true;
+    ok &= cudaFuncSetAttribute(k_tree_attn_mma<128, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, 4 * TA_BLK * 128 * 2) == cudaSuccess;
+    ok &= cudaFuncSetAttribute(k_tree_attn_mma<128, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, 4 * TA_BLK * 128 * 2) == cudaSuccess;
+    ok &= cudaFuncSetAttribute(k_tree_attn_mma<64, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, 4 * TA_BLK * 64 * 2) == cudaSuccess;
+    ok &= cudaFuncSetAttribute(k_tree_attn_mma<64, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, 4 * TA_BLK * 64 * 2) == cudaSuccess;
+    return ok;
 }
 
 void launch_tree_attention(aded_model* m, aded_kv* kv, int layer, int batch, int rows, int max_tree, cudaStream_t st) {
