@@ -38,6 +38,34 @@ template <typename T> __device__ __forceinline__ T from_f32(float v);
 template <> __device__ __forceinline__ float from_f32<float>(float v) { return v; }
 template <> __device__ __forceinline__ bf16 from_f32<bf16>(float v) { return __float2bfloat16_rn(v); }
 
+// ---- programmatic dependent launch ---------------------------------------------------------
+// Every kernel of a pass is launched with the programmatic-serialisation attribute and begins with
+// pdl_enter(): it lets the next kernel of the stream start launching at once (its blocks become
+// resident and run their own preamble) and then waits until the previous kernel has finished and
+// its writes are visible.  Nothing may be read from or written to global memory that another kernel
+// of the pass touches before pdl_wait() -- the weight-streaming GEMM alone does work before it: it
+// prefetches weights, which no kernel writes.
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_enter() { pdl_launch_dependents(); pdl_wait(); }
+
+bool pdl_enabled();
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_k(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = pdl_enabled() ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+
 // ---- per-call row bookkeeping (device arrays sized for max_rows / max_batch) --------------
 struct RowMeta {
     int32_t* seq;      // [R] sequence of the row

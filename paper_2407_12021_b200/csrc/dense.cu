@@ -29,6 +29,7 @@ __device__ __forceinline__ float block_sum(float v, float* red) {
 template <typename T>
 __global__ void k_embed(const T* __restrict__ table, const CallPtrs* __restrict__ call, T* __restrict__ h,
                         int d, const int32_t* status) {
+    pdl_enter();
     if (*status != 0) return;
     const int32_t* __restrict__ tokens = call->tokens;
     const int r = blockIdx.x;
@@ -40,6 +41,7 @@ __global__ void k_embed(const T* __restrict__ table, const CallPtrs* __restrict_
 // thousands of radians, where float argument reduction would cost several bf16 ulps.
 __global__ void k_rope_table(const int32_t* __restrict__ pos, float* __restrict__ cs, float* __restrict__ sn,
                              int half, double theta, const int32_t* status) {
+    pdl_enter();
     if (*status != 0) return;
     const int r = blockIdx.x;
     for (int i = threadIdx.x; i < half; i += blockDim.x) {
@@ -60,6 +62,7 @@ template <typename T>
 __global__ void __launch_bounds__(256) k_add_rmsnorm(T* __restrict__ h, GemmOut y, int has_y, const T* __restrict__ gain,
                                                      T* __restrict__ x, int d, float eps, float* __restrict__ ssq,
                                                      int32_t* __restrict__ row_count, const int32_t* status) {
+    pdl_enter();
     if (*status != 0) return;
     __shared__ float red[32];
     __shared__ int s_last;
@@ -115,6 +118,7 @@ template <typename T>
 __global__ void __launch_bounds__(256) k_gemm_plain(const T* __restrict__ x, const T* __restrict__ w,
                                                     float* __restrict__ y, int rows, int n, int k,
                                                     const int32_t* status) {
+    pdl_enter();
     if (*status != 0) return;
     __shared__ float sx[16][64 + 4];
     __shared__ float sw[16][64 + 4];
@@ -157,6 +161,7 @@ __global__ void k_rope_kv(GemmOut qkv, const float* __restrict__ cs, const float
                           T* __restrict__ q, char* const* __restrict__ base, const int32_t* __restrict__ cap,
                           const int32_t* __restrict__ len, const int32_t* __restrict__ row_seq,
                           const int32_t* __restrict__ row_local, int layer, int H, int hd, const int32_t* status) {
+    pdl_enter();
     if (*status != 0) return;
     const int r = blockIdx.x, hh = blockIdx.y, half = hd >> 1, d = H * hd;
     const int b = row_seq[r];
@@ -187,6 +192,7 @@ __global__ void k_rope_kv(GemmOut qkv, const float* __restrict__ cs, const float
 // act = round(silu(gate) * up), gate = gu[:, :F], up = gu[:, F:].
 template <typename T>
 __global__ void k_swiglu(GemmOut gu, T* __restrict__ act, int F, const int32_t* status) {
+    pdl_enter();
     if (*status != 0) return;
     const int r = blockIdx.y;
     const int c = blockIdx.x * blockDim.x + threadIdx.x;
@@ -200,6 +206,7 @@ __global__ void k_swiglu(GemmOut gu, T* __restrict__ act, int F, const int32_t* 
 // thread per row) takes the best of the chunks in ascending column order.
 __global__ void __launch_bounds__(256) k_argmax_chunks(GemmOut logits, float* __restrict__ pv, int32_t* __restrict__ pi,
                                                        int V, int chunk, const int32_t* status) {
+    pdl_enter();
     if (*status != 0) return;
     __shared__ float sv[8];
     __shared__ int si[8];
@@ -229,6 +236,7 @@ __global__ void __launch_bounds__(256) k_argmax_chunks(GemmOut logits, float* __
 
 __global__ void k_argmax_final(const float* __restrict__ pv, const int32_t* __restrict__ pi, int32_t* __restrict__ best,
                                int chunks, int rows, const int32_t* status) {
+    pdl_enter();
     if (*status != 0) return;
     const int r = blockIdx.x * blockDim.x + threadIdx.x;
     if (r >= rows) return;
@@ -243,6 +251,7 @@ __global__ void k_argmax_final(const float* __restrict__ pv, const int32_t* __re
 }
 
 __global__ void k_materialize(GemmOut src, float* __restrict__ dst, int n, const int32_t* status) {
+    pdl_enter();
     if (*status != 0) return;
     const int r = blockIdx.y;
     const int c = blockIdx.x * blockDim.x + threadIdx.x;
@@ -255,12 +264,12 @@ __global__ void k_materialize(GemmOut src, float* __restrict__ dst, int n, const
 
 void launch_embed(aded_model* m, int rows, cudaStream_t st) {
     const int d = m->cfg.d_model;
-    BY_DTYPE(m, (k_embed<bf16><<<rows, 256, 0, st>>>((const bf16*)m->top.embed, m->call_dev, (bf16*)m->h, d, m->status)),
-             (k_embed<float><<<rows, 256, 0, st>>>((const float*)m->top.embed, m->call_dev, (float*)m->h, d, m->status)));
+    BY_DTYPE(m, (launch_k(k_embed<bf16>, rows, 256, 0, st, (const bf16*)m->top.embed, m->call_dev, (bf16*)m->h, d, m->status)),
+             (launch_k(k_embed<float>, rows, 256, 0, st, (const float*)m->top.embed, m->call_dev, (float*)m->h, d, m->status)));
 }
 
 void launch_rope_table(aded_model* m, int rows, cudaStream_t st) {
-    k_rope_table<<<rows, 64, 0, st>>>(m->rows.pos, m->rope_cos, m->rope_sin, m->cfg.head_dim / 2,
+    launch_k(k_rope_table, rows, 64, 0, st, m->rows.pos, m->rope_cos, m->rope_sin, m->cfg.head_dim / 2,
                                       (double)m->cfg.rope_theta, m->status);
 }
 
@@ -270,14 +279,14 @@ void launch_add_rmsnorm(aded_model* m, const GemmOut* y, const void* gain, int r
     const GemmOut& yy = y ? *y : none;
     const int has = y != nullptr;
     dim3 grid((d + 255) / 256, rows);
-    BY_DTYPE(m, (k_add_rmsnorm<bf16><<<grid, 256, 0, st>>>((bf16*)m->h, yy, has, (const bf16*)gain, (bf16*)m->x, d, m->cfg.rms_eps, m->norm_ssq, m->norm_count, m->status)),
-             (k_add_rmsnorm<float><<<grid, 256, 0, st>>>((float*)m->h, yy, has, (const float*)gain, (float*)m->x, d, m->cfg.rms_eps, m->norm_ssq, m->norm_count, m->status)));
+    BY_DTYPE(m, (launch_k(k_add_rmsnorm<bf16>, grid, 256, 0, st, (bf16*)m->h, yy, has, (const bf16*)gain, (bf16*)m->x, d, m->cfg.rms_eps, m->norm_ssq, m->norm_count, m->status)),
+             (launch_k(k_add_rmsnorm<float>, grid, 256, 0, st, (float*)m->h, yy, has, (const float*)gain, (float*)m->x, d, m->cfg.rms_eps, m->norm_ssq, m->norm_count, m->status)));
 }
 
 static void launch_gemm_plain(aded_model* m, const void* x, const void* w, float* y, int rows, int n, int k, cudaStream_t st) {
     dim3 grid((n + 63) / 64, (rows + 63) / 64);
-    BY_DTYPE(m, (k_gemm_plain<bf16><<<grid, 256, 0, st>>>((const bf16*)x, (const bf16*)w, y, rows, n, k, m->status)),
-             (k_gemm_plain<float><<<grid, 256, 0, st>>>((const float*)x, (const float*)w, y, rows, n, k, m->status)));
+    BY_DTYPE(m, (launch_k(k_gemm_plain<bf16>, grid, 256, 0, st, (const bf16*)x, (const bf16*)w, y, rows, n, k, m->status)),
+             (launch_k(k_gemm_plain<float>, grid, 256, 0, st, (const float*)x, (const float*)w, y, rows, n, k, m->status)));
 }
 
 GemmOut launch_gemm(aded_model* m, int w_map, int x_map, const void* x, const void* w, float* y, int rows, int n, int k,
@@ -307,21 +316,21 @@ GemmOut launch_gemm(aded_model* m, int w_map, int x_map, const void* x, const vo
 
 void launch_materialize(aded_model* m, const GemmOut& src, float* dst, int rows, cudaStream_t st) {
     dim3 grid((src.n + 255) / 256, rows);
-    k_materialize<<<grid, 256, 0, st>>>(src, dst, src.n, m->status);
+    launch_k(k_materialize, grid, 256, 0, st, src, dst, src.n, m->status);
 }
 
 void launch_rope_kv(aded_model* m, aded_kv* kv, const GemmOut& qkv, int layer, int rows, cudaStream_t st) {
     dim3 grid(rows, m->cfg.n_heads);
     const int H = m->cfg.n_heads, hd = m->cfg.head_dim;
-    BY_DTYPE(m, (k_rope_kv<bf16><<<grid, 64, 0, st>>>(qkv, m->rope_cos, m->rope_sin, (bf16*)m->q, kv->base_dev, kv->cap_dev, kv->len_dev, m->rows.seq, m->rows.local, layer, H, hd, m->status)),
-             (k_rope_kv<float><<<grid, 64, 0, st>>>(qkv, m->rope_cos, m->rope_sin, (float*)m->q, kv->base_dev, kv->cap_dev, kv->len_dev, m->rows.seq, m->rows.local, layer, H, hd, m->status)));
+    BY_DTYPE(m, (launch_k(k_rope_kv<bf16>, grid, 64, 0, st, qkv, m->rope_cos, m->rope_sin, (bf16*)m->q, kv->base_dev, kv->cap_dev, kv->len_dev, m->rows.seq, m->rows.local, layer, H, hd, m->status)),
+             (launch_k(k_rope_kv<float>, grid, 64, 0, st, qkv, m->rope_cos, m->rope_sin, (float*)m->q, kv->base_dev, kv->cap_dev, kv->len_dev, m->rows.seq, m->rows.local, layer, H, hd, m->status)));
 }
 
 void launch_swiglu(aded_model* m, const GemmOut& gu, int rows, cudaStream_t st) {
     const int F = m->cfg.d_ffn;
     dim3 grid((F + 255) / 256, rows);
-    BY_DTYPE(m, (k_swiglu<bf16><<<grid, 256, 0, st>>>(gu, (bf16*)m->act, F, m->status)),
-             (k_swiglu<float><<<grid, 256, 0, st>>>(gu, (float*)m->act, F, m->status)));
+    BY_DTYPE(m, (launch_k(k_swiglu<bf16>, grid, 256, 0, st, gu, (bf16*)m->act, F, m->status)),
+             (launch_k(k_swiglu<float>, grid, 256, 0, st, gu, (float*)m->act, F, m->status)));
 }
 
 void launch_argmax(aded_model* m, const GemmOut& logits, int rows, cudaStream_t st) {
@@ -329,8 +338,8 @@ void launch_argmax(aded_model* m, const GemmOut& logits, int rows, cudaStream_t 
     const int chunks = ARGMAX_CHUNKS;
     const int chunk = ((V + chunks - 1) / chunks + 127) / 128 * 128;   // whole 128-column tiles per block
     dim3 grid(chunks, rows);
-    k_argmax_chunks<<<grid, 256, 0, st>>>(logits, m->argmax_val, m->argmax_idx, V, chunk, m->status);
-    k_argmax_final<<<(rows + 127) / 128, 128, 0, st>>>(m->argmax_val, m->argmax_idx, m->best, chunks, rows, m->status);
+    launch_k(k_argmax_chunks, grid, 256, 0, st, logits, m->argmax_val, m->argmax_idx, V, chunk, m->status);
+    launch_k(k_argmax_final, (rows + 127) / 128, 128, 0, st, m->argmax_val, m->argmax_idx, m->best, chunks, rows, m->status);
 }
 
 }  // namespace aded

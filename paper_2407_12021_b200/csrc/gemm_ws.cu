@@ -14,6 +14,9 @@
 //   * a CTA stores the fp32 partial tile of each of its segments to a slot; the kernel that consumes
 //     the result adds a tile's slots in CTA order -- a fixed order, so results do not depend on
 //     timing, and the GEMM itself ends without counters, fences or dependent reads;
+//   * the kernel is launched with programmatic dependent launch: its blocks become resident while
+//     the previous kernel drains, set up barriers and TMEM, and already stream their first W tiles;
+//     only the loads of x wait for the previous kernel;
 //   * warp 0 issues TMA loads, warp 1 issues MMAs, warps 2..5 drain TMEM and run the epilogue; two
 //     TMEM accumulators let the MMAs of the next segment run under the epilogue of the last.
 // Every mbarrier wait is bounded; a wait that runs out raises ADED_ERR_TIMEOUT in the status word
@@ -132,6 +135,7 @@ k_gemm_ws(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUt
     uint32_t* s_tmem = (uint32_t*)(acc_empty + 2);
     volatile int* s_flag = (volatile int*)(s_tmem + 1);   // [0] abort, [2] live
 
+    pdl_launch_dependents();   // the next kernel may start its preamble; it waits for this one's results itself
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const long long units = (long long)p.n_tiles * p.kb;
     const long long G = gridDim.x;
@@ -163,9 +167,25 @@ k_gemm_ws(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUt
             asm volatile("prefetch.tensormap [%0];" ::"l"(&map_x) : "memory");
             uint64_t pol_stream;
             asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol_stream));
-            int s = 0;
-            uint32_t ph = 0;
-            for (long long u = u0; u < u1 && !s_flag[0]; ++u) {
+            // Weights do not depend on the previous kernel: fill the pipeline with W tiles first, then
+            // wait for the previous kernel (which produces x) and add the x tiles of those stages.
+            const long long n_units = u1 - u0;
+            const int ahead = (int)(n_units < p.stages ? n_units : p.stages);
+            for (int i = 0; i < ahead; ++i) {
+                const long long u = u0 + i;
+                const int tile = (int)(u / p.kb), kb = (int)(u % p.kb);
+                mbar_expect_tx(&full[i], stage_bytes);
+                tma_load_2d_hint(&map_w, &full[i], base + (size_t)i * stage_bytes, kb * WS_BK, tile * WS_BM, pol_stream);
+            }
+            pdl_wait();
+            for (int i = 0; i < ahead; ++i) {
+                const int kb = (int)((u0 + i) % p.kb);
+                uint8_t* sb = base + (size_t)i * stage_bytes + a_bytes;
+                for (int r = 0; r < p.rb; r += 16) tma_load_2d(&map_x, &full[i], sb + r * 128, kb * WS_BK, p.row0 + r);
+            }
+            int s = ahead == p.stages ? 0 : ahead;
+            uint32_t ph = ahead == p.stages ? 1 : 0;
+            for (long long u = u0 + ahead; u < u1 && !s_flag[0]; ++u) {
                 const int tile = (int)(u / p.kb), kb = (int)(u % p.kb);
                 if (!mbar_wait(&empty[s], ph ^ 1)) { s_flag[0] = 1; atomicCAS(p.status, 0, (int)ADED_ERR_TIMEOUT); break; }
                 uint8_t* sa = base + (size_t)s * stage_bytes;
@@ -341,8 +361,7 @@ cudaError_t ws_launch(const CUtensorMap& map_w, const CUtensorMap& map_x, int ro
     p.slots = slots + (size_t)(row0 / 128) * (size_t)(p.n_tiles + grid) * 128 * WS_BM;
     p.status = status;
     const size_t smem = (size_t)p.stages * stage_bytes + 1024 + 256;
-    k_gemm_ws<<<grid, WS_THREADS, smem, st>>>(map_w, map_x, p);
-    return cudaGetLastError();
+    return launch_k(k_gemm_ws, dim3(grid), dim3(WS_THREADS), smem, st, map_w, map_x, p);
 }
 
 }  // namespace aded

@@ -18,6 +18,11 @@ void note_cuda_error(cudaError_t e, const char* what) {
     cudaGetLastError();
 }
 
+bool pdl_enabled() {
+    static const bool on = getenv("ADED_NO_PDL") == nullptr;
+    return on;
+}
+
 static std::atomic<uint64_t> g_launches{0};
 void note_launch(int n) { g_launches.fetch_add((uint64_t)n, std::memory_order_relaxed); }
 

@@ -12,6 +12,7 @@ __global__ void k_tree_prologue(const CallPtrs* __restrict__ call,
                                 const int32_t* __restrict__ row_off, const int32_t* __restrict__ len,
                                 const int32_t* __restrict__ cap, int vocab, int chain_mode,
                                 RowMeta rows, int32_t* status) {
+    pdl_enter();
     const int32_t* __restrict__ tokens = call->tokens;
     const int32_t* __restrict__ parents = call->parents;
     const int b = blockIdx.x;
@@ -64,6 +65,7 @@ __global__ void k_accept(const CallPtrs* __restrict__ call,
                          const int32_t* __restrict__ depth, const int32_t* __restrict__ len,
                          int32_t* __restrict__ path, int32_t* __restrict__ new_len,
                          const int32_t* status, int batch) {
+    pdl_enter();
     const int32_t* __restrict__ tokens = call->tokens;
     const int32_t* __restrict__ parents = call->parents;
     int32_t* __restrict__ out_tokens = call->out_tokens;
@@ -108,6 +110,7 @@ template <typename T>
 __global__ void k_compact(char* const* __restrict__ base, const int32_t* __restrict__ cap,
                           const int32_t* __restrict__ len, const int32_t* __restrict__ new_len,
                           const int32_t* __restrict__ path, int hd, const int32_t* status) {
+    pdl_enter();
     if (*status != 0) return;
     const int b = blockIdx.y;
     const int n_acc = new_len[b] - len[b];
@@ -124,18 +127,19 @@ __global__ void k_compact(char* const* __restrict__ base, const int32_t* __restr
 
 __global__ void k_commit(int32_t* len, const int32_t* __restrict__ new_len, const int32_t* __restrict__ row_off,
                          int chain_mode, const int32_t* status, int batch) {
+    pdl_enter();
     const int b = blockIdx.x * blockDim.x + threadIdx.x;
     if (b >= batch || *status != 0) return;
     len[b] = chain_mode ? len[b] + (row_off[b + 1] - row_off[b]) : new_len[b];
 }
 
 void launch_tree_prologue(aded_model* m, aded_kv* kv, int batch, int chain_mode, cudaStream_t st) {
-    k_tree_prologue<<<batch, ADED_MAX_NODES, 0, st>>>(m->call_dev, m->seqs.row_off, kv->len_dev, kv->cap_dev,
+    launch_k(k_tree_prologue, batch, ADED_MAX_NODES, 0, st, m->call_dev, m->seqs.row_off, kv->len_dev, kv->cap_dev,
                                                       m->cfg.vocab, chain_mode, m->rows, m->status);
 }
 
 void launch_accept(aded_model* m, aded_kv* kv, int batch, cudaStream_t st) {
-    k_accept<<<(batch + 31) / 32, 32, 0, st>>>(m->call_dev, m->seqs.row_off, m->best, m->rows.depth,
+    launch_k(k_accept, (batch + 31) / 32, 32, 0, st, m->call_dev, m->seqs.row_off, m->best, m->rows.depth,
                                                kv->len_dev, m->seqs.path, m->seqs.new_len, m->status, batch);
 }
 
@@ -143,13 +147,13 @@ void launch_compact_commit(aded_model* m, aded_kv* kv, int batch, int chain_mode
     if (!chain_mode) {
         dim3 grid(m->cfg.n_layers * 2 * m->cfg.n_heads, batch);
         if (m->cfg.dtype == ADED_BF16)
-            k_compact<bf16><<<grid, 128, 0, st>>>(kv->base_dev, kv->cap_dev, kv->len_dev, m->seqs.new_len,
+            launch_k(k_compact<bf16>, grid, 128, 0, st, kv->base_dev, kv->cap_dev, kv->len_dev, m->seqs.new_len,
                                                   m->seqs.path, m->cfg.head_dim, m->status);
         else
-            k_compact<float><<<grid, 128, 0, st>>>(kv->base_dev, kv->cap_dev, kv->len_dev, m->seqs.new_len,
+            launch_k(k_compact<float>, grid, 128, 0, st, kv->base_dev, kv->cap_dev, kv->len_dev, m->seqs.new_len,
                                                    m->seqs.path, m->cfg.head_dim, m->status);
     }
-    k_commit<<<(batch + 31) / 32, 32, 0, st>>>(kv->len_dev, m->seqs.new_len, m->seqs.row_off, chain_mode,
+    launch_k(k_commit, (batch + 31) / 32, 32, 0, st, kv->len_dev, m->seqs.new_len, m->seqs.row_off, chain_mode,
                                                m->status, batch);
 }
 

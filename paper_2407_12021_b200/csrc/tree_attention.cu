@@ -25,6 +25,7 @@ __global__ void __launch_bounds__(128) k_tree_attn_plain(
         const T* __restrict__ q, T* __restrict__ out, char* const* __restrict__ base,
         const int32_t* __restrict__ cap, const int32_t* __restrict__ len, const int32_t* __restrict__ row_seq,
         const uint64_t* __restrict__ anc, int layer, int H, int rows, float scale, const int32_t* status) {
+    pdl_enter();
     if (*status != 0) return;
     constexpr int PER = HD / 32;
     const int warp = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
@@ -126,6 +127,7 @@ struct AttnArgs {
 
 template <int HD, int NW>
 __global__ void __launch_bounds__(NW * 32) k_tree_attn_mma(AttnArgs a) {
+    pdl_enter();
     if (*a.status != 0) return;
     constexpr int KSTEPS = HD / 16;        // k steps of Q K^T
     constexpr int ONT = HD / 8;            // n tiles of the output
@@ -313,6 +315,7 @@ template <int HD>
 __global__ void __launch_bounds__(HD) k_tree_attn_merge(const float* __restrict__ part_o, const float* __restrict__ part_ml,
                                                        bf16* __restrict__ out, int n_splits, int rows, int H,
                                                        const int32_t* status) {
+    pdl_enter();
     if (*status != 0) return;
     const int r = blockIdx.x, hh = blockIdx.y, e = threadIdx.x;
     const size_t pstride = (size_t)rows * H, idx = (size_t)r * H + hh;
@@ -352,10 +355,10 @@ static void launch_mma(aded_model* m, aded_kv* kv, int layer, int batch, int row
     a.status = m->status;
     dim3 grid(m->cfg.n_heads, splits, batch);
     const size_t smem = (size_t)4 * TA_BLK * HD * sizeof(bf16);
-    if (max_tree <= 64) k_tree_attn_mma<HD, 4><<<grid, 128, smem, st>>>(a);
-    else k_tree_attn_mma<HD, 8><<<grid, 256, smem, st>>>(a);
+    if (max_tree <= 64) launch_k(k_tree_attn_mma<HD, 4>, grid, 128, smem, st, a);
+    else launch_k(k_tree_attn_mma<HD, 8>, grid, 256, smem, st, a);
     dim3 mgrid(rows, m->cfg.n_heads);
-    k_tree_attn_merge<HD><<<mgrid, HD, 0, st>>>(m->att_o, m->att_ml, (bf16*)m->attn, splits, rows, m->cfg.n_heads, m->status);
+    launch_k(k_tree_attn_merge<HD>, mgrid, HD, 0, st, m->att_o, m->att_ml, (bf16*)m->attn, splits, rows, m->cfg.n_heads, m->status);
 }
 
 // Raises the split-KV kernels' dynamic shared-memory limit; once per process, before any launch.
@@ -379,7 +382,7 @@ void launch_tree_attention(aded_model* m, aded_kv* kv, int layer, int batch, int
     const int warps = rows * H;
     const int blocks = (warps + 3) / 4;
 #define ATTN(T, HD)                                                                                          \
-    k_tree_attn_plain<T, HD><<<blocks, 128, 0, st>>>((const T*)m->q, (T*)m->attn, kv->base_dev, kv->cap_dev, \
+    launch_k(k_tree_attn_plain<T, HD>, blocks, 128, 0, st, (const T*)m->q, (T*)m->attn, kv->base_dev, kv->cap_dev, \
                                                      kv->len_dev, m->rows.seq, m->rows.anc, layer, H, rows,  \
                                                      scale, m->status)
     if (m->cfg.dtype == ADED_BF16) {
