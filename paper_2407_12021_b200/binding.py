@@ -103,7 +103,7 @@ class Model:
         self.handle, self._keep, self.cfg = handle, keep, cfg
 
     def __del__(self):
-        if getattr(self, "handle", None):
+        if getattr(self, "handle", None) and _lib is not None:
             _lib.aded_model_destroy(self.handle)
             self.handle = None
 
@@ -113,7 +113,7 @@ class KV:
         self.handle, self.model, self.batch = handle, model, batch
 
     def __del__(self):
-        if getattr(self, "handle", None):
+        if getattr(self, "handle", None) and _lib is not None:
             _lib.aded_kv_destroy(self.handle)
             self.handle = None
 
@@ -123,7 +123,7 @@ class Trigram:
         self.handle, self.cfg = handle, cfg
 
     def __del__(self):
-        if getattr(self, "handle", None):
+        if getattr(self, "handle", None) and _lib is not None:
             _lib.aded_trigram_destroy(self.handle)
             self.handle = None
 

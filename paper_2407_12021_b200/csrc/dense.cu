@@ -275,6 +275,7 @@ void launch_rope_table(aded_model* m, int rows, cudaStream_t st) {
 
 void launch_add_rmsnorm(aded_model* m, const GemmOut* y, const void* gain, int rows, cudaStream_t st) {
     const int d = m->cfg.d_model;
+    if (y && y->mode == 1 && m->cfg.dtype == ADED_BF16) { launch_add_rmsnorm_ws(m, *y, gain, rows, st); return; }
     GemmOut none = {};
     const GemmOut& yy = y ? *y : none;
     const int has = y != nullptr;
@@ -290,7 +291,7 @@ static void launch_gemm_plain(aded_model* m, const void* x, const void* w, float
 }
 
 GemmOut launch_gemm(aded_model* m, int w_map, int x_map, const void* x, const void* w, float* y, int rows, int n, int k,
-                    cudaStream_t st) {
+                    cudaStream_t st, int next_map, int next_n, int next_k) {
     GemmOut out = {};
     out.n = n;
     out.rows = rows;
@@ -298,7 +299,9 @@ GemmOut launch_gemm(aded_model* m, int w_map, int x_map, const void* x, const vo
         // tensor-core path, 128 rows of x per pass over the weights; the result stays in slots
         for (int row0 = 0; row0 < rows; row0 += 128) {
             const int part = rows - row0 < 128 ? rows - row0 : 128;
-            ws_launch(m->ws_maps[w_map], m->ws_maps[x_map], part, row0, n, k, m->ws_slots, m->status, m->device, st);
+            const bool last_pass = row0 + 128 >= rows;
+            ws_launch(m->ws_maps[w_map], m->ws_maps[x_map], part, row0, n, k, m->ws_slots, m->status, m->device, st,
+                      last_pass && next_map >= 0 ? &m->ws_maps[next_map] : nullptr, next_n, next_k);
         }
         out.mode = 1;
         out.slots = m->ws_slots;
@@ -320,6 +323,7 @@ void launch_materialize(aded_model* m, const GemmOut& src, float* dst, int rows,
 }
 
 void launch_rope_kv(aded_model* m, aded_kv* kv, const GemmOut& qkv, int layer, int rows, cudaStream_t st) {
+    if (qkv.mode == 1 && m->cfg.dtype == ADED_BF16) { launch_rope_kv_ws(m, kv, qkv, layer, rows, st); return; }
     dim3 grid(rows, m->cfg.n_heads);
     const int H = m->cfg.n_heads, hd = m->cfg.head_dim;
     BY_DTYPE(m, (launch_k(k_rope_kv<bf16>, grid, 64, 0, st, qkv, m->rope_cos, m->rope_sin, (bf16*)m->q, kv->base_dev, kv->cap_dev, kv->len_dev, m->rows.seq, m->rows.local, layer, H, hd, m->status)),
@@ -327,6 +331,7 @@ void launch_rope_kv(aded_model* m, aded_kv* kv, const GemmOut& qkv, int layer, i
 }
 
 void launch_swiglu(aded_model* m, const GemmOut& gu, int rows, cudaStream_t st) {
+    if (gu.mode == 1 && m->cfg.dtype == ADED_BF16) { launch_swiglu_ws(m, gu, rows, st); return; }
     const int F = m->cfg.d_ffn;
     dim3 grid((F + 255) / 256, rows);
     BY_DTYPE(m, (launch_k(k_swiglu<bf16>, grid, 256, 0, st, gu, (bf16*)m->act, F, m->status)),

@@ -1,0 +1,164 @@
+// bf16 consumers of the tensor-core GEMM's partial tiles, four columns per thread.
+//
+// Same arithmetic as the generic kernels in dense.cu (residual add + RMSNorm, rotary + K/V write,
+// SwiGLU), specialised for the case that matters for speed: the projection result lives in slots
+// (gemm_out.cuh) and the model is bf16.  Each thread gathers four adjacent columns of every
+// contributing slot with 16-byte loads that are all in flight at once, so a kernel is one or two
+// memory round trips deep instead of one per contributor.
+#include "aded_internal.cuh"
+
+namespace aded {
+
+__device__ __forceinline__ float4 f4_add(float4 a, float4 b) { return make_float4(a.x + b.x, a.y + b.y, a.z + b.z, a.w + b.w); }
+
+// Columns col .. col+3 (col % 4 == 0) of tile t, row r: slots added in CTA order.
+__device__ __forceinline__ float4 gemm_out_at4(const GemmOut& o, const TileRef& t, int r, int col) {
+    const int rb = gemm_block_rb(o, r);
+    const size_t region = (size_t)(r >> 7) * (size_t)(o.n_tiles + o.g) * 128 * 128;
+    const float* p = o.slots + region + ((size_t)t.first_slot * rb + (r & 127)) * 128 + col;
+    const size_t stride = (size_t)rb * 128;
+    float4 sum = make_float4(0.f, 0.f, 0.f, 0.f);
+    int i = 0;
+    for (; i + 4 <= t.count; i += 4) {     // four loads in flight, added in order
+        const float4 a = __ldcg(reinterpret_cast<const float4*>(p + (size_t)i * stride));
+        const float4 b = __ldcg(reinterpret_cast<const float4*>(p + (size_t)(i + 1) * stride));
+        const float4 c = __ldcg(reinterpret_cast<const float4*>(p + (size_t)(i + 2) * stride));
+        const float4 d = __ldcg(reinterpret_cast<const float4*>(p + (size_t)(i + 3) * stride));
+        sum = f4_add(f4_add(f4_add(f4_add(sum, a), b), c), d);
+    }
+    for (; i < t.count; ++i) sum = f4_add(sum, __ldcg(reinterpret_cast<const float4*>(p + (size_t)i * stride)));
+    return sum;
+}
+
+__device__ __forceinline__ uint2 pack4_bf16(float a, float b, float c, float d) {
+    const __nv_bfloat162 lo = __floats2bfloat162_rn(a, b), hi = __floats2bfloat162_rn(c, d);
+    uint2 u;
+    u.x = *reinterpret_cast<const uint32_t*>(&lo);
+    u.y = *reinterpret_cast<const uint32_t*>(&hi);
+    return u;
+}
+__device__ __forceinline__ float4 unpack4_bf16(uint2 u) {
+    const __nv_bfloat162 lo = *reinterpret_cast<const __nv_bfloat162*>(&u.x), hi = *reinterpret_cast<const __nv_bfloat162*>(&u.y);
+    return make_float4(__low2float(lo), __high2float(lo), __low2float(hi), __high2float(hi));
+}
+
+__device__ __forceinline__ float warp_sum_f(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+// Residual add + RMSNorm (see k_add_rmsnorm): grid (chunks of 1024 columns, rows), 256 threads,
+// four columns per thread; the chunk that finishes a row last normalises the whole row.
+__global__ void __launch_bounds__(256) k_add_rmsnorm_ws(bf16* __restrict__ h, GemmOut y, const bf16* __restrict__ gain,
+                                                        bf16* __restrict__ x, int d, float eps, float* __restrict__ ssq,
+                                                        int32_t* __restrict__ row_count, const int32_t* status) {
+    pdl_enter();
+    if (*status != 0) return;
+    __shared__ float red[8];
+    __shared__ int s_last;
+    const int r = blockIdx.y, c = (blockIdx.x * 256 + threadIdx.x) * 4;
+    float sq = 0.f;
+    if (c < d) {
+        uint2* hp = reinterpret_cast<uint2*>(h + (size_t)r * d + c);
+        const float4 hv = unpack4_bf16(*hp);
+        const float4 add = gemm_out_at4(y, y.tiles[c >> 7], r, c & 127);
+        const uint2 nv = pack4_bf16(hv.x + add.x, hv.y + add.y, hv.z + add.z, hv.w + add.w);
+        *hp = nv;
+        const float4 v = unpack4_bf16(nv);
+        sq = v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
+    }
+    sq = warp_sum_f(sq);
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = sq;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        float tot = 0.f;
+        for (int i = 0; i < 8; ++i) tot += red[i];
+        ssq[r * 32 + blockIdx.x] = tot;
+        __threadfence();
+        const int prev = atomicAdd(&row_count[r], 1);
+        s_last = prev == (int)gridDim.x - 1;
+        if (s_last) row_count[r] = 0;
+    }
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();
+    float total = 0.f;
+    for (int i = 0; i < (int)gridDim.x; ++i) total += __ldcg(ssq + r * 32 + i);
+    const float inv = rsqrtf(total / (float)d + eps);
+    const uint2* hr = reinterpret_cast<const uint2*>(h + (size_t)r * d);
+    const uint2* gr = reinterpret_cast<const uint2*>(gain);
+    uint2* xr = reinterpret_cast<uint2*>(x + (size_t)r * d);
+    for (int cc = threadIdx.x; cc < d / 4; cc += 256) {
+        const float4 hv = unpack4_bf16(__ldcg(hr + cc)), gv = unpack4_bf16(gr[cc]);
+        xr[cc] = pack4_bf16(hv.x * inv * gv.x, hv.y * inv * gv.y, hv.z * inv * gv.z, hv.w * inv * gv.w);
+    }
+}
+
+// act = round(silu(gate) * up): grid (chunks of 1024 columns, rows), four columns per thread.
+__global__ void __launch_bounds__(256) k_swiglu_ws(GemmOut gu, bf16* __restrict__ act, int F, const int32_t* status) {
+    pdl_enter();
+    if (*status != 0) return;
+    const int r = blockIdx.y, c = (blockIdx.x * 256 + threadIdx.x) * 4;
+    if (c >= F) return;
+    const float4 g = gemm_out_at4(gu, gu.tiles[c >> 7], r, c & 127);
+    const float4 u = gemm_out_at4(gu, gu.tiles[(F + c) >> 7], r, (F + c) & 127);
+    *reinterpret_cast<uint2*>(act + (size_t)r * F + c) =
+        pack4_bf16(g.x / (1.f + expf(-g.x)) * u.x, g.y / (1.f + expf(-g.y)) * u.y,
+                   g.z / (1.f + expf(-g.z)) * u.z, g.w / (1.f + expf(-g.w)) * u.w);
+}
+
+// Rotary embedding + K/V write (see k_rope_kv): block = (row, head), hd/8 threads, each owning four
+// adjacent rotary pairs (i .. i+3, i+half .. i+half+3).
+__global__ void k_rope_kv_ws(GemmOut qkv, const float* __restrict__ cs, const float* __restrict__ sn,
+                             bf16* __restrict__ q, char* const* __restrict__ base, const int32_t* __restrict__ cap,
+                             const int32_t* __restrict__ len, const int32_t* __restrict__ row_seq,
+                             const int32_t* __restrict__ row_local, int layer, int H, int hd, const int32_t* status) {
+    pdl_enter();
+    if (*status != 0) return;
+    const int r = blockIdx.x, hh = blockIdx.y, half = hd >> 1, d = H * hd;
+    const int i = threadIdx.x * 4;
+    if (i >= half) return;
+    const int b = row_seq[r];
+    const size_t slot = (size_t)len[b] + row_local[r];
+    const size_t cp = cap[b];
+    bf16* kdst = reinterpret_cast<bf16*>(base[b]) + ((((size_t)layer * 2 + 0) * H + hh) * cp + slot) * hd;
+    bf16* vdst = reinterpret_cast<bf16*>(base[b]) + ((((size_t)layer * 2 + 1) * H + hh) * cp + slot) * hd;
+    const int cq = hh * hd, ck = d + hh * hd, cv = 2 * d + hh * hd;
+    const TileRef tq = qkv.tiles[cq >> 7], tk = qkv.tiles[ck >> 7], tv = qkv.tiles[cv >> 7];
+    const float4 q0 = gemm_out_at4(qkv, tq, r, (cq + i) & 127), q1 = gemm_out_at4(qkv, tq, r, (cq + i + half) & 127);
+    const float4 k0 = gemm_out_at4(qkv, tk, r, (ck + i) & 127), k1 = gemm_out_at4(qkv, tk, r, (ck + i + half) & 127);
+    const float4 v0 = gemm_out_at4(qkv, tv, r, (cv + i) & 127), v1 = gemm_out_at4(qkv, tv, r, (cv + i + half) & 127);
+    const float4 c = *reinterpret_cast<const float4*>(cs + r * half + i), s = *reinterpret_cast<const float4*>(sn + r * half + i);
+    bf16* qd = q + (size_t)r * d + hh * hd;
+    *reinterpret_cast<uint2*>(qd + i) = pack4_bf16(q0.x * c.x - q1.x * s.x, q0.y * c.y - q1.y * s.y, q0.z * c.z - q1.z * s.z, q0.w * c.w - q1.w * s.w);
+    *reinterpret_cast<uint2*>(qd + i + half) = pack4_bf16(q1.x * c.x + q0.x * s.x, q1.y * c.y + q0.y * s.y, q1.z * c.z + q0.z * s.z, q1.w * c.w + q0.w * s.w);
+    *reinterpret_cast<uint2*>(kdst + i) = pack4_bf16(k0.x * c.x - k1.x * s.x, k0.y * c.y - k1.y * s.y, k0.z * c.z - k1.z * s.z, k0.w * c.w - k1.w * s.w);
+    *reinterpret_cast<uint2*>(kdst + i + half) = pack4_bf16(k1.x * c.x + k0.x * s.x, k1.y * c.y + k0.y * s.y, k1.z * c.z + k0.z * s.z, k1.w * c.w + k0.w * s.w);
+    *reinterpret_cast<uint2*>(vdst + i) = pack4_bf16(v0.x, v0.y, v0.z, v0.w);
+    *reinterpret_cast<uint2*>(vdst + i + half) = pack4_bf16(v1.x, v1.y, v1.z, v1.w);
+}
+
+// ---- launchers (callers have checked: bf16 model, result in slots) ----------------------------
+void launch_add_rmsnorm_ws(aded_model* m, const GemmOut& y, const void* gain, int rows, cudaStream_t st) {
+    const int d = m->cfg.d_model;
+    dim3 grid((d + 1023) / 1024, rows);
+    launch_k(k_add_rmsnorm_ws, grid, dim3(256), 0, st, (bf16*)m->h, y, (const bf16*)gain, (bf16*)m->x, d, m->cfg.rms_eps,
+             m->norm_ssq, m->norm_count, m->status);
+}
+
+void launch_swiglu_ws(aded_model* m, const GemmOut& gu, int rows, cudaStream_t st) {
+    const int F = m->cfg.d_ffn;
+    dim3 grid((F + 1023) / 1024, rows);
+    launch_k(k_swiglu_ws, grid, dim3(256), 0, st, gu, (bf16*)m->act, F, m->status);
+}
+
+void launch_rope_kv_ws(aded_model* m, aded_kv* kv, const GemmOut& qkv, int layer, int rows, cudaStream_t st) {
+    dim3 grid(rows, m->cfg.n_heads);
+    launch_k(k_rope_kv_ws, grid, dim3(32), 0, st, qkv, (const float*)m->rope_cos, (const float*)m->rope_sin, (bf16*)m->q,
+             (char* const*)kv->base_dev, (const int32_t*)kv->cap_dev, (const int32_t*)kv->len_dev,
+             (const int32_t*)m->rows.seq, (const int32_t*)m->rows.local, layer, m->cfg.n_heads, m->cfg.head_dim,
+             (const int32_t*)m->status);
+}
+
+}  // namespace aded
