@@ -137,10 +137,7 @@ struct aded_model {
     float* dbg_logits;
     int32_t* dbg_best;
 
-    // split-KV attention partials (bf16 models)
-    float* att_o;       // [splits][R][H][hd] unnormalised outputs
-    float* att_ml;      // [splits][R][H][2]  running max (log2 domain) and sum
-    int32_t att_splits_max;
+    bool att_mma;       // bf16 models: tensor-core split-KV attention kernel
 
     // tensor-core GEMM path (bf16 models): TMA descriptors and split-tile scratch
     bool ws_ready;

@@ -48,61 +48,69 @@ __device__ __forceinline__ float warp_sum_f(float v) {
     return v;
 }
 
-// Residual add + RMSNorm (see k_add_rmsnorm): grid (chunks of 1024 columns, rows), 256 threads,
-// four columns per thread; the chunk that finishes a row last normalises the whole row.
-__global__ void __launch_bounds__(256) k_add_rmsnorm_ws(bf16* __restrict__ h, GemmOut y, const bf16* __restrict__ gain,
-                                                        bf16* __restrict__ x, int d, float eps, float* __restrict__ ssq,
-                                                        int32_t* __restrict__ row_count, const int32_t* status) {
-    pdl_enter();
+// Residual add + RMSNorm (see k_add_rmsnorm): one block of 1024 threads per row, four columns per
+// thread and pass (two passes cover d up to 8192).  The row stays in registers between the sum of
+// squares and the scaling, so the kernel is: gather the projection's slots, one block reduction,
+// store h and x.  The contributor table and the gain are not written by any kernel of the pass and
+// are fetched before waiting for the previous kernel.
+__global__ void __launch_bounds__(1024) k_add_rmsnorm_ws(bf16* __restrict__ h, GemmOut y, const bf16* __restrict__ gain,
+                                                         bf16* __restrict__ x, int d, float eps, const int32_t* status) {
+    pdl_launch_dependents();
+    __shared__ float red[32];
+    const int r = blockIdx.x;
+    TileRef tr[2];
+    float4 gv[2];
+#pragma unroll
+    for (int i = 0; i < 2; ++i) {
+        const int c = (i * 1024 + threadIdx.x) * 4;
+        if (c < d) {
+            tr[i] = y.tiles[c >> 7];
+            gv[i] = unpack4_bf16(*reinterpret_cast<const uint2*>(gain + c));
+        }
+    }
+    pdl_wait();
     if (*status != 0) return;
-    __shared__ float red[8];
-    __shared__ int s_last;
-    const int r = blockIdx.y, c = (blockIdx.x * 256 + threadIdx.x) * 4;
+    float4 v[2];
     float sq = 0.f;
-    if (c < d) {
-        uint2* hp = reinterpret_cast<uint2*>(h + (size_t)r * d + c);
-        const float4 hv = unpack4_bf16(*hp);
-        const float4 add = gemm_out_at4(y, y.tiles[c >> 7], r, c & 127);
-        const uint2 nv = pack4_bf16(hv.x + add.x, hv.y + add.y, hv.z + add.z, hv.w + add.w);
-        *hp = nv;
-        const float4 v = unpack4_bf16(nv);
-        sq = v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
+#pragma unroll
+    for (int i = 0; i < 2; ++i) {
+        const int c = (i * 1024 + threadIdx.x) * 4;
+        if (c < d) {
+            uint2* hp = reinterpret_cast<uint2*>(h + (size_t)r * d + c);
+            const float4 hv = unpack4_bf16(*hp);
+            const float4 add = gemm_out_at4(y, tr[i], r, c & 127);
+            const uint2 nv = pack4_bf16(hv.x + add.x, hv.y + add.y, hv.z + add.z, hv.w + add.w);
+            *hp = nv;
+            v[i] = unpack4_bf16(nv);
+            sq += v[i].x * v[i].x + v[i].y * v[i].y + v[i].z * v[i].z + v[i].w * v[i].w;
+        }
     }
     sq = warp_sum_f(sq);
     if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = sq;
     __syncthreads();
-    if (threadIdx.x == 0) {
-        float tot = 0.f;
-        for (int i = 0; i < 8; ++i) tot += red[i];
-        ssq[r * 32 + blockIdx.x] = tot;
-        __threadfence();
-        const int prev = atomicAdd(&row_count[r], 1);
-        s_last = prev == (int)gridDim.x - 1;
-        if (s_last) row_count[r] = 0;
-    }
-    __syncthreads();
-    if (!s_last) return;
-    __threadfence();
     float total = 0.f;
-    for (int i = 0; i < (int)gridDim.x; ++i) total += __ldcg(ssq + r * 32 + i);
+#pragma unroll
+    for (int i = 0; i < 32; ++i) total += red[i];      // same order in every thread
     const float inv = rsqrtf(total / (float)d + eps);
-    const uint2* hr = reinterpret_cast<const uint2*>(h + (size_t)r * d);
-    const uint2* gr = reinterpret_cast<const uint2*>(gain);
-    uint2* xr = reinterpret_cast<uint2*>(x + (size_t)r * d);
-    for (int cc = threadIdx.x; cc < d / 4; cc += 256) {
-        const float4 hv = unpack4_bf16(__ldcg(hr + cc)), gv = unpack4_bf16(gr[cc]);
-        xr[cc] = pack4_bf16(hv.x * inv * gv.x, hv.y * inv * gv.y, hv.z * inv * gv.z, hv.w * inv * gv.w);
+#pragma unroll
+    for (int i = 0; i < 2; ++i) {
+        const int c = (i * 1024 + threadIdx.x) * 4;
+        if (c < d)
+            *reinterpret_cast<uint2*>(x + (size_t)r * d + c) =
+                pack4_bf16(v[i].x * inv * gv[i].x, v[i].y * inv * gv[i].y, v[i].z * inv * gv[i].z, v[i].w * inv * gv[i].w);
     }
 }
 
 // act = round(silu(gate) * up): grid (chunks of 1024 columns, rows), four columns per thread.
 __global__ void __launch_bounds__(256) k_swiglu_ws(GemmOut gu, bf16* __restrict__ act, int F, const int32_t* status) {
-    pdl_enter();
-    if (*status != 0) return;
+    pdl_launch_dependents();
     const int r = blockIdx.y, c = (blockIdx.x * 256 + threadIdx.x) * 4;
-    if (c >= F) return;
-    const float4 g = gemm_out_at4(gu, gu.tiles[c >> 7], r, c & 127);
-    const float4 u = gemm_out_at4(gu, gu.tiles[(F + c) >> 7], r, (F + c) & 127);
+    TileRef tg = {0, 0}, tu = {0, 0};
+    if (c < F) { tg = gu.tiles[c >> 7]; tu = gu.tiles[(F + c) >> 7]; }   // the table is constant: read it before waiting
+    pdl_wait();
+    if (*status != 0 || c >= F) return;
+    const float4 g = gemm_out_at4(gu, tg, r, c & 127);
+    const float4 u = gemm_out_at4(gu, tu, r, (F + c) & 127);
     *reinterpret_cast<uint2*>(act + (size_t)r * F + c) =
         pack4_bf16(g.x / (1.f + expf(-g.x)) * u.x, g.y / (1.f + expf(-g.y)) * u.y,
                    g.z / (1.f + expf(-g.z)) * u.z, g.w / (1.f + expf(-g.w)) * u.w);
@@ -114,18 +122,18 @@ __global__ void k_rope_kv_ws(GemmOut qkv, const float* __restrict__ cs, const fl
                              bf16* __restrict__ q, char* const* __restrict__ base, const int32_t* __restrict__ cap,
                              const int32_t* __restrict__ len, const int32_t* __restrict__ row_seq,
                              const int32_t* __restrict__ row_local, int layer, int H, int hd, const int32_t* status) {
-    pdl_enter();
-    if (*status != 0) return;
+    pdl_launch_dependents();
     const int r = blockIdx.x, hh = blockIdx.y, half = hd >> 1, d = H * hd;
     const int i = threadIdx.x * 4;
-    if (i >= half) return;
+    const int cq = hh * hd, ck = d + hh * hd, cv = 2 * d + hh * hd;
+    const TileRef tq = qkv.tiles[cq >> 7], tk = qkv.tiles[ck >> 7], tv = qkv.tiles[cv >> 7];   // constant table
+    pdl_wait();
+    if (*status != 0 || i >= half) return;
     const int b = row_seq[r];
     const size_t slot = (size_t)len[b] + row_local[r];
     const size_t cp = cap[b];
     bf16* kdst = reinterpret_cast<bf16*>(base[b]) + ((((size_t)layer * 2 + 0) * H + hh) * cp + slot) * hd;
     bf16* vdst = reinterpret_cast<bf16*>(base[b]) + ((((size_t)layer * 2 + 1) * H + hh) * cp + slot) * hd;
-    const int cq = hh * hd, ck = d + hh * hd, cv = 2 * d + hh * hd;
-    const TileRef tq = qkv.tiles[cq >> 7], tk = qkv.tiles[ck >> 7], tv = qkv.tiles[cv >> 7];
     const float4 q0 = gemm_out_at4(qkv, tq, r, (cq + i) & 127), q1 = gemm_out_at4(qkv, tq, r, (cq + i + half) & 127);
     const float4 k0 = gemm_out_at4(qkv, tk, r, (ck + i) & 127), k1 = gemm_out_at4(qkv, tk, r, (ck + i + half) & 127);
     const float4 v0 = gemm_out_at4(qkv, tv, r, (cv + i) & 127), v1 = gemm_out_at4(qkv, tv, r, (cv + i + half) & 127);
@@ -142,9 +150,8 @@ __global__ void k_rope_kv_ws(GemmOut qkv, const float* __restrict__ cs, const fl
 // ---- launchers (callers have checked: bf16 model, result in slots) ----------------------------
 void launch_add_rmsnorm_ws(aded_model* m, const GemmOut& y, const void* gain, int rows, cudaStream_t st) {
     const int d = m->cfg.d_model;
-    dim3 grid((d + 1023) / 1024, rows);
-    launch_k(k_add_rmsnorm_ws, grid, dim3(256), 0, st, (bf16*)m->h, y, (const bf16*)gain, (bf16*)m->x, d, m->cfg.rms_eps,
-             m->norm_ssq, m->norm_count, m->status);
+    launch_k(k_add_rmsnorm_ws, dim3(rows), dim3(1024), 0, st, (bf16*)m->h, y, (const bf16*)gain, (bf16*)m->x, d, m->cfg.rms_eps,
+             (const int32_t*)m->status);
 }
 
 void launch_swiglu_ws(aded_model* m, const GemmOut& gu, int rows, cudaStream_t st) {

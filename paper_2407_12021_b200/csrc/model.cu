@@ -108,14 +108,7 @@ static aded_status alloc_model(aded_model* m) {
     ADED_CUDA_TRY(cudaMemset(m->attn, 0, R * d * m->elem));
     ADED_CUDA_TRY(cudaMemset(m->act, 0, R * F * m->elem));
 
-    m->att_o = nullptr;
-    m->att_ml = nullptr;
-    m->att_splits_max = 1;
-    if (c.dtype == ADED_BF16 && !getenv("ADED_PLAIN_ATTN") && attn_prepare()) {
-        m->att_splits_max = R <= 128 ? 16 : (int)(16 * 128 / R > 0 ? 16 * 128 / R : 1);
-        TRY(dev_alloc(m, &m->att_o, (size_t)m->att_splits_max * R * d));
-        TRY(dev_alloc(m, &m->att_ml, (size_t)m->att_splits_max * R * c.n_heads * 2));
-    }
+    m->att_mma = c.dtype == ADED_BF16 && !getenv("ADED_PLAIN_ATTN") && attn_prepare();
 
     // tensor-core GEMM path: bf16 models whose every matrix tiles into 128-row x 64-column blocks
     m->ws_ready = false;
@@ -158,7 +151,7 @@ static aded_status alloc_model(aded_model* m) {
 static int pass_launches(const aded_model* m, int rows, int chain_mode) {
     const int gemm_passes = (rows + 127) / 128;   // the tensor-core GEMM runs once per 128 rows
     const int per_gemm = m->ws_ready ? gemm_passes : 1;
-    int n = 4 + m->cfg.n_layers * (4 * per_gemm + 3 + (m->att_o ? 2 : 1));
+    int n = 4 + m->cfg.n_layers * (4 * per_gemm + 3 + 1);
     n += chain_mode ? 1 : per_gemm + 5;
     return n;
 }
@@ -186,7 +179,7 @@ static aded_status enqueue_pass(aded_model* m, aded_kv* kv, const int32_t* offse
         GemmOut o;
         { Span sp(m, PROF_GEMM, 1, st); o = launch_gemm(m, 4 * l + WS_MAP_QKV, xm, m->x, w.wqkv, m->y32, rows, 3 * d, d, st, 4 * l + WS_MAP_O, d, d); }
         { Span sp(m, PROF_OTHER, 1, st); launch_rope_kv(m, kv, o, l, rows, st); }
-        { Span sp(m, PROF_ATTN, 2, st); launch_tree_attention(m, kv, l, batch, rows, max_tree, st); }
+        { Span sp(m, PROF_ATTN, 1, st); launch_tree_attention(m, kv, l, batch, rows, max_tree, st); }
         { Span sp(m, PROF_GEMM, 1, st); o = launch_gemm(m, 4 * l + WS_MAP_O, xm + 1, m->attn, w.wo, m->y32, rows, d, d, st, 4 * l + WS_MAP_GU, 2 * F, d); }
         { Span sp(m, PROF_OTHER, 1, st); launch_add_rmsnorm(m, &o, w.norm2, rows, st); }
         { Span sp(m, PROF_GEMM, 1, st); o = launch_gemm(m, 4 * l + WS_MAP_GU, xm, m->x, w.wgu, m->y32, rows, 2 * F, d, st, 4 * l + WS_MAP_D, d, F); }

@@ -9,8 +9,10 @@
 // warps share through shared memory (double-buffered cp.async).  Scores S = Q K^T and O += P V
 // are m16n8k16 bf16 MMAs with fp32 accumulators; the online softmax keeps a running maximum and
 // sum per row in registers (quad shuffles).  Only the blocks that reach past L apply the ancestor
-// bit mask.  Each split writes an unnormalised partial (O, max, sum); a merge kernel combines the
-// splits and rounds to bf16.  The key range is derived on the device from the committed length.
+// bit mask.  The splits of one (sequence, head) form a thread-block cluster: each keeps its
+// unnormalised partial (O, max, sum) in shared memory and the cluster combines them through
+// distributed shared memory, so partials never touch global memory and no merge kernel runs.  The
+// key range is derived on the device from the committed length.
 //
 // fp32 models use the plain one-warp-per-(row, head) kernel below.
 #include "aded_internal.cuh"
@@ -113,8 +115,7 @@ __device__ __forceinline__ bf16* tile_chunk(bf16* tile, int row, int chunk) {
 
 struct AttnArgs {
     const bf16* q;                 // [R][H][HD]
-    float* part_o;                 // [S][R][H][HD]
-    float* part_ml;                // [S][R][H][2]  (running max in the log2 domain, sum)
+    bf16* out;                     // [R][H][HD] attention output
     char* const* base;
     const int32_t* cap;
     const int32_t* len;
@@ -151,14 +152,6 @@ __global__ void __launch_bounds__(NW * 32) k_tree_attn_mma(AttnArgs a) {
     // this thread's two query rows (local node indices) and their global rows
     const int i0 = warp * 16 + g, i1 = i0 + 8;
     const bool v0 = i0 < T, v1 = i1 < T;
-    const size_t pstride = (size_t)a.rows_total * a.H;            // (row, head) pairs per split
-    if (blk0 >= blk1) {                                           // nothing in this split
-        if (tig == 0) {
-            if (v0) { float* ml = a.part_ml + ((size_t)split * pstride + (size_t)(off + i0) * a.H + hh) * 2; ml[0] = -INFINITY; ml[1] = 0.f; }
-            if (v1) { float* ml = a.part_ml + ((size_t)split * pstride + (size_t)(off + i1) * a.H + hh) * 2; ml[0] = -INFINITY; ml[1] = 0.f; }
-        }
-        return;
-    }
     const bf16* kg = reinterpret_cast<const bf16*>(a.base[b]) + (((size_t)a.layer * 2 + 0) * a.H + hh) * cp * HD;
     const bf16* vg = reinterpret_cast<const bf16*>(a.base[b]) + (((size_t)a.layer * 2 + 1) * a.H + hh) * cp * HD;
 
@@ -200,7 +193,7 @@ __global__ void __launch_bounds__(NW * 32) k_tree_attn_mma(AttnArgs a) {
         cp_async_commit();
     };
 
-    load_block(blk0, 0);
+    if (blk0 < blk1) load_block(blk0, 0);   // (a split past the last key block has nothing to do but still joins the merge)
     for (int blk = blk0; blk < blk1; ++blk) {
         const int buf = (blk - blk0) & 1;
         if (blk + 1 < blk1) { load_block(blk + 1, buf ^ 1); cp_async_wait<1>(); } else { cp_async_wait<0>(); }
@@ -289,55 +282,112 @@ __global__ void __launch_bounds__(NW * 32) k_tree_attn_mma(AttnArgs a) {
         }
         __syncthreads();   // the buffer is refilled two iterations later by load_block(blk + 2, buf)
     }
-    // ---- write the split's partial result ----
+    // ---- merge the splits of this (sequence, head) across the cluster ----
+    // Every CTA parks its unnormalised partial (O, running max, sum) in its own shared memory; after a
+    // cluster barrier CTA j combines rows j, j + S, ... from all S CTAs' shared memory (distributed
+    // shared memory reads), out = sum_s O_s 2^(m_s - M) / sum_s l_s 2^(m_s - M), rounds to bf16 and
+    // writes the attention output.  No partial ever goes to global memory.
     lrow0 += __shfl_xor_sync(0xffffffffu, lrow0, 1);
     lrow0 += __shfl_xor_sync(0xffffffffu, lrow0, 2);
     lrow1 += __shfl_xor_sync(0xffffffffu, lrow1, 1);
     lrow1 += __shfl_xor_sync(0xffffffffu, lrow1, 2);
-    if (v0) {
-        const size_t idx = (size_t)split * pstride + (size_t)(off + i0) * a.H + hh;
-        float* po = a.part_o + idx * HD;
+    __syncthreads();                                   // all warps are done with the K/V tiles
+    float* so = reinterpret_cast<float*>(smem_raw);    // [NW*16][HD]
+    float* sml = so + NW * 16 * HD;                    // [NW*16][2]
+    {
+        const int r0 = warp * 16 + g, r1 = r0 + 8;
 #pragma unroll
-        for (int n = 0; n < ONT; ++n) *reinterpret_cast<float2*>(po + n * 8 + 2 * tig) = make_float2(oacc[n][0], oacc[n][1]);
-        if (tig == 0) { a.part_ml[idx * 2] = mrow0; a.part_ml[idx * 2 + 1] = lrow0; }
+        for (int n = 0; n < ONT; ++n) {
+            *reinterpret_cast<float2*>(so + (size_t)r0 * HD + n * 8 + 2 * tig) = make_float2(oacc[n][0], oacc[n][1]);
+            *reinterpret_cast<float2*>(so + (size_t)r1 * HD + n * 8 + 2 * tig) = make_float2(oacc[n][2], oacc[n][3]);
+        }
+        if (tig == 0) {
+            sml[r0 * 2] = mrow0; sml[r0 * 2 + 1] = lrow0;
+            sml[r1 * 2] = mrow1; sml[r1 * 2 + 1] = lrow1;
+        }
     }
-    if (v1) {
-        const size_t idx = (size_t)split * pstride + (size_t)(off + i1) * a.H + hh;
-        float* po = a.part_o + idx * HD;
-#pragma unroll
-        for (int n = 0; n < ONT; ++n) *reinterpret_cast<float2*>(po + n * 8 + 2 * tig) = make_float2(oacc[n][2], oacc[n][3]);
-        if (tig == 0) { a.part_ml[idx * 2] = mrow1; a.part_ml[idx * 2 + 1] = lrow1; }
+    const int S = a.n_splits;
+    if (S > 1) {
+        asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+        asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+    } else {
+        __syncthreads();
+    }
+    const uint32_t so_addr = (uint32_t)__cvta_generic_to_shared(so), sml_addr = (uint32_t)__cvta_generic_to_shared(sml);
+    constexpr int QUADS = HD / 4;                      // float4 groups per row
+    for (int item = threadIdx.x; item < ((T - split + S - 1) / S) * QUADS; item += NW * 32) {
+        const int row = split + (item / QUADS) * S, c4 = (item % QUADS) * 4;
+        float ms[8], ls[8];
+        float M = -INFINITY;
+        for (int s2 = 0; s2 < S; ++s2) {
+            uint32_t remote;
+            asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(sml_addr + (uint32_t)row * 8), "r"(s2));
+            asm volatile("ld.shared::cluster.v2.f32 {%0, %1}, [%2];" : "=f"(ms[s2]), "=f"(ls[s2]) : "r"(remote));
+            M = fmaxf(M, ms[s2]);
+        }
+        float4 num = make_float4(0.f, 0.f, 0.f, 0.f);
+        float den = 0.f;
+        for (int s2 = 0; s2 < S; ++s2) {
+            if (ms[s2] == -INFINITY) continue;
+            const float w = exp2f(ms[s2] - M);
+            uint32_t remote;
+            asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(so_addr + (uint32_t)(row * HD + c4) * 4), "r"(s2));
+            float4 o;
+            asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(o.x), "=f"(o.y), "=f"(o.z), "=f"(o.w) : "r"(remote));
+            den += ls[s2] * w;
+            num.x += o.x * w; num.y += o.y * w; num.z += o.z * w; num.w += o.w * w;
+        }
+        const float inv = 1.f / den;
+        bf16* dst = a.out + ((size_t)(off + row) * a.H + hh) * HD + c4;
+        const __nv_bfloat162 lo = __floats2bfloat162_rn(num.x * inv, num.y * inv), hi = __floats2bfloat162_rn(num.z * inv, num.w * inv);
+        uint2 u;
+        u.x = *reinterpret_cast<const uint32_t*>(&lo);
+        u.y = *reinterpret_cast<const uint32_t*>(&hi);
+        *reinterpret_cast<uint2*>(dst) = u;
+    }
+    if (S > 1) {   // nobody may leave while a neighbour still reads its shared memory
+        asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+        asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
     }
 }
 
-// Combines the splits of one (row, head): out = sum_s O_s 2^(m_s - M) / sum_s l_s 2^(m_s - M).
-template <int HD>
-__global__ void __launch_bounds__(HD) k_tree_attn_merge(const float* __restrict__ part_o, const float* __restrict__ part_ml,
-                                                       bf16* __restrict__ out, int n_splits, int rows, int H,
-                                                       const int32_t* status) {
-    pdl_enter();
-    if (*status != 0) return;
-    const int r = blockIdx.x, hh = blockIdx.y, e = threadIdx.x;
-    const size_t pstride = (size_t)rows * H, idx = (size_t)r * H + hh;
-    float M = -INFINITY;
-    for (int s = 0; s < n_splits; ++s) M = fmaxf(M, part_ml[((size_t)s * pstride + idx) * 2]);
-    float num = 0.f, den = 0.f;
-    for (int s = 0; s < n_splits; ++s) {
-        const float m = part_ml[((size_t)s * pstride + idx) * 2];
-        if (m == -INFINITY) continue;
-        const float w = exp2f(m - M);
-        den += part_ml[((size_t)s * pstride + idx) * 2 + 1] * w;
-        num += part_o[((size_t)s * pstride + idx) * HD + e] * w;
+template <int HD, int NW>
+static size_t attn_smem() {
+    const size_t kv = (size_t)4 * TA_BLK * HD * sizeof(bf16), merge = (size_t)NW * 16 * (HD + 2) * sizeof(float);
+    return kv > merge ? kv : merge;
+}
+
+template <int HD, int NW>
+static void launch_mma_nw(aded_model* m, AttnArgs& a, int batch, int splits, cudaStream_t st) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(m->cfg.n_heads, splits, batch);
+    cfg.blockDim = dim3(NW * 32);
+    cfg.dynamicSmemBytes = attn_smem<HD, NW>();
+    cfg.stream = st;
+    cudaLaunchAttribute attr[2];
+    int n = 0;
+    if (splits > 1) {
+        attr[n].id = cudaLaunchAttributeClusterDimension;
+        attr[n].val.clusterDim.x = 1;
+        attr[n].val.clusterDim.y = splits;
+        attr[n].val.clusterDim.z = 1;
+        ++n;
     }
-    out[idx * HD + e] = __float2bfloat16_rn(num / den);
+    if (pdl_enabled()) {
+        attr[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[n].val.programmaticStreamSerializationAllowed = 1;
+        ++n;
+    }
+    cfg.attrs = attr;
+    cfg.numAttrs = n;
+    cudaLaunchKernelEx(&cfg, k_tree_attn_mma<HD, NW>, a);
 }
 
 template <int HD>
 static void launch_mma(aded_model* m, aded_kv* kv, int layer, int batch, int rows, int max_tree, cudaStream_t st) {
     AttnArgs a;
     a.q = (const bf16*)m->q;
-    a.part_o = m->att_o;
-    a.part_ml = m->att_ml;
+    a.out = (bf16*)m->attn;
     a.base = kv->base_dev;
     a.cap = kv->cap_dev;
     a.len = kv->len_dev;
@@ -345,35 +395,31 @@ static void launch_mma(aded_model* m, aded_kv* kv, int layer, int batch, int row
     a.anc = m->rows.anc;
     a.layer = layer;
     a.H = m->cfg.n_heads;
-    // enough (head, split) CTAs for about two per SM, within what the partial buffers hold
-    int splits = (ws_grid_limit(m->device) + m->cfg.n_heads * batch - 1) / (m->cfg.n_heads * batch);
-    if (splits > m->att_splits_max) splits = m->att_splits_max;
-    if (splits < 1) splits = 1;
+    // key splits per (sequence, head): a power of two up to 8 (one thread-block cluster), enough for
+    // about three quarters of the two-per-SM CTA slots
+    int splits = 1;
+    while (splits < 8 && m->cfg.n_heads * batch * splits * 4 < ws_grid_limit(m->device) * 3) splits *= 2;
     a.n_splits = splits;
     a.rows_total = rows;
     a.scale_log2 = 1.4426950408889634f / sqrtf((float)HD);
     a.status = m->status;
-    dim3 grid(m->cfg.n_heads, splits, batch);
-    const size_t smem = (size_t)4 * TA_BLK * HD * sizeof(bf16);
-    if (max_tree <= 64) launch_k(k_tree_attn_mma<HD, 4>, grid, 128, smem, st, a);
-    else launch_k(k_tree_attn_mma<HD, 8>, grid, 256, smem, st, a);
-    dim3 mgrid(rows, m->cfg.n_heads);
-    launch_k(k_tree_attn_merge<HD>, mgrid, HD, 0, st, m->att_o, m->att_ml, (bf16*)m->attn, splits, rows, m->cfg.n_heads, m->status);
+    if (max_tree <= 64) launch_mma_nw<HD, 4>(m, a, batch, splits, st);
+    else launch_mma_nw<HD, 8>(m, a, batch, splits, st);
 }
 
 // Raises the split-KV kernels' dynamic shared-memory limit; once per process, before any launch.
 bool attn_prepare() {
     bool ok = true;
-    ok &= cudaFuncSetAttribute(k_tree_attn_mma<128, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, 4 * TA_BLK * 128 * 2) == cudaSuccess;
-    ok &= cudaFuncSetAttribute(k_tree_attn_mma<128, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, 4 * TA_BLK * 128 * 2) == cudaSuccess;
-    ok &= cudaFuncSetAttribute(k_tree_attn_mma<64, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, 4 * TA_BLK * 64 * 2) == cudaSuccess;
-    ok &= cudaFuncSetAttribute(k_tree_attn_mma<64, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, 4 * TA_BLK * 64 * 2) == cudaSuccess;
+    ok &= cudaFuncSetAttribute(k_tree_attn_mma<128, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attn_smem<128, 4>()) == cudaSuccess;
+    ok &= cudaFuncSetAttribute(k_tree_attn_mma<128, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attn_smem<128, 8>()) == cudaSuccess;
+    ok &= cudaFuncSetAttribute(k_tree_attn_mma<64, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attn_smem<64, 4>()) == cudaSuccess;
+    ok &= cudaFuncSetAttribute(k_tree_attn_mma<64, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attn_smem<64, 8>()) == cudaSuccess;
     return ok;
 }
 
 void launch_tree_attention(aded_model* m, aded_kv* kv, int layer, int batch, int rows, int max_tree, cudaStream_t st) {
     const int H = m->cfg.n_heads, hd = m->cfg.head_dim;
-    if (m->cfg.dtype == ADED_BF16 && m->att_o != nullptr) {
+    if (m->cfg.dtype == ADED_BF16 && m->att_mma) {
         if (hd == 128) launch_mma<128>(m, kv, layer, batch, rows, max_tree, st);
         else launch_mma<64>(m, kv, layer, batch, rows, max_tree, st);
         return;
