@@ -179,6 +179,31 @@ aded_status aded_profile_end(aded_model* m, float* out_ms_host, int32_t* out_lau
 /* Kernels launched by this library in this process so far (all handles). */
 uint64_t aded_launch_count(void);
 
+/* Greedy token choice without any allocation.  (The paper has no counterpart of this call; it is
+ * the library's per-node greedy choice -- largest fp32 logit, lowest token id among equals -- offered
+ * on its own.)
+ *
+ * For callers that cannot allocate device memory: a process whose device heap is wholly reserved by
+ * another component (for instance a framework's caching allocator, so that a cudaMalloc made by this
+ * library could fail or stall), or a latency-critical loop that bans allocation calls because
+ * cudaMalloc and cudaFree synchronise the device.  Such callers cannot create a model handle, but
+ * can still pick tokens from logits they computed elsewhere.
+ *   logits_dev    [rows][vocab] fp32, row-major, device memory
+ *   out_best_dev  [rows] int32, device memory: index of each row's largest logit
+ * The call uses no handle and calls no cudaMalloc, cudaFree or other allocating routine.  Its
+ * intermediate results live in a fixed 16 KiB array inside the library's device image (every
+ * device that loads the library holds it until the process exits), which bounds the size:
+ * rows <= ADED_NOALLOC_MAX_ROWS, otherwise ADED_ERR_INVALID_ARG and nothing is launched.
+ * The first call on each device looks up the array's device address (with that device current);
+ * make that first call outside any stream capture.  All calls share the one array: it keeps the
+ * previous call's contents, which is harmless because every entry is rewritten before it is read,
+ * but two calls whose kernels overlap on the GPU (different streams, no dependency) race on it --
+ * keep calls on one stream or order them with events.  Work is enqueued on `stream`; the call does
+ * not synchronise. */
+#define ADED_NOALLOC_MAX_ROWS 128
+aded_status aded_greedy_noalloc(const float* logits_dev, int32_t rows, int32_t vocab, int32_t* out_best_dev,
+                                void* stream);
+
 /* Read and clear the model's device status word; synchronises `stream`. */
 aded_status aded_model_poll_status(aded_model* m, aded_status* out_host, void* stream);
 

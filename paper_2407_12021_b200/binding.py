@@ -25,7 +25,7 @@ STATUS_NAMES = {0: "ADED_OK", 1: "ADED_ERR_INVALID_ARG", 2: "ADED_ERR_BAD_TREE",
 EXPORTS = [
     "aded_model_create", "aded_model_destroy", "aded_kv_create", "aded_kv_destroy", "aded_kv_len",
     "aded_kv_load", "aded_kv_set_len", "aded_kv_read", "aded_append", "aded_verify", "aded_verify_batch", "aded_verify_host",
-    "aded_debug_capture", "aded_debug_gemm", "aded_profile_begin", "aded_profile_end", "aded_launch_count", "aded_model_poll_status", "aded_trigram_create", "aded_trigram_destroy",
+    "aded_debug_capture", "aded_debug_gemm", "aded_greedy_noalloc", "aded_profile_begin", "aded_profile_end", "aded_launch_count", "aded_model_poll_status", "aded_trigram_create", "aded_trigram_destroy",
     "aded_trigram_update", "aded_trigram_update_host", "aded_trigram_topk", "aded_trigram_topk_host",
     "aded_trigram_get", "aded_trigram_stats", "aded_trigram_poll_status", "aded_status_string",
 ]
@@ -254,6 +254,23 @@ def aded_debug_gemm(model: Model, layer: int, which: int, x: torch.Tensor) -> to
     _check(_lib.aded_debug_gemm(model.handle, c_int32(layer), c_int32(which), _ptr(x), c_int32(x.shape[0]), _ptr(y),
                                 _stream()), "aded_debug_gemm")
     return y
+
+
+ADED_NOALLOC_MAX_ROWS = 128
+
+
+def aded_greedy_noalloc(logits: torch.Tensor, out_best: torch.Tensor) -> None:
+    """Greedy token per row of a [rows, vocab] fp32 CUDA logits tensor into out_best ([rows] int32 CUDA),
+    without a handle and without any allocation (for callers whose device memory is owned by another
+    allocator, or whose decode loop may not call cudaMalloc).  rows <= ADED_NOALLOC_MAX_ROWS.  Calls
+    share one fixed scratch array inside the library: keep them on one stream."""
+    if not (logits.is_cuda and logits.dtype == torch.float32 and logits.is_contiguous() and logits.dim() == 2):
+        raise TypeError("logits must be a contiguous fp32 CUDA tensor [rows, vocab]")
+    _dev_i32(out_best, "out_best")
+    if out_best.numel() < logits.shape[0]:
+        raise ValueError("out_best is shorter than the number of rows")
+    _check(_lib.aded_greedy_noalloc(_ptr(logits), c_int32(logits.shape[0]), c_int32(logits.shape[1]), _ptr(out_best),
+                                    _stream()), "aded_greedy_noalloc")
 
 
 def aded_profile_begin(model: Model) -> None:
