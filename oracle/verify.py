@@ -11,8 +11,8 @@ The model is a Llama-style decoder (pre-norm RMSNorm, rotary embedding on pairs
 (i, i + hd/2), multi-head attention, SwiGLU FFN, untied LM head), which is the family the
 paper evaluates.  All arithmetic is float64.  For bf16 models activations are rounded to
 bf16 at the points where a bf16 inference pipeline stores them (norm outputs, q/k/v after
-rotation, attention output, the SwiGLU product, the residual stream); attention
-probabilities and logits are never rounded.  For fp32 models nothing is rounded.
+rotation, the softmax numerators that multiply V, attention output, the SwiGLU product, the
+residual stream); logits are never rounded.  For fp32 models nothing is rounded.
 """
 from __future__ import annotations
 
@@ -90,6 +90,20 @@ def silu(x: np.ndarray) -> np.ndarray:
 def softmax(s: np.ndarray) -> np.ndarray:
     e = np.exp(s - np.max(s, axis=-1, keepdims=True))
     return e / np.sum(e, axis=-1, keepdims=True)
+
+
+def attention_weights(s: np.ndarray, bf16: bool) -> np.ndarray:
+    """Softmax weights of scaled scores s [..., n].  Exact for fp32 models.  For bf16 models the
+    weights that multiply V are bf16 numbers, as in a bf16 tensor-core pipeline: with t = s * log2(e)
+    and the power-of-two reference M = ceil(max t), each numerator 2^(t - M) is rounded to bf16 while
+    the denominator sums the unrounded numerators.  (A power-of-two reference makes the rounding
+    independent of the order in which keys are visited: rescaling by 2^k commutes with rounding.)"""
+    if not bf16:
+        return softmax(s)
+    t = s * np.log2(np.e)
+    m = np.ceil(np.max(t, axis=-1, keepdims=True))
+    e = np.exp2(t - m)
+    return round_bf16(e) / np.sum(e, axis=-1, keepdims=True)
 
 
 # --------------------------------------------------------------------------
@@ -209,7 +223,7 @@ def forward_tree(arch: Arch, w: Weights, cache: Cache, tokens: Sequence[int],
             keys = np.concatenate([cache.k[l], k[paths[i]].transpose(1, 0, 2)], axis=1)   # [H, n, hd]
             vals = np.concatenate([cache.v[l], v[paths[i]].transpose(1, 0, 2)], axis=1)
             s = np.einsum("hd,hnd->hn", q[i], keys) * scale
-            o[i] = np.einsum("hn,hnd->hd", softmax(s), vals)
+            o[i] = np.einsum("hn,hnd->hd", attention_weights(s, arch.bf16), vals)
         o = r(o).reshape(T, d)
         h = r(h + o @ p["wo"].T)
         x = r(rmsnorm(h, p["norm2"], arch.rms_eps))

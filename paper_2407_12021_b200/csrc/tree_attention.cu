@@ -7,8 +7,10 @@
 // bf16 models: split-KV kernel on tensor cores.  A CTA owns (sequence, head, key split); each of
 // its warps owns 16 tree nodes (query rows) and walks the split's keys in blocks of 64 that all
 // warps share through shared memory (double-buffered cp.async).  Scores S = Q K^T and O += P V
-// are m16n8k16 bf16 MMAs with fp32 accumulators; the online softmax keeps a running maximum and
-// sum per row in registers (quad shuffles).  Only the blocks that reach past L apply the ancestor
+// are m16n8k16 bf16 MMAs with fp32 accumulators; the online softmax keeps a running reference and
+// sum per row in registers (quad shuffles).  Numerators are 2^(t - M) with t the score in the log2
+// domain and M = ceil(max t) an integer, rounded to bf16 for the P V product while the row sum keeps
+// them unrounded; integer references make all rescaling exact.  Only the blocks that reach past L apply the ancestor
 // bit mask.  The splits of one (sequence, head) form a thread-block cluster: each keeps its
 // unnormalised partial (O, max, sum) in shared memory and the cluster combines them through
 // distributed shared memory, so partials never touch global memory and no merge kernel runs.  The
@@ -244,7 +246,10 @@ __global__ void __launch_bounds__(NW * 32) k_tree_attn_mma(AttnArgs a) {
         bm0 = fmaxf(bm0, __shfl_xor_sync(0xffffffffu, bm0, 2));
         bm1 = fmaxf(bm1, __shfl_xor_sync(0xffffffffu, bm1, 1));
         bm1 = fmaxf(bm1, __shfl_xor_sync(0xffffffffu, bm1, 2));
-        const float nm0 = fmaxf(mrow0, bm0), nm1 = fmaxf(mrow1, bm1);
+        // The running reference is the maximum rounded UP to an integer (scores are in the log2
+        // domain), so every rescale below is an exact power of two and the bf16 rounding of the
+        // numerators 2^(t - M) does not depend on how the keys are split or ordered.
+        const float nm0 = fmaxf(mrow0, ceilf(bm0)), nm1 = fmaxf(mrow1, ceilf(bm1));
         const float use0 = nm0 == -INFINITY ? 0.f : nm0, use1 = nm1 == -INFINITY ? 0.f : nm1;
         const float corr0 = exp2f(mrow0 - use0), corr1 = exp2f(mrow1 - use1);
         mrow0 = nm0;

@@ -306,3 +306,32 @@ def test_cache_after_verify_holds_the_accepted_path_not_the_first_nodes():
     for l in range(SMALL.n_layers):
         assert np.allclose(cache.k[l], ar_cache.k[l][:, :n], rtol=1e-9, atol=1e-11)
         assert np.allclose(cache.v[l], ar_cache.v[l][:, :n], rtol=1e-9, atol=1e-11)
+
+
+def test_bf16_attention_weights_are_softmax_with_rounded_numerators():
+    rng = np.random.default_rng(7)
+    s = rng.normal(size=(5, 301)) * 3
+    w = ov.attention_weights(s, True)
+    exact = torch.softmax(torch.from_numpy(s), -1).numpy()
+    assert np.allclose(w, exact, rtol=2.0 ** -8, atol=0)          # one bf16 rounding per weight
+    assert np.all(np.abs(w.sum(-1) - 1) < 2.0 ** -9)
+    assert np.array_equal(ov.attention_weights(s, False), ov.softmax(s))
+    # numerators are bf16 numbers relative to a power-of-two reference >= the row maximum
+    t = s * np.log2(np.e)
+    m = np.ceil(t.max(-1, keepdims=True))
+    num = w * np.exp2(t - m).sum(-1, keepdims=True)
+    assert np.allclose(num, ov.round_bf16(num), rtol=1e-12) and num.max() <= 1.0
+    # the result does not depend on key order or on processing the keys in pieces with their own
+    # (integer) references and rescaling -- rescaling by powers of two commutes with the rounding
+    perm = rng.permutation(301)
+    assert np.allclose(ov.attention_weights(s[:, perm], True), w[:, perm], rtol=1e-13, atol=0)   # (the sum's order moves the last bit)
+    pieces = [slice(0, 64), slice(64, 200), slice(200, 301)]
+    nums, dens, refs = [], [], []
+    for sl in pieces:
+        mp = np.ceil(t[:, sl].max(-1, keepdims=True))
+        e = np.exp2(t[:, sl] - mp)
+        nums.append(ov.round_bf16(e)); dens.append(e.sum(-1, keepdims=True)); refs.append(mp)
+    top = np.maximum.reduce(refs)
+    merged = np.concatenate([n * np.exp2(r - top) for n, r in zip(nums, refs)], axis=-1)
+    den = sum(d * np.exp2(r - top) for d, r in zip(dens, refs))
+    assert np.allclose(merged / den, w, rtol=1e-13, atol=0)
