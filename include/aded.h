@@ -179,6 +179,17 @@ aded_status aded_profile_end(aded_model* m, float* out_ms_host, int32_t* out_lau
 /* Kernels launched by this library in this process so far (all handles). */
 uint64_t aded_launch_count(void);
 
+/* Ask the next verify call to also store the residual stream before the first layer and after
+ * every layer: hidden_dev receives [n_layers + 1][rows][d_model] in the model dtype.  Lets a checker
+ * re-run any single layer from the inputs the device actually had.  Parity checks only. */
+aded_status aded_debug_capture_hidden(aded_model* m, void* hidden_dev);
+
+/* Copy out one of the model's activation buffers as the last verify/append call left it (after
+ * its last layer): which = 0 residual stream h [rows, d], 1 normalised input x [rows, d], 2 rotated
+ * queries q [rows, d], 3 attention output [rows, d], 4 SwiGLU product [rows, F]; model dtype.
+ * Stage-by-stage parity checks only. */
+aded_status aded_debug_read_buffer(aded_model* m, int32_t which, int32_t rows, void* out_dev, void* stream);
+
 /* Greedy token choice without any allocation.  (The paper has no counterpart of this call; it is
  * the library's per-node greedy choice -- largest fp32 logit, lowest token id among equals -- offered
  * on its own.)

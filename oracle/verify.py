@@ -193,49 +193,61 @@ class Cache:
 # --------------------------------------------------------------------------
 # the forward pass over a token tree
 # --------------------------------------------------------------------------
+def decoder_layer(arch: Arch, p: Dict[str, np.ndarray], cache_k: np.ndarray, cache_v: np.ndarray,
+                  h: np.ndarray, paths: Sequence[Sequence[int]], pos: np.ndarray, trace: Optional[dict] = None):
+    """One decoder layer over the tree's hidden states h [T, d].  cache_k / cache_v [H, L, hd] are the
+    layer's committed keys/values.  Returns (h_out [T, d], k [T, H, hd], v [T, H, hd])."""
+    r = round_bf16 if arch.bf16 else (lambda a: a)
+    T = h.shape[0]
+    H, hd, d, F = arch.n_heads, arch.head_dim, arch.d_model, arch.d_ffn
+    scale = 1.0 / np.sqrt(hd)
+    wq, wk, wv = p["wqkv"][:d], p["wqkv"][d:2 * d], p["wqkv"][2 * d:]
+    x = r(rmsnorm(h, p["norm1"], arch.rms_eps))
+    q = r(rope((x @ wq.T).reshape(T, H, hd), pos, arch.rope_theta))
+    k = r(rope((x @ wk.T).reshape(T, H, hd), pos, arch.rope_theta))
+    v = r((x @ wv.T).reshape(T, H, hd))
+    o = np.zeros((T, H, hd))
+    for i in range(T):
+        # keys node i may see: every cached position, then its ancestors and itself
+        keys = np.concatenate([cache_k, k[paths[i]].transpose(1, 0, 2)], axis=1)   # [H, n, hd]
+        vals = np.concatenate([cache_v, v[paths[i]].transpose(1, 0, 2)], axis=1)
+        s = np.einsum("hd,hnd->hn", q[i], keys) * scale
+        o[i] = np.einsum("hn,hnd->hd", attention_weights(s, arch.bf16), vals)
+    o = r(o).reshape(T, d)
+    h = r(h + o @ p["wo"].T)
+    x = r(rmsnorm(h, p["norm2"], arch.rms_eps))
+    gate, up = x @ p["wgu"][:F].T, x @ p["wgu"][F:].T
+    a = r(silu(gate) * up)
+    h = r(h + a @ p["wd"].T)
+    if trace is not None:      # intermediates, for stage-by-stage comparisons
+        trace.update(q=q.reshape(T, d), attn=o, act=a, h=h)
+    return h, k, v
+
+
+def lm_head(arch: Arch, w: Weights, h: np.ndarray) -> np.ndarray:
+    """Logits of hidden states h [T, d]: final RMSNorm, then the (untied) output projection."""
+    r = round_bf16 if arch.bf16 else (lambda a: a)
+    x = r(rmsnorm(h, w.top("final_norm"), arch.rms_eps))
+    return x @ w.top("lm_head").T
+
+
 def forward_tree(arch: Arch, w: Weights, cache: Cache, tokens: Sequence[int],
-                 parents: Sequence[int], want_logits: bool = True):
+                 parents: Sequence[int], want_logits: bool = True, trace: Optional[dict] = None):
     """Score every tree node in one pass.
 
     Returns (logits [T, V] or None, k_new, v_new) where k_new[l], v_new[l] are the tree
-    nodes' keys/values of layer l, shape [H, T, hd].  The cache is not modified.
+    nodes' keys/values of layer l, shape [H, T, hd].  The cache is not modified.  `trace`, when
+    given, receives the last layer's intermediates.
     """
-    r = round_bf16 if arch.bf16 else (lambda a: a)
-    T = len(tokens)
-    H, hd, d, F = arch.n_heads, arch.head_dim, arch.d_model, arch.d_ffn
     paths, depth = paths_and_depths(parents)
-    L = cache.length
-    pos = L + np.asarray(depth)                       # a node sits `depth` tokens after the context
-    scale = 1.0 / np.sqrt(hd)
-
+    pos = cache.length + np.asarray(depth)            # a node sits `depth` tokens after the context
     h = w.embed_rows(tokens)                          # residual stream [T, d]
     k_new, v_new = [], []
     for l in range(arch.n_layers):
-        p = w.layer(l)
-        wq, wk, wv = p["wqkv"][:d], p["wqkv"][d:2 * d], p["wqkv"][2 * d:]
-        x = r(rmsnorm(h, p["norm1"], arch.rms_eps))
-        q = r(rope((x @ wq.T).reshape(T, H, hd), pos, arch.rope_theta))
-        k = r(rope((x @ wk.T).reshape(T, H, hd), pos, arch.rope_theta))
-        v = r((x @ wv.T).reshape(T, H, hd))
-        o = np.zeros((T, H, hd))
-        for i in range(T):
-            # keys node i may see: every cached position, then its ancestors and itself
-            keys = np.concatenate([cache.k[l], k[paths[i]].transpose(1, 0, 2)], axis=1)   # [H, n, hd]
-            vals = np.concatenate([cache.v[l], v[paths[i]].transpose(1, 0, 2)], axis=1)
-            s = np.einsum("hd,hnd->hn", q[i], keys) * scale
-            o[i] = np.einsum("hn,hnd->hd", attention_weights(s, arch.bf16), vals)
-        o = r(o).reshape(T, d)
-        h = r(h + o @ p["wo"].T)
-        x = r(rmsnorm(h, p["norm2"], arch.rms_eps))
-        gate, up = x @ p["wgu"][:F].T, x @ p["wgu"][F:].T
-        a = r(silu(gate) * up)
-        h = r(h + a @ p["wd"].T)
+        h, k, v = decoder_layer(arch, w.layer(l), cache.k[l], cache.v[l], h, paths, pos, trace)
         k_new.append(k.transpose(1, 0, 2).copy())
         v_new.append(v.transpose(1, 0, 2).copy())
-    logits = None
-    if want_logits:
-        x = r(rmsnorm(h, w.top("final_norm"), arch.rms_eps))
-        logits = x @ w.top("lm_head").T
+    logits = lm_head(arch, w, h) if want_logits else None
     return logits, k_new, v_new
 
 

@@ -25,7 +25,7 @@ STATUS_NAMES = {0: "ADED_OK", 1: "ADED_ERR_INVALID_ARG", 2: "ADED_ERR_BAD_TREE",
 EXPORTS = [
     "aded_model_create", "aded_model_destroy", "aded_kv_create", "aded_kv_destroy", "aded_kv_len",
     "aded_kv_load", "aded_kv_set_len", "aded_kv_read", "aded_append", "aded_verify", "aded_verify_batch", "aded_verify_host",
-    "aded_debug_capture", "aded_debug_gemm", "aded_greedy_noalloc", "aded_profile_begin", "aded_profile_end", "aded_launch_count", "aded_model_poll_status", "aded_trigram_create", "aded_trigram_destroy",
+    "aded_debug_capture", "aded_debug_capture_hidden", "aded_debug_gemm", "aded_debug_read_buffer", "aded_greedy_noalloc", "aded_profile_begin", "aded_profile_end", "aded_launch_count", "aded_model_poll_status", "aded_trigram_create", "aded_trigram_destroy",
     "aded_trigram_update", "aded_trigram_update_host", "aded_trigram_topk", "aded_trigram_topk_host",
     "aded_trigram_get", "aded_trigram_stats", "aded_trigram_poll_status", "aded_status_string",
 ]
@@ -254,6 +254,23 @@ def aded_debug_gemm(model: Model, layer: int, which: int, x: torch.Tensor) -> to
     _check(_lib.aded_debug_gemm(model.handle, c_int32(layer), c_int32(which), _ptr(x), c_int32(x.shape[0]), _ptr(y),
                                 _stream()), "aded_debug_gemm")
     return y
+
+
+def aded_debug_capture_hidden(model: Model, hidden: torch.Tensor) -> None:
+    """hidden: CUDA tensor [n_layers + 1, rows, d] in the model dtype; filled by the next verify call."""
+    assert hidden.is_cuda and hidden.is_contiguous()
+    _check(_lib.aded_debug_capture_hidden(model.handle, _ptr(hidden)), "aded_debug_capture_hidden")
+
+
+def aded_debug_read_buffer(model: Model, which: int, rows: int) -> torch.Tensor:
+    """Activation buffer after the last call's last layer: 0 h, 1 x, 2 q, 3 attention output, 4 SwiGLU product."""
+    cfg = model.cfg
+    width = cfg.d_ffn if which == 4 else cfg.d_model
+    dt = torch.bfloat16 if cfg.dtype == ADED_BF16 else torch.float32
+    out = torch.empty((rows, width), dtype=dt, device="cuda")
+    _check(_lib.aded_debug_read_buffer(model.handle, c_int32(which), c_int32(rows), _ptr(out), _stream()),
+           "aded_debug_read_buffer")
+    return out
 
 
 ADED_NOALLOC_MAX_ROWS = 128

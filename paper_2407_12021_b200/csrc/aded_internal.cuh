@@ -136,6 +136,7 @@ struct aded_model {
 
     float* dbg_logits;
     int32_t* dbg_best;
+    void* dbg_hidden;   // [n_layers + 1][rows][d] copies of the residual stream (debug capture)
 
     bool att_mma;       // bf16 models: tensor-core split-KV attention kernel
 

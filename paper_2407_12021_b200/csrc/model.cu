@@ -174,6 +174,8 @@ static aded_status enqueue_pass(aded_model* m, aded_kv* kv, const int32_t* offse
         launch_rope_table(m, rows, st);
         launch_add_rmsnorm(m, (const GemmOut*)nullptr, m->layers[0].norm1, rows, st);
     }
+    const size_t hid_bytes = (size_t)rows * d * m->elem;
+    if (m->dbg_hidden) ADED_CUDA_TRY(cudaMemcpyAsync(m->dbg_hidden, m->h, hid_bytes, cudaMemcpyDeviceToDevice, st));
     for (int l = 0; l < c.n_layers; ++l) {
         const aded_layer_weights& w = m->layers[l];
         GemmOut o;
@@ -191,6 +193,9 @@ static aded_status enqueue_pass(aded_model* m, aded_kv* kv, const int32_t* offse
         } }
         const void* next_gain = l + 1 < c.n_layers ? m->layers[l + 1].norm1 : m->top.final_norm;
         { Span sp(m, PROF_OTHER, 1, st); launch_add_rmsnorm(m, &o, next_gain, rows, st); }
+        if (m->dbg_hidden)
+            ADED_CUDA_TRY(cudaMemcpyAsync((char*)m->dbg_hidden + (size_t)(l + 1) * hid_bytes, m->h, hid_bytes,
+                                          cudaMemcpyDeviceToDevice, st));
     }
     if (!chain_mode) {
         GemmOut lg;
@@ -257,11 +262,12 @@ static aded_status forward(aded_model* m, aded_kv* kv, const int32_t* tokens, co
 
     cudaStreamCaptureStatus cap_state = cudaStreamCaptureStatusNone;
     cudaStreamIsCapturing(st, &cap_state);
-    const bool direct = !m->graphs_on || m->dbg_logits || m->dbg_best || cap_state != cudaStreamCaptureStatusNone;
+    const bool direct = !m->graphs_on || m->dbg_logits || m->dbg_best || m->dbg_hidden || cap_state != cudaStreamCaptureStatusNone;
     if (direct) {
         aded_status s = enqueue_pass(m, kv, offsets_host, batch, rows, max_tree, chain_mode, st);
         m->dbg_logits = nullptr;
         m->dbg_best = nullptr;
+        m->dbg_hidden = nullptr;
         return s;
     }
     std::vector<int64_t> key;
@@ -350,6 +356,7 @@ aded_status aded_model_create(const aded_model_config* cfg, const aded_weights* 
     m->elem = cfg->dtype == ADED_BF16 ? 2 : 4;
     m->dbg_logits = nullptr;
     m->dbg_best = nullptr;
+    m->dbg_hidden = nullptr;
     m->prof_on = false;
     m->capture_spans = nullptr;
     m->prof_pending = -1;
@@ -571,6 +578,21 @@ aded_status aded_debug_gemm(aded_model* m, int32_t layer, int32_t which, const v
     const GemmOut o = launch_gemm(m, w_map, x_map, xbuf, w, ybuf, rows, n, k, st);
     launch_materialize(m, o, y_dev, rows, st);
     ADED_CUDA_TRY(cudaGetLastError());
+    return ADED_OK;
+}
+
+aded_status aded_debug_capture_hidden(aded_model* m, void* hidden_dev) {
+    if (!m) return ADED_ERR_INVALID_ARG;
+    m->dbg_hidden = hidden_dev;
+    return ADED_OK;
+}
+
+aded_status aded_debug_read_buffer(aded_model* m, int32_t which, int32_t rows, void* out_dev, void* stream) {
+    if (!m || !out_dev || which < 0 || which > 4 || rows < 1 || rows > m->cfg.max_rows) return ADED_ERR_INVALID_ARG;
+    const void* src = which == 0 ? m->h : which == 1 ? m->x : which == 2 ? m->q : which == 3 ? m->attn : m->act;
+    const size_t width = which == 4 ? m->cfg.d_ffn : m->cfg.d_model;
+    ADED_CUDA_TRY(cudaMemcpyAsync(out_dev, src, (size_t)rows * width * m->elem, cudaMemcpyDeviceToDevice,
+                                  static_cast<cudaStream_t>(stream)));
     return ADED_OK;
 }
 
