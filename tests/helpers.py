@@ -73,10 +73,15 @@ def compare_step(shape, gpu: Dict, cpu: Dict, tokens, parents, where: str = "") 
     rel = np.max(np.abs(lg - lc), axis=1) / np.max(np.abs(lc), axis=1)
     assert np.all(rel <= tol), f"{where}: logits off by {rel.max():.3e} (row {int(rel.argmax())}), tolerance {tol}"
     margin = ov.top2_margin(lc)
+    delta = np.max(np.abs(lg - lc), axis=1)            # measured logit deviation of every row
     diff = np.nonzero(gpu["best"] != cpu["best"])[0]
     for i in diff:
-        assert margin[i] < MARGIN_EXEMPT, (f"{where}: greedy token of node {i} differs "
-                                           f"({gpu['best'][i]} vs {cpu['best'][i]}) with top-2 margin {margin[i]:.3e}")
+        # A different greedy token is acceptable only at a near-tie: the checker's margin is below the
+        # fixed threshold, or below what this row's measured logit deviation (itself inside the logit
+        # tolerance, checked above) can explain -- two logits can each move by delta.
+        assert margin[i] < max(MARGIN_EXEMPT, 2 * delta[i]), (
+            f"{where}: greedy token of node {i} differs ({gpu['best'][i]} vs {cpu['best'][i]}) with top-2 margin "
+            f"{margin[i]:.3e}, logit deviation {delta[i]:.3e}")
     # the accepted sequence must equal the checker's walk over the GPU's own per-node choices;
     # when no node differed that is the checker's answer itself
     path, out = ov.accept_walk(tokens, parents, gpu["best"])
@@ -84,7 +89,9 @@ def compare_step(shape, gpu: Dict, cpu: Dict, tokens, parents, where: str = "") 
     assert gpu["accept_len"] == len(out)
     if len(diff) == 0:
         assert gpu["out_tokens"] == cpu["out_tokens"] and gpu["accept_len"] == cpu["accept_len"]
-    return {"logit_rel": float(rel.max()), "flipped": int(len(diff)), "min_margin": float(margin.min())}
+    beyond = int(sum(margin[i] >= MARGIN_EXEMPT for i in diff))
+    return {"logit_rel": float(rel.max()), "flipped": int(len(diff)), "flipped_beyond_1e-2": beyond,
+            "min_margin": float(margin.min())}
 
 
 def compare_cache(shape, sess: GpuSession, cache: ov.Cache, pos0: int, n: int, layers: Sequence[int], where=""):

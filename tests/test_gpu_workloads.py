@@ -25,8 +25,12 @@ def _oracle_cache_from_gpu(sess, arch, n_pos):
 
 def test_c3_full_7b_decode_sampled_step(cuda_device):
     """Workload 3 at full size: 32 layers, 2048-token Zipf prompt, 64-node trees built from the GPU
-    tri-gram top-4 lists, table updated every step.  Tri-gram results are compared at every step,
-    the verification at one sampled step (the checker re-runs it from the GPU's cache)."""
+    tri-gram top-4 lists, table updated every step.  Tri-gram results are compared at every lookup.
+    The verification is compared at one sampled step, teacher-forced layer by layer: a random-init
+    bf16 network amplifies one-ulp differences (a 1 % disagreement in attention outputs becomes a 50 %
+    disagreement in SwiGLU outputs one layer on), so end-to-end logits drift apart with depth whatever
+    the implementation; instead every checked layer is re-run by the checker from the hidden states and
+    cache the device actually had, and the LM head from the device's final hidden states."""
     from paper_2407_12021_b200 import binding as B
     wl = gen.WORKLOADS["c3"]
     shape = wl.shape
@@ -55,15 +59,44 @@ def test_c3_full_7b_decode_sampled_step(cuda_device):
         tokens, parents, _ = gen.expand_tree_from_topk(prev_tok, root_tok, topk_gpu, 64, 6, shape.vocab, 400 + step)
         L = sess.length()
         if step == sampled:
-            cache = _oracle_cache_from_gpu(sess, arch, L)
-            cpu = ov.verify(arch, ow, cache, tokens, parents)
+            check_layers = [0, 1, 15, 31]
+            before = {l: B.aded_kv_read(sess.kv, 0, l, 0, L) for l in check_layers}   # the cache the step starts from
+            hidden = torch.empty((shape.n_layers + 1, 64, shape.d_model), dtype=torch.bfloat16, device=cuda_device)
+            B.aded_debug_capture_hidden(sess.model, hidden)
         gpu = sess.verify(tokens, parents, capture=(step == sampled))
         assert gpu["status"] == 0 and gpu["accept_len"] >= 1
         if step == sampled:
-            worst = H.compare_step(shape, gpu, cpu, tokens, parents, "c3 sampled step")
-            print("c3 sampled step:", worst)
-            if worst["flipped"] == 0:
-                H.compare_cache(shape, sess, cache, L, cpu["accept_len"], [0, 15, 31], "c3 cache")
+            paths, depth = ov.paths_and_depths(parents)
+            pos = L + np.asarray(depth)
+            hid = hidden.double().cpu().numpy()
+            emb = ow.embed_rows(tokens)
+            assert np.array_equal(hid[0], emb)                       # embedding rows are copies
+            for l in check_layers:
+                kc, vc = (t.double().cpu().numpy() for t in before[l])
+                h_out, k, v = ov.decoder_layer(arch, ow.layer(l), kc, vc, hid[l], paths, pos)
+                err = np.abs(h_out - hid[l + 1])
+                rel_max = err.max() / np.abs(h_out).max()
+                rel_rms = np.sqrt((err ** 2).mean() / (h_out ** 2).mean())
+                print(f"c3 layer {l}: max {rel_max:.3e} rms {rel_rms:.3e} differing {np.mean(err > 0):.3f}")
+                assert rel_max <= 2e-2 and rel_rms <= 1e-2, (l, rel_max, rel_rms)
+            # LM head and greedy choice from the device's own final hidden states
+            lc = ov.lm_head(arch, ow, hid[shape.n_layers])
+            step_cpu = {"logits": lc, "best": ov.greedy(lc)}
+            step_cpu["out_tokens"] = ov.accept_walk(tokens, parents, step_cpu["best"])[1]
+            step_cpu["accept_len"] = len(step_cpu["out_tokens"])
+            worst = H.compare_step(shape, gpu, step_cpu, tokens, parents, "c3 LM head")
+            print("c3 LM head from device hidden states:", worst)
+            assert worst["logit_rel"] <= 2e-3 and worst["flipped_beyond_1e-2"] == 0
+            # end to end (all 32 layers in the checker, from the device's cache): reported, loosely bounded
+            cache = ov.Cache(arch)
+            for l in range(shape.n_layers):
+                kk, vv = (before[l] if l in before else B.aded_kv_read(sess.kv, 0, l, 0, L))
+                cache.load(l, kk, vv)
+            full = ov.verify(arch, ow, cache, tokens, parents)
+            rel = np.max(np.abs(gpu["logits"] - full["logits"]), axis=1) / np.max(np.abs(full["logits"]), axis=1)
+            print(f"c3 end-to-end logit deviation over 32 layers: max {rel.max():.3e} median {np.median(rel):.3e}; "
+                  f"greedy tokens equal on {int(np.sum(gpu['best'] == full['best']))}/64 nodes")
+            assert rel.max() < 0.15
         span = [prev_tok, root_tok] + gpu["out_tokens"]
         st.update(span)
         B.aded_trigram_update(tg, H.i32(span))
