@@ -284,7 +284,7 @@ def run_ours(args, rank, world):
         "launches": launches, "h2d": h2d / steps, "d2h": d2h / steps, "setup_s": setup_s,
         "roofline": {"bound": "hbm", "kernel": "projection/FFN/LM-head GEMM", "achieved": round(achieved, 1),
                      "peak": pk["hbm_gbs"], "peak_source": pk["source"], "unit": "GB/s",
-                     "frac": round(achieved / pk["hbm_gbs"], 4), "traffic": None,
+                     "frac": round(achieved / pk["hbm_gbs"], 4), "traffic": gemm_traffic_per_launch(shape),
                      "algorithmic_bytes_per_launch": gemm_bytes_step // gemm_launches_step,
                      "avg_launch_us": round(gemm_ms_launch * 1e3, 2),
                      "time_share": {k: round(v / max(sum(prof_ms.values()), 1e-9), 4) for k, v in prof_ms.items()},
@@ -326,6 +326,39 @@ def cpu_oracle_sample(shape, wl, weights, context, layers_timed=2, threads=None)
     return step_s, f"1 verify step ({wl.tree_nodes}-node tree, context {context}): {sub.n_layers} of {shape.n_layers} layers + LM head timed ({t_layers + t_head:.1f} s), scaled to {shape.n_layers} layers"
 
 
+def aggregate_over_ranks(ms, e2e_ms, accepted, world, device):
+    """Replicas are independent: the job's time is the slowest rank's, its tokens the sum over ranks."""
+    if world <= 1:
+        return ms, e2e_ms, accepted
+    t = torch.tensor([ms, e2e_ms], dtype=torch.float64, device=device)
+    torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
+    a = torch.tensor([accepted], dtype=torch.float64, device=device)
+    torch.distributed.all_reduce(a, op=torch.distributed.ReduceOp.SUM)
+    return float(t[0]), float(t[1]), float(a[0])
+
+
+def gemm_traffic_per_launch(shape):
+    """DRAM bytes per GEMM launch from the committed ncu capture (profiles/k_gemm_ws_traffic.json), averaged
+    over the launches of one step; None when the capture does not belong to the current kernel source."""
+    import hashlib
+    path = os.path.join(ROOT, "profiles", "k_gemm_ws_traffic.json")
+    src = os.path.join(ROOT, "paper_2407_12021_b200", "csrc", "gemm_ws.cu")
+    if not (os.path.exists(path) and os.path.exists(src)):
+        return None
+    with open(path) as f:
+        rec = json.load(f)
+    with open(src, "rb") as f:
+        if hashlib.sha256(f.read()).hexdigest() != rec.get("gemm_ws_sha256"):
+            return None
+    per = rec.get("dram_bytes_per_launch", {})
+    d, f_, v = shape.d_model, shape.d_ffn, shape.vocab
+    keys = [f"{3 * d}x{d}", f"{d}x{d}", f"{2 * f_}x{d}", f"{d}x{f_}", f"{v}x{d}"]
+    if any(k not in per for k in keys):
+        return None
+    total = shape.n_layers * sum(per[k] for k in keys[:4]) + per[keys[4]]
+    return int(total / (4 * shape.n_layers + 1))
+
+
 def main():
     args = parse_args()
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -362,15 +395,9 @@ def main():
     if world > 1:
         torch.distributed.init_process_group("nccl", device_id=torch.device("cuda", int(os.environ.get("LOCAL_RANK", 0))))
     res = run_ours(args, rank, world)
-    ms, e2e_ms, acc = res["ms"], res["e2e_ms"], res["accepted"]
-    if world > 1:
-        t = torch.tensor([ms, e2e_ms], dtype=torch.float64, device="cuda")
-        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
-        a = torch.tensor([acc], dtype=torch.float64, device="cuda")
-        torch.distributed.all_reduce(a, op=torch.distributed.ReduceOp.SUM)
-        ms, e2e_ms, acc_total = float(t[0]), float(t[1]), float(a[0])
-    else:
-        acc_total = acc
+    acc = res["accepted"]
+    ms, e2e_ms, acc_total = aggregate_over_ranks(res["ms"], res["e2e_ms"], acc, world,
+                                                 torch.device("cuda", int(os.environ.get("LOCAL_RANK", 0))))
     if rank != 0:
         torch.distributed.destroy_process_group()
         return

@@ -187,9 +187,8 @@ void launch_rope_table(aded_model* m, int rows, cudaStream_t st);
 void launch_add_rmsnorm(aded_model* m, const GemmOut* y, const void* gain, int rows, cudaStream_t st);
 // w_map / x_map: indices into m->ws_maps of the operands' TMA descriptors (-1: none, plain kernel).
 // `y` is the fp32 buffer the plain kernel writes; the returned descriptor says where the result is.
-// next_map / next_n / next_k: the projection that runs after this one (-1: none), for L2 prefetch.
 GemmOut launch_gemm(aded_model* m, int w_map, int x_map, const void* x, const void* w, float* y, int rows, int n, int k,
-                    cudaStream_t st, int next_map = -1, int next_n = 0, int next_k = 0);
+                    cudaStream_t st);
 void launch_rope_kv(aded_model* m, aded_kv* kv, const GemmOut& qkv, int layer, int rows, cudaStream_t st);
 void launch_swiglu(aded_model* m, const GemmOut& gu, int rows, cudaStream_t st);
 void launch_argmax(aded_model* m, const GemmOut& logits, int rows, cudaStream_t st);
@@ -209,11 +208,8 @@ bool attn_prepare();
 int ws_grid_limit(int device);
 int ws_grid(int device, int n, int k);
 size_t ws_slot_floats(int device, int max_n, int max_rows);
-// map_next (may be NULL): weights of the projection that follows, [next_n, next_k]; its first tiles
-// are prefetched into L2 at the end of this launch
 cudaError_t ws_launch(const CUtensorMap& map_w, const CUtensorMap& map_x, int rows, int row0, int n, int k,
-                      float* slots, int32_t* status, int device, cudaStream_t st, const CUtensorMap* map_next,
-                      int next_n, int next_k);
+                      float* slots, int32_t* status, int device, cudaStream_t st);
 enum { WS_MAP_QKV = 0, WS_MAP_O = 1, WS_MAP_GU = 2, WS_MAP_D = 3 };   // per-layer map order
 
 // tree_attention.cu

@@ -291,7 +291,7 @@ static void launch_gemm_plain(aded_model* m, const void* x, const void* w, float
 }
 
 GemmOut launch_gemm(aded_model* m, int w_map, int x_map, const void* x, const void* w, float* y, int rows, int n, int k,
-                    cudaStream_t st, int next_map, int next_n, int next_k) {
+                    cudaStream_t st) {
     GemmOut out = {};
     out.n = n;
     out.rows = rows;
@@ -299,9 +299,7 @@ GemmOut launch_gemm(aded_model* m, int w_map, int x_map, const void* x, const vo
         // tensor-core path, 128 rows of x per pass over the weights; the result stays in slots
         for (int row0 = 0; row0 < rows; row0 += 128) {
             const int part = rows - row0 < 128 ? rows - row0 : 128;
-            const bool last_pass = row0 + 128 >= rows;
-            ws_launch(m->ws_maps[w_map], m->ws_maps[x_map], part, row0, n, k, m->ws_slots, m->status, m->device, st,
-                      last_pass && next_map >= 0 ? &m->ws_maps[next_map] : nullptr, next_n, next_k);
+            ws_launch(m->ws_maps[w_map], m->ws_maps[x_map], part, row0, n, k, m->ws_slots, m->status, m->device, st);
         }
         out.mode = 1;
         out.slots = m->ws_slots;

@@ -16,7 +16,8 @@
 //     timing, and the GEMM itself ends without counters, fences or dependent reads;
 //   * the kernel is launched with programmatic dependent launch: its blocks become resident while
 //     the previous kernel drains, set up barriers and TMEM, and already stream their first W tiles;
-//     only the loads of x wait for the previous kernel;
+//     only the loads of x wait for the previous kernel.  (Also tried: TMA L2 prefetches of the next
+//     projection's first tiles at the end of the kernel -- no measurable gain, removed.)
 //   * warp 0 issues TMA loads, warp 1 issues MMAs, warps 2..5 drain TMEM and run the epilogue; two
 //     TMEM accumulators let the MMAs of the next segment run under the epilogue of the last.
 // Every mbarrier wait is bounded; a wait that runs out raises ADED_ERR_TIMEOUT in the status word
@@ -45,10 +46,6 @@ struct WsParams {
     int tmem_cols;       // power of two >= 2 * rb
     float* slots;        // this row block's slot region: [n_tiles + gridDim.x][rb][128] fp32
     int32_t* status;
-    // L2 prefetch of the weights the NEXT projection will read first (0 units: none)
-    int pf_units;        // units per CTA of the next GEMM to prefetch
-    int pf_tiles, pf_kb; // its tile and k-block counts
-    int pf_grid;         // its CTA count
 };
 
 // ---- PTX wrappers -------------------------------------------------------------------------
@@ -89,9 +86,6 @@ __device__ __forceinline__ void tma_load_2d_hint(const CUtensorMap* map, uint64_
         "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%3, %4}], [%2], %5;"
         ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "l"(policy) : "memory");
 }
-__device__ __forceinline__ void tma_prefetch_l2_2d(const CUtensorMap* map, int c0, int c1) {
-    asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global.tile [%0, {%1, %2}];" ::"l"(map), "r"(c0), "r"(c1) : "memory");
-}
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_commit(uint64_t* bar) {
@@ -129,8 +123,7 @@ __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr) {
 }
 
 __global__ void __launch_bounds__(WS_THREADS, 2)
-k_gemm_ws(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_x,
-          const __grid_constant__ CUtensorMap map_next, WsParams p) {
+k_gemm_ws(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_x, WsParams p) {
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     // carve: stages x (W tile 16 KB | x tile rb*128 B), then barriers
     uint8_t* base = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
@@ -202,16 +195,6 @@ k_gemm_ws(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUt
                 tma_load_2d_hint(&map_w, &full[s], sa, kb * WS_BK, tile * WS_BM, pol_stream);
                 for (int r = 0; r < p.rb; r += 16) tma_load_2d(&map_x, &full[s], sb + r * 128, kb * WS_BK, p.row0 + r);
                 if (++s == p.stages) { s = 0; ph ^= 1; }
-            }
-            // HBM would idle during the short kernels that follow: ask L2 for the first W tiles each
-            // CTA of the next projection will want (its work split is known in advance).
-            if (p.pf_units > 0 && (int)blockIdx.x < p.pf_grid) {
-                const long long nu = (long long)p.pf_tiles * p.pf_kb;
-                const long long n0 = ws_start(blockIdx.x, nu, p.pf_grid);
-                long long n1 = ws_start(blockIdx.x + 1, nu, p.pf_grid);
-                if (n1 > n0 + p.pf_units) n1 = n0 + p.pf_units;
-                for (long long u = n0; u < n1; ++u)
-                    tma_prefetch_l2_2d(&map_next, (int)(u % p.pf_kb) * WS_BK, (int)(u / p.pf_kb) * WS_BM);
             }
         }
     } else if (warp == 1) {
@@ -361,8 +344,7 @@ bool ws_supported(int n, int k) { return n % WS_BM == 0 && k % WS_BK == 0 && k >
 // One pass: rows [row0, row0 + rows) of x (rows <= 128) against all of W.  Partial tiles go to the
 // slot region of row block row0 / 128.
 cudaError_t ws_launch(const CUtensorMap& map_w, const CUtensorMap& map_x, int rows, int row0, int n, int k,
-                      float* slots, int32_t* status, int device, cudaStream_t st, const CUtensorMap* map_next,
-                      int next_n, int next_k) {
+                      float* slots, int32_t* status, int device, cudaStream_t st) {
     WsParams p;
     p.rows = rows;
     p.rb = (rows + 15) / 16 * 16;
@@ -381,16 +363,8 @@ cudaError_t ws_launch(const CUtensorMap& map_w, const CUtensorMap& map_x, int ro
     const int grid = ws_grid(device, n, k);
     p.slots = slots + (size_t)(row0 / 128) * (size_t)(p.n_tiles + grid) * 128 * WS_BM;
     p.status = status;
-    p.pf_units = 0;
-    p.pf_tiles = p.pf_kb = p.pf_grid = 1;
-    if (map_next != nullptr && ws_supported(next_n, next_k)) {
-        p.pf_units = 6;
-        p.pf_tiles = next_n / WS_BM;
-        p.pf_kb = next_k / WS_BK;
-        p.pf_grid = ws_grid(device, next_n, next_k);
-    }
     const size_t smem = (size_t)p.stages * stage_bytes + 1024 + 256;
-    return launch_k(k_gemm_ws, dim3(grid), dim3(WS_THREADS), smem, st, map_w, map_x, map_next ? *map_next : map_w, p);
+    return launch_k(k_gemm_ws, dim3(grid), dim3(WS_THREADS), smem, st, map_w, map_x, p);
 }
 
 }  // namespace aded

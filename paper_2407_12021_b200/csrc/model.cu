@@ -179,18 +179,14 @@ static aded_status enqueue_pass(aded_model* m, aded_kv* kv, const int32_t* offse
     for (int l = 0; l < c.n_layers; ++l) {
         const aded_layer_weights& w = m->layers[l];
         GemmOut o;
-        { Span sp(m, PROF_GEMM, 1, st); o = launch_gemm(m, 4 * l + WS_MAP_QKV, xm, m->x, w.wqkv, m->y32, rows, 3 * d, d, st, 4 * l + WS_MAP_O, d, d); }
+        { Span sp(m, PROF_GEMM, 1, st); o = launch_gemm(m, 4 * l + WS_MAP_QKV, xm, m->x, w.wqkv, m->y32, rows, 3 * d, d, st); }
         { Span sp(m, PROF_OTHER, 1, st); launch_rope_kv(m, kv, o, l, rows, st); }
         { Span sp(m, PROF_ATTN, 1, st); launch_tree_attention(m, kv, l, batch, rows, max_tree, st); }
-        { Span sp(m, PROF_GEMM, 1, st); o = launch_gemm(m, 4 * l + WS_MAP_O, xm + 1, m->attn, w.wo, m->y32, rows, d, d, st, 4 * l + WS_MAP_GU, 2 * F, d); }
+        { Span sp(m, PROF_GEMM, 1, st); o = launch_gemm(m, 4 * l + WS_MAP_O, xm + 1, m->attn, w.wo, m->y32, rows, d, d, st); }
         { Span sp(m, PROF_OTHER, 1, st); launch_add_rmsnorm(m, &o, w.norm2, rows, st); }
-        { Span sp(m, PROF_GEMM, 1, st); o = launch_gemm(m, 4 * l + WS_MAP_GU, xm, m->x, w.wgu, m->y32, rows, 2 * F, d, st, 4 * l + WS_MAP_D, d, F); }
+        { Span sp(m, PROF_GEMM, 1, st); o = launch_gemm(m, 4 * l + WS_MAP_GU, xm, m->x, w.wgu, m->y32, rows, 2 * F, d, st); }
         { Span sp(m, PROF_OTHER, 1, st); launch_swiglu(m, o, rows, st); }
-        { Span sp(m, PROF_GEMM, 1, st); {
-            const bool more = l + 1 < c.n_layers;
-            const int nm = more ? 4 * (l + 1) + WS_MAP_QKV : (chain_mode ? -1 : 4 * c.n_layers);
-            o = launch_gemm(m, 4 * l + WS_MAP_D, xm + 2, m->act, w.wd, m->y32, rows, d, F, st, nm, more ? 3 * d : c.vocab, d);
-        } }
+        { Span sp(m, PROF_GEMM, 1, st); o = launch_gemm(m, 4 * l + WS_MAP_D, xm + 2, m->act, w.wd, m->y32, rows, d, F, st); }
         const void* next_gain = l + 1 < c.n_layers ? m->layers[l + 1].norm1 : m->top.final_norm;
         { Span sp(m, PROF_OTHER, 1, st); launch_add_rmsnorm(m, &o, next_gain, rows, st); }
         if (m->dbg_hidden)
