@@ -6,7 +6,7 @@
 //
 // bf16 models: split-KV kernel on tensor cores.  A CTA owns (sequence, head, key split); each of
 // its warps owns 16 tree nodes (query rows) and walks the split's keys in blocks of 64 that all
-// warps share through shared memory (double-buffered cp.async).  Scores S = Q K^T and O += P V
+// warps share through shared memory (three-deep cp.async pipeline).  Scores S = Q K^T and O += P V
 // are m16n8k16 bf16 MMAs with fp32 accumulators; the online softmax keeps a running reference and
 // sum per row in registers (quad shuffles).  Numerators are 2^(t - M) with t the score in the log2
 // domain and M = ceil(max t) an integer, rounded to bf16 for the P V product while the row sum keeps
@@ -80,6 +80,7 @@ __global__ void __launch_bounds__(128) k_tree_attn_plain(
 // tensor-core split-KV kernel (bf16)
 // ------------------------------------------------------------------------------------------
 constexpr int TA_BLK = 64;   // keys per shared-memory block
+constexpr int TA_STAGES = 3; // key blocks in flight per CTA (cp.async pipeline depth)
 
 __device__ __forceinline__ void cp_async16(void* smem, const void* gmem) {
     const uint32_t s = (uint32_t)__cvta_generic_to_shared(smem);
@@ -136,8 +137,8 @@ __global__ void __launch_bounds__(NW * 32) k_tree_attn_mma(AttnArgs a) {
     constexpr int ONT = HD / 8;            // n tiles of the output
     constexpr int CHUNKS = HD / 8;         // 16-byte chunks per row
     extern __shared__ __align__(128) uint8_t smem_raw[];
-    bf16* sk = reinterpret_cast<bf16*>(smem_raw);                 // [2][TA_BLK][HD]
-    bf16* sv = sk + 2 * TA_BLK * HD;                              // [2][TA_BLK][HD]
+    bf16* sk = reinterpret_cast<bf16*>(smem_raw);                 // [TA_STAGES][TA_BLK][HD]
+    bf16* sv = sk + TA_STAGES * TA_BLK * HD;                      // [TA_STAGES][TA_BLK][HD]
 
     const int hh = blockIdx.x, split = blockIdx.y, b = blockIdx.z;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, tig = lane & 3;
@@ -195,11 +196,22 @@ __global__ void __launch_bounds__(NW * 32) k_tree_attn_mma(AttnArgs a) {
         cp_async_commit();
     };
 
-    if (blk0 < blk1) load_block(blk0, 0);   // (a split past the last key block has nothing to do but still joins the merge)
+    // Pipeline: TA_STAGES - 1 blocks are in flight while one is being used.  Every iteration commits
+    // exactly one group (an empty one past the end), so "all but the newest TA_STAGES - 2 groups have
+    // landed" always means the current block has.  (A split past the last key block has nothing to do
+    // but still joins the merge.)
+#pragma unroll
+    for (int s = 0; s < TA_STAGES - 1; ++s) {
+        if (blk0 + s < blk1) load_block(blk0 + s, s); else cp_async_commit();
+    }
     for (int blk = blk0; blk < blk1; ++blk) {
-        const int buf = (blk - blk0) & 1;
-        if (blk + 1 < blk1) { load_block(blk + 1, buf ^ 1); cp_async_wait<1>(); } else { cp_async_wait<0>(); }
-        __syncthreads();
+        const int buf = (blk - blk0) % TA_STAGES;
+        cp_async_wait<TA_STAGES - 2>();
+        __syncthreads();                      // block `blk` is visible; everyone is done with block blk - 1
+        {
+            const int nxt = blk + TA_STAGES - 1;   // goes into the buffer block blk - 1 used
+            if (nxt < blk1) load_block(nxt, (nxt - blk0) % TA_STAGES); else cp_async_commit();
+        }
         bf16* tk = sk + (size_t)buf * TA_BLK * HD;
         bf16* tv = sv + (size_t)buf * TA_BLK * HD;
 
@@ -285,7 +297,6 @@ __global__ void __launch_bounds__(NW * 32) k_tree_attn_mma(AttnArgs a) {
                 mma_bf16_16816(oacc[2 * np + 1], pf[kk], vb[2], vb[3]);
             }
         }
-        __syncthreads();   // the buffer is refilled two iterations later by load_block(blk + 2, buf)
     }
     // ---- merge the splits of this (sequence, head) across the cluster ----
     // Every CTA parks its unnormalised partial (O, running max, sum) in its own shared memory; after a
@@ -358,7 +369,7 @@ __global__ void __launch_bounds__(NW * 32) k_tree_attn_mma(AttnArgs a) {
 
 template <int HD, int NW>
 static size_t attn_smem() {
-    const size_t kv = (size_t)4 * TA_BLK * HD * sizeof(bf16), merge = (size_t)NW * 16 * (HD + 2) * sizeof(float);
+    const size_t kv = (size_t)2 * TA_STAGES * TA_BLK * HD * sizeof(bf16), merge = (size_t)NW * 16 * (HD + 2) * sizeof(float);
     return kv > merge ? kv : merge;
 }
 
