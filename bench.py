@@ -297,7 +297,7 @@ def run_ours(args, rank, world):
     return result
 
 
-def cpu_oracle_sample(shape, wl, weights, context, layers_timed=2, threads=None):
+def cpu_oracle_sample(shape, wl, weights, context, layers_timed=6, threads=None):
     """Times the CPU checker on a bounded sample of one verify step: `layers_timed` decoder layers over
     the workload's tree and context, plus the LM head; scaled to the full depth."""
     import numpy as np
