@@ -159,6 +159,23 @@ def test_verify_host_entry_point(cuda_device):
     assert int(n[0]) == cpu["accept_len"] and out[:int(n[0])].tolist() == cpu["out_tokens"]
 
 
+def test_graph_replay_gives_the_same_steps(cuda_device, monkeypatch):
+    """A model created with ADED_GRAPH set captures the pass once per call shape and replays it; the
+    decoded steps must equal those of the checker, replay after replay."""
+    monkeypatch.setenv("ADED_GRAPH", "1")
+    shape, arch, ow, cache, sess, prompt = _c1_setup(cuda_device, seed=23)
+    monkeypatch.delenv("ADED_GRAPH")
+    root = prompt[-1]
+    for step in range(4):      # the same tree shape every step: one capture, three replays
+        tokens, parents = gen.make_tree(16, 4, 4, shape.vocab, 40 + step, root_token=root)
+        cpu = ov.verify(arch, ow, cache, tokens, parents)
+        gpu = sess.verify(tokens, parents, capture=False)
+        assert gpu["status"] == 0
+        assert gpu["accept_len"] == cpu["accept_len"] and gpu["out_tokens"] == cpu["out_tokens"], f"step {step}"
+        assert sess.length() == cache.length
+        root = cpu["out_tokens"][-1]
+
+
 def test_c2_one_7b_layer_bf16(cuda_device):
     """Workload 2: one Llama-2-7B-shaped layer + LM head in bf16, cache pre-filled with 1024 N(0,1)
     positions, 64-node depth-6 tree with branching <= 4."""
