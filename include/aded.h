@@ -251,6 +251,48 @@ aded_status aded_trigram_stats(const aded_trigram* t, uint64_t* out_entries_host
 /* Read and clear the store's device status word; synchronises `stream`. */
 aded_status aded_trigram_poll_status(aded_trigram* t, aded_status* out_host, void* stream);
 
+/* ---- draft retrieval and the decoding step on the device ------------------------------------
+ * Figure 1's loop -- update the tri-gram matrix, retrieve candidate continuations from it with the
+ * last two tokens of the text, hand them to the model as one prefix-sharing pseudo-sequence
+ * ("Draft Construction and Verification"), feed the model's output back -- without a host round
+ * trip between its stages. */
+#define ADED_DRAFT_MAX_K 8
+
+/* Draft tree of exactly n_nodes (1..ADED_MAX_NODES) nodes for the context
+ * (context_dev[0], context_dev[1]) = (second-last, last) token of the text.  Node 0 holds the last
+ * token.  Nodes are visited in index order; a visited node of depth < max_depth whose parent holds
+ * u and which holds w gets one child per entry of the top-k (k in 1..ADED_DRAFT_MAX_K) list of
+ * context (u, w), in rank order, appended at the end, until the tree is full: indices are
+ * breadth-first, parents[i] < i, siblings differ.  When the table runs dry the tree is completed
+ * from filler_dev[0 .. n_filler) (tokens in [0, vocab), supplied by the caller; the paper has no
+ * such step, it keeps the launch shape constant): nodes are visited round-robin and a visited
+ * node with depth < max_depth and fewer than k children gets the next filler token none of its
+ * children holds (tokens passed over are consumed).
+ * Outputs (device): tree_tokens[n_nodes], tree_parents[n_nodes], n_from_table[1] (may be NULL):
+ * how many nodes came from the table.  If the filler runs out or no node has room left the
+ * store's status word becomes ADED_ERR_INVALID_ARG and tree_tokens[0] is set to -1, which the
+ * verification step rejects.  Asynchronous on `stream`. */
+aded_status aded_draft_tree(const aded_trigram* t, const int32_t* context_dev, int32_t n_nodes, int32_t max_depth,
+                            int32_t k, const int32_t* filler_dev, int32_t n_filler, int32_t* tree_tokens_dev,
+                            int32_t* tree_parents_dev, int32_t* n_from_table_dev, void* stream);
+
+/* One decoding step, all on the device and asynchronous on `stream`:
+ *   aded_draft_tree from context_dev  ->  aded_verify (out_tokens_dev[n_nodes], out_accept_len_dev[1])
+ *   ->  aded_trigram_update over (context, emitted tokens)  ->  context_dev <- last two tokens of the
+ *   text after the step.
+ * A step whose verification failed (status word of the model set) emits nothing, leaves the cache,
+ * the table and the context as they were and writes accept length 0.  n_nodes <= max_rows.
+ * n_from_table_dev may be NULL. */
+aded_status aded_decode_step(aded_model* m, aded_kv* kv, aded_trigram* t, int32_t* context_dev, int32_t n_nodes,
+                             int32_t max_depth, int32_t k, const int32_t* filler_dev, int32_t n_filler,
+                             int32_t* out_tokens_dev, int32_t* out_accept_len_dev, int32_t* n_from_table_dev,
+                             void* stream);
+/* Same with the filler, the emitted tokens and the accept length in host memory (pinned for the
+ * copies to be asynchronous); n_filler <= 4 * ADED_MAX_NODES; returns after `stream` has finished. */
+aded_status aded_decode_step_host(aded_model* m, aded_kv* kv, aded_trigram* t, int32_t* context_dev, int32_t n_nodes,
+                                  int32_t max_depth, int32_t k, const int32_t* filler_host, int32_t n_filler,
+                                  int32_t* out_tokens_host, int32_t* out_accept_len_host, void* stream);
+
 const char* aded_status_string(aded_status s);
 
 #ifdef __cplusplus

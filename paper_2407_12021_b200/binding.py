@@ -27,7 +27,8 @@ EXPORTS = [
     "aded_kv_load", "aded_kv_set_len", "aded_kv_read", "aded_append", "aded_verify", "aded_verify_batch", "aded_verify_host",
     "aded_debug_capture", "aded_debug_capture_hidden", "aded_debug_gemm", "aded_debug_read_buffer", "aded_greedy_noalloc", "aded_profile_begin", "aded_profile_end", "aded_launch_count", "aded_model_poll_status", "aded_trigram_create", "aded_trigram_destroy",
     "aded_trigram_update", "aded_trigram_update_host", "aded_trigram_topk", "aded_trigram_topk_host",
-    "aded_trigram_get", "aded_trigram_stats", "aded_trigram_poll_status", "aded_status_string",
+    "aded_trigram_get", "aded_trigram_stats", "aded_trigram_poll_status", "aded_draft_tree", "aded_decode_step",
+    "aded_decode_step_host", "aded_status_string",
 ]
 
 
@@ -373,6 +374,60 @@ def aded_trigram_poll_status(t: Trigram) -> int:
     out = c_int32()
     _check(_lib.aded_trigram_poll_status(t.handle, ctypes.byref(out), _stream()), "aded_trigram_poll_status")
     return out.value
+
+
+def aded_draft_tree(t: Trigram, context_dev: torch.Tensor, n_nodes: int, max_depth: int, k: int,
+                    filler_dev: Optional[torch.Tensor], tree_tokens: torch.Tensor, tree_parents: torch.Tensor,
+                    n_from_table: Optional[torch.Tensor] = None) -> None:
+    """context_dev [2] int32 CUDA (second-last, last token); filler_dev int32 CUDA or None;
+    tree_tokens / tree_parents [n_nodes] int32 CUDA; n_from_table [1] int32 CUDA or None."""
+    _dev_i32(context_dev, "context"), _dev_i32(tree_tokens, "tree_tokens"), _dev_i32(tree_parents, "tree_parents")
+    if context_dev.numel() < 2 or tree_tokens.numel() < n_nodes or tree_parents.numel() < n_nodes:
+        raise ValueError("arrays are too short")
+    nf = 0
+    if filler_dev is not None:
+        _dev_i32(filler_dev, "filler")
+        nf = filler_dev.numel()
+    if n_from_table is not None:
+        _dev_i32(n_from_table, "n_from_table")
+    _check(_lib.aded_draft_tree(t.handle, _ptr(context_dev), c_int32(n_nodes), c_int32(max_depth), c_int32(k),
+                                _ptr(filler_dev), c_int32(nf), _ptr(tree_tokens), _ptr(tree_parents),
+                                _ptr(n_from_table), _stream()), "aded_draft_tree")
+
+
+def aded_decode_step(model: Model, kv: KV, t: Trigram, context_dev: torch.Tensor, n_nodes: int, max_depth: int, k: int,
+                     filler_dev: Optional[torch.Tensor], out_tokens: torch.Tensor, out_accept_len: torch.Tensor,
+                     n_from_table: Optional[torch.Tensor] = None) -> None:
+    """One decoding step on the device; context_dev [2] int32 CUDA is read and advanced."""
+    _dev_i32(context_dev, "context"), _dev_i32(out_tokens, "out_tokens"), _dev_i32(out_accept_len, "out_accept_len")
+    if context_dev.numel() < 2 or out_tokens.numel() < n_nodes or out_accept_len.numel() < 1:
+        raise ValueError("arrays are too short")
+    nf = 0
+    if filler_dev is not None:
+        _dev_i32(filler_dev, "filler")
+        nf = filler_dev.numel()
+    if n_from_table is not None:
+        _dev_i32(n_from_table, "n_from_table")
+    _check(_lib.aded_decode_step(model.handle, kv.handle, t.handle, _ptr(context_dev), c_int32(n_nodes),
+                                 c_int32(max_depth), c_int32(k), _ptr(filler_dev), c_int32(nf), _ptr(out_tokens),
+                                 _ptr(out_accept_len), _ptr(n_from_table), _stream()), "aded_decode_step")
+
+
+def aded_decode_step_host(model: Model, kv: KV, t: Trigram, context_dev: torch.Tensor, n_nodes: int, max_depth: int,
+                          k: int, filler_host: Optional[torch.Tensor], out_tokens_host: torch.Tensor,
+                          out_accept_len_host: torch.Tensor) -> None:
+    """Same with filler, emitted tokens and accept length in (pinned) host memory; returns when done."""
+    _dev_i32(context_dev, "context"), _host_i32(out_tokens_host, "out_tokens"), _host_i32(out_accept_len_host, "out_accept_len")
+    if context_dev.numel() < 2 or out_tokens_host.numel() < n_nodes or out_accept_len_host.numel() < 1:
+        raise ValueError("arrays are too short")
+    nf = 0
+    if filler_host is not None:
+        _host_i32(filler_host, "filler")
+        nf = filler_host.numel()
+    _check(_lib.aded_decode_step_host(model.handle, kv.handle, t.handle, _ptr(context_dev), c_int32(n_nodes),
+                                      c_int32(max_depth), c_int32(k), _ptr(filler_host), c_int32(nf),
+                                      _ptr(out_tokens_host), _ptr(out_accept_len_host), _stream()),
+           "aded_decode_step_host")
 
 
 def aded_status_string(status: int) -> str:

@@ -81,8 +81,10 @@ __global__ void k_tg_init(Bucket* b, size_t n) {
 
 // Algorithm 2, one thread per window.  Duplicate windows inside one call are independent atomic
 // adds, so the result is min(count + multiplicity, cap) whatever the thread order.
-__global__ void k_tg_update(TgView t, const int32_t* __restrict__ tok, int n) {
+// `n_dev` (may be NULL): the span length lives on the device (at most n).
+__global__ void k_tg_update(TgView t, const int32_t* __restrict__ tok, int n, const int32_t* __restrict__ n_dev) {
     const int i = blockIdx.x * blockDim.x + threadIdx.x + 2;
+    if (n_dev && *n_dev < n) n = *n_dev;
     if (i >= n || *t.status != 0) return;
     const int a = tok[i - 2], b = tok[i - 1], c = tok[i];
     if (a < 0 || b < 0 || c < 0 || a >= t.vocab || b >= t.vocab || c >= t.vocab) {
@@ -136,6 +138,36 @@ __global__ void k_tg_update(TgView t, const int32_t* __restrict__ tok, int n) {
     atomicCAS(t.status, 0, (int)ADED_ERR_TIMEOUT);
 }
 
+// One selection round of a warp over the chain that starts at `home`: the largest packed
+// (count, ~token) strictly below `prev`, or 0 when nothing is left; `total` = sum of the counts.
+__device__ __forceinline__ unsigned long long tg_select_round(const TgView& t, int64_t home, unsigned long long prev,
+                                                              int lane, uint32_t* total_out) {
+    unsigned long long best = 0;
+    uint32_t total = 0;
+    int64_t cur = home;
+    for (uint32_t hop = 0; cur >= 0 && hop <= t.n_over; ++hop) {
+        const Bucket* bk = t.buckets + cur;
+        if (lane < 6) {
+            const int32_t tk = bk->e[lane].tok;
+            const uint32_t cn = bk->e[lane].cnt;
+            if (tk >= 0) {
+                total += cn;
+                const unsigned long long key = ((unsigned long long)cn << 32) | (0xFFFFFFFFu - (uint32_t)tk);
+                if (cn >= t.min_count && cn > 0 && key < prev && key > best) best = key;
+            }
+        }
+        const uint32_t nxt = bk->next;
+        cur = nxt == 0 ? -1 : (int64_t)nxt;
+    }
+    for (int o = 16; o > 0; o >>= 1) {
+        const unsigned long long ob = __shfl_xor_sync(0xffffffffu, best, o);
+        if (ob > best) best = ob;
+        total += __shfl_xor_sync(0xffffffffu, total, o);
+    }
+    if (total_out) *total_out = total;
+    return best;
+}
+
 // One warp per query.  k selection rounds over the context's chain; a round picks the largest
 // packed (count, ~token) strictly below the previous pick, which yields count descending, token
 // ascending among equals, without storing the list.
@@ -149,34 +181,141 @@ __global__ void k_tg_topk(TgView t, const int32_t* __restrict__ ctx, int q, int 
     if (a >= 0 && b >= 0 && a < t.vocab && b < t.vocab) home = tg_find_home(t, tg_key(a, b), false);
     unsigned long long prev = ~0ull;
     for (int round = 0; round < k; ++round) {
-        unsigned long long best = 0;
-        uint32_t total = 0;
-        int64_t cur = home;
-        for (uint32_t hop = 0; cur >= 0 && hop <= t.n_over; ++hop) {
-            const Bucket* bk = t.buckets + cur;
-            if (lane < 6) {
-                const int32_t tk = bk->e[lane].tok;
-                const uint32_t cn = bk->e[lane].cnt;
-                if (tk >= 0) {
-                    total += cn;
-                    const unsigned long long key = ((unsigned long long)cn << 32) | (0xFFFFFFFFu - (uint32_t)tk);
-                    if (cn >= t.min_count && cn > 0 && key < prev && key > best) best = key;
-                }
-            }
-            const uint32_t nxt = bk->next;
-            cur = nxt == 0 ? -1 : (int64_t)nxt;
-        }
-        for (int o = 16; o > 0; o >>= 1) {
-            const unsigned long long ob = __shfl_xor_sync(0xffffffffu, best, o);
-            if (ob > best) best = ob;
-            total += __shfl_xor_sync(0xffffffffu, total, o);
-        }
+        uint32_t total;
+        const unsigned long long best = tg_select_round(t, home, prev, lane, &total);
         if (lane == 0) {
             out_tok[(size_t)w * k + round] = best ? (int32_t)(0xFFFFFFFFu - (uint32_t)best) : -1;
             out_cnt[(size_t)w * k + round] = (uint32_t)(best >> 32);
             if (round == 0 && out_total) out_total[w] = total;
         }
         prev = best ? best : 0;   // nothing left: later rounds find nothing either
+    }
+}
+
+// Draft tree of n_nodes nodes for the context (ctx[0], ctx[1]); one block of 32 warps.
+// Level by level: every node of the current level gets its top-k list (one warp per node), then
+// one thread appends the lists in node order, rank order -- the same tree as visiting the nodes in
+// index order.  The filler pass (one thread; child lists kept in shared memory) hangs caller-
+// supplied tokens under nodes with room, round-robin, until the tree is full.
+constexpr int DRAFT_MAX_FILLER = 4 * ADED_MAX_NODES;
+
+__global__ void __launch_bounds__(1024)
+k_draft_tree(TgView t, const int32_t* __restrict__ ctx, int n_nodes, int max_depth, int k,
+             const int32_t* __restrict__ filler, int n_filler, int32_t* __restrict__ out_tok,
+             int32_t* __restrict__ out_par, int32_t* __restrict__ out_real) {
+    __shared__ int32_t s_tok[ADED_MAX_NODES], s_par[ADED_MAX_NODES], s_dep[ADED_MAX_NODES], s_nkid[ADED_MAX_NODES];
+    __shared__ int32_t s_cand[ADED_MAX_NODES * ADED_DRAFT_MAX_K];   // top-k lists, later the child tokens of every node
+    __shared__ int32_t s_fill[DRAFT_MAX_FILLER];
+    __shared__ int s_n, s_lo, s_hi, s_fail;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int prev_token = ctx[0];
+    if (threadIdx.x == 0) {
+        s_tok[0] = ctx[1];
+        s_par[0] = -1;
+        s_dep[0] = 0;
+        s_n = 1;
+        s_lo = 0;
+        s_hi = 1;
+        s_fail = 0;
+    }
+    for (int i = threadIdx.x; i < n_filler; i += blockDim.x) s_fill[i] = filler[i];
+    for (int i = threadIdx.x; i < ADED_MAX_NODES; i += blockDim.x) s_nkid[i] = 0;
+    __syncthreads();
+    for (int d = 0; d < max_depth; ++d) {
+        const int lo = s_lo, hi = s_hi;
+        if (lo >= hi || s_n >= n_nodes) break;
+        for (int node = lo + warp; node < hi; node += 32) {
+            const int u = node == 0 ? prev_token : s_tok[s_par[node]], w = s_tok[node];
+            int64_t home = -1;
+            if (u >= 0 && w >= 0 && u < t.vocab && w < t.vocab) home = tg_find_home(t, tg_key(u, w), false);
+            unsigned long long prev = ~0ull;
+            for (int round = 0; round < k; ++round) {
+                const unsigned long long best = tg_select_round(t, home, prev, lane, nullptr);
+                if (lane == 0) s_cand[node * ADED_DRAFT_MAX_K + round] = best ? (int32_t)(0xFFFFFFFFu - (uint32_t)best) : -1;
+                prev = best ? best : 0;
+            }
+        }
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            int n = s_n;
+            for (int node = lo; node < hi && n < n_nodes; ++node) {
+                for (int j = 0; j < k && n < n_nodes; ++j) {
+                    const int32_t c = s_cand[node * ADED_DRAFT_MAX_K + j];
+                    if (c < 0) break;
+                    s_tok[n] = c;
+                    s_par[n] = node;
+                    s_dep[n] = d + 1;
+                    s_nkid[node] = j + 1;    // s_cand[node][0 .. j] are this node's child tokens
+                    ++n;
+                }
+            }
+            s_lo = hi;
+            s_hi = n;
+            s_n = n;
+        }
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) {
+        int n = s_n;
+        if (out_real) *out_real = n;
+        if (filler && n < n_nodes) {
+            int pos = 0, p = 0, idle = 0;
+            while (n < n_nodes) {
+                const int nk = s_nkid[p];
+                if (s_dep[p] < max_depth && nk < k) {
+                    int32_t f = -1;
+                    for (; pos < n_filler; ++pos) {
+                        f = s_fill[pos];
+                        bool clash = false;
+                        for (int j = 0; j < nk; ++j) clash |= s_cand[p * ADED_DRAFT_MAX_K + j] == f;
+                        if (!clash) break;
+                    }
+                    if (pos >= n_filler || f < 0 || f >= t.vocab) { s_fail = 1; break; }
+                    ++pos;
+                    s_cand[p * ADED_DRAFT_MAX_K + nk] = f;
+                    s_nkid[p] = nk + 1;
+                    s_tok[n] = f;
+                    s_par[n] = p;
+                    s_dep[n] = s_dep[p] + 1;
+                    s_nkid[n] = 0;
+                    ++n;
+                    idle = 0;
+                } else if (++idle > n) {
+                    s_fail = 1;
+                    break;
+                }
+                p = (p + 1) % n;
+            }
+            s_n = n;
+        }
+        if (s_fail) atomicCAS(t.status, 0, (int)ADED_ERR_INVALID_ARG);
+    }
+    __syncthreads();
+    const int n = s_n;
+    for (int i = threadIdx.x; i < n_nodes; i += blockDim.x) {
+        out_tok[i] = (i < n && !(s_fail && i == 0)) ? s_tok[i] : -1;
+        out_par[i] = i < n ? s_par[i] : -1;
+    }
+}
+
+// After a verification step: the span the table learns from (context + emitted tokens) and the
+// context of the next step.  A failed step (accept length < 1) leaves the context and an empty span.
+__global__ void k_decode_advance(const int32_t* __restrict__ out_tok, int32_t* __restrict__ out_len, int32_t* ctx,
+                                 int32_t* __restrict__ span, int32_t* __restrict__ span_len, int max_emit) {
+    __shared__ int32_t s_ctx[2];
+    int a = *out_len;
+    if (a > max_emit) a = max_emit;
+    if (threadIdx.x < 2) s_ctx[threadIdx.x] = ctx[threadIdx.x];
+    __syncthreads();
+    if (a < 1) {
+        if (threadIdx.x == 0) { *span_len = 0; *out_len = 0; }
+        return;
+    }
+    for (int i = threadIdx.x; i < a + 2; i += blockDim.x) span[i] = i < 2 ? s_ctx[i] : out_tok[i - 2];
+    if (threadIdx.x == 0) {
+        *span_len = a + 2;
+        ctx[0] = a >= 2 ? out_tok[a - 2] : s_ctx[1];
+        ctx[1] = out_tok[a - 1];
     }
 }
 
@@ -216,11 +355,15 @@ struct aded_trigram {
     uint32_t* stage_u;
     size_t stage_n;
     unsigned long long* stats_dev;
+    int32_t* step_i;     // decoding step: span [ADED_MAX_NODES + 2], span length [1], filler staging
 };
 
 using namespace aded;
 
 static constexpr size_t TG_STAGE = 1 << 16;
+// step_i layout: span, span length, tokens from the table, filler staging
+static constexpr int STEP_SPAN = 0, STEP_LEN = ADED_MAX_NODES + 2, STEP_REAL = STEP_LEN + 1, STEP_FILL = STEP_REAL + 1;
+static constexpr int STEP_INTS = STEP_FILL + DRAFT_MAX_FILLER;
 
 extern "C" {
 
@@ -235,6 +378,7 @@ aded_status aded_trigram_create(const aded_trigram_config* cfg, aded_trigram** o
     t->stage_i = nullptr;
     t->stage_u = nullptr;
     t->stats_dev = nullptr;
+    t->step_i = nullptr;
     t->view = TgView();
     const size_t n_home = (size_t)1 << cfg->log2_buckets, n = n_home + (size_t)cfg->overflow_buckets;
     bool ok = cudaGetDevice(&t->device) == cudaSuccess;
@@ -245,6 +389,7 @@ aded_status aded_trigram_create(const aded_trigram_config* cfg, aded_trigram** o
     if (ok) ok = cudaMalloc((void**)&t->stage_i, TG_STAGE * sizeof(int32_t)) == cudaSuccess;
     if (ok) ok = cudaMalloc((void**)&t->stage_u, TG_STAGE * sizeof(uint32_t)) == cudaSuccess;
     if (ok) ok = cudaMalloc((void**)&t->stats_dev, 2 * sizeof(unsigned long long)) == cudaSuccess;
+    if (ok) ok = cudaMalloc((void**)&t->step_i, STEP_INTS * sizeof(int32_t)) == cudaSuccess;
     if (!ok) {
         cudaGetLastError();
         aded_trigram_destroy(t);
@@ -276,6 +421,7 @@ aded_status aded_trigram_destroy(aded_trigram* t) {
     if (t->stage_i) cudaFree(t->stage_i);
     if (t->stage_u) cudaFree(t->stage_u);
     if (t->stats_dev) cudaFree(t->stats_dev);
+    if (t->step_i) cudaFree(t->step_i);
     delete t;
     return ADED_OK;
 }
@@ -285,7 +431,7 @@ aded_status aded_trigram_update(aded_trigram* t, const int32_t* tokens_dev, int3
     if (n < 3) return ADED_OK;
     const int windows = n - 2;
     note_launch();
-    k_tg_update<<<(windows + 255) / 256, 256, 0, static_cast<cudaStream_t>(stream)>>>(t->view, tokens_dev, n);
+    k_tg_update<<<(windows + 255) / 256, 256, 0, static_cast<cudaStream_t>(stream)>>>(t->view, tokens_dev, n, nullptr);
     ADED_CUDA_TRY(cudaGetLastError());
     return ADED_OK;
 }
@@ -343,6 +489,60 @@ aded_status aded_trigram_topk_host(const aded_trigram* t, const int32_t* ctx_hos
             ADED_CUDA_TRY(cudaMemcpyAsync(out_total_host + lo, tot_d, (size_t)qq * sizeof(uint32_t), cudaMemcpyDeviceToHost, st));
         ADED_CUDA_TRY(cudaStreamSynchronize(st));
     }
+    return ADED_OK;
+}
+
+aded_status aded_draft_tree(const aded_trigram* t, const int32_t* context_dev, int32_t n_nodes, int32_t max_depth,
+                            int32_t k, const int32_t* filler_dev, int32_t n_filler, int32_t* tree_tokens_dev,
+                            int32_t* tree_parents_dev, int32_t* n_from_table_dev, void* stream) {
+    if (!t || !context_dev || !tree_tokens_dev || !tree_parents_dev) return ADED_ERR_INVALID_ARG;
+    if (n_nodes < 1 || n_nodes > ADED_MAX_NODES || max_depth < 0 || k < 1 || k > ADED_DRAFT_MAX_K) return ADED_ERR_INVALID_ARG;
+    if (n_filler < 0 || n_filler > DRAFT_MAX_FILLER || (n_filler > 0 && !filler_dev)) return ADED_ERR_INVALID_ARG;
+    note_launch();
+    k_draft_tree<<<1, 1024, 0, static_cast<cudaStream_t>(stream)>>>(t->view, context_dev, n_nodes, max_depth, k,
+                                                                    n_filler > 0 ? filler_dev : nullptr, n_filler,
+                                                                    tree_tokens_dev, tree_parents_dev, n_from_table_dev);
+    ADED_CUDA_TRY(cudaGetLastError());
+    return ADED_OK;
+}
+
+aded_status aded_decode_step(aded_model* m, aded_kv* kv, aded_trigram* t, int32_t* context_dev, int32_t n_nodes,
+                             int32_t max_depth, int32_t k, const int32_t* filler_dev, int32_t n_filler,
+                             int32_t* out_tokens_dev, int32_t* out_accept_len_dev, int32_t* n_from_table_dev,
+                             void* stream) {
+    if (!m || !kv || !t || !context_dev || !out_tokens_dev || !out_accept_len_dev) return ADED_ERR_INVALID_ARG;
+    if (n_nodes < 1 || n_nodes > ADED_MAX_NODES || n_nodes > m->cfg.max_rows) return ADED_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    aded_status s = aded_draft_tree(t, context_dev, n_nodes, max_depth, k, filler_dev, n_filler, m->tokens, m->parents,
+                                    n_from_table_dev ? n_from_table_dev : t->step_i + STEP_REAL, stream);
+    if (s != ADED_OK) return s;
+    s = aded_verify(m, kv, m->tokens, m->parents, n_nodes, out_tokens_dev, out_accept_len_dev, stream);
+    if (s != ADED_OK) return s;
+    note_launch(2);
+    k_decode_advance<<<1, 160, 0, st>>>(out_tokens_dev, out_accept_len_dev, context_dev, t->step_i + STEP_SPAN,
+                                        t->step_i + STEP_LEN, n_nodes);
+    k_tg_update<<<(ADED_MAX_NODES + 255) / 256, 256, 0, st>>>(t->view, t->step_i + STEP_SPAN, n_nodes + 2,
+                                                              t->step_i + STEP_LEN);
+    ADED_CUDA_TRY(cudaGetLastError());
+    return ADED_OK;
+}
+
+aded_status aded_decode_step_host(aded_model* m, aded_kv* kv, aded_trigram* t, int32_t* context_dev, int32_t n_nodes,
+                                  int32_t max_depth, int32_t k, const int32_t* filler_host, int32_t n_filler,
+                                  int32_t* out_tokens_host, int32_t* out_accept_len_host, void* stream) {
+    if (!m || !t || !out_tokens_host || !out_accept_len_host) return ADED_ERR_INVALID_ARG;
+    if (n_filler < 0 || n_filler > DRAFT_MAX_FILLER || (n_filler > 0 && !filler_host)) return ADED_ERR_INVALID_ARG;
+    if (n_nodes < 1 || n_nodes > m->cfg.max_rows) return ADED_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (n_filler > 0)
+        ADED_CUDA_TRY(cudaMemcpyAsync(t->step_i + STEP_FILL, filler_host, (size_t)n_filler * sizeof(int32_t),
+                                      cudaMemcpyHostToDevice, st));
+    const aded_status s = aded_decode_step(m, kv, t, context_dev, n_nodes, max_depth, k, t->step_i + STEP_FILL, n_filler,
+                                           m->out_tokens, m->out_len, nullptr, stream);
+    if (s != ADED_OK) return s;
+    ADED_CUDA_TRY(cudaMemcpyAsync(out_tokens_host, m->out_tokens, (size_t)n_nodes * sizeof(int32_t), cudaMemcpyDeviceToHost, st));
+    ADED_CUDA_TRY(cudaMemcpyAsync(out_accept_len_host, m->out_len, sizeof(int32_t), cudaMemcpyDeviceToHost, st));
+    ADED_CUDA_TRY(cudaStreamSynchronize(st));
     return ADED_OK;
 }
 
