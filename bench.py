@@ -2,14 +2,14 @@
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c3|c2|c4] [--impl ours|reference]
 
-A step is one decode step of the loop: tri-gram top-k lookups for the draft tree, the 64-node tree
-verification (all layers, LM head, greedy choice, approval, cache compaction) and the tri-gram
-count update from the emitted tokens.  Two passes over the same deterministic decode:
-  * end to end: every call takes HOST buffers (`*_host` entry points), the draft tree is built on
-    the host from the returned top-k lists; this pass also records each step's tree;
-  * device resident: the cache and the table are rolled back, the recorded trees, lookup contexts
-    and update spans are uploaded once, and the same steps run from device memory only.  The
-    emitted tokens must equal the first pass's.
+A step is one decode step of the loop: the 64-node draft tree retrieved from the tri-gram table
+with the last two tokens of the text, its verification (all layers, LM head, greedy choice,
+approval, cache compaction), the tri-gram count update from the emitted tokens and the next
+context -- one library call, every stage on the device.  Two passes over the same deterministic decode:
+  * end to end: `aded_decode_step_host` -- the step's filler tokens come from pinned host memory,
+    the emitted tokens and the accept length are read back to the host before the next step starts;
+  * device resident: the cache and the table are rolled back and the same steps run through
+    `aded_decode_step` from device memory only.  The emitted tokens must equal the first pass's.
 With --gpus N every rank runs an independent replica (nothing in the step is exchanged).
 """
 from __future__ import annotations
@@ -96,39 +96,6 @@ class ClockSampler:
                 "reasons": reasons, "samples": len(sm)}
 
 
-def build_tree_host(B, tg, prev_tok, root_tok, wl, vocab, step, pin):
-    """Breadth-first draft tree from top-k lists, one host round trip per tree level."""
-    cache = {}
-
-    def lookup_level(ctxs):
-        q = len(ctxs)
-        pin["ctx"][:q] = torch.tensor(ctxs, dtype=torch.int32)
-        B.aded_trigram_topk_host(tg, pin["ctx"][:q], wl.topk, pin["tok"][:q], pin["cnt"][:q])
-        for i, c in enumerate(ctxs):
-            cache[c] = pin["tok"][i].tolist()
-
-    def topk(a, b):
-        if (a, b) not in cache:
-            lookup_level([(a, b)])
-        return cache[(a, b)]
-
-    # prefetch level by level: expand once to learn the frontier's contexts, batch the misses
-    frontier = [(prev_tok, root_tok)]
-    for _ in range(wl.tree_depth):
-        miss = [c for c in dict.fromkeys(frontier) if c not in cache]
-        if miss:
-            lookup_level(miss)
-        nxt = []
-        for (a, b) in frontier:
-            nxt += [(b, t) for t in cache[(a, b)] if t >= 0]
-        frontier = nxt[:wl.tree_nodes]
-        if not frontier:
-            break
-    tokens, parents, real = gen.expand_tree_from_topk(prev_tok, root_tok, topk, wl.tree_nodes, wl.tree_depth, vocab,
-                                                      SEED + step, fill=True)
-    return tokens, parents, real, list(cache.keys())
-
-
 def run_ours(args, rank, world):
     from paper_2407_12021_b200 import build as libbuild
     if rank == 0:
@@ -170,22 +137,19 @@ def run_ours(args, rank, world):
         return t
 
     n = wl.tree_nodes
-    pin = {"ctx": torch.empty((4 * n, 2), dtype=torch.int32).pin_memory(),
-           "tok": torch.empty((4 * n, wl.topk), dtype=torch.int32).pin_memory(),
-           "cnt": torch.empty((4 * n, wl.topk), dtype=torch.int32).pin_memory(),
-           "tree_tok": torch.empty(n, dtype=torch.int32).pin_memory(),
-           "tree_par": torch.empty(n, dtype=torch.int32).pin_memory(),
-           "out": torch.empty(n, dtype=torch.int32).pin_memory(),
-           "len": torch.empty(1, dtype=torch.int32).pin_memory(),
-           "span": torch.empty(n + 2, dtype=torch.int32).pin_memory()}
+    nf = 4 * n
+    fill_h = torch.stack([gen.zipf_tokens(nf, shape.vocab, SEED + rank, 9000 + s).to(torch.int32) for s in range(total)]).pin_memory()
+    fill_d = fill_h.to(dev)
+    out_h = torch.empty(n, dtype=torch.int32).pin_memory()
+    len_h = torch.empty(1, dtype=torch.int32).pin_memory()
+    ctx0 = prompt[-2:].to(torch.int32).to(dev)
 
-    # ---------------- pass 1: end to end through the *_host entry points; records the decode ----------
+    # ---------------- pass 1: end to end, one host-buffer call per step; records the decode ----------
     tg = fresh_table()
+    ctx = ctx0.clone()
     torch.cuda.synchronize()
     rec = []
-    prev_tok, root_tok = int(prompt[-2]), int(prompt[-1])
     ev = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
-    h2d = d2h = 0
     sampler = ClockSampler(dev.index or 0)
     accepted_e2e = 0
     for step in range(total):
@@ -194,45 +158,29 @@ def run_ours(args, rank, world):
                 torch.distributed.barrier()
             torch.cuda.synchronize()
             ev[0].record()
-            h2d = d2h = 0
-        tokens, parents, real, ctxs = build_tree_host(B, tg, prev_tok, root_tok, wl, shape.vocab, step, pin)
-        pin["tree_tok"][:] = torch.tensor(tokens, dtype=torch.int32)
-        pin["tree_par"][:] = torch.tensor(parents, dtype=torch.int32)
-        B.aded_verify_host(model, kv, pin["tree_tok"], pin["tree_par"], pin["out"], pin["len"])
-        a = int(pin["len"][0])
-        assert a >= 1, B.aded_model_poll_status(model)
-        out = pin["out"][:a].tolist()
-        span = [prev_tok, root_tok] + out
-        pin["span"][:len(span)] = torch.tensor(span, dtype=torch.int32)
-        B.aded_trigram_update_host(tg, pin["span"][:len(span)])
-        h2d += 4 * (2 * n + len(span) + 2 * len(ctxs))
-        d2h += 4 * (n + 1 + 2 * wl.topk * len(ctxs))
-        rec.append({"tokens": tokens, "parents": parents, "out": out, "ctxs": ctxs, "span": span, "real": real})
+        B.aded_decode_step_host(model, kv, tg, ctx, n, wl.tree_depth, wl.topk, fill_h[step], out_h, len_h)
+        a = int(len_h[0])
+        assert a >= 1, (B.aded_model_poll_status(model), B.aded_trigram_poll_status(tg))
+        rec.append(out_h[:a].tolist())
         if step >= warm:
             accepted_e2e += a
-        chain = [root_tok] + out
-        prev_tok, root_tok = chain[-2], chain[-1]
     ev[1].record()
     torch.cuda.synchronize()
     e2e_ms = ev[0].elapsed_time(ev[1])
+    h2d, d2h = 4 * nf, 4 * (n + 1)
     assert B.aded_trigram_poll_status(tg) == 0 and B.aded_model_poll_status(model) == 0
 
     # ---------------- pass 2: the same decode from device-resident inputs ---------------------------------
-    d_tok = torch.tensor([r["tokens"] for r in rec], dtype=torch.int32, device=dev)
-    d_par = torch.tensor([r["parents"] for r in rec], dtype=torch.int32, device=dev)
     d_out = torch.zeros((total, n), dtype=torch.int32, device=dev)
     d_len = torch.zeros((total, 1), dtype=torch.int32, device=dev)
-    d_ctx = [torch.tensor(r["ctxs"], dtype=torch.int32, device=dev) for r in rec]
-    d_span = [torch.tensor(r["span"], dtype=torch.int32, device=dev) for r in rec]
-    qmax = max(len(r["ctxs"]) for r in rec)
-    d_tk = torch.empty((qmax, wl.topk), dtype=torch.int32, device=dev)
-    d_cn = torch.empty((qmax, wl.topk), dtype=torch.int32, device=dev)
+    d_real = torch.zeros((total, 1), dtype=torch.int32, device=dev)
 
     def replay(profile):
-        """Rolls cache and table back to the end of the prompt and runs all steps from device memory.
-        profile=False is the timed run; profile=True repeats it with per-kernel event timing."""
+        """Rolls cache, table and context back to the end of the prompt and runs all steps from device
+        memory.  profile=False is the timed run; profile=True repeats it with per-kernel event timing."""
         B.aded_kv_set_len(kv, 0, base_len)
         table = fresh_table()
+        ctx.copy_(ctx0)
         d_out.zero_()
         d_len.zero_()
         torch.cuda.synchronize()
@@ -247,9 +195,8 @@ def run_ours(args, rank, world):
                 if profile:
                     B.aded_profile_begin(model)
                 step_ev[0].record()
-            B.aded_trigram_topk(table, d_ctx[step], wl.topk, d_tk, d_cn)
-            B.aded_verify(model, kv, d_tok[step], d_par[step], d_out[step], d_len[step])
-            B.aded_trigram_update(table, d_span[step])
+            B.aded_decode_step(model, kv, table, ctx, n, wl.tree_depth, wl.topk, fill_d[step], d_out[step], d_len[step],
+                               d_real[step])
             if step >= warm:
                 step_ev[step - warm + 1].record()
         torch.cuda.synchronize()
@@ -259,7 +206,7 @@ def run_ours(args, rank, world):
         launches = B.aded_launch_count() - launches0
         lens = d_len[:, 0].tolist()
         for step in range(total):   # the replay must reproduce the recorded decode
-            assert d_out[step, :lens[step]].tolist() == rec[step]["out"], f"replay diverged at step {step}"
+            assert d_out[step, :lens[step]].tolist() == rec[step], f"replay diverged at step {step}"
         per_step = [step_ev[i].elapsed_time(step_ev[i + 1]) for i in range(steps)]
         return step_ev[0].elapsed_time(step_ev[-1]), per_step, launches, sum(lens[warm:]), prof
 
@@ -281,7 +228,7 @@ def run_ours(args, rank, world):
     whole = step_bytes / (dev_ms / steps * 1e-3) / 1e9
     result = {
         "ms": dev_ms, "e2e_ms": e2e_ms, "accepted": accepted, "per_step": per_step, "clocks": clocks,
-        "launches": launches, "h2d": h2d / steps, "d2h": d2h / steps, "setup_s": setup_s,
+        "launches": launches, "h2d": h2d, "d2h": d2h, "setup_s": setup_s,
         "roofline": {"bound": "hbm", "kernel": "projection/FFN/LM-head GEMM", "achieved": round(achieved, 1),
                      "peak": pk["hbm_gbs"], "peak_source": pk["source"], "unit": "GB/s",
                      "frac": round(achieved / pk["hbm_gbs"], 4), "traffic": gemm_traffic_per_launch(shape),
@@ -291,7 +238,7 @@ def run_ours(args, rank, world):
                      "whole_step": {"bytes": int(step_bytes), "achieved_gbs": round(whole, 1),
                                     "frac_of_measured_peak": round(whole / pk["hbm_gbs"], 4),
                                     "frac_of_8tbs": round(whole / 8000.0, 4)}},
-        "shape": shape, "wl": wl, "context": context, "from_topk": statistics.mean(r["real"] for r in rec[warm:]),
+        "shape": shape, "wl": wl, "context": context, "from_topk": float(d_real[warm:].float().mean()),
         "weights": w, "prompt": prompt,
     }
     return result
@@ -407,7 +354,7 @@ def main():
         "warmup": max(args.warmup, 3), "ms_per_step": ms / steps, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": shape.dtype, "data": "synthetic",
         "config": {"workload": f"{args.workload}: {shape.name} ({shape.n_layers} layers, d={shape.d_model}, vocab {shape.vocab}), "
-                               f"Zipf(1.1) prompt {res['context']}, {wl.tree_nodes}-node depth-{wl.tree_depth} trees from tri-gram top-{wl.topk}, "
+                               f"Zipf(1.1) prompt {res['context']}, {wl.tree_nodes}-node depth-{wl.tree_depth} trees retrieved on the device from tri-gram top-{wl.topk}, "
                                "greedy, batch 1, table updated every step",
                    "l2": "inputs larger than L2 (every step streams all weights)", "replicas": world,
                    "accept_len_mean": acc / steps, "tree_nodes_from_topk_mean": res["from_topk"],
