@@ -69,7 +69,7 @@ __global__ void __launch_bounds__(1024) k_add_rmsnorm_ws(bf16* __restrict__ h, G
         }
     }
     pdl_wait();
-    if (*status != 0) return;
+    const int pass_status = *status;     // acted on before the first store; the loads below are valid in any case
     float4 v[2];
     float sq = 0.f;
 #pragma unroll
@@ -80,7 +80,7 @@ __global__ void __launch_bounds__(1024) k_add_rmsnorm_ws(bf16* __restrict__ h, G
             const float4 hv = unpack4_bf16(*hp);
             const float4 add = gemm_out_at4(y, tr[i], r, c & 127);
             const uint2 nv = pack4_bf16(hv.x + add.x, hv.y + add.y, hv.z + add.z, hv.w + add.w);
-            *hp = nv;
+            if (pass_status == 0) *hp = nv;
             v[i] = unpack4_bf16(nv);
             sq += v[i].x * v[i].x + v[i].y * v[i].y + v[i].z * v[i].z + v[i].w * v[i].w;
         }
@@ -92,6 +92,7 @@ __global__ void __launch_bounds__(1024) k_add_rmsnorm_ws(bf16* __restrict__ h, G
 #pragma unroll
     for (int i = 0; i < 32; ++i) total += red[i];      // same order in every thread
     const float inv = rsqrtf(total / (float)d + eps);
+    if (pass_status != 0) return;
 #pragma unroll
     for (int i = 0; i < 2; ++i) {
         const int c = (i * 1024 + threadIdx.x) * 4;
@@ -108,9 +109,11 @@ __global__ void __launch_bounds__(256) k_swiglu_ws(GemmOut gu, bf16* __restrict_
     TileRef tg = {0, 0}, tu = {0, 0};
     if (c < F) { tg = gu.tiles[c >> 7]; tu = gu.tiles[(F + c) >> 7]; }   // the table is constant: read it before waiting
     pdl_wait();
-    if (*status != 0 || c >= F) return;
+    if (c >= F) return;
+    const int pass_status = *status;     // checked before the store, not before the loads
     const float4 g = gemm_out_at4(gu, tg, r, c & 127);
     const float4 u = gemm_out_at4(gu, tu, r, (F + c) & 127);
+    if (pass_status != 0) return;
     *reinterpret_cast<uint2*>(act + (size_t)r * F + c) =
         pack4_bf16(g.x / (1.f + expf(-g.x)) * u.x, g.y / (1.f + expf(-g.y)) * u.y,
                    g.z / (1.f + expf(-g.z)) * u.z, g.w / (1.f + expf(-g.w)) * u.w);
@@ -128,7 +131,8 @@ __global__ void k_rope_kv_ws(GemmOut qkv, const float* __restrict__ cs, const fl
     const int cq = hh * hd, ck = d + hh * hd, cv = 2 * d + hh * hd;
     const TileRef tq = qkv.tiles[cq >> 7], tk = qkv.tiles[ck >> 7], tv = qkv.tiles[cv >> 7];   // constant table
     pdl_wait();
-    if (*status != 0 || i >= half) return;
+    if (i >= half) return;
+    const int pass_status = *status;     // checked before the stores, not before the loads
     const int b = row_seq[r];
     const size_t slot = (size_t)len[b] + row_local[r];
     const size_t cp = cap[b];
@@ -138,6 +142,7 @@ __global__ void k_rope_kv_ws(GemmOut qkv, const float* __restrict__ cs, const fl
     const float4 k0 = gemm_out_at4(qkv, tk, r, (ck + i) & 127), k1 = gemm_out_at4(qkv, tk, r, (ck + i + half) & 127);
     const float4 v0 = gemm_out_at4(qkv, tv, r, (cv + i) & 127), v1 = gemm_out_at4(qkv, tv, r, (cv + i + half) & 127);
     const float4 c = *reinterpret_cast<const float4*>(cs + r * half + i), s = *reinterpret_cast<const float4*>(sn + r * half + i);
+    if (pass_status != 0) return;
     bf16* qd = q + (size_t)r * d + hh * hd;
     *reinterpret_cast<uint2*>(qd + i) = pack4_bf16(q0.x * c.x - q1.x * s.x, q0.y * c.y - q1.y * s.y, q0.z * c.z - q1.z * s.z, q0.w * c.w - q1.w * s.w);
     *reinterpret_cast<uint2*>(qd + i + half) = pack4_bf16(q1.x * c.x + q0.x * s.x, q1.y * c.y + q0.y * s.y, q1.z * c.z + q0.z * s.z, q1.w * c.w + q0.w * s.w);

@@ -132,7 +132,11 @@ struct AttnArgs {
 template <int HD, int NW>
 __global__ void __launch_bounds__(NW * 32) k_tree_attn_mma(AttnArgs a) {
     pdl_enter();
-    if (*a.status != 0) return;
+    // The status word is fetched along with the rest of the call's metadata and acted on before the
+    // first store, so that it does not cost a memory round trip of its own.  Until then nothing is
+    // written, and every load below stays inside the cache block and the row arrays whatever a failed
+    // earlier kernel left in them (positions are clamped to the capacity).
+    const int pass_status = *a.status;
     constexpr int KSTEPS = HD / 16;        // k steps of Q K^T
     constexpr int ONT = HD / 8;            // n tiles of the output
     constexpr int CHUNKS = HD / 8;         // 16-byte chunks per row
@@ -189,7 +193,7 @@ __global__ void __launch_bounds__(NW * 32) k_tree_attn_mma(AttnArgs a) {
         bf16* dv = sv + (size_t)buf * TA_BLK * HD;
         for (int e = threadIdx.x; e < TA_BLK * CHUNKS; e += NW * 32) {
             const int row = e / CHUNKS, chunk = e % CHUNKS;
-            const int pos = min(p0 + row, n_keys - 1);
+            const int pos = min(min(p0 + row, n_keys - 1), (int)cp - 1);
             cp_async16(tile_chunk<HD>(dk, row, chunk), kg + (size_t)pos * HD + chunk * 8);
             cp_async16(tile_chunk<HD>(dv, row, chunk), vg + (size_t)pos * HD + chunk * 8);
         }
@@ -303,6 +307,7 @@ __global__ void __launch_bounds__(NW * 32) k_tree_attn_mma(AttnArgs a) {
     // cluster barrier CTA j combines rows j, j + S, ... from all S CTAs' shared memory (distributed
     // shared memory reads), out = sum_s O_s 2^(m_s - M) / sum_s l_s 2^(m_s - M), rounds to bf16 and
     // writes the attention output.  No partial ever goes to global memory.
+    if (pass_status != 0) return;     // uniform over the cluster: nobody waits for a CTA that left
     lrow0 += __shfl_xor_sync(0xffffffffu, lrow0, 1);
     lrow0 += __shfl_xor_sync(0xffffffffu, lrow0, 2);
     lrow1 += __shfl_xor_sync(0xffffffffu, lrow1, 1);
@@ -333,25 +338,34 @@ __global__ void __launch_bounds__(NW * 32) k_tree_attn_mma(AttnArgs a) {
     constexpr int QUADS = HD / 4;                      // float4 groups per row
     for (int item = threadIdx.x; item < ((T - split + S - 1) / S) * QUADS; item += NW * 32) {
         const int row = split + (item / QUADS) * S, c4 = (item % QUADS) * 4;
+        // all remote reads of an item are issued before any is used (S <= 8 partials)
         float ms[8], ls[8];
+        float4 os[8];
         float M = -INFINITY;
-        for (int s2 = 0; s2 < S; ++s2) {
-            uint32_t remote;
-            asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(sml_addr + (uint32_t)row * 8), "r"(s2));
-            asm volatile("ld.shared::cluster.v2.f32 {%0, %1}, [%2];" : "=f"(ms[s2]), "=f"(ls[s2]) : "r"(remote));
-            M = fmaxf(M, ms[s2]);
+#pragma unroll
+        for (int s2 = 0; s2 < 8; ++s2) {
+            ms[s2] = -INFINITY;
+            ls[s2] = 0.f;
+            os[s2] = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (s2 < S) {
+                uint32_t rm, ro;
+                asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(rm) : "r"(sml_addr + (uint32_t)row * 8), "r"(s2));
+                asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(ro) : "r"(so_addr + (uint32_t)(row * HD + c4) * 4), "r"(s2));
+                asm volatile("ld.shared::cluster.v2.f32 {%0, %1}, [%2];" : "=f"(ms[s2]), "=f"(ls[s2]) : "r"(rm));
+                asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];"
+                             : "=f"(os[s2].x), "=f"(os[s2].y), "=f"(os[s2].z), "=f"(os[s2].w) : "r"(ro));
+            }
         }
+#pragma unroll
+        for (int s2 = 0; s2 < 8; ++s2) M = fmaxf(M, ms[s2]);
         float4 num = make_float4(0.f, 0.f, 0.f, 0.f);
         float den = 0.f;
-        for (int s2 = 0; s2 < S; ++s2) {
-            if (ms[s2] == -INFINITY) continue;
+#pragma unroll
+        for (int s2 = 0; s2 < 8; ++s2) {
+            if (ms[s2] == -INFINITY) continue;     // an empty split (or s2 >= S) holds no keys of this row
             const float w = exp2f(ms[s2] - M);
-            uint32_t remote;
-            asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(so_addr + (uint32_t)(row * HD + c4) * 4), "r"(s2));
-            float4 o;
-            asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(o.x), "=f"(o.y), "=f"(o.z), "=f"(o.w) : "r"(remote));
             den += ls[s2] * w;
-            num.x += o.x * w; num.y += o.y * w; num.z += o.z * w; num.w += o.w * w;
+            num.x += os[s2].x * w; num.y += os[s2].y * w; num.z += os[s2].z * w; num.w += os[s2].w * w;
         }
         const float inv = 1.f / den;
         bf16* dst = a.out + ((size_t)(off + row) * a.H + hh) * HD + c4;
