@@ -9,6 +9,7 @@
 #include <vector>
 
 #include "aded.h"
+#include "fused_ws.cuh"
 #include "gemm_out.cuh"
 
 #define ADED_CUDA_TRY(expr)                      \
@@ -146,6 +147,12 @@ struct aded_model {
     float* ws_slots;                    // partial result tiles (see gemm_out.cuh)
     aded::TileRef* ws_tiles[5];         // contributor tables of the wqkv, wo, wgu, wd and LM-head results
 
+    // persistent projection kernel (fused_ws.cu): passes of at most 128 rows
+    bool fw_ready;
+    CUtensorMap* fw_maps;               // device copy of ws_maps
+    uint32_t* fw_counters;              // [FW_COUNTERS] grid-barrier counters, zeroed at the start of a pass
+    aded::TileRef* fw_tiles[5];         // contributor tables for results split over the full grid
+
     float* norm_ssq;        // [R][32] per-chunk sums of squares of the RMSNorm kernel
     int32_t* norm_count;    // [R] chunk arrival counters, zero between launches
     float* argmax_val;      // [R][ARGMAX_CHUNKS] best logit of each column chunk
@@ -211,6 +218,10 @@ size_t ws_slot_floats(int device, int max_n, int max_rows);
 cudaError_t ws_launch(const CUtensorMap& map_w, const CUtensorMap& map_x, int rows, int row0, int n, int k,
                       float* slots, int32_t* status, int device, cudaStream_t st);
 enum { WS_MAP_QKV = 0, WS_MAP_O = 1, WS_MAP_GU = 2, WS_MAP_D = 3 };   // per-layer map order
+
+// fused_ws.cu
+bool fw_prepare(int device);
+cudaError_t fw_launch(aded_model* m, aded_kv* kv, const FwPair* pairs, int n_pairs, int rows, int launch_index, cudaStream_t st);
 
 // tree_attention.cu
 // max_tree: most nodes any sequence's tree has in this call

@@ -9,39 +9,6 @@
 
 namespace aded {
 
-__device__ __forceinline__ float4 f4_add(float4 a, float4 b) { return make_float4(a.x + b.x, a.y + b.y, a.z + b.z, a.w + b.w); }
-
-// Columns col .. col+3 (col % 4 == 0) of tile t, row r: slots added in CTA order.
-__device__ __forceinline__ float4 gemm_out_at4(const GemmOut& o, const TileRef& t, int r, int col) {
-    const int rb = gemm_block_rb(o, r);
-    const size_t region = (size_t)(r >> 7) * (size_t)(o.n_tiles + o.g) * 128 * 128;
-    const float* p = o.slots + region + ((size_t)t.first_slot * rb + (r & 127)) * 128 + col;
-    const size_t stride = (size_t)rb * 128;
-    float4 sum = make_float4(0.f, 0.f, 0.f, 0.f);
-    int i = 0;
-    for (; i + 4 <= t.count; i += 4) {     // four loads in flight, added in order
-        const float4 a = __ldcg(reinterpret_cast<const float4*>(p + (size_t)i * stride));
-        const float4 b = __ldcg(reinterpret_cast<const float4*>(p + (size_t)(i + 1) * stride));
-        const float4 c = __ldcg(reinterpret_cast<const float4*>(p + (size_t)(i + 2) * stride));
-        const float4 d = __ldcg(reinterpret_cast<const float4*>(p + (size_t)(i + 3) * stride));
-        sum = f4_add(f4_add(f4_add(f4_add(sum, a), b), c), d);
-    }
-    for (; i < t.count; ++i) sum = f4_add(sum, __ldcg(reinterpret_cast<const float4*>(p + (size_t)i * stride)));
-    return sum;
-}
-
-__device__ __forceinline__ uint2 pack4_bf16(float a, float b, float c, float d) {
-    const __nv_bfloat162 lo = __floats2bfloat162_rn(a, b), hi = __floats2bfloat162_rn(c, d);
-    uint2 u;
-    u.x = *reinterpret_cast<const uint32_t*>(&lo);
-    u.y = *reinterpret_cast<const uint32_t*>(&hi);
-    return u;
-}
-__device__ __forceinline__ float4 unpack4_bf16(uint2 u) {
-    const __nv_bfloat162 lo = *reinterpret_cast<const __nv_bfloat162*>(&u.x), hi = *reinterpret_cast<const __nv_bfloat162*>(&u.y);
-    return make_float4(__low2float(lo), __high2float(lo), __low2float(hi), __high2float(hi));
-}
-
 __device__ __forceinline__ float warp_sum_f(float v) {
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);

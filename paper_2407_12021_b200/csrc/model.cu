@@ -112,6 +112,7 @@ static aded_status alloc_model(aded_model* m) {
 
     // tensor-core GEMM path: bf16 models whose every matrix tiles into 128-row x 64-column blocks
     m->ws_ready = false;
+    m->fw_ready = false;
     if (c.dtype == ADED_BF16 && !getenv("ADED_PLAIN_GEMM") && ws_supported(3 * (int)d, (int)d) && ws_supported((int)d, (int)d) &&
         ws_supported(2 * (int)F, (int)d) && ws_supported((int)d, (int)F) && ws_supported((int)V, (int)d)) {
         const int L = c.n_layers;
@@ -142,13 +143,36 @@ static aded_status alloc_model(aded_model* m) {
                 ADED_CUDA_TRY(cudaMemcpy(m->ws_tiles[i], table.data(), nt * sizeof(TileRef), cudaMemcpyHostToDevice));
             }
             m->ws_ready = true;
+            // persistent kernel: device copy of the descriptors, barrier counters, tables for the full-grid split
+            if (!getenv("ADED_NO_FUSED") && d % 4 == 0 && (c.head_dim / 2) % 4 == 0 && fw_prepare(m->device)) {
+                TRY(dev_alloc(m, &m->fw_maps, m->ws_maps.size()));
+                ADED_CUDA_TRY(cudaMemcpy(m->fw_maps, m->ws_maps.data(), m->ws_maps.size() * sizeof(CUtensorMap), cudaMemcpyHostToDevice));
+                TRY(dev_alloc(m, &m->fw_counters, (size_t)FW_COUNTERS));
+                ADED_CUDA_TRY(cudaMemset(m->fw_counters, 0, FW_COUNTERS * sizeof(uint32_t)));
+                const int g = ws_grid_limit(m->device);
+                for (int i = 0; i < 5; ++i) {
+                    const int nt = shapes[i][0] / 128, kb = shapes[i][1] / 64;
+                    std::vector<TileRef> table(nt);
+                    for (int t = 0; t < nt; ++t) table[t] = gemm_tile_ref(nt, kb, g, t);
+                    TRY(dev_alloc(m, &m->fw_tiles[i], (size_t)nt));
+                    ADED_CUDA_TRY(cudaMemcpy(m->fw_tiles[i], table.data(), nt * sizeof(TileRef), cudaMemcpyHostToDevice));
+                }
+                m->fw_ready = true;
+            }
         }
     }
     return ADED_OK;
 }
 
+// The persistent projection kernel takes passes of at most 128 rows (one row block) with fewer
+// launches than barrier counters; the debug capture of the residual stream needs the layer-by-layer path.
+static bool use_fused(const aded_model* m, int rows) {
+    return m->fw_ready && rows <= 128 && !m->dbg_hidden && m->cfg.n_layers + 1 <= FW_COUNTERS;
+}
+
 // Kernels one pass launches (what enqueue_pass enqueues), for the launch counter of graph replays.
 static int pass_launches(const aded_model* m, int rows, int chain_mode) {
+    if (use_fused(m, rows)) return 4 + 1 + 2 * m->cfg.n_layers + (chain_mode ? 1 : 5);
     const int gemm_passes = (rows + 127) / 128;   // the tensor-core GEMM runs once per 128 rows
     const int per_gemm = m->ws_ready ? gemm_passes : 1;
     int n = 4 + m->cfg.n_layers * (4 * per_gemm + 3 + 1);
@@ -167,6 +191,7 @@ static aded_status enqueue_pass(aded_model* m, aded_kv* kv, const int32_t* offse
     const int xm = 4 * c.n_layers + 1;   // TMA descriptor indices of x, attn, act
     ADED_CUDA_TRY(cudaMemcpyAsync(m->seqs.row_off, offsets_src, (batch + 1) * sizeof(int32_t),
                                   cudaMemcpyHostToDevice, st));
+    if (use_fused(m, rows)) ADED_CUDA_TRY(cudaMemsetAsync(m->fw_counters, 0, FW_COUNTERS * sizeof(uint32_t), st));
     {
         Span sp(m, PROF_OTHER, 4, st);
         launch_tree_prologue(m, kv, batch, chain_mode, st);
@@ -176,7 +201,57 @@ static aded_status enqueue_pass(aded_model* m, aded_kv* kv, const int32_t* offse
     }
     const size_t hid_bytes = (size_t)rows * d * m->elem;
     if (m->dbg_hidden) ADED_CUDA_TRY(cudaMemcpyAsync(m->dbg_hidden, m->h, hid_bytes, cudaMemcpyDeviceToDevice, st));
-    for (int l = 0; l < c.n_layers; ++l) {
+    const bool fused = use_fused(m, rows);
+    GemmOut fused_logits = {};
+    if (fused) {
+        // Persistent-kernel path: [QKV_0, rotary] | attention_0 | [O, norm, gate/up, SwiGLU, down, norm,
+        // QKV_1, rotary] | attention_1 | ... | [O, norm, gate/up, SwiGLU, down, final norm, LM head].
+        const int F2 = 2 * F;
+        auto pair = [&](int map_w, int map_x, int n, int k, int table, int post, int layer, const void* gain) {
+            FwPair pr;
+            pr.map_w = map_w;
+            pr.map_x = map_x;
+            pr.n_tiles = n / 128;
+            pr.kb = k / 64;
+            pr.tiles = m->fw_tiles[table];
+            pr.post = post;
+            pr.layer = layer;
+            pr.gain = gain;
+            return pr;
+        };
+        int launch_index = 0;
+        {
+            const FwPair first = pair(WS_MAP_QKV, xm, 3 * d, d, 0, FW_POST_ROPE_KV, 0, nullptr);
+            Span sp(m, PROF_GEMM, 1, st);
+            ADED_CUDA_TRY(fw_launch(m, kv, &first, 1, rows, launch_index++, st));
+            note_launch();
+        }
+        for (int l = 0; l < c.n_layers; ++l) {
+            const aded_layer_weights& w = m->layers[l];
+            { Span sp(m, PROF_ATTN, 1, st); launch_tree_attention(m, kv, l, batch, rows, max_tree, st); }
+            const bool last = l + 1 == c.n_layers;
+            FwPair prs[FW_MAX_PAIRS];
+            int np = 0;
+            prs[np++] = pair(4 * l + WS_MAP_O, xm + 1, d, d, 1, FW_POST_ADD_NORM, 0, w.norm2);
+            prs[np++] = pair(4 * l + WS_MAP_GU, xm, F2, d, 2, FW_POST_SWIGLU, 0, nullptr);
+            prs[np++] = pair(4 * l + WS_MAP_D, xm + 2, d, F, 3, FW_POST_ADD_NORM, 0, last ? m->top.final_norm : m->layers[l + 1].norm1);
+            if (!last) prs[np++] = pair(4 * (l + 1) + WS_MAP_QKV, xm, 3 * d, d, 0, FW_POST_ROPE_KV, l + 1, nullptr);
+            else if (!chain_mode) prs[np++] = pair(4 * c.n_layers, xm, c.vocab, d, 4, FW_POST_NONE, 0, nullptr);
+            Span sp(m, PROF_GEMM, 1, st);
+            ADED_CUDA_TRY(fw_launch(m, kv, prs, np, rows, launch_index++, st));
+            note_launch();
+        }
+        fused_logits.y = nullptr;
+        fused_logits.slots = m->ws_slots;
+        fused_logits.tiles = m->fw_tiles[4];
+        fused_logits.mode = 1;
+        fused_logits.n = c.vocab;
+        fused_logits.n_tiles = c.vocab / 128;
+        fused_logits.kb = d / 64;
+        fused_logits.g = ws_grid_limit(m->device);
+        fused_logits.rows = rows;
+    }
+    for (int l = 0; l < c.n_layers && !fused; ++l) {
         const aded_layer_weights& w = m->layers[l];
         GemmOut o;
         { Span sp(m, PROF_GEMM, 1, st); o = launch_gemm(m, 4 * l + WS_MAP_QKV, xm, m->x, w.wqkv, m->y32, rows, 3 * d, d, st); }
@@ -194,8 +269,8 @@ static aded_status enqueue_pass(aded_model* m, aded_kv* kv, const int32_t* offse
                                           cudaMemcpyDeviceToDevice, st));
     }
     if (!chain_mode) {
-        GemmOut lg;
-        { Span sp(m, PROF_GEMM, 1, st); lg = launch_gemm(m, 4 * c.n_layers, xm, m->x, m->top.lm_head, m->logits, rows, c.vocab, d, st); }
+        GemmOut lg = fused_logits;
+        if (!fused) { Span sp(m, PROF_GEMM, 1, st); lg = launch_gemm(m, 4 * c.n_layers, xm, m->x, m->top.lm_head, m->logits, rows, c.vocab, d, st); }
         Span sp(m, PROF_OTHER, 3, st);
         launch_argmax(m, lg, rows, st);
         if (m->dbg_logits) launch_materialize(m, lg, m->dbg_logits, rows, st);
