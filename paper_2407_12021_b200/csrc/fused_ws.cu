@@ -155,9 +155,10 @@ __device__ __forceinline__ void load_x_stage(const CUtensorMap* mx, uint64_t* ba
     for (int r = 0; r < rb; r += 16) tma_load_2d(mx, bar, sb + r * 128, kb * FW_BK, r);
 }
 
-// 128 registers per thread at most: register files are handed out in units of four warps, so a CTA
-// of six warps counts as eight and two CTAs fit on an SM only up to 65536 / (2 * 8 * 32) registers.
-__global__ void __launch_bounds__(256, 2) k_fused_ws(const __grid_constant__ FwParams p) {
+// Registers are capped at 112 per thread: the register file is handed out in units of four warps, so
+// a CTA of six warps counts as eight, and at 128 registers (2 x 8 x 32 x 128 = the whole file) the
+// occupancy query still reports one CTA per SM.
+__global__ void __maxnreg__(112) k_fused_ws(const __grid_constant__ FwParams p) {
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     uint8_t* base = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     const uint32_t a_bytes = FW_BM * 128, b_bytes = (uint32_t)p.rb * 128, stage_bytes = a_bytes + b_bytes;
@@ -396,20 +397,31 @@ static size_t fw_smem(int rb, int* stages_out) {
     return (size_t)stages * stage_bytes + 1024 + 256;
 }
 
-// The grid barrier needs every CTA resident: two per SM must fit.
+// The grid barrier needs every CTA resident: two per SM must fit.  The runtime's occupancy query
+// answers one CTA per SM for this kernel whatever block size and shared memory are asked about (it
+// seems not to model kernels that allocate tensor memory), so the check is done by hand from the
+// device's limits: registers are granted per group of four warps, shared memory per CTA plus the
+// reserved kilobyte, tensor memory 512 columns per SM.
 bool fw_prepare(int device) {
-    (void)device;
-    cudaError_t e = cudaFuncSetAttribute(k_fused_ws, cudaFuncAttributeMaxDynamicSharedMemorySize, 112 * 1024);
-    int per_sm = 0;
-    if (e == cudaSuccess) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_fused_ws, FW_THREADS, fw_smem(128, nullptr));
-    if (getenv("ADED_VERBOSE")) {
-        cudaFuncAttributes fa = {};
-        cudaFuncGetAttributes(&fa, k_fused_ws);
-        fprintf(stderr, "[aded] persistent projection kernel: %s, %d CTAs per SM (%d registers, %zu bytes local)\n",
-                cudaGetErrorString(e), per_sm, fa.numRegs, fa.localSizeBytes);
+    if (cudaFuncSetAttribute(k_fused_ws, cudaFuncAttributeMaxDynamicSharedMemorySize, 112 * 1024) != cudaSuccess) {
+        cudaGetLastError();
+        return false;
     }
-    if (e != cudaSuccess) { cudaGetLastError(); return false; }
-    return per_sm >= 2;
+    cudaFuncAttributes fa = {};
+    if (cudaFuncGetAttributes(&fa, k_fused_ws) != cudaSuccess) { cudaGetLastError(); return false; }
+    int regs_sm = 0, smem_sm = 0, smem_res = 0, threads_sm = 0;
+    cudaDeviceGetAttribute(&regs_sm, cudaDevAttrMaxRegistersPerMultiprocessor, device);
+    cudaDeviceGetAttribute(&smem_sm, cudaDevAttrMaxSharedMemoryPerMultiprocessor, device);
+    cudaDeviceGetAttribute(&smem_res, cudaDevAttrReservedSharedMemoryPerBlock, device);
+    cudaDeviceGetAttribute(&threads_sm, cudaDevAttrMaxThreadsPerMultiProcessor, device);
+    const int warps = (FW_THREADS / 32 + 3) / 4 * 4;
+    const long long regs_cta = (long long)warps * 32 * ((fa.numRegs + 7) / 8 * 8);
+    const long long smem_cta = (long long)fw_smem(128, nullptr) + fa.sharedSizeBytes + smem_res;
+    const bool ok = 2 * regs_cta < regs_sm && 2 * smem_cta <= smem_sm && 2 * FW_THREADS <= threads_sm;
+    if (getenv("ADED_VERBOSE"))
+        fprintf(stderr, "[aded] persistent projection kernel: %d registers, %lld of %d registers and %lld of %d bytes of shared memory for two CTAs: %s\n",
+                fa.numRegs, 2 * regs_cta, regs_sm, 2 * smem_cta, smem_sm, ok ? "used" : "not used");
+    return ok;
 }
 
 cudaError_t fw_launch(aded_model* m, aded_kv* kv, const FwPair* pairs, int n_pairs, int rows, int launch_index, cudaStream_t st) {
