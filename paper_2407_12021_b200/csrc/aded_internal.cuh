@@ -151,7 +151,6 @@ struct aded_model {
     bool fw_ready;
     CUtensorMap* fw_maps;               // device copy of ws_maps
     uint32_t* fw_counters;              // [FW_COUNTERS] grid-barrier counters, zeroed at the start of a pass
-    aded::TileRef* fw_tiles[5];         // contributor tables for results split over the full grid
 
     float* norm_ssq;        // [R][32] per-chunk sums of squares of the RMSNorm kernel
     int32_t* norm_count;    // [R] chunk arrival counters, zero between launches

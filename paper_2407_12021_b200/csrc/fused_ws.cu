@@ -18,7 +18,7 @@
 // Per CTA (192 threads, two CTAs per SM, grid = 2 x SMs; all CTAs are resident, which the barrier
 // needs): warp 0 TMA producer, warp 1 MMA issuer (tcgen05, fp32 accumulators in TMEM, two of them),
 // warps 2..5 epilogue and small steps.  GEMM work split, slots and contributor tables: gemm_out.cuh
-// and gemm_ws.cu (same scheme, always split over the full grid).  The arithmetic of the small steps
+// and gemm_ws.cu (same scheme).  The arithmetic of the small steps
 // is that of dense_ws.cu.  Every wait is bounded; one that runs out raises ADED_ERR_TIMEOUT and the
 // CTA unwinds (the others see the status word and unwind too).
 #include <cuda.h>
@@ -150,6 +150,21 @@ __device__ __forceinline__ void post_rope_kv(const FwParams& p, const GemmOut& q
     }
 }
 
+// Work units of this CTA in one projection.  A projection with fewer units than CTAs is split over
+// as many CTAs as it has units (the others idle), so that a tile's contributors are consecutive
+// CTAs -- the same split, and the same contributor tables, as the stand-alone GEMM's.
+__device__ __forceinline__ int fw_range(const FwPair& pr, long long G, long long& u0, long long& u1) {
+    const long long units = (long long)pr.n_tiles * pr.kb;
+    const long long g = units < G ? units : G;
+    if ((long long)blockIdx.x < g) {
+        u0 = ws_start(blockIdx.x, units, g);
+        u1 = ws_start(blockIdx.x + 1, units, g);
+    } else {
+        u0 = u1 = 0;
+    }
+    return (int)g;
+}
+
 // x tiles of one stage: rb rows x 64 columns of the activation matrix, 16 rows per TMA box.
 __device__ __forceinline__ void load_x_stage(const CUtensorMap* mx, uint64_t* bar, uint8_t* sb, int kb, int rb) {
     for (int r = 0; r < rb; r += 16) tma_load_2d(mx, bar, sb + r * 128, kb * FW_BK, r);
@@ -208,12 +223,14 @@ __global__ void __maxnreg__(112) k_fused_ws(const __grid_constant__ FwParams p) 
                 const CUtensorMap* mx = p.maps + pr.map_x;
                 asm volatile("prefetch.tensormap [%0];" ::"l"(mw) : "memory");
                 asm volatile("prefetch.tensormap [%0];" ::"l"(mx) : "memory");
-                const long long units = (long long)pr.n_tiles * pr.kb;
-                const long long u0 = ws_start(blockIdx.x, units, G), u1 = ws_start(blockIdx.x + 1, units, G);
+                long long u0, u1;
+                fw_range(pr, G, u0, u1);
                 // x of projection i exists once the step before it has finished on every CTA: for the
-                // first projection that is the previous kernel, afterwards 2 i G arrivals at the counter
-                // (G after each earlier projection, G after each earlier step).
-                const uint32_t target = (uint32_t)(2 * i * G);
+                // first projection that is the previous kernel, afterwards i G arrivals at the counter
+                // of finished steps.  (Steps and projections count separately: a CTA without work in a
+                // projection arrives at its barrier at once, and one shared count could reach the target
+                // while another CTA is still inside the step.)
+                const uint32_t target = (uint32_t)(i * G);
                 bool x_ready = false;
                 for (long long u = u0; u <= u1 && !s_flag[0]; ++u) {
                     const bool last = u == u1;          // one extra round that only settles the pending stages
@@ -223,10 +240,10 @@ __global__ void __maxnreg__(112) k_fused_ws(const __grid_constant__ FwParams p) 
                         if (i == 0) {
                             if (must) { pdl_wait(); ok = true; }
                         } else if (must) {
-                            ok = counter_wait(p.counter, target, p.status);
+                            ok = counter_wait(p.counter + 1, target, p.status);
                             if (!ok) { s_flag[0] = 1; atomicCAS(p.status, 0, (int)ADED_ERR_TIMEOUT); break; }
                         } else {
-                            ok = ld_acquire(p.counter) >= target;
+                            ok = ld_acquire(p.counter + 1) >= target;
                         }
                         if (ok) {
                             fence_async_global();
@@ -265,8 +282,8 @@ __global__ void __maxnreg__(112) k_fused_ws(const __grid_constant__ FwParams p) 
             int seg = 0;
             for (int i = 0; i < p.n_pairs && !s_flag[0]; ++i) {
                 const FwPair& pr = p.pair[i];
-                const long long units = (long long)pr.n_tiles * pr.kb;
-                const long long u0 = ws_start(blockIdx.x, units, G), u1 = ws_start(blockIdx.x + 1, units, G);
+                long long u0, u1;
+                fw_range(pr, G, u0, u1);
                 long long u = u0;
                 while (u < u1 && !s_flag[0]) {
                     const int kb0 = (int)(u % pr.kb);
@@ -314,8 +331,8 @@ __global__ void __maxnreg__(112) k_fused_ws(const __grid_constant__ FwParams p) 
         for (int i = 0; i < p.n_pairs && live; ++i) {
             if (epi_agree_abort(s_flag, et)) break;
             const FwPair& pr = p.pair[i];
-            const long long units = (long long)pr.n_tiles * pr.kb;
-            const long long u0 = ws_start(blockIdx.x, units, G), u1 = ws_start(blockIdx.x + 1, units, G);
+            long long u0, u1;
+            const int g_eff = fw_range(pr, G, u0, u1);
             long long u = u0;
             while (u < u1) {
                 const int tile = (int)(u / pr.kb), kb0 = (int)(u % pr.kb);
@@ -346,7 +363,7 @@ __global__ void __maxnreg__(112) k_fused_ws(const __grid_constant__ FwParams p) 
             if (et == 0) {
                 if (!s_flag[0]) {
                     red_release(p.counter);
-                    if (!counter_wait(p.counter, (uint32_t)((2 * i + 1) * G), p.status)) {
+                    if (!counter_wait(p.counter, (uint32_t)((i + 1) * G), p.status)) {
                         s_flag[0] = 1;
                         atomicCAS(p.status, 0, (int)ADED_ERR_TIMEOUT);
                     }
@@ -362,7 +379,7 @@ __global__ void __maxnreg__(112) k_fused_ws(const __grid_constant__ FwParams p) 
             o.n = pr.n_tiles * FW_BM;
             o.n_tiles = pr.n_tiles;
             o.kb = pr.kb;
-            o.g = (int)G;
+            o.g = g_eff;
             o.rows = p.rows;
             if (pr.post == FW_POST_ADD_NORM) post_add_norm(p, o, reinterpret_cast<const bf16*>(pr.gain), et, s_red);
             else if (pr.post == FW_POST_SWIGLU) post_swiglu(p, o, et);
@@ -371,7 +388,7 @@ __global__ void __maxnreg__(112) k_fused_ws(const __grid_constant__ FwParams p) 
             __threadfence();
             fence_async_global();
             epi_sync();
-            if (et == 0) red_release(p.counter);
+            if (et == 0) red_release(p.counter + 1);
         }
     }
 
@@ -435,7 +452,7 @@ cudaError_t fw_launch(aded_model* m, aded_kv* kv, const FwPair* pairs, int n_pai
     while (p.tmem_cols < 2 * p.rb) p.tmem_cols *= 2;
     p.maps = m->fw_maps;
     p.slots = m->ws_slots;
-    p.counter = m->fw_counters + (launch_index % FW_COUNTERS);
+    p.counter = m->fw_counters + 2 * (launch_index % FW_COUNTERS);
     p.status = m->status;
     p.h = (bf16*)m->h;
     p.x = (bf16*)m->x;

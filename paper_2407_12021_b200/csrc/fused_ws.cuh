@@ -10,7 +10,7 @@
 namespace aded {
 
 constexpr int FW_MAX_PAIRS = 4;
-constexpr int FW_COUNTERS = 64;        // barrier counters per pass, one per launch
+constexpr int FW_COUNTERS = 64;        // launches per pass that get barrier counters (a pair each)
 
 enum { FW_POST_NONE = 0, FW_POST_ADD_NORM = 1, FW_POST_SWIGLU = 2, FW_POST_ROPE_KV = 3 };
 
@@ -18,7 +18,7 @@ enum { FW_POST_NONE = 0, FW_POST_ADD_NORM = 1, FW_POST_SWIGLU = 2, FW_POST_ROPE_
 struct FwPair {
     int map_w, map_x;          // indices into the device array of TMA descriptors
     int n_tiles, kb;           // W is [128 * n_tiles, 64 * kb]
-    const TileRef* tiles;      // contributor table of the result (split over the full grid)
+    const TileRef* tiles;      // contributor table of the result
     int post;                  // FW_POST_*
     int layer;                 // FW_POST_ROPE_KV: layer whose K/V rows are written
     const void* gain;          // FW_POST_ADD_NORM: RMSNorm gain [d]
@@ -30,7 +30,7 @@ struct FwParams {
     int rows, rb, stages, tmem_cols;
     const CUtensorMap* maps;
     float* slots;
-    uint32_t* counter;         // this launch's barrier counter, zero at launch
+    uint32_t* counter;         // this launch's two barrier counters (projections done, steps done), zero at launch
     int32_t* status;
     __nv_bfloat16 *h, *x, *q, *act;
     int d, F, H, hd;

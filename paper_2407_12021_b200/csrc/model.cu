@@ -143,20 +143,13 @@ static aded_status alloc_model(aded_model* m) {
                 ADED_CUDA_TRY(cudaMemcpy(m->ws_tiles[i], table.data(), nt * sizeof(TileRef), cudaMemcpyHostToDevice));
             }
             m->ws_ready = true;
-            // persistent kernel: device copy of the descriptors, barrier counters, tables for the full-grid split
-            if (!getenv("ADED_NO_FUSED") && d % 4 == 0 && (c.head_dim / 2) % 4 == 0 && fw_prepare(m->device)) {
+            // persistent kernel (opt-in with ADED_FUSED=1 while it is slower than the separate kernels):
+            // device copy of the descriptors, barrier counters
+            if (getenv("ADED_FUSED") && d % 4 == 0 && (c.head_dim / 2) % 4 == 0 && fw_prepare(m->device)) {
                 TRY(dev_alloc(m, &m->fw_maps, m->ws_maps.size()));
                 ADED_CUDA_TRY(cudaMemcpy(m->fw_maps, m->ws_maps.data(), m->ws_maps.size() * sizeof(CUtensorMap), cudaMemcpyHostToDevice));
-                TRY(dev_alloc(m, &m->fw_counters, (size_t)FW_COUNTERS));
-                ADED_CUDA_TRY(cudaMemset(m->fw_counters, 0, FW_COUNTERS * sizeof(uint32_t)));
-                const int g = ws_grid_limit(m->device);
-                for (int i = 0; i < 5; ++i) {
-                    const int nt = shapes[i][0] / 128, kb = shapes[i][1] / 64;
-                    std::vector<TileRef> table(nt);
-                    for (int t = 0; t < nt; ++t) table[t] = gemm_tile_ref(nt, kb, g, t);
-                    TRY(dev_alloc(m, &m->fw_tiles[i], (size_t)nt));
-                    ADED_CUDA_TRY(cudaMemcpy(m->fw_tiles[i], table.data(), nt * sizeof(TileRef), cudaMemcpyHostToDevice));
-                }
+                TRY(dev_alloc(m, &m->fw_counters, (size_t)2 * FW_COUNTERS));
+                ADED_CUDA_TRY(cudaMemset(m->fw_counters, 0, 2 * FW_COUNTERS * sizeof(uint32_t)));
                 m->fw_ready = true;
             }
         }
@@ -191,7 +184,7 @@ static aded_status enqueue_pass(aded_model* m, aded_kv* kv, const int32_t* offse
     const int xm = 4 * c.n_layers + 1;   // TMA descriptor indices of x, attn, act
     ADED_CUDA_TRY(cudaMemcpyAsync(m->seqs.row_off, offsets_src, (batch + 1) * sizeof(int32_t),
                                   cudaMemcpyHostToDevice, st));
-    if (use_fused(m, rows)) ADED_CUDA_TRY(cudaMemsetAsync(m->fw_counters, 0, FW_COUNTERS * sizeof(uint32_t), st));
+    if (use_fused(m, rows)) ADED_CUDA_TRY(cudaMemsetAsync(m->fw_counters, 0, 2 * FW_COUNTERS * sizeof(uint32_t), st));
     {
         Span sp(m, PROF_OTHER, 4, st);
         launch_tree_prologue(m, kv, batch, chain_mode, st);
@@ -213,7 +206,7 @@ static aded_status enqueue_pass(aded_model* m, aded_kv* kv, const int32_t* offse
             pr.map_x = map_x;
             pr.n_tiles = n / 128;
             pr.kb = k / 64;
-            pr.tiles = m->fw_tiles[table];
+            pr.tiles = m->ws_tiles[table];
             pr.post = post;
             pr.layer = layer;
             pr.gain = gain;
@@ -243,12 +236,12 @@ static aded_status enqueue_pass(aded_model* m, aded_kv* kv, const int32_t* offse
         }
         fused_logits.y = nullptr;
         fused_logits.slots = m->ws_slots;
-        fused_logits.tiles = m->fw_tiles[4];
+        fused_logits.tiles = m->ws_tiles[4];
         fused_logits.mode = 1;
         fused_logits.n = c.vocab;
         fused_logits.n_tiles = c.vocab / 128;
         fused_logits.kb = d / 64;
-        fused_logits.g = ws_grid_limit(m->device);
+        fused_logits.g = ws_grid(m->device, c.vocab, d);
         fused_logits.rows = rows;
     }
     for (int l = 0; l < c.n_layers && !fused; ++l) {
