@@ -131,7 +131,52 @@ struct AttnArgs {
 
 template <int HD, int NW>
 __global__ void __launch_bounds__(NW * 32) k_tree_attn_mma(AttnArgs a) {
-    pdl_enter();
+    pdl_launch_dependents();
+    constexpr int CHUNKS = HD / 8;         // 16-byte chunks per row
+    extern __shared__ __align__(128) uint8_t smem_raw[];
+    bf16* sk = reinterpret_cast<bf16*>(smem_raw);                 // [TA_STAGES][TA_BLK][HD]
+    bf16* sv = sk + TA_STAGES * TA_BLK * HD;                      // [TA_STAGES][TA_BLK][HD]
+    // Before waiting for the previous kernel (which writes the tree's own K/V rows and q): start
+    // fetching this CTA's first key blocks if they lie entirely in the committed part of the cache,
+    // which no kernel of this pass writes.  The committed length and the tree size are read here on
+    // trust -- nothing orders this read after the kernels that wrote them -- and read again after the
+    // wait: the early blocks are used only if both reads agree, otherwise they are fetched again.
+    // The cache block's address and capacity never change after the cache was created.
+    const int pre_hh = blockIdx.x, pre_b = blockIdx.z;
+    const size_t pre_cp = a.cap[pre_b];
+    const bf16* pre_kg = reinterpret_cast<const bf16*>(a.base[pre_b]) + (((size_t)a.layer * 2 + 0) * a.H + pre_hh) * pre_cp * HD;
+    const bf16* pre_vg = reinterpret_cast<const bf16*>(a.base[pre_b]) + (((size_t)a.layer * 2 + 1) * a.H + pre_hh) * pre_cp * HD;
+    __shared__ int s_pre[2];               // one thread reads, so that the whole CTA acts on the same values
+    if (threadIdx.x == 0) {
+        s_pre[0] = __ldcg(a.len + pre_b);
+        s_pre[1] = __ldcg(a.row_off + pre_b + 1) - __ldcg(a.row_off + pre_b);
+    }
+    __syncthreads();
+    const int pre_L = s_pre[0], pre_T = s_pre[1];
+    int pre_blk0 = 0, n_pre = 0;
+    if (pre_L >= 0 && pre_T >= 1 && pre_T <= ADED_MAX_NODES && (size_t)pre_L + pre_T <= pre_cp) {
+        const int nb_p = (pre_L + pre_T + TA_BLK - 1) / TA_BLK;
+        const int bps_p = (nb_p + a.n_splits - 1) / a.n_splits;
+        pre_blk0 = blockIdx.y * bps_p;
+        const int blk1_p = min(nb_p, pre_blk0 + bps_p);
+#pragma unroll
+        for (int st = 0; st < TA_STAGES - 1; ++st) {
+            const int blk = pre_blk0 + st;
+            if (n_pre == st && blk < blk1_p && (blk + 1) * TA_BLK <= pre_L) {
+                bf16* dk = sk + (size_t)st * TA_BLK * HD;
+                bf16* dv = sv + (size_t)st * TA_BLK * HD;
+                for (int e = threadIdx.x; e < TA_BLK * CHUNKS; e += NW * 32) {
+                    const int row = e / CHUNKS, chunk = e % CHUNKS;
+                    const size_t pos = (size_t)blk * TA_BLK + row;
+                    cp_async16(tile_chunk<HD>(dk, row, chunk), pre_kg + pos * HD + chunk * 8);
+                    cp_async16(tile_chunk<HD>(dv, row, chunk), pre_vg + pos * HD + chunk * 8);
+                }
+                cp_async_commit();
+                ++n_pre;
+            }
+        }
+    }
+    pdl_wait();
     // The status word is fetched along with the rest of the call's metadata and acted on before the
     // first store, so that it does not cost a memory round trip of its own.  Until then nothing is
     // written, and every load below stays inside the cache block and the row arrays whatever a failed
@@ -139,16 +184,12 @@ __global__ void __launch_bounds__(NW * 32) k_tree_attn_mma(AttnArgs a) {
     const int pass_status = *a.status;
     constexpr int KSTEPS = HD / 16;        // k steps of Q K^T
     constexpr int ONT = HD / 8;            // n tiles of the output
-    constexpr int CHUNKS = HD / 8;         // 16-byte chunks per row
-    extern __shared__ __align__(128) uint8_t smem_raw[];
-    bf16* sk = reinterpret_cast<bf16*>(smem_raw);                 // [TA_STAGES][TA_BLK][HD]
-    bf16* sv = sk + TA_STAGES * TA_BLK * HD;                      // [TA_STAGES][TA_BLK][HD]
 
     const int hh = blockIdx.x, split = blockIdx.y, b = blockIdx.z;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, tig = lane & 3;
     const int off = a.row_off[b];
     const int T = a.row_off[b + 1] - off;
-    const int L = a.len[b];
+    const int L = __ldcg(a.len + b);
     const size_t cp = a.cap[b];
     const int n_keys = L + T;
     const int nb = (n_keys + TA_BLK - 1) / TA_BLK;
@@ -204,8 +245,15 @@ __global__ void __launch_bounds__(NW * 32) k_tree_attn_mma(AttnArgs a) {
     // exactly one group (an empty one past the end), so "all but the newest TA_STAGES - 2 groups have
     // landed" always means the current block has.  (A split past the last key block has nothing to do
     // but still joins the merge.)
+    if (n_pre > 0 && (L != pre_L || T != pre_T || blk0 != pre_blk0)) {
+        // the early reads were stale: let the early copies land, then fetch the right blocks over them
+        cp_async_wait<0>();
+        __syncthreads();
+        n_pre = 0;
+    }
 #pragma unroll
     for (int s = 0; s < TA_STAGES - 1; ++s) {
+        if (s < n_pre) continue;           // already in flight
         if (blk0 + s < blk1) load_block(blk0 + s, s); else cp_async_commit();
     }
     for (int blk = blk0; blk < blk1; ++blk) {
