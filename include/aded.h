@@ -159,6 +159,29 @@ aded_status aded_verify_host(aded_model* m, aded_kv* kv, const int32_t* tree_tok
                              const int32_t* tree_parents_host, int32_t n_nodes, int32_t* out_tokens_host,
                              int32_t* out_accept_len_host, void* stream);
 
+/* Sampling-mode verification ("Draft Construction and Verification": at every position a token is
+ * sampled from the model's distribution and compared with the draft token; Figure 5: temperature and
+ * top-p).  Same as aded_verify, except that node i's token is drawn with the uniform number u_dev[i]
+ * (float32 in [0, 1), device, n_nodes of them, supplied by the caller -- the library draws no random
+ * numbers) from softmax(logits / temperature) restricted to the top-p nucleus, by the rule of
+ * aded_sample_tokens.  temperature > 0, 2^-16 <= top_p <= 1, vocab <= 32768, else
+ * ADED_ERR_INVALID_ARG / ADED_ERR_UNSUPPORTED. */
+aded_status aded_verify_sampled(aded_model* m, aded_kv* kv, const int32_t* tree_tokens_dev,
+                                const int32_t* tree_parents_dev, int32_t n_nodes, float temperature, float top_p,
+                                const float* u_dev, int32_t* out_tokens_dev, int32_t* out_accept_len_dev, void* stream);
+
+/* The drawing rule alone: out_tokens_dev[r] for r < rows from logits_dev[r][0 .. vocab) (float32, row
+ * stride vocab, finite or -inf) and u_dev[r].  The paper does not fix a rule; this one is exact
+ * integer arithmetic after one rounded exponential per logit, so two implementations agree bit for
+ * bit:  m = max logit;  t = fl32(fl32(l - m) * fl32(log2(e) / temperature));  n = floor(t), f = t - n;
+ * r = 2^f by a fixed degree-6 polynomial in float32 (Horner, every product and sum rounded);
+ * weight q = floor(r * 2^30) >> (-n);  need = ceil(sum q * floor(top_p * 65536) / 65536);  nucleus =
+ * shortest prefix in (q descending, id ascending) order with mass >= need, Z its mass;  target =
+ * floor(Z * floor(u * 2^24) / 2^24);  result = first nucleus token in id order whose running mass
+ * exceeds target.  Asynchronous on `stream`. */
+aded_status aded_sample_tokens(const float* logits_dev, int32_t rows, int32_t vocab, float temperature, float top_p,
+                               const float* u_dev, int32_t* out_tokens_dev, void* stream);
+
 /* Ask the next verify call to also write every node's logits ([rows][vocab] fp32, may be NULL)
  * and greedy token ([rows] int32, may be NULL) to the given device buffers.  Parity checks only. */
 aded_status aded_debug_capture(aded_model* m, float* logits_dev, int32_t* best_dev);

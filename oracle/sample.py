@@ -10,7 +10,7 @@ exponential per logit, so that two implementations that follow it agree bit for 
   2. n = floor(t_v), f = t_v - n (exact);  r = P(f), the degree-6 polynomial below evaluated by
      Horner's rule in float32 with separately rounded multiplications and additions (1 <= r < 2,
      relative error against 2^f below 1e-7);  weight q_v = floor(r * 2^30) >> (-n)  (0 for n < -40):
-     an unsigned fixed-point value of 2^t_v with 30 fractional bits
+     an unsigned fixed-point value of 2^t_v with 30 fractional bits; a logit of -inf has weight 0
   3. total = sum q_v;  need = ceil(total * floor(top_p * 65536) / 65536)
   4. nucleus = shortest prefix of the tokens ordered by (q descending, id ascending) whose weights
      sum to at least need;  Z = its sum
@@ -38,7 +38,8 @@ def weights(logits: Sequence[float], temperature: float) -> np.ndarray:
     l = np.asarray(logits, dtype=f32)
     m = l.max()
     c = f32(f32(LOG2E) / f32(temperature))
-    t = ((l - m).astype(f32) * c).astype(f32)
+    dead = np.isneginf(l)                      # a logit of -inf has weight 0
+    t = ((np.where(dead, m, l) - m).astype(f32) * c).astype(f32)
     n = np.floor(t)
     f = (t - n).astype(f32)
     r = np.full_like(f, f32(EXP2_COEF[6]))
@@ -48,6 +49,7 @@ def weights(logits: Sequence[float], temperature: float) -> np.ndarray:
     big = np.floor(r.astype(np.float64) * 2.0 ** 30).astype(np.uint64)
     shift = (-n).astype(np.int64)
     q = np.where(shift <= 40, big >> np.minimum(shift, 40).astype(np.uint64), 0).astype(np.uint64)
+    q[dead] = 0
     return q
 
 
@@ -68,8 +70,8 @@ def nucleus(q: np.ndarray, top_p: float) -> List[int]:
 
 def sample(logits: Sequence[float], temperature: float, top_p: float, u: float) -> int:
     """One token drawn by the rule of the module header."""
-    if not (temperature > 0.0 and 0.0 < top_p <= 1.0 and 0.0 <= u < 1.0):
-        raise ValueError("temperature > 0, 0 < top_p <= 1, 0 <= u < 1")
+    if not (temperature > 0.0 and 2.0 ** -16 <= top_p <= 1.0 and 0.0 <= u < 1.0):
+        raise ValueError("temperature > 0, 2^-16 <= top_p <= 1, 0 <= u < 1")
     q = weights(logits, temperature)
     members = sorted(nucleus(q, top_p))
     z = sum(int(q[v]) for v in members)
@@ -81,6 +83,14 @@ def sample(logits: Sequence[float], temperature: float, top_p: float, u: float) 
         if run > target:
             return v
     raise AssertionError("unreachable: target < Z")
+
+
+def chooser(temperature: float, top_p: float, u: Sequence[float]):
+    """Per-node token choice for oracle.verify.verify(choose=...): node i draws with u[i] from its
+    logits rounded to float32 (the precision the rule is stated in)."""
+    def choose(logits: np.ndarray) -> np.ndarray:
+        return sample_rows(np.asarray(logits, dtype=np.float32), temperature, top_p, u)
+    return choose
 
 
 def sample_rows(logits: np.ndarray, temperature: float, top_p: float, u: Sequence[float]) -> np.ndarray:

@@ -276,11 +276,12 @@ def accept_walk(tokens: Sequence[int], parents: Sequence[int], best: Sequence[in
         path.append(cur)
 
 
-def verify(arch: Arch, w: Weights, cache: Cache, tokens: Sequence[int], parents: Sequence[int]):
+def verify(arch: Arch, w: Weights, cache: Cache, tokens: Sequence[int], parents: Sequence[int], choose=None):
     """One verification step.  Appends the accepted path's K/V to the cache (root first) and
-    returns a dict with out_tokens, accept_len, path, best (per-node greedy token), logits."""
+    returns a dict with out_tokens, accept_len, path, best (per-node chosen token), logits.
+    `choose` maps the logits [n, V] to one token per node; the default is the greedy choice."""
     logits, k_new, v_new = forward_tree(arch, w, cache, tokens, parents)
-    best = greedy(logits)
+    best = greedy(logits) if choose is None else np.asarray(choose(logits), dtype=np.int64)
     path, out = accept_walk(tokens, parents, best)
     for l in range(arch.n_layers):
         cache.k[l] = np.concatenate([cache.k[l], k_new[l][:, path]], axis=1)

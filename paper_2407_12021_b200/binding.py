@@ -28,7 +28,7 @@ EXPORTS = [
     "aded_debug_capture", "aded_debug_capture_hidden", "aded_debug_gemm", "aded_debug_read_buffer", "aded_greedy_noalloc", "aded_profile_begin", "aded_profile_end", "aded_launch_count", "aded_model_poll_status", "aded_trigram_create", "aded_trigram_destroy",
     "aded_trigram_update", "aded_trigram_update_host", "aded_trigram_topk", "aded_trigram_topk_host",
     "aded_trigram_get", "aded_trigram_stats", "aded_trigram_poll_status", "aded_draft_tree", "aded_decode_step",
-    "aded_decode_step_host", "aded_status_string",
+    "aded_decode_step_host", "aded_verify_sampled", "aded_sample_tokens", "aded_status_string",
 ]
 
 
@@ -428,6 +428,34 @@ def aded_decode_step_host(model: Model, kv: KV, t: Trigram, context_dev: torch.T
                                       c_int32(max_depth), c_int32(k), _ptr(filler_host), c_int32(nf),
                                       _ptr(out_tokens_host), _ptr(out_accept_len_host), _stream()),
            "aded_decode_step_host")
+
+
+def _dev_f32(t: torch.Tensor, what: str) -> torch.Tensor:
+    if not (t.is_cuda and t.dtype == torch.float32 and t.is_contiguous()):
+        raise TypeError(f"{what} must be a contiguous CUDA float32 tensor")
+    return t
+
+
+def aded_verify_sampled(model: Model, kv: KV, tree_tokens: torch.Tensor, tree_parents: torch.Tensor, temperature: float,
+                        top_p: float, u: torch.Tensor, out_tokens: torch.Tensor, out_accept_len: torch.Tensor) -> None:
+    """aded_verify with node i's token drawn with u[i] (CUDA float32 [n_nodes]) instead of the greedy choice."""
+    _dev_i32(tree_tokens, "tree_tokens"), _dev_i32(tree_parents, "tree_parents")
+    _dev_i32(out_tokens, "out_tokens"), _dev_i32(out_accept_len, "out_accept_len"), _dev_f32(u, "u")
+    n = tree_tokens.numel()
+    if tree_parents.numel() != n or out_tokens.numel() < n or out_accept_len.numel() < 1 or u.numel() < n:
+        raise ValueError("array lengths do not match the tree")
+    _check(_lib.aded_verify_sampled(model.handle, kv.handle, _ptr(tree_tokens), _ptr(tree_parents), c_int32(n),
+                                    c_float(temperature), c_float(top_p), _ptr(u), _ptr(out_tokens), _ptr(out_accept_len),
+                                    _stream()), "aded_verify_sampled")
+
+
+def aded_sample_tokens(logits: torch.Tensor, temperature: float, top_p: float, u: torch.Tensor, out_tokens: torch.Tensor) -> None:
+    """logits CUDA float32 [rows, vocab]; u CUDA float32 [rows]; out_tokens CUDA int32 [rows]."""
+    _dev_f32(logits, "logits"), _dev_f32(u, "u"), _dev_i32(out_tokens, "out_tokens")
+    if logits.dim() != 2 or u.numel() < logits.shape[0] or out_tokens.numel() < logits.shape[0]:
+        raise ValueError("logits must be [rows, vocab] with one u and one output per row")
+    _check(_lib.aded_sample_tokens(_ptr(logits), c_int32(logits.shape[0]), c_int32(logits.shape[1]), c_float(temperature),
+                                   c_float(top_p), _ptr(u), _ptr(out_tokens), _stream()), "aded_sample_tokens")
 
 
 def aded_status_string(status: int) -> str:

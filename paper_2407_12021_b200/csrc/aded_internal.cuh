@@ -135,6 +135,11 @@ struct aded_model {
     aded::CallPtrs* call_dev;   // device copy of the current call's array pointers
     std::vector<void*> owned;   // everything cudaMalloc'ed for this handle
 
+    // sampling-mode verification (aded_verify_sampled): armed for one call
+    bool samp_on;
+    float samp_temp, samp_top_p;
+    const float* samp_u;        // caller's [rows] uniform numbers (device)
+
     float* dbg_logits;
     int32_t* dbg_best;
     void* dbg_hidden;   // [n_layers + 1][rows][d] copies of the residual stream (debug capture)
@@ -221,6 +226,11 @@ enum { WS_MAP_QKV = 0, WS_MAP_O = 1, WS_MAP_GU = 2, WS_MAP_D = 3 };   // per-lay
 // fused_ws.cu
 bool fw_prepare(int device);
 cudaError_t fw_launch(aded_model* m, aded_kv* kv, const FwPair* pairs, int n_pairs, int rows, int launch_index, cudaStream_t st);
+
+// sample.cu
+bool sample_supported(int vocab);
+cudaError_t launch_sample_rows(const float* logits, int rows, int vocab, int ld, float temperature, float top_p, const float* u,
+                               int32_t* out, const int32_t* status, cudaStream_t st);
 
 // tree_attention.cu
 // max_tree: most nodes any sequence's tree has in this call

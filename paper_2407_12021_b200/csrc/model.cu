@@ -265,7 +265,14 @@ static aded_status enqueue_pass(aded_model* m, aded_kv* kv, const int32_t* offse
         GemmOut lg = fused_logits;
         if (!fused) { Span sp(m, PROF_GEMM, 1, st); lg = launch_gemm(m, 4 * c.n_layers, xm, m->x, m->top.lm_head, m->logits, rows, c.vocab, d, st); }
         Span sp(m, PROF_OTHER, 3, st);
-        launch_argmax(m, lg, rows, st);
+        if (m->samp_on) {
+            // sampling mode: the logits as a dense matrix, then one drawn token per node in place of the greedy one
+            launch_materialize(m, lg, m->logits, rows, st);
+            ADED_CUDA_TRY(launch_sample_rows(m->logits, rows, c.vocab, c.vocab, m->samp_temp, m->samp_top_p, m->samp_u, m->best,
+                                             m->status, st));
+        } else {
+            launch_argmax(m, lg, rows, st);
+        }
         if (m->dbg_logits) launch_materialize(m, lg, m->dbg_logits, rows, st);
         if (m->dbg_best)
             ADED_CUDA_TRY(cudaMemcpyAsync(m->dbg_best, m->best, (size_t)rows * sizeof(int32_t),
@@ -327,7 +334,7 @@ static aded_status forward(aded_model* m, aded_kv* kv, const int32_t* tokens, co
 
     cudaStreamCaptureStatus cap_state = cudaStreamCaptureStatusNone;
     cudaStreamIsCapturing(st, &cap_state);
-    const bool direct = !m->graphs_on || m->dbg_logits || m->dbg_best || m->dbg_hidden || cap_state != cudaStreamCaptureStatusNone;
+    const bool direct = !m->graphs_on || m->samp_on || m->dbg_logits || m->dbg_best || m->dbg_hidden || cap_state != cudaStreamCaptureStatusNone;
     if (direct) {
         aded_status s = enqueue_pass(m, kv, offsets_host, batch, rows, max_tree, chain_mode, st);
         m->dbg_logits = nullptr;
@@ -422,6 +429,10 @@ aded_status aded_model_create(const aded_model_config* cfg, const aded_weights* 
     m->dbg_logits = nullptr;
     m->dbg_best = nullptr;
     m->dbg_hidden = nullptr;
+    m->samp_on = false;
+    m->samp_temp = 1.f;
+    m->samp_top_p = 1.f;
+    m->samp_u = nullptr;
     m->prof_on = false;
     m->capture_spans = nullptr;
     m->prof_pending = -1;
@@ -603,6 +614,22 @@ aded_status aded_verify(aded_model* m, aded_kv* kv, const int32_t* tree_tokens_d
     const int32_t off[2] = {0, n_nodes};
     return aded_verify_batch(m, kv, off, tree_tokens_dev, tree_parents_dev, out_tokens_dev, n_nodes,
                              out_accept_len_dev, stream);
+}
+
+aded_status aded_verify_sampled(aded_model* m, aded_kv* kv, const int32_t* tree_tokens_dev,
+                                const int32_t* tree_parents_dev, int32_t n_nodes, float temperature, float top_p,
+                                const float* u_dev, int32_t* out_tokens_dev, int32_t* out_accept_len_dev, void* stream) {
+    if (!m || !u_dev) return ADED_ERR_INVALID_ARG;
+    if (!(temperature > 0.f) || !(top_p >= 1.f / 65536.f) || !(top_p <= 1.f)) return ADED_ERR_INVALID_ARG;
+    if (!sample_supported(m->cfg.vocab)) return ADED_ERR_UNSUPPORTED;
+    m->samp_on = true;
+    m->samp_temp = temperature;
+    m->samp_top_p = top_p;
+    m->samp_u = u_dev;
+    const aded_status s = aded_verify(m, kv, tree_tokens_dev, tree_parents_dev, n_nodes, out_tokens_dev, out_accept_len_dev, stream);
+    m->samp_on = false;
+    m->samp_u = nullptr;
+    return s;
 }
 
 aded_status aded_verify_host(aded_model* m, aded_kv* kv, const int32_t* tree_tokens_host,

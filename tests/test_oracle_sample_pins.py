@@ -16,6 +16,7 @@ def test_power_of_two_weights_by_hand():
     assert q.tolist() == [2 ** 30, 2 ** 29, 2 ** 28, 2 ** 27]
     # shifts: 2^-41 and below leave nothing of the 31-bit mantissa
     assert osmp.weights([5, 5, -25, -26, -200], T1).tolist() == [2 ** 30, 2 ** 30, 1, 0, 0]
+    assert osmp.weights([0, -np.inf, -1], T1).tolist() == [2 ** 30, 0, 2 ** 29]
     # top-p 0.5: the first token alone carries 8/15 of the mass
     assert osmp.nucleus(q, 0.5) == [0]
     assert all(osmp.sample([0, -1, -2, -3], T1, 0.5, u) == 0 for u in (0.0, 0.3, 0.999))
