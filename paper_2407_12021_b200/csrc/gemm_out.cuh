@@ -94,15 +94,19 @@ __device__ __forceinline__ float4 gemm_out_at4(const GemmOut& o, const TileRef& 
     const float* p = o.slots + region + ((size_t)t.first_slot * rb + (r & 127)) * 128 + col;
     const size_t stride = (size_t)rb * 128;
     float4 sum = make_float4(0.f, 0.f, 0.f, 0.f);
-    int i = 0;
-    for (; i + 4 <= t.count; i += 4) {     // four loads in flight, added in order
-        const float4 a = __ldcg(reinterpret_cast<const float4*>(p + (size_t)i * stride));
-        const float4 b = __ldcg(reinterpret_cast<const float4*>(p + (size_t)(i + 1) * stride));
-        const float4 c = __ldcg(reinterpret_cast<const float4*>(p + (size_t)(i + 2) * stride));
-        const float4 d = __ldcg(reinterpret_cast<const float4*>(p + (size_t)(i + 3) * stride));
-        sum = f4_add(f4_add(f4_add(f4_add(sum, a), b), c), d);
+    // Up to GO_BATCH contributors are fetched at once (predicated loads, no branch between them) and
+    // then added in CTA order: a projection with few tiles (O, down: 32 tiles over 296 CTAs) has about
+    // ten contributors per tile, and a loop that fetched them four at a time cost three L2 round trips.
+    constexpr int GO_BATCH = 12;
+    for (int i0 = 0; i0 < t.count; i0 += GO_BATCH) {
+        float4 v[GO_BATCH];
+#pragma unroll
+        for (int j = 0; j < GO_BATCH; ++j)
+            v[j] = i0 + j < t.count ? __ldcg(reinterpret_cast<const float4*>(p + (size_t)(i0 + j) * stride)) : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+        for (int j = 0; j < GO_BATCH; ++j)
+            if (i0 + j < t.count) sum = f4_add(sum, v[j]);
     }
-    for (; i < t.count; ++i) sum = f4_add(sum, __ldcg(reinterpret_cast<const float4*>(p + (size_t)i * stride)));
     return sum;
 }
 
