@@ -176,6 +176,50 @@ def test_graph_replay_gives_the_same_steps(cuda_device, monkeypatch):
         root = cpu["out_tokens"][-1]
 
 
+@pytest.mark.parametrize("heads,hd,layers,ffn", [(4, 64, 2, 384), (8, 128, 3, 2048)])
+def test_persistent_projection_kernel_matches_separate_kernels(cuda_device, monkeypatch, heads, hd, layers, ffn):
+    """A model created with ADED_FUSED set runs the projections of a layer and the steps between them in
+    one persistent kernel with grid barriers.  Same arithmetic and the same order of the partial
+    sums of every projection; only the RMSNorm's sum of squares is added up in another order (128
+    threads per row instead of 1024), so activations and cache rows of the first layer may differ in the last bf16 bit, later ones by what
+    that grows to.
+    Also covers projections with fewer work units than CTAs."""
+    from paper_2407_12021_b200 import binding as B
+    shape = gen.ModelShape(f"bf16-{heads}x{hd}", layers, heads * hd, heads, hd, ffn, 1024, "bf16")
+    w = H.weights_to(gen.model_weights(shape, 77), cuda_device)
+    prompt = gen.zipf_tokens(91, shape.vocab, 77, 50).to(torch.int32).cuda()
+    tokens, parents = gen.make_tree(48, 5, 4, shape.vocab, 78, root_token=int(prompt[-1]))
+    results = []
+    for fused in (False, True):
+        if fused:
+            monkeypatch.setenv("ADED_FUSED", "1")
+        else:
+            monkeypatch.delenv("ADED_FUSED", raising=False)
+        m = B.aded_model_create(shape, w, max_rows=128, max_batch=1)
+        kv = B.aded_kv_create(m, [512])
+        n0 = B.aded_launch_count()
+        B.aded_append(m, kv, prompt[:-1].contiguous())
+        launches = B.aded_launch_count() - n0
+        out = torch.full((48,), -7, dtype=torch.int32, device="cuda")
+        alen = torch.full((1,), -7, dtype=torch.int32, device="cuda")
+        B.aded_verify(m, kv, H.i32(tokens), H.i32(parents), out, alen)
+        torch.cuda.synchronize()
+        assert B.aded_model_poll_status(m) == 0
+        bufs = [B.aded_debug_read_buffer(m, i, 48).clone() for i in range(5)]
+        n = B.aded_kv_len(kv, 0)
+        rows = [t.clone() for l in range(layers) for t in B.aded_kv_read(kv, 0, l, 0, n)]
+        torch.cuda.synchronize()
+        results.append((launches, out.tolist(), int(alen[0]), n, bufs, rows))
+    monkeypatch.delenv("ADED_FUSED", raising=False)
+    (l0, out0, a0, n0_, b0, r0), (l1, out1, a1, n1, b1, r1) = results
+    assert l1 < l0, "the persistent kernel was not used"
+    assert (out0, a0, n0_) == (out1, a1, n1)
+    for x, y in zip(b0 + r0, b1 + r1):
+        x, y = x.float(), y.float()
+        # a last-bit difference after one layer grows through the next ones (a random-init network amplifies one-ulp differences)
+        assert (x - y).abs().max() <= 2e-2 * x.abs().max()
+
+
 def test_c2_one_7b_layer_bf16(cuda_device):
     """Workload 2: one Llama-2-7B-shaped layer + LM head in bf16, cache pre-filled with 1024 N(0,1)
     positions, 64-node depth-6 tree with branching <= 4."""
