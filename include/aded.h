@@ -274,6 +274,30 @@ aded_status aded_trigram_stats(const aded_trigram* t, uint64_t* out_entries_host
 /* Read and clear the store's device status word; synchronises `stream`. */
 aded_status aded_trigram_poll_status(aded_trigram* t, aded_status* out_host, void* stream);
 
+/* ---- keeping and trimming the table (the tri-gram matrix is "initialised from a corpus" and kept
+ * between runs; "threshold for the elimination of tri-gram probability", Detailed Experimental
+ * Settings) ------------------------------------------------------------------------------------ */
+
+/* Every stored tri-gram whose count is >= min_count: keys_dev[3*i .. 3*i+2] = (w_{i-2}, w_{i-1}, w_i),
+ * counts_dev[i] = its count, in no particular order.  *n_out_host = how many there are; only the
+ * first max_entries are written (call with max_entries = 0 to size the arrays).  Synchronises. */
+aded_status aded_trigram_export(const aded_trigram* t, uint32_t min_count, int32_t* keys_dev, uint32_t* counts_dev,
+                                uint64_t max_entries, uint64_t* n_out_host, void* stream);
+/* Adds n exported entries to the table: counts of tri-grams already present add up (saturating at
+ * the cap).  Asynchronous. */
+aded_status aded_trigram_import(aded_trigram* t, const int32_t* keys_dev, const uint32_t* counts_dev, uint64_t n,
+                                void* stream);
+/* Empties the table (the status word is kept).  Asynchronous. */
+aded_status aded_trigram_clear(aded_trigram* t, void* stream);
+/* Removes every tri-gram whose count is below min_count and gives its buckets back: the table is
+ * rebuilt from the entries that stay.  Allocates a scratch copy of them; synchronises. */
+aded_status aded_trigram_prune(aded_trigram* t, uint32_t min_count, void* stream);
+/* Writes / reads the table's entries to / from a file on the host ("ADEDTG01", vocab, entry count,
+ * keys, counts; native byte order).  Loading ADDS the file's entries to the table (clear it first for
+ * a copy) and refuses a file written for another vocabulary size.  Both synchronise. */
+aded_status aded_trigram_save(const aded_trigram* t, const char* path, void* stream);
+aded_status aded_trigram_load(aded_trigram* t, const char* path, void* stream);
+
 /* ---- draft retrieval and the decoding step on the device ------------------------------------
  * Figure 1's loop -- update the tri-gram matrix, retrieve candidate continuations from it with the
  * last two tokens of the text, hand them to the model as one prefix-sharing pseudo-sequence

@@ -52,5 +52,18 @@ class TrigramStore:
         cnts = [n for _, n in items] + [0] * (k - len(items))
         return toks, cnts
 
+    def prune(self, min_count: int) -> None:
+        """Removes every tri-gram whose count is below min_count (the "threshold for the elimination of
+        tri-gram probability" of the experimental settings, on the count scale); contexts left without a
+        continuation disappear."""
+        self.table = {ctx: kept for ctx, kept in
+                      ((ctx, {c: n for c, n in row.items() if n >= min_count}) for ctx, row in self.table.items()) if kept}
+
+    def merge(self, entries: Dict[Tuple[int, int, int], int]) -> None:
+        """Adds stored entries (as returned by entries()) to the table: counts add up, saturating at the cap."""
+        for (a, b, c), n in entries.items():
+            row = self.table.setdefault((int(a), int(b)), {})
+            row[int(c)] = min(row.get(int(c), 0) + int(n), self.cap)
+
     def entries(self) -> Dict[Tuple[int, int, int], int]:
         return {(a, b, c): n for (a, b), row in self.table.items() for c, n in row.items()}

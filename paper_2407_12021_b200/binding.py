@@ -28,7 +28,8 @@ EXPORTS = [
     "aded_debug_capture", "aded_debug_capture_hidden", "aded_debug_gemm", "aded_debug_read_buffer", "aded_greedy_noalloc", "aded_profile_begin", "aded_profile_end", "aded_launch_count", "aded_model_poll_status", "aded_trigram_create", "aded_trigram_destroy",
     "aded_trigram_update", "aded_trigram_update_host", "aded_trigram_topk", "aded_trigram_topk_host",
     "aded_trigram_get", "aded_trigram_stats", "aded_trigram_poll_status", "aded_draft_tree", "aded_decode_step",
-    "aded_decode_step_host", "aded_verify_sampled", "aded_sample_tokens", "aded_status_string",
+    "aded_decode_step_host", "aded_verify_sampled", "aded_sample_tokens", "aded_trigram_export",
+    "aded_trigram_import", "aded_trigram_clear", "aded_trigram_prune", "aded_trigram_save", "aded_trigram_load", "aded_status_string",
 ]
 
 
@@ -456,6 +457,46 @@ def aded_sample_tokens(logits: torch.Tensor, temperature: float, top_p: float, u
         raise ValueError("logits must be [rows, vocab] with one u and one output per row")
     _check(_lib.aded_sample_tokens(_ptr(logits), c_int32(logits.shape[0]), c_int32(logits.shape[1]), c_float(temperature),
                                    c_float(top_p), _ptr(u), _ptr(out_tokens), _stream()), "aded_sample_tokens")
+
+
+def aded_trigram_export(t: Trigram, min_count: int = 0):
+    """(keys [n, 3] int32, counts [n] int32 holding uint32 bit patterns) of the entries with count >= min_count, on the device."""
+    n = c_uint64()
+    _check(_lib.aded_trigram_export(t.handle, c_uint32(min_count), None, None, c_uint64(0), ctypes.byref(n), _stream()),
+           "aded_trigram_export")
+    keys = torch.empty((n.value, 3), dtype=torch.int32, device="cuda")
+    counts = torch.empty((n.value,), dtype=torch.int32, device="cuda")
+    if n.value:
+        m = c_uint64()
+        _check(_lib.aded_trigram_export(t.handle, c_uint32(min_count), _ptr(keys), _ptr(counts), c_uint64(n.value),
+                                        ctypes.byref(m), _stream()), "aded_trigram_export")
+        if m.value != n.value:
+            raise RuntimeError("the table changed during the export")
+    return keys, counts
+
+
+def aded_trigram_import(t: Trigram, keys: torch.Tensor, counts: torch.Tensor) -> None:
+    _dev_i32(keys, "keys"), _dev_i32(counts, "counts")
+    n = counts.numel()
+    if keys.numel() != 3 * n:
+        raise ValueError("keys must hold three tokens per count")
+    _check(_lib.aded_trigram_import(t.handle, _ptr(keys), _ptr(counts), c_uint64(n), _stream()), "aded_trigram_import")
+
+
+def aded_trigram_clear(t: Trigram) -> None:
+    _check(_lib.aded_trigram_clear(t.handle, _stream()), "aded_trigram_clear")
+
+
+def aded_trigram_prune(t: Trigram, min_count: int) -> None:
+    _check(_lib.aded_trigram_prune(t.handle, c_uint32(min_count), _stream()), "aded_trigram_prune")
+
+
+def aded_trigram_save(t: Trigram, path: str) -> None:
+    _check(_lib.aded_trigram_save(t.handle, path.encode(), _stream()), "aded_trigram_save")
+
+
+def aded_trigram_load(t: Trigram, path: str) -> None:
+    _check(_lib.aded_trigram_load(t.handle, path.encode(), _stream()), "aded_trigram_load")
 
 
 def aded_status_string(status: int) -> str:

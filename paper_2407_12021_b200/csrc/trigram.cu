@@ -8,7 +8,9 @@
 // continuations are therefore reachable from one hash probe, which is what top-k needs, and an
 // update is one probe plus one atomic add.
 #include <cstdio>
+#include <cstring>
 #include <new>
+#include <vector>
 
 #include "aded_internal.cuh"
 
@@ -79,18 +81,9 @@ __global__ void k_tg_init(Bucket* b, size_t n) {
     }
 }
 
-// Algorithm 2, one thread per window.  Duplicate windows inside one call are independent atomic
-// adds, so the result is min(count + multiplicity, cap) whatever the thread order.
-// `n_dev` (may be NULL): the span length lives on the device (at most n).
-__global__ void k_tg_update(TgView t, const int32_t* __restrict__ tok, int n, const int32_t* __restrict__ n_dev) {
-    const int i = blockIdx.x * blockDim.x + threadIdx.x + 2;
-    if (n_dev && *n_dev < n) n = *n_dev;
-    if (i >= n || *t.status != 0) return;
-    const int a = tok[i - 2], b = tok[i - 1], c = tok[i];
-    if (a < 0 || b < 0 || c < 0 || a >= t.vocab || b >= t.vocab || c >= t.vocab) {
-        atomicCAS(t.status, 0, (int)ADED_ERR_INVALID_ARG);
-        return;
-    }
+// Raises the count of tri-gram (a, b, c) by `inc` (1 <= inc <= cap), inserting it if absent; counts
+// saturate at the cap.  Independent atomic adds: the result does not depend on the thread order.
+__device__ __forceinline__ void tg_add(const TgView& t, int a, int b, int c, uint32_t inc) {
     const unsigned long long key = tg_key(a, b);
     int64_t cur = tg_find_home(t, key, true);
     if (cur < 0) { atomicCAS(t.status, 0, (int)ADED_ERR_TABLE_FULL); return; }
@@ -101,8 +94,8 @@ __global__ void k_tg_update(TgView t, const int32_t* __restrict__ tok, int n, co
             int32_t have = *reinterpret_cast<volatile int32_t*>(&bk->e[e].tok);
             if (have == -1) have = atomicCAS(&bk->e[e].tok, -1, c) == -1 ? c : *reinterpret_cast<volatile int32_t*>(&bk->e[e].tok);
             if (have == c) {
-                const uint32_t old = atomicAdd(&bk->e[e].cnt, 1u);
-                if (old >= t.cap) atomicMin(&bk->e[e].cnt, t.cap);
+                const uint32_t old = atomicAdd(&bk->e[e].cnt, inc);
+                if (old > t.cap - inc) atomicMin(&bk->e[e].cnt, t.cap);   // inc <= cap (callers clamp)
                 return;
             }
         }
@@ -136,6 +129,60 @@ __global__ void k_tg_update(TgView t, const int32_t* __restrict__ tok, int n, co
         cur = nxt;
     }
     atomicCAS(t.status, 0, (int)ADED_ERR_TIMEOUT);
+}
+
+// Algorithm 2, one thread per window.  Duplicate windows inside one call are independent atomic
+// adds, so the result is min(count + multiplicity, cap) whatever the thread order.
+// `n_dev` (may be NULL): the span length lives on the device (at most n).
+__global__ void k_tg_update(TgView t, const int32_t* __restrict__ tok, int n, const int32_t* __restrict__ n_dev) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x + 2;
+    if (n_dev && *n_dev < n) n = *n_dev;
+    if (i >= n || *t.status != 0) return;
+    const int a = tok[i - 2], b = tok[i - 1], c = tok[i];
+    if (a < 0 || b < 0 || c < 0 || a >= t.vocab || b >= t.vocab || c >= t.vocab) {
+        atomicCAS(t.status, 0, (int)ADED_ERR_INVALID_ARG);
+        return;
+    }
+    tg_add(t, a, b, c, 1u);
+}
+
+// Every stored tri-gram with count >= min_count as (a, b, c) and its count, in no particular order;
+// *n_out counts all of them, only the first `max_entries` are written.
+__global__ void k_tg_export(TgView t, uint32_t min_count, int32_t* __restrict__ keys, uint32_t* __restrict__ counts,
+                            unsigned long long max_entries, unsigned long long* n_out) {
+    const size_t n = (size_t)t.n_home + t.n_over;
+    for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
+        const Bucket* bk = t.buckets + i;
+        const unsigned long long key = bk->key;
+        if (key == TG_EMPTY) continue;
+        for (int e = 0; e < 6; ++e) {
+            const int32_t tk = bk->e[e].tok;
+            const uint32_t cn = bk->e[e].cnt;
+            if (tk < 0 || cn < min_count || cn == 0) continue;
+            const unsigned long long at = atomicAdd(n_out, 1ull);
+            if (at < max_entries) {
+                keys[3 * at + 0] = (int32_t)(key >> 32);
+                keys[3 * at + 1] = (int32_t)(key & 0xFFFFFFFFu);
+                keys[3 * at + 2] = tk;
+                counts[at] = cn;
+            }
+        }
+    }
+}
+
+// Adds exported entries to a table (counts add up, saturating).
+__global__ void k_tg_import(TgView t, const int32_t* __restrict__ keys, const uint32_t* __restrict__ counts, unsigned long long n) {
+    const unsigned long long i = blockIdx.x * (unsigned long long)blockDim.x + threadIdx.x;
+    if (i >= n || *t.status != 0) return;
+    const int a = keys[3 * i], b = keys[3 * i + 1], c = keys[3 * i + 2];
+    uint32_t inc = counts[i];
+    if (a < 0 || b < 0 || c < 0 || a >= t.vocab || b >= t.vocab || c >= t.vocab) {
+        atomicCAS(t.status, 0, (int)ADED_ERR_INVALID_ARG);
+        return;
+    }
+    if (inc == 0) return;
+    if (inc > t.cap) inc = t.cap;
+    tg_add(t, a, b, c, inc);
 }
 
 // One selection round of a warp over the chain that starts at `home`: the largest packed
@@ -544,6 +591,144 @@ aded_status aded_decode_step_host(aded_model* m, aded_kv* kv, aded_trigram* t, i
     ADED_CUDA_TRY(cudaMemcpyAsync(out_accept_len_host, m->out_len, sizeof(int32_t), cudaMemcpyDeviceToHost, st));
     ADED_CUDA_TRY(cudaStreamSynchronize(st));
     return ADED_OK;
+}
+
+// ---- persistence and pruning -----------------------------------------------------------------------
+aded_status aded_trigram_export(const aded_trigram* t, uint32_t min_count, int32_t* keys_dev, uint32_t* counts_dev,
+                                uint64_t max_entries, uint64_t* n_out_host, void* stream) {
+    if (!t || !n_out_host || (max_entries > 0 && (!keys_dev || !counts_dev))) return ADED_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    unsigned long long n = 0;
+    ADED_CUDA_TRY(cudaMemsetAsync(t->stats_dev, 0, sizeof n, st));
+    note_launch();
+    k_tg_export<<<1024, 256, 0, st>>>(t->view, min_count, keys_dev, counts_dev, max_entries, t->stats_dev);
+    ADED_CUDA_TRY(cudaMemcpyAsync(&n, t->stats_dev, sizeof n, cudaMemcpyDeviceToHost, st));
+    ADED_CUDA_TRY(cudaStreamSynchronize(st));
+    *n_out_host = n;
+    return ADED_OK;
+}
+
+aded_status aded_trigram_import(aded_trigram* t, const int32_t* keys_dev, const uint32_t* counts_dev, uint64_t n, void* stream) {
+    if (!t || (n > 0 && (!keys_dev || !counts_dev))) return ADED_ERR_INVALID_ARG;
+    if (n == 0) return ADED_OK;
+    note_launch();
+    k_tg_import<<<(unsigned int)((n + 255) / 256), 256, 0, static_cast<cudaStream_t>(stream)>>>(t->view, keys_dev, counts_dev, n);
+    ADED_CUDA_TRY(cudaGetLastError());
+    return ADED_OK;
+}
+
+aded_status aded_trigram_clear(aded_trigram* t, void* stream) {
+    if (!t) return ADED_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    note_launch();
+    k_tg_init<<<1024, 256, 0, st>>>(t->view.buckets, (size_t)t->view.n_home + t->view.n_over);
+    ADED_CUDA_TRY(cudaMemsetAsync(t->view.over_used, 0, sizeof(uint32_t), st));
+    ADED_CUDA_TRY(cudaGetLastError());
+    return ADED_OK;
+}
+
+// Scratch copy of the entries with count >= min_count; the caller frees *keys / *counts.
+static aded_status tg_snapshot(const aded_trigram* t, uint32_t min_count, int32_t** keys, uint32_t** counts, uint64_t* n, void* stream) {
+    *keys = nullptr;
+    *counts = nullptr;
+    uint64_t total = 0;
+    aded_status s = aded_trigram_export(t, min_count, nullptr, nullptr, 0, &total, stream);
+    if (s != ADED_OK) return s;
+    *n = total;
+    if (total == 0) return ADED_OK;
+    if (cudaMalloc((void**)keys, total * 3 * sizeof(int32_t)) != cudaSuccess || cudaMalloc((void**)counts, total * sizeof(uint32_t)) != cudaSuccess) {
+        cudaGetLastError();
+        if (*keys) cudaFree(*keys);
+        *keys = nullptr;
+        return ADED_ERR_OOM;
+    }
+    uint64_t again = 0;
+    s = aded_trigram_export(t, min_count, *keys, *counts, total, &again, stream);
+    if (s == ADED_OK && again != total) s = ADED_ERR_INVALID_ARG;     // the table changed between the two passes
+    if (s != ADED_OK) { cudaFree(*keys); cudaFree(*counts); *keys = nullptr; *counts = nullptr; }
+    return s;
+}
+
+aded_status aded_trigram_prune(aded_trigram* t, uint32_t min_count, void* stream) {
+    if (!t) return ADED_ERR_INVALID_ARG;
+    int32_t* keys;
+    uint32_t* counts;
+    uint64_t n;
+    aded_status s = tg_snapshot(t, min_count, &keys, &counts, &n, stream);
+    if (s != ADED_OK) return s;
+    s = aded_trigram_clear(t, stream);
+    if (s == ADED_OK) s = aded_trigram_import(t, keys, counts, n, stream);
+    cudaStreamSynchronize(static_cast<cudaStream_t>(stream));
+    if (keys) cudaFree(keys);
+    if (counts) cudaFree(counts);
+    return s;
+}
+
+static const char TG_MAGIC[8] = {'A', 'D', 'E', 'D', 'T', 'G', '0', '1'};
+
+aded_status aded_trigram_save(const aded_trigram* t, const char* path, void* stream) {
+    if (!t || !path) return ADED_ERR_INVALID_ARG;
+    int32_t* keys;
+    uint32_t* counts;
+    uint64_t n;
+    aded_status s = tg_snapshot(t, 0, &keys, &counts, &n, stream);
+    if (s != ADED_OK) return s;
+    std::vector<int32_t> hk(n * 3);
+    std::vector<uint32_t> hc(n);
+    bool ok = true;
+    if (n) {
+        ok = cudaMemcpy(hk.data(), keys, n * 3 * sizeof(int32_t), cudaMemcpyDeviceToHost) == cudaSuccess &&
+             cudaMemcpy(hc.data(), counts, n * sizeof(uint32_t), cudaMemcpyDeviceToHost) == cudaSuccess;
+        cudaFree(keys);
+        cudaFree(counts);
+    }
+    if (!ok) { cudaGetLastError(); return ADED_ERR_CUDA; }
+    FILE* f = fopen(path, "wb");
+    if (!f) return ADED_ERR_INVALID_ARG;
+    const int32_t vocab = t->cfg.vocab;
+    ok = fwrite(TG_MAGIC, 1, 8, f) == 8 && fwrite(&vocab, sizeof vocab, 1, f) == 1 && fwrite(&n, sizeof n, 1, f) == 1 &&
+         (n == 0 || (fwrite(hk.data(), sizeof(int32_t), n * 3, f) == n * 3 && fwrite(hc.data(), sizeof(uint32_t), n, f) == n));
+    ok = (fclose(f) == 0) && ok;
+    return ok ? ADED_OK : ADED_ERR_INVALID_ARG;
+}
+
+aded_status aded_trigram_load(aded_trigram* t, const char* path, void* stream) {
+    if (!t || !path) return ADED_ERR_INVALID_ARG;
+    FILE* f = fopen(path, "rb");
+    if (!f) return ADED_ERR_INVALID_ARG;
+    char magic[8];
+    int32_t vocab = 0;
+    uint64_t n = 0;
+    bool ok = fread(magic, 1, 8, f) == 8 && memcmp(magic, TG_MAGIC, 8) == 0 && fread(&vocab, sizeof vocab, 1, f) == 1 &&
+              fread(&n, sizeof n, 1, f) == 1 && vocab == t->cfg.vocab && n <= ((uint64_t)1 << 34);
+    std::vector<int32_t> hk;
+    std::vector<uint32_t> hc;
+    if (ok && n) {
+        hk.resize(n * 3);
+        hc.resize(n);
+        ok = fread(hk.data(), sizeof(int32_t), n * 3, f) == n * 3 && fread(hc.data(), sizeof(uint32_t), n, f) == n;
+    }
+    fclose(f);
+    if (!ok) return ADED_ERR_INVALID_ARG;
+    if (n == 0) return ADED_OK;
+    int32_t* keys = nullptr;
+    uint32_t* counts = nullptr;
+    if (cudaMalloc((void**)&keys, n * 3 * sizeof(int32_t)) != cudaSuccess || cudaMalloc((void**)&counts, n * sizeof(uint32_t)) != cudaSuccess) {
+        cudaGetLastError();
+        if (keys) cudaFree(keys);
+        return ADED_ERR_OOM;
+    }
+    aded_status s = ADED_OK;
+    if (cudaMemcpy(keys, hk.data(), n * 3 * sizeof(int32_t), cudaMemcpyHostToDevice) != cudaSuccess ||
+        cudaMemcpy(counts, hc.data(), n * sizeof(uint32_t), cudaMemcpyHostToDevice) != cudaSuccess) {
+        cudaGetLastError();
+        s = ADED_ERR_CUDA;
+    }
+    if (s == ADED_OK) s = aded_trigram_import(t, keys, counts, n, stream);
+    cudaStreamSynchronize(static_cast<cudaStream_t>(stream));
+    cudaFree(keys);
+    cudaFree(counts);
+    return s;
 }
 
 aded_status aded_trigram_get(const aded_trigram* t, int32_t a, int32_t b, int32_t c, uint32_t* out_count_host, void* stream) {

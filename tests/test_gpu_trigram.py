@@ -127,3 +127,62 @@ def test_large_table_bulk_update_and_queries(cuda_device):
     ctxs.sort(key=lambda ab: -len(st.table[ab]))
     sample = ctxs[:64] + ctxs[1000::997][:400]
     _check_against(B, t, st, sample, ks=(4,))
+
+
+def _entries_gpu(B, t, min_count=0):
+    keys, counts = B.aded_trigram_export(t, min_count)
+    torch.cuda.synchronize()
+    k, c = keys.cpu().tolist(), counts.cpu().tolist()
+    out = {tuple(kk): cc for kk, cc in zip(k, c)}
+    assert len(out) == len(k), "an entry was exported twice"
+    return out
+
+
+def test_export_prune_save_load(cuda_device, tmp_path):
+    """Table persistence and the elimination threshold: exported entries, the pruned table and a table
+    read back from a file equal the checker's, bit for bit; the pruned table keeps working."""
+    from paper_2407_12021_b200 import binding as B
+    vocab = 60
+    toks = gen.zipf_tokens(6000, vocab, 41, 1)
+    st = TrigramStore(cap=50)
+    st.update(toks.tolist())
+    t = B.aded_trigram_create(vocab, log2_buckets=12, overflow_buckets=4096, cap=50)
+    B.aded_trigram_update(t, toks.cuda())
+    assert _entries_gpu(B, t) == st.entries()
+    assert _entries_gpu(B, t, 12) == {k: n for k, n in st.entries().items() if n >= 12}
+    path = str(tmp_path / "table.bin")
+    B.aded_trigram_save(t, path)
+    # a copy read from the file
+    t2 = B.aded_trigram_create(vocab, log2_buckets=13, overflow_buckets=8192, cap=50)   # another geometry than the source
+    B.aded_trigram_load(t2, path)
+    assert _entries_gpu(B, t2) == st.entries()
+    # loading again adds the counts (saturating)
+    B.aded_trigram_load(t2, path)
+    twice = TrigramStore(cap=50)
+    twice.merge(st.entries())
+    twice.merge(st.entries())
+    assert _entries_gpu(B, t2) == twice.entries()
+    # a file for another vocabulary is refused
+    from paper_2407_12021_b200.binding import AdedError
+    t3 = B.aded_trigram_create(vocab + 1, log2_buckets=10, overflow_buckets=64)
+    with pytest.raises(AdedError):
+        B.aded_trigram_load(t3, path)
+    with pytest.raises(AdedError):
+        B.aded_trigram_load(t2, str(tmp_path / "missing.bin"))
+    # elimination threshold 12 (the paper's setting): the table is rebuilt from what stays
+    _, buckets_before = B.aded_trigram_stats(t)
+    B.aded_trigram_prune(t, 12)
+    st.prune(12)
+    assert _entries_gpu(B, t) == st.entries()
+    entries_after, buckets_after = B.aded_trigram_stats(t)
+    assert entries_after == len(st.entries()) and buckets_after < buckets_before
+    ctxs = list(st.table.keys())[:200] + [(vocab - 1, vocab - 1)]
+    _check_against(B, t, st, ctxs, ks=(1, 4))
+    # and keeps counting: no duplicate entries appear where pruned ones used to be
+    more = gen.zipf_tokens(3000, vocab, 42, 1)
+    B.aded_trigram_update(t, more.cuda())
+    st.update(more.tolist())
+    assert _entries_gpu(B, t) == st.entries()
+    B.aded_trigram_clear(t)
+    assert _entries_gpu(B, t) == {} and B.aded_trigram_stats(t) == (0, 0)
+    assert B.aded_trigram_poll_status(t) == 0 and B.aded_trigram_poll_status(t2) == 0

@@ -80,3 +80,17 @@ def test_topk_equals_full_sort_with_tie_rule():
     # the count filter drops rare continuations
     st.update([1, 1, 7])
     assert st.topk(1, 1, 4, min_count=2) == ([7, -1, -1, -1], [2, 0, 0, 0])
+
+
+def test_prune_and_merge_by_hand():
+    from oracle.trigram import TrigramStore
+    s = TrigramStore(cap=10)
+    s.update([1, 2, 3, 1, 2, 3, 1, 2, 4])          # (1,2,3) x2, (2,3,1) x2, (3,1,2) x2, (1,2,4) x1
+    assert s.entries() == {(1, 2, 3): 2, (2, 3, 1): 2, (3, 1, 2): 2, (1, 2, 4): 1}
+    s.prune(2)
+    assert s.entries() == {(1, 2, 3): 2, (2, 3, 1): 2, (3, 1, 2): 2}
+    assert s.topk(1, 2, 3) == ([3, -1, -1], [2, 0, 0])
+    s.merge({(1, 2, 3): 9, (7, 7, 7): 4})
+    assert s.entries() == {(1, 2, 3): 10, (2, 3, 1): 2, (3, 1, 2): 2, (7, 7, 7): 4}      # 2 + 9 saturates at the cap
+    s.prune(11)
+    assert s.entries() == {} and s.table == {}
