@@ -323,6 +323,24 @@ aded_status aded_draft_tree(const aded_trigram* t, const int32_t* context_dev, i
                             int32_t k, const int32_t* filler_dev, int32_t n_filler, int32_t* tree_tokens_dev,
                             int32_t* tree_parents_dev, int32_t* n_from_table_dev, void* stream);
 
+/* The draft maker of the paper: Monte Carlo tree search over tri-gram continuations (Eq. 2-3,
+ * Algorithm 1) from the context (context_dev[0], context_dev[1]).  `iterations` (1..160; the paper
+ * uses 150) rounds of selection by the PUCT score with constants c1, c2 (32 and 8 in the paper),
+ * expansion of all candidate words of the reached node (its top-k list, k in 1..ADED_DRAFT_MAX_K),
+ * simulation up to `length` (1..8; the paper: 4) tokens after the root by drawing from top-k lists in
+ * proportion to the counts with the uniform numbers u_dev[iteration * length + draw] (float32 in
+ * [0, 1), supplied by the caller), and back propagation of 1 + the sum of the state's Eq. 1
+ * probabilities.  The leaves of the search tree are ranked by mean score (earlier-created first on
+ * ties); the best n_candidates (the paper: 24; n_candidates * length + 1 <= ADED_MAX_NODES) are
+ * written as sentence_tokens_dev[r][length] (-1 padded) with sentence_scores_dev[r], and merged
+ * into one prefix tree tree_tokens_dev / tree_parents_dev (breadth-first, *n_nodes_dev nodes, node 0
+ * the last token of the text) ready for aded_verify.  All scores are IEEE doubles computed one
+ * rounded operation at a time.  One warp; asynchronous on `stream`. */
+aded_status aded_mcts_draft(const aded_trigram* t, const int32_t* context_dev, int32_t iterations, int32_t length,
+                            int32_t n_candidates, int32_t k, float c1, float c2, const float* u_dev, int32_t* tree_tokens_dev,
+                            int32_t* tree_parents_dev, int32_t* n_nodes_dev, int32_t* sentence_tokens_dev,
+                            double* sentence_scores_dev, int32_t* n_sentences_dev, void* stream);
+
 /* One decoding step, all on the device and asynchronous on `stream`:
  *   aded_draft_tree from context_dev  ->  aded_verify (out_tokens_dev[n_nodes], out_accept_len_dev[1])
  *   ->  aded_trigram_update over (context, emitted tokens)  ->  context_dev <- last two tokens of the

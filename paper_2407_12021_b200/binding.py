@@ -29,7 +29,7 @@ EXPORTS = [
     "aded_trigram_update", "aded_trigram_update_host", "aded_trigram_topk", "aded_trigram_topk_host",
     "aded_trigram_get", "aded_trigram_stats", "aded_trigram_poll_status", "aded_draft_tree", "aded_decode_step",
     "aded_decode_step_host", "aded_verify_sampled", "aded_sample_tokens", "aded_trigram_export",
-    "aded_trigram_import", "aded_trigram_clear", "aded_trigram_prune", "aded_trigram_save", "aded_trigram_load", "aded_status_string",
+    "aded_trigram_import", "aded_mcts_draft", "aded_trigram_clear", "aded_trigram_prune", "aded_trigram_save", "aded_trigram_load", "aded_status_string",
 ]
 
 
@@ -497,6 +497,27 @@ def aded_trigram_save(t: Trigram, path: str) -> None:
 
 def aded_trigram_load(t: Trigram, path: str) -> None:
     _check(_lib.aded_trigram_load(t.handle, path.encode(), _stream()), "aded_trigram_load")
+
+
+def aded_mcts_draft(t: Trigram, context_dev: torch.Tensor, iterations: int, length: int, n_candidates: int, k: int,
+                    u: torch.Tensor, c1: float = 32.0, c2: float = 8.0):
+    """Runs the tree search; returns (tokens, parents, sentences) as Python lists after synchronising:
+    the merged prefix tree and the ranked sentences [(tokens after the root, mean score)]."""
+    _dev_i32(context_dev, "context"), _dev_f32(u, "u")
+    if u.numel() < iterations * length:
+        raise ValueError("u must hold iterations * length numbers")
+    tok = torch.full((ADED_MAX_NODES,), -9, dtype=torch.int32, device="cuda")
+    par = torch.full((ADED_MAX_NODES,), -9, dtype=torch.int32, device="cuda")
+    n = torch.zeros(2, dtype=torch.int32, device="cuda")
+    st = torch.full((n_candidates, length), -9, dtype=torch.int32, device="cuda")
+    sc = torch.zeros(n_candidates, dtype=torch.float64, device="cuda")
+    _check(_lib.aded_mcts_draft(t.handle, _ptr(context_dev), c_int32(iterations), c_int32(length), c_int32(n_candidates),
+                                c_int32(k), c_float(c1), c_float(c2), _ptr(u), _ptr(tok), _ptr(par), c_void_p(n.data_ptr()),
+                                _ptr(st), _ptr(sc), c_void_p(n.data_ptr() + 4), _stream()), "aded_mcts_draft")
+    torch.cuda.synchronize()
+    nn, ns = int(n[0]), int(n[1])
+    sentences = [([x for x in st[r].tolist() if x >= 0], float(sc[r])) for r in range(ns)]
+    return tok[:nn].tolist(), par[:nn].tolist(), sentences
 
 
 def aded_status_string(status: int) -> str:

@@ -7,6 +7,7 @@
 // and six (token, count) entries that fill front to back and are never removed.  All contexts'
 // continuations are therefore reachable from one hash probe, which is what top-k needs, and an
 // update is one probe plus one atomic add.
+#include <cmath>
 #include <cstdio>
 #include <cstring>
 #include <new>
@@ -392,6 +393,283 @@ __global__ void k_tg_stats(TgView t, unsigned long long* out) {
     atomicAdd(out + 1, used);
 }
 
+
+// ---- draft maker: Monte Carlo tree search (Eq. 2-3, Algorithm 1) -----------------------------------
+// One warp runs the search; every lane executes the same scalar logic on the tree in shared memory
+// (lane 0 alone writes), the lanes cooperate only in the table lookups.  A lookup reads the context's
+// chain once into shared memory and then selects the k best entries there.  Floating point is IEEE
+// double, one rounded operation at a time (no fused multiply-add), so that the search can be
+// reproduced bit for bit; the exploration factor E of Eq. 3 depends on an integer only and comes
+// from a table the host computes.
+constexpr int MC_MAX_ITER = 160, MC_MAX_K = ADED_DRAFT_MAX_K, MC_MAX_LEN = 8;
+constexpr int MC_MAX_NODES = 1 + MC_MAX_ITER * MC_MAX_K;
+constexpr int MC_CHAIN = 192;          // entries of a context held in shared memory (32 buckets)
+constexpr int MC_CACHE = 64;           // remembered lookups (direct mapped): a search meets the same contexts again and again
+
+struct McParams {
+    int iterations, length, n_candidates, k;
+    double e_table[MC_MAX_ITER + 1];   // E for sum N = 0 .. iterations
+};
+
+struct McLookup {                      // top-k list of one context
+    int n;                             // valid entries
+    int32_t word[MC_MAX_K];
+    uint32_t count[MC_MAX_K];
+    uint32_t total;                    // sum over ALL continuations of the context (Eq. 1's denominator)
+};
+
+// All 32 lanes call this with the same (a, b); the result is identical in every lane.
+__device__ __forceinline__ void mc_lookup(const TgView& t, int a, int b, int k, int lane, int32_t* s_tok, uint32_t* s_cnt,
+                                          McLookup& out) {
+    out.n = 0;
+    out.total = 0;
+    int64_t home = -1;
+    if (a >= 0 && b >= 0 && a < t.vocab && b < t.vocab) home = tg_find_home(t, tg_key(a, b), false);
+    if (home < 0) return;
+    // pass 1: the chain into shared memory (six entries per bucket, lanes 0..5 read them)
+    int n_ent = 0;
+    bool overflow = false;
+    int64_t cur = home;
+    for (uint32_t hop = 0; cur >= 0 && hop <= t.n_over; ++hop) {
+        const Bucket* bk = t.buckets + cur;
+        if (n_ent + 6 > MC_CHAIN) { overflow = true; break; }
+        if (lane < 6) { s_tok[n_ent + lane] = bk->e[lane].tok; s_cnt[n_ent + lane] = bk->e[lane].cnt; }
+        n_ent += 6;
+        const uint32_t nxt = bk->next;
+        cur = nxt == 0 ? -1 : (int64_t)nxt;
+    }
+    __syncwarp();
+    unsigned long long prev = ~0ull;
+    if (overflow) {                    // a very long chain: select round by round from global memory
+        for (int round = 0; round < k; ++round) {
+            uint32_t total;
+            const unsigned long long best = tg_select_round(t, home, prev, lane, &total);
+            out.total = total;
+            if (!best) break;
+            out.word[out.n] = (int32_t)(0xFFFFFFFFu - (uint32_t)best);
+            out.count[out.n] = (uint32_t)(best >> 32);
+            ++out.n;
+            prev = best;
+        }
+        return;
+    }
+    uint32_t total = 0;
+    for (int i = lane; i < n_ent; i += 32)
+        if (s_tok[i] >= 0) total += s_cnt[i];
+    for (int o = 16; o > 0; o >>= 1) total += __shfl_xor_sync(0xffffffffu, total, o);
+    out.total = total;
+    for (int round = 0; round < k; ++round) {
+        unsigned long long best = 0;
+        for (int i = lane; i < n_ent; i += 32) {
+            const int32_t tk = s_tok[i];
+            const uint32_t cn = s_cnt[i];
+            if (tk < 0 || cn == 0 || cn < t.min_count) continue;
+            const unsigned long long key = ((unsigned long long)cn << 32) | (0xFFFFFFFFu - (uint32_t)tk);
+            if (key < prev && key > best) best = key;
+        }
+        for (int o = 16; o > 0; o >>= 1) {
+            const unsigned long long ob = __shfl_xor_sync(0xffffffffu, best, o);
+            if (ob > best) best = ob;
+        }
+        if (!best) break;
+        out.word[out.n] = (int32_t)(0xFFFFFFFFu - (uint32_t)best);
+        out.count[out.n] = (uint32_t)(best >> 32);
+        ++out.n;
+        prev = best;
+    }
+    __syncwarp();
+}
+
+// mc_lookup through the cache of remembered contexts (the table does not change during a search).
+__device__ __forceinline__ void mc_lookup_cached(const TgView& t, int a, int b, int k, int lane, int32_t* s_tok, uint32_t* s_cnt,
+                                                 unsigned long long* s_ckey, McLookup* s_cval, McLookup& out) {
+    const unsigned long long key = tg_key(a, b);
+    const int slot = (int)(tg_hash(key) & (MC_CACHE - 1));
+    if (s_ckey[slot] == key) { out = s_cval[slot]; return; }
+    mc_lookup(t, a, b, k, lane, s_tok, s_cnt, out);
+    __syncwarp();
+    if (lane == 0) { s_cval[slot] = out; s_ckey[slot] = key; }
+    __syncwarp();
+}
+
+__host__ __device__ constexpr size_t mc_cache_offset() {
+    return (((size_t)MC_MAX_NODES * (8 + 4 * 4 + 2 * 2 + 2 * 1) + (size_t)MC_CHAIN * 8 + ADED_MAX_NODES * 2) + 15) & ~(size_t)15;
+}
+
+__global__ void __launch_bounds__(32)
+k_mcts_draft(TgView t, const __grid_constant__ McParams p, const int32_t* __restrict__ ctx, const float* __restrict__ u,
+             int32_t* __restrict__ out_tok, int32_t* __restrict__ out_par, int32_t* __restrict__ out_n,
+             int32_t* __restrict__ sent_tok, double* __restrict__ sent_score, int32_t* __restrict__ out_n_sent) {
+    extern __shared__ __align__(16) uint8_t mc_smem[];
+    // 8-byte, then 4-byte, then 2-byte, then 1-byte arrays, so that each starts aligned
+    double* s_score = reinterpret_cast<double*>(mc_smem);                 // [MC_MAX_NODES] sum of scores
+    int32_t* s_tok = reinterpret_cast<int32_t*>(s_score + MC_MAX_NODES);  // token
+    int32_t* s_visits = s_tok + MC_MAX_NODES;
+    uint32_t* s_cnt = reinterpret_cast<uint32_t*>(s_visits + MC_MAX_NODES);   // count of the node's token in its parent's context
+    uint32_t* s_ctxtot = s_cnt + MC_MAX_NODES;                            // expanded nodes: total of their own context
+    int32_t* s_ltok = reinterpret_cast<int32_t*>(s_ctxtot + MC_MAX_NODES);    // lookup scratch
+    uint32_t* s_lcnt = reinterpret_cast<uint32_t*>(s_ltok + MC_CHAIN);
+    int16_t* s_par = reinterpret_cast<int16_t*>(s_lcnt + MC_CHAIN);
+    int16_t* s_first = s_par + MC_MAX_NODES;                              // first child (children are consecutive)
+    int16_t* s_queue = s_first + MC_MAX_NODES;                            // [ADED_MAX_NODES] breadth-first order of the result
+    uint8_t* s_nkid = reinterpret_cast<uint8_t*>(s_queue + ADED_MAX_NODES);
+    uint8_t* s_flag = s_nkid + MC_MAX_NODES;                              // bit 0 expanded, bit 1 chosen, bit 2 kept
+    unsigned long long* s_ckey = reinterpret_cast<unsigned long long*>(mc_smem + mc_cache_offset());   // [MC_CACHE] context of a remembered lookup
+    McLookup* s_cval = reinterpret_cast<McLookup*>(s_ckey + MC_CACHE);
+    for (int i = threadIdx.x; i < MC_CACHE; i += 32) s_ckey[i] = TG_EMPTY;
+    float* s_u = reinterpret_cast<float*>(s_cval + MC_CACHE);            // the caller's uniform numbers
+    for (int i = threadIdx.x; i < p.iterations * p.length; i += 32) s_u[i] = u[i];
+
+    const int lane = threadIdx.x;
+    const int prev_token = ctx[0], root_token = ctx[1];
+    int n_nodes = 1;
+    if (lane == 0) {
+        s_tok[0] = root_token; s_par[0] = -1; s_first[0] = 0; s_nkid[0] = 0; s_flag[0] = 0;
+        s_visits[0] = 0; s_score[0] = 0.0; s_cnt[0] = 0; s_ctxtot[0] = 0;
+    }
+    __syncwarp();
+    McLookup lk;
+    for (int it = 0; it < p.iterations; ++it) {
+        int node = 0, len = 1;
+        int state[MC_MAX_LEN + 1];
+        double sp[MC_MAX_LEN + 1];          // Eq. 1 probability of state[i] given its two predecessors
+        state[0] = root_token;
+        bool end = false;
+        // selection
+        while ((s_flag[node] & 1) && s_nkid[node] > 0 && !end) {
+            // one lane per child (at most eight): the double divisions run side by side
+            const int first = s_first[node], nk = s_nkid[node];
+            const bool mine = lane < nk;
+            const int c = first + (mine ? lane : 0);
+            const int nv = mine ? s_visits[c] : 0;
+            int n_sum = nv;
+            for (int o = 16; o > 0; o >>= 1) n_sum += __shfl_xor_sync(0xffffffffu, n_sum, o);
+            const double e = p.e_table[n_sum], root_n = sqrt((double)n_sum), tot = (double)s_ctxtot[node];
+            const double q = nv ? __ddiv_rn(s_score[c], (double)nv) : 0.0;
+            const double pr = __ddiv_rn((double)s_cnt[c], tot);
+            double best_s = __dadd_rn(q, __ddiv_rn(__dmul_rn(__dmul_rn(e, pr), root_n), __dadd_rn(1.0, (double)nv)));
+            double best_p = pr;
+            int best = mine ? c : -1;
+            for (int o = 16; o > 0; o >>= 1) {
+                const double os = __shfl_xor_sync(0xffffffffu, best_s, o), op = __shfl_xor_sync(0xffffffffu, best_p, o);
+                const int ob = __shfl_xor_sync(0xffffffffu, best, o);
+                if (ob >= 0 && (best < 0 || os > best_s || (os == best_s && ob < best))) { best = ob; best_s = os; best_p = op; }
+            }
+            node = best;
+            state[len] = s_tok[node];
+            sp[len] = best_p;
+            ++len;
+            if (len == p.length + 1) end = true;
+        }
+        // expansion
+        if (!(s_flag[node] & 1) && !end) {
+            const int a = node == 0 ? prev_token : s_tok[s_par[node]], b = s_tok[node];
+            mc_lookup_cached(t, a, b, p.k, lane, s_ltok, s_lcnt, s_ckey, s_cval, lk);
+            if (lane == 0) {
+                s_flag[node] |= 1;
+                s_ctxtot[node] = lk.total;
+                s_first[node] = (int16_t)n_nodes;
+                s_nkid[node] = (uint8_t)lk.n;
+                for (int j = 0; j < lk.n; ++j) {
+                    const int c = n_nodes + j;
+                    s_tok[c] = lk.word[j]; s_par[c] = (int16_t)node; s_first[c] = 0; s_nkid[c] = 0; s_flag[c] = 0;
+                    s_visits[c] = 0; s_score[c] = 0.0; s_cnt[c] = lk.count[j]; s_ctxtot[c] = 0;
+                }
+            }
+            __syncwarp();
+            if (lk.n > 0) {
+                n_nodes += lk.n;
+                node = n_nodes - 1;                       // the last child created
+                state[len] = s_tok[node];
+                sp[len] = __ddiv_rn((double)s_cnt[node], (double)lk.total);
+                ++len;
+            }
+        }
+        // simulation
+        int draws = 0;
+        while (len < p.length + 1) {
+            const int a = len >= 2 ? state[len - 2] : prev_token, b = state[len - 1];
+            mc_lookup_cached(t, a, b, p.k, lane, s_ltok, s_lcnt, s_ckey, s_cval, lk);
+            if (lk.n == 0) break;
+            unsigned long long total = 0;
+            for (int j = 0; j < lk.n; ++j) total += lk.count[j];
+            unsigned long long u24 = __float2uint_rd(__fmul_rn(s_u[it * p.length + draws], 16777216.f));
+            if (u24 > 16777215ull) u24 = 16777215ull;
+            const unsigned long long target = (total * u24) >> 24;
+            unsigned long long run = 0;
+            int pick = lk.n - 1;
+            for (int j = 0; j < lk.n; ++j) {
+                run += lk.count[j];
+                if (run > target) { pick = j; break; }
+            }
+            state[len] = lk.word[pick];
+            sp[len] = __ddiv_rn((double)lk.count[pick], (double)lk.total);
+            ++len;
+            ++draws;
+        }
+        // back propagation
+        double sc = 1.0;
+        for (int i = 1; i < len; ++i) sc = __dadd_rn(sc, sp[i]);
+        if (lane == 0) {
+            for (int cur = node; cur >= 0; cur = s_par[cur]) {
+                s_visits[cur] += 1;
+                s_score[cur] = __dadd_rn(s_score[cur], sc);
+            }
+        }
+        __syncwarp();
+    }
+
+    // ranking: leaves of the search tree by mean score (descending), earlier nodes first on ties
+    int n_sent = 0;
+    for (int r = 0; r < p.n_candidates; ++r) {
+        double best_m = -1.0;
+        int best_i = -1;
+        for (int i = 1 + lane; i < n_nodes; i += 32) {
+            if (s_nkid[i] != 0 || (s_flag[i] & 2)) continue;
+            const double m = s_visits[i] ? __ddiv_rn(s_score[i], (double)s_visits[i]) : 0.0;
+            if (best_i < 0 || m > best_m) { best_m = m; best_i = i; }     // i ascends within a lane: first wins ties
+        }
+        for (int o = 16; o > 0; o >>= 1) {
+            const double om = __shfl_xor_sync(0xffffffffu, best_m, o);
+            const int oi = __shfl_xor_sync(0xffffffffu, best_i, o);
+            if (oi >= 0 && (best_i < 0 || om > best_m || (om == best_m && oi < best_i))) { best_m = om; best_i = oi; }
+        }
+        if (best_i < 0) break;
+        if (lane == 0) {
+            s_flag[best_i] |= 2;
+            int path[MC_MAX_LEN], d = 0;
+            for (int j = best_i; j > 0; j = s_par[j]) { s_flag[j] |= 4; path[d++] = s_tok[j]; }
+            for (int j = 0; j < p.length; ++j) sent_tok[r * p.length + j] = j < d ? path[d - 1 - j] : -1;
+            sent_score[r] = best_m;
+        }
+        __syncwarp();
+        ++n_sent;
+    }
+    // prefix tree of the chosen sentences, breadth first, children in creation order
+    if (lane == 0) {
+        int count = 1;
+        s_queue[0] = 0;
+        out_tok[0] = root_token;
+        out_par[0] = -1;
+        for (int head = 0; head < count; ++head) {
+            const int nd = s_queue[head];
+            for (int c = s_first[nd]; c < s_first[nd] + s_nkid[nd]; ++c) {
+                if (!(s_flag[c] & 4) || count >= ADED_MAX_NODES) continue;
+                s_queue[count] = (int16_t)c;
+                out_tok[count] = s_tok[c];
+                out_par[count] = head;
+                ++count;
+            }
+        }
+        *out_n = count;
+        *out_n_sent = n_sent;
+    }
+}
+
+static size_t mc_smem_bytes() {
+    return mc_cache_offset() + (size_t)MC_CACHE * (8 + sizeof(McLookup)) + (size_t)MC_MAX_ITER * MC_MAX_LEN * sizeof(float);
+}
+
 }  // namespace aded
 
 struct aded_trigram {
@@ -549,6 +827,35 @@ aded_status aded_draft_tree(const aded_trigram* t, const int32_t* context_dev, i
     k_draft_tree<<<1, 1024, 0, static_cast<cudaStream_t>(stream)>>>(t->view, context_dev, n_nodes, max_depth, k,
                                                                     n_filler > 0 ? filler_dev : nullptr, n_filler,
                                                                     tree_tokens_dev, tree_parents_dev, n_from_table_dev);
+    ADED_CUDA_TRY(cudaGetLastError());
+    return ADED_OK;
+}
+
+aded_status aded_mcts_draft(const aded_trigram* t, const int32_t* context_dev, int32_t iterations, int32_t length,
+                            int32_t n_candidates, int32_t k, float c1, float c2, const float* u_dev, int32_t* tree_tokens_dev,
+                            int32_t* tree_parents_dev, int32_t* n_nodes_dev, int32_t* sentence_tokens_dev,
+                            double* sentence_scores_dev, int32_t* n_sentences_dev, void* stream) {
+    if (!t || !context_dev || !u_dev || !tree_tokens_dev || !tree_parents_dev || !n_nodes_dev || !sentence_tokens_dev ||
+        !sentence_scores_dev || !n_sentences_dev)
+        return ADED_ERR_INVALID_ARG;
+    if (iterations < 1 || iterations > MC_MAX_ITER || length < 1 || length > MC_MAX_LEN || k < 1 || k > MC_MAX_K ||
+        n_candidates < 1 || n_candidates * length + 1 > ADED_MAX_NODES || !(c2 > 0.f))
+        return ADED_ERR_INVALID_ARG;
+    static bool prepared = false;
+    if (!prepared) {
+        ADED_CUDA_TRY(cudaFuncSetAttribute(k_mcts_draft, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)mc_smem_bytes()));
+        prepared = true;
+    }
+    McParams p;
+    p.iterations = iterations;
+    p.length = length;
+    p.n_candidates = n_candidates;
+    p.k = k;
+    for (int n = 0; n <= MC_MAX_ITER; ++n) p.e_table[n] = (double)c1 + std::log(((double)n + (double)c2 + 1.0) / (double)c2);   // Eq. 3
+    note_launch();
+    k_mcts_draft<<<1, 32, mc_smem_bytes(), static_cast<cudaStream_t>(stream)>>>(t->view, p, context_dev, u_dev, tree_tokens_dev,
+                                                                               tree_parents_dev, n_nodes_dev, sentence_tokens_dev,
+                                                                               sentence_scores_dev, n_sentences_dev);
     ADED_CUDA_TRY(cudaGetLastError());
     return ADED_OK;
 }
