@@ -4,7 +4,7 @@
 Algorithm 1 is followed phase by phase -- selection by the PUCT score, expansion of every candidate
 word of the reached node, simulation by drawing continuations from the tri-gram statistics, back
 propagation of a score built from the tri-gram probabilities, ranking of the found sentences -- with
-these readings where the listing or the text leave a choice (the design doc lists them):
+these readings where the listing or the text leave a choice:
 
   * a node stands for a token; its context is (token of its parent, its token), the root's context is
     the last two tokens of the text; its candidate words are the top-k list of that context (rank order);
