@@ -104,6 +104,12 @@ __device__ __forceinline__ void mma_bf16_16816(float* c, const uint32_t* a, uint
                  : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
                  : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
+// 2^x for x <= 0 by the hardware approximation (2 ulp; results below 2^-126 flush to zero).
+__device__ __forceinline__ float ex2_fast(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
     return *reinterpret_cast<uint32_t*>(&v);
@@ -291,7 +297,7 @@ __global__ void __launch_bounds__(NW * 32) k_tree_attn_mma(AttnArgs a) {
         for (int n = 0; n < TA_BLK / 8; ++n) {
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
-                float s = sacc[n][e] * a.scale_log2;
+                float s = sacc[n][e];          // raw dot product; the scale (> 0) is applied to the maximum and inside the exponent
                 if (need_mask) {
                     const int pos = p0 + n * 8 + 2 * tig + (e & 1);
                     const int j = pos - L;
@@ -313,8 +319,11 @@ __global__ void __launch_bounds__(NW * 32) k_tree_attn_mma(AttnArgs a) {
         // The running reference is the maximum rounded UP to an integer (scores are in the log2
         // domain), so every rescale below is an exact power of two and the bf16 rounding of the
         // numerators 2^(t - M) does not depend on how the keys are split or ordered.
-        const float nm0 = fmaxf(mrow0, ceilf(bm0)), nm1 = fmaxf(mrow1, ceilf(bm1));
+        const float nm0 = fmaxf(mrow0, ceilf(bm0 * a.scale_log2)), nm1 = fmaxf(mrow1, ceilf(bm1 * a.scale_log2));
         const float use0 = nm0 == -INFINITY ? 0.f : nm0, use1 = nm1 == -INFINITY ? 0.f : nm1;
+        // the partial sums need rescaling only when a row's reference moved (rare after the first block:
+        // it is an integer); a row without any key yet holds zeros, which need none
+        const bool moved = (mrow0 != nm0 && mrow0 != -INFINITY) || (mrow1 != nm1 && mrow1 != -INFINITY);
         const float corr0 = exp2f(mrow0 - use0), corr1 = exp2f(mrow1 - use1);
         mrow0 = nm0;
         mrow1 = nm1;
@@ -322,20 +331,24 @@ __global__ void __launch_bounds__(NW * 32) k_tree_attn_mma(AttnArgs a) {
         uint32_t pf[TA_BLK / 16][4];
 #pragma unroll
         for (int n = 0; n < TA_BLK / 8; ++n) {
-            const float e0 = exp2f(sacc[n][0] - use0), e1 = exp2f(sacc[n][1] - use0);
-            const float e2 = exp2f(sacc[n][2] - use1), e3 = exp2f(sacc[n][3] - use1);
+            const float e0 = ex2_fast(fmaf(sacc[n][0], a.scale_log2, -use0)), e1 = ex2_fast(fmaf(sacc[n][1], a.scale_log2, -use0));
+            const float e2 = ex2_fast(fmaf(sacc[n][2], a.scale_log2, -use1)), e3 = ex2_fast(fmaf(sacc[n][3], a.scale_log2, -use1));
             ps0 += e0 + e1;
             ps1 += e2 + e3;
             pf[n >> 1][(n & 1) * 2 + 0] = pack_bf16(e0, e1);
             pf[n >> 1][(n & 1) * 2 + 1] = pack_bf16(e2, e3);
         }
-        lrow0 = lrow0 * corr0 + ps0;
-        lrow1 = lrow1 * corr1 + ps1;
+        if (__any_sync(0xffffffffu, moved)) {
+            lrow0 *= corr0;
+            lrow1 *= corr1;
 #pragma unroll
-        for (int n = 0; n < ONT; ++n) {
-            oacc[n][0] *= corr0; oacc[n][1] *= corr0;
-            oacc[n][2] *= corr1; oacc[n][3] *= corr1;
+            for (int n = 0; n < ONT; ++n) {
+                oacc[n][0] *= corr0; oacc[n][1] *= corr0;
+                oacc[n][2] *= corr1; oacc[n][3] *= corr1;
+            }
         }
+        lrow0 += ps0;
+        lrow1 += ps1;
         // ---- O += P V ----
 #pragma unroll
         for (int kk = 0; kk < TA_BLK / 16; ++kk) {
