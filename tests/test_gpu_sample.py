@@ -114,3 +114,38 @@ def test_sampled_verification_steps(cuda_device):
             pytest.skip("a fragile draw changed the accepted path; the remaining steps would compare different texts")
     assert not_greedy >= 3, "the temperature is so low that sampling never left the greedy token"
     assert fragile <= 2
+
+
+def test_sampled_step_on_the_tensor_core_path(cuda_device):
+    """bf16 model (projections and LM head on the tensor-core GEMM, logits gathered from its partial
+    tiles): the tokens the sampled step drew equal the library's stand-alone drawing call on the step's
+    own logits (that call is checked bit for bit against the checker on seeded logits above), and the
+    emitted sequence is the approval walk over those draws."""
+    from paper_2407_12021_b200 import binding as B
+    shape = gen.ModelShape("bf16-4x64", 2, 256, 4, 64, 384, 1024, "bf16")
+    w = gen.model_weights(shape, 91)
+    sess = H.GpuSession(shape, H.weights_to(w, cuda_device), capacity=400)
+    prompt = gen.zipf_tokens(90, shape.vocab, 91, 50).tolist()
+    sess.append(prompt[:-1])
+    n = 40
+    for step, (temp, top_p) in enumerate([(1.0, 0.9), (0.3, 1.0), (2.0, 0.5)]):
+        tokens, parents = gen.make_tree(n, 5, 4, shape.vocab, 92 + step, root_token=prompt[-1])
+        u = torch.tensor(gen.uniform01(n, 93, step).numpy().astype(np.float32), device="cuda")
+        logits = torch.empty((n, shape.vocab), dtype=torch.float32, device="cuda")
+        best = torch.empty((n,), dtype=torch.int32, device="cuda")
+        out = torch.full((n,), -7, dtype=torch.int32, device="cuda")
+        alen = torch.full((1,), -7, dtype=torch.int32, device="cuda")
+        length_before = sess.length()
+        B.aded_debug_capture(sess.model, logits, best)
+        B.aded_verify_sampled(sess.model, sess.kv, H.i32(tokens), H.i32(parents), temp, top_p, u, out, alen)
+        torch.cuda.synchronize()
+        assert B.aded_model_poll_status(sess.model) == 0
+        again = torch.full((n,), -5, dtype=torch.int32, device="cuda")
+        B.aded_sample_tokens(logits, temp, top_p, u, again)
+        torch.cuda.synchronize()
+        assert torch.equal(again, best)
+        path, want_out = ov.accept_walk(tokens, parents, best.cpu().numpy().astype(np.int64))
+        a = int(alen[0])
+        assert a == len(want_out) and out[:a].tolist() == want_out
+        assert sess.length() == length_before + a
+        B.aded_kv_set_len(sess.kv, 0, length_before)
