@@ -131,6 +131,7 @@ struct AttnArgs {
     const int32_t* row_off;
     const uint64_t* anc;
     int layer, H, n_splits, rows_total;
+    int row_blocks;                // CTAs (of NW * 16 query rows each) per sequence and key split; grid.z = batch * row_blocks
     float scale_log2;              // softmax scale * log2(e)
     const int32_t* status;
 };
@@ -148,7 +149,7 @@ __global__ void __launch_bounds__(NW * 32) k_tree_attn_mma(AttnArgs a) {
     // trust -- nothing orders this read after the kernels that wrote them -- and read again after the
     // wait: the early blocks are used only if both reads agree, otherwise they are fetched again.
     // The cache block's address and capacity never change after the cache was created.
-    const int pre_hh = blockIdx.x, pre_b = blockIdx.z;
+    const int pre_hh = blockIdx.x, pre_b = blockIdx.z / a.row_blocks;
     const size_t pre_cp = a.cap[pre_b];
     const bf16* pre_kg = reinterpret_cast<const bf16*>(a.base[pre_b]) + (((size_t)a.layer * 2 + 0) * a.H + pre_hh) * pre_cp * HD;
     const bf16* pre_vg = reinterpret_cast<const bf16*>(a.base[pre_b]) + (((size_t)a.layer * 2 + 1) * a.H + pre_hh) * pre_cp * HD;
@@ -191,7 +192,8 @@ __global__ void __launch_bounds__(NW * 32) k_tree_attn_mma(AttnArgs a) {
     constexpr int KSTEPS = HD / 16;        // k steps of Q K^T
     constexpr int ONT = HD / 8;            // n tiles of the output
 
-    const int hh = blockIdx.x, split = blockIdx.y, b = blockIdx.z;
+    const int hh = blockIdx.x, split = blockIdx.y, b = blockIdx.z / a.row_blocks;
+    const int row_base = (blockIdx.z % a.row_blocks) * NW * 16;    // first query row (node of the tree) of this CTA
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, tig = lane & 3;
     const int off = a.row_off[b];
     const int T = a.row_off[b + 1] - off;
@@ -204,7 +206,7 @@ __global__ void __launch_bounds__(NW * 32) k_tree_attn_mma(AttnArgs a) {
     const int blk1 = min(nb, blk0 + bps);
 
     // this thread's two query rows (local node indices) and their global rows
-    const int i0 = warp * 16 + g, i1 = i0 + 8;
+    const int i0 = row_base + warp * 16 + g, i1 = i0 + 8;
     const bool v0 = i0 < T, v1 = i1 < T;
     const bf16* kg = reinterpret_cast<const bf16*>(a.base[b]) + (((size_t)a.layer * 2 + 0) * a.H + hh) * cp * HD;
     const bf16* vg = reinterpret_cast<const bf16*>(a.base[b]) + (((size_t)a.layer * 2 + 1) * a.H + hh) * cp * HD;
@@ -397,8 +399,9 @@ __global__ void __launch_bounds__(NW * 32) k_tree_attn_mma(AttnArgs a) {
     }
     const uint32_t so_addr = (uint32_t)__cvta_generic_to_shared(so), sml_addr = (uint32_t)__cvta_generic_to_shared(sml);
     constexpr int QUADS = HD / 4;                      // float4 groups per row
-    for (int item = threadIdx.x; item < ((T - split + S - 1) / S) * QUADS; item += NW * 32) {
-        const int row = split + (item / QUADS) * S, c4 = (item % QUADS) * 4;
+    const int t_here = min(max(T - row_base, 0), NW * 16);         // query rows of this CTA
+    for (int item = threadIdx.x; item < ((t_here - split + S - 1) / S) * QUADS; item += NW * 32) {
+        const int row = split + (item / QUADS) * S, c4 = (item % QUADS) * 4;       // row inside this CTA's block
         // all remote reads of an item are issued before any is used (S <= 8 partials)
         float ms[8], ls[8];
         float4 os[8];
@@ -429,7 +432,7 @@ __global__ void __launch_bounds__(NW * 32) k_tree_attn_mma(AttnArgs a) {
             num.x += os[s2].x * w; num.y += os[s2].y * w; num.z += os[s2].z * w; num.w += os[s2].w * w;
         }
         const float inv = 1.f / den;
-        bf16* dst = a.out + ((size_t)(off + row) * a.H + hh) * HD + c4;
+        bf16* dst = a.out + ((size_t)(off + row_base + row) * a.H + hh) * HD + c4;
         const __nv_bfloat162 lo = __floats2bfloat162_rn(num.x * inv, num.y * inv), hi = __floats2bfloat162_rn(num.z * inv, num.w * inv);
         uint2 u;
         u.x = *reinterpret_cast<const uint32_t*>(&lo);
@@ -451,7 +454,7 @@ static size_t attn_smem() {
 template <int HD, int NW>
 static void launch_mma_nw(aded_model* m, AttnArgs& a, int batch, int splits, cudaStream_t st) {
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(m->cfg.n_heads, splits, batch);
+    cfg.gridDim = dim3(m->cfg.n_heads, splits, batch * a.row_blocks);
     cfg.blockDim = dim3(NW * 32);
     cfg.dynamicSmemBytes = attn_smem<HD, NW>();
     cfg.stream = st;
@@ -486,25 +489,25 @@ static void launch_mma(aded_model* m, aded_kv* kv, int layer, int batch, int row
     a.anc = m->rows.anc;
     a.layer = layer;
     a.H = m->cfg.n_heads;
-    // key splits per (sequence, head): a power of two up to 8 (one thread-block cluster), enough for
-    // about three quarters of the two-per-SM CTA slots
-    int splits = 1;
-    while (splits < 8 && m->cfg.n_heads * batch * splits * 4 < ws_grid_limit(m->device) * 3) splits *= 2;
+    // Trees of more than 64 nodes are worked as two blocks of 64 query rows by separate CTAs (four
+    // warps and two CTAs per SM as for small trees; an eight-warp CTA holds a whole SM's registers and
+    // left the launch at one CTA per SM in two waves).  Key splits per (sequence, head, row block): up
+    // to 8 (one thread-block cluster), as many as keep the launch within the two-per-SM CTA slots.
+    a.row_blocks = max_tree <= 64 ? 1 : 2;
+    int splits = ws_grid_limit(m->device) / (m->cfg.n_heads * batch * a.row_blocks);
+    splits = splits < 1 ? 1 : splits > 8 ? 8 : splits;
     a.n_splits = splits;
     a.rows_total = rows;
     a.scale_log2 = 1.4426950408889634f / sqrtf((float)HD);
     a.status = m->status;
-    if (max_tree <= 64) launch_mma_nw<HD, 4>(m, a, batch, splits, st);
-    else launch_mma_nw<HD, 8>(m, a, batch, splits, st);
+    launch_mma_nw<HD, 4>(m, a, batch, splits, st);
 }
 
 // Raises the split-KV kernels' dynamic shared-memory limit; once per process, before any launch.
 bool attn_prepare() {
     bool ok = true;
     ok &= cudaFuncSetAttribute(k_tree_attn_mma<128, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attn_smem<128, 4>()) == cudaSuccess;
-    ok &= cudaFuncSetAttribute(k_tree_attn_mma<128, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attn_smem<128, 8>()) == cudaSuccess;
     ok &= cudaFuncSetAttribute(k_tree_attn_mma<64, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attn_smem<64, 4>()) == cudaSuccess;
-    ok &= cudaFuncSetAttribute(k_tree_attn_mma<64, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attn_smem<64, 8>()) == cudaSuccess;
     return ok;
 }
 
