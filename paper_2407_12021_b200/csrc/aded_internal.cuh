@@ -209,6 +209,9 @@ void launch_materialize(aded_model* m, const GemmOut& src, float* dst, int rows,
 // dense_ws.cu: bf16 consumers of slot-resident projection results
 void launch_add_rmsnorm_ws(aded_model* m, const GemmOut& y, const void* gain, int rows, cudaStream_t st);
 void launch_swiglu_ws(aded_model* m, const GemmOut& gu, int rows, cudaStream_t st);
+bool embed_norm_ws_supported(const aded_model* m);
+// embedding lookup and the first RMSNorm in one kernel
+void launch_embed_norm_ws(aded_model* m, const void* gain, int rows, cudaStream_t st);
 void launch_rope_kv_ws(aded_model* m, aded_kv* kv, const GemmOut& qkv, int layer, int rows, cudaStream_t st);
 
 // gemm_ws.cu

@@ -69,6 +69,54 @@ __global__ void __launch_bounds__(1024) k_add_rmsnorm_ws(bf16* __restrict__ h, G
     }
 }
 
+// Embedding lookup + the first layer's RMSNorm in one kernel (bf16): h = embed[token], x = norm(h).
+// One block of 1024 threads per row, four columns per thread and pass, as k_add_rmsnorm_ws.
+__global__ void __launch_bounds__(1024) k_embed_norm_ws(const bf16* __restrict__ table, const CallPtrs* __restrict__ call,
+                                                        bf16* __restrict__ h, const bf16* __restrict__ gain, bf16* __restrict__ x,
+                                                        int d, int vocab, float eps, const int32_t* status) {
+    pdl_launch_dependents();
+    __shared__ float red[32];
+    const int r = blockIdx.x;
+    float4 gv[2];
+#pragma unroll
+    for (int i = 0; i < 2; ++i) {
+        const int c = (i * 1024 + threadIdx.x) * 4;
+        if (c < d) gv[i] = unpack4_bf16(*reinterpret_cast<const uint2*>(gain + c));
+    }
+    pdl_wait();
+    const int pass_status = *status;
+    int tok = call->tokens[r];
+    if (tok < 0 || tok >= vocab) tok = 0;          // a token outside the vocabulary has been reported by the tree check
+    const bf16* src = table + (size_t)tok * d;
+    float4 v[2];
+    float sq = 0.f;
+#pragma unroll
+    for (int i = 0; i < 2; ++i) {
+        const int c = (i * 1024 + threadIdx.x) * 4;
+        if (c < d) {
+            const uint2 raw = *reinterpret_cast<const uint2*>(src + c);
+            if (pass_status == 0) *reinterpret_cast<uint2*>(h + (size_t)r * d + c) = raw;
+            v[i] = unpack4_bf16(raw);
+            sq += v[i].x * v[i].x + v[i].y * v[i].y + v[i].z * v[i].z + v[i].w * v[i].w;
+        }
+    }
+    sq = warp_sum_f(sq);
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = sq;
+    __syncthreads();
+    float total = 0.f;
+#pragma unroll
+    for (int i = 0; i < 32; ++i) total += red[i];
+    const float inv = rsqrtf(total / (float)d + eps);
+    if (pass_status != 0) return;
+#pragma unroll
+    for (int i = 0; i < 2; ++i) {
+        const int c = (i * 1024 + threadIdx.x) * 4;
+        if (c < d)
+            *reinterpret_cast<uint2*>(x + (size_t)r * d + c) =
+                pack4_bf16(v[i].x * inv * gv[i].x, v[i].y * inv * gv[i].y, v[i].z * inv * gv[i].z, v[i].w * inv * gv[i].w);
+    }
+}
+
 // act = round(silu(gate) * up): grid (chunks of 1024 columns, rows), four columns per thread.
 __global__ void __launch_bounds__(256) k_swiglu_ws(GemmOut gu, bf16* __restrict__ act, int F, const int32_t* status) {
     pdl_launch_dependents();
@@ -124,6 +172,15 @@ void launch_add_rmsnorm_ws(aded_model* m, const GemmOut& y, const void* gain, in
     const int d = m->cfg.d_model;
     launch_k(k_add_rmsnorm_ws, dim3(rows), dim3(1024), 0, st, (bf16*)m->h, y, (const bf16*)gain, (bf16*)m->x, d, m->cfg.rms_eps,
              (const int32_t*)m->status);
+}
+
+bool embed_norm_ws_supported(const aded_model* m) {
+    return m->cfg.dtype == ADED_BF16 && m->cfg.d_model % 4 == 0 && m->cfg.d_model <= 8192;
+}
+
+void launch_embed_norm_ws(aded_model* m, const void* gain, int rows, cudaStream_t st) {
+    launch_k(k_embed_norm_ws, dim3(rows), dim3(1024), 0, st, (const bf16*)m->top.embed, (const CallPtrs*)m->call_dev, (bf16*)m->h,
+             (const bf16*)gain, (bf16*)m->x, m->cfg.d_model, m->cfg.vocab, m->cfg.rms_eps, (const int32_t*)m->status);
 }
 
 void launch_swiglu_ws(aded_model* m, const GemmOut& gu, int rows, cudaStream_t st) {

@@ -165,10 +165,11 @@ static bool use_fused(const aded_model* m, int rows) {
 
 // Kernels one pass launches (what enqueue_pass enqueues), for the launch counter of graph replays.
 static int pass_launches(const aded_model* m, int rows, int chain_mode) {
-    if (use_fused(m, rows)) return 4 + 1 + 2 * m->cfg.n_layers + (chain_mode ? 1 : 5);
+    const int head = embed_norm_ws_supported(m) ? 3 : 4;
+    if (use_fused(m, rows)) return head + 1 + 2 * m->cfg.n_layers + (chain_mode ? 1 : 5);
     const int gemm_passes = (rows + 127) / 128;   // the tensor-core GEMM runs once per 128 rows
     const int per_gemm = m->ws_ready ? gemm_passes : 1;
-    int n = 4 + m->cfg.n_layers * (4 * per_gemm + 3 + 1);
+    int n = head + m->cfg.n_layers * (4 * per_gemm + 3 + 1);
     n += chain_mode ? 1 : per_gemm + 5;
     return n;
 }
@@ -186,11 +187,16 @@ static aded_status enqueue_pass(aded_model* m, aded_kv* kv, const int32_t* offse
                                   cudaMemcpyHostToDevice, st));
     if (use_fused(m, rows)) ADED_CUDA_TRY(cudaMemsetAsync(m->fw_counters, 0, 2 * FW_COUNTERS * sizeof(uint32_t), st));
     {
-        Span sp(m, PROF_OTHER, 4, st);
+        const bool one = embed_norm_ws_supported(m);
+        Span sp(m, PROF_OTHER, one ? 3 : 4, st);
         launch_tree_prologue(m, kv, batch, chain_mode, st);
-        launch_embed(m, rows, st);
         launch_rope_table(m, rows, st);
-        launch_add_rmsnorm(m, (const GemmOut*)nullptr, m->layers[0].norm1, rows, st);
+        if (one) {
+            launch_embed_norm_ws(m, m->layers[0].norm1, rows, st);
+        } else {
+            launch_embed(m, rows, st);
+            launch_add_rmsnorm(m, (const GemmOut*)nullptr, m->layers[0].norm1, rows, st);
+        }
     }
     const size_t hid_bytes = (size_t)rows * d * m->elem;
     if (m->dbg_hidden) ADED_CUDA_TRY(cudaMemcpyAsync(m->dbg_hidden, m->h, hid_bytes, cudaMemcpyDeviceToDevice, st));
