@@ -214,9 +214,20 @@ __global__ void __launch_bounds__(256) k_argmax_chunks(GemmOut logits, float* __
     const int c0 = blockIdx.x * chunk, c1 = min(V, c0 + chunk);
     float bv = -INFINITY;
     int bi = 0x7fffffff;
-    for (int c = c0 + threadIdx.x; c < c1; c += 256) {
-        const float v = gemm_out_load(logits, r, c);
-        if (v > bv) { bv = v; bi = c; }   // c ascends per thread: first maximum kept
+    if (logits.mode == 1 && (V & 3) == 0) {
+        // partial tiles: four adjacent columns per thread and step, all contributors fetched at once
+        for (int c = c0 + threadIdx.x * 4; c < c1; c += 1024) {
+            const float4 v = gemm_out_at4(logits, logits.tiles[c >> 7], r, c & 127);
+            if (v.x > bv) { bv = v.x; bi = c; }       // columns ascend per thread: first maximum kept
+            if (v.y > bv) { bv = v.y; bi = c + 1; }
+            if (v.z > bv) { bv = v.z; bi = c + 2; }
+            if (v.w > bv) { bv = v.w; bi = c + 3; }
+        }
+    } else {
+        for (int c = c0 + threadIdx.x; c < c1; c += 256) {
+            const float v = gemm_out_load(logits, r, c);
+            if (v > bv) { bv = v; bi = c; }   // c ascends per thread: first maximum kept
+        }
     }
     for (int o = 16; o > 0; o >>= 1) {
         const float ov = __shfl_xor_sync(0xffffffffu, bv, o);

@@ -71,23 +71,34 @@ __global__ void k_accept(const CallPtrs* __restrict__ call,
     int32_t* __restrict__ out_tokens = call->out_tokens;
     int32_t* __restrict__ out_len = call->out_len;
     const int out_stride = call->out_stride;
-    const int b = blockIdx.x * blockDim.x + threadIdx.x;
+    // one block per sequence: the tree's arrays are fetched by all threads at once, then one thread walks
+    const int b = blockIdx.x;
     if (b >= batch) return;
-    if (*status != 0) {
+    __shared__ int32_t s_par[ADED_MAX_NODES], s_tok[ADED_MAX_NODES], s_best[ADED_MAX_NODES], s_dep[ADED_MAX_NODES];
+    const int pass_status = *status;
+    const int off = row_off[b];
+    const int T = min(row_off[b + 1] - off, (int)ADED_MAX_NODES);
+    for (int i = threadIdx.x; i < T; i += blockDim.x) {
+        s_par[i] = parents[off + i];
+        s_tok[i] = tokens[off + i];
+        s_best[i] = best[off + i];
+        s_dep[i] = depth[off + i];
+    }
+    __syncthreads();
+    if (threadIdx.x != 0) return;
+    if (pass_status != 0) {
         out_len[b] = 0;
         new_len[b] = len[b];
         return;
     }
-    const int off = row_off[b];
-    const int T = row_off[b + 1] - off;
     uint64_t ok_lo = 1ull, ok_hi = 0ull;   // approved set; the root always is
     int deepest = 0, deepest_depth = 0;
     for (int i = 1; i < T; ++i) {
-        const int p = parents[off + i];
+        const int p = s_par[i];
         const bool p_ok = p < 64 ? (ok_lo >> p) & 1 : (ok_hi >> (p - 64)) & 1;
-        if (p_ok && tokens[off + i] == best[off + p]) {
+        if (p_ok && s_tok[i] == s_best[p]) {
             if (i < 64) ok_lo |= 1ull << i; else ok_hi |= 1ull << (i - 64);
-            const int d = depth[off + i];
+            const int d = s_dep[i];
             if (d > deepest_depth) { deepest_depth = d; deepest = i; }
         }
     }
@@ -95,8 +106,8 @@ __global__ void k_accept(const CallPtrs* __restrict__ call,
     int cur = deepest;
     for (int j = deepest_depth; j >= 0; --j) {
         path[b * ADED_MAX_NODES + j] = cur;
-        out_tokens[(size_t)b * out_stride + j] = best[off + cur];
-        cur = parents[off + cur];
+        out_tokens[(size_t)b * out_stride + j] = s_best[cur];
+        cur = s_par[cur];
     }
     out_len[b] = deepest_depth + 1;
     new_len[b] = len[b] + deepest_depth + 1;
@@ -139,7 +150,7 @@ void launch_tree_prologue(aded_model* m, aded_kv* kv, int batch, int chain_mode,
 }
 
 void launch_accept(aded_model* m, aded_kv* kv, int batch, cudaStream_t st) {
-    launch_k(k_accept, (batch + 31) / 32, 32, 0, st, m->call_dev, m->seqs.row_off, m->best, m->rows.depth,
+    launch_k(k_accept, batch, 128, 0, st, m->call_dev, m->seqs.row_off, m->best, m->rows.depth,
                                                kv->len_dev, m->seqs.path, m->seqs.new_len, m->status, batch);
 }
 
