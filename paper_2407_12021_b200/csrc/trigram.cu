@@ -493,7 +493,7 @@ __device__ __forceinline__ void mc_lookup_cached(const TgView& t, int a, int b, 
 }
 
 __host__ __device__ constexpr size_t mc_cache_offset() {
-    return (((size_t)MC_MAX_NODES * (8 + 4 * 4 + 2 * 2 + 2 * 1) + (size_t)MC_CHAIN * 8 + ADED_MAX_NODES * 2) + 15) & ~(size_t)15;
+    return (((size_t)MC_MAX_NODES * (2 * 8 + 2 * 4 + 2 * 2 + 2 * 1) + (size_t)MC_CHAIN * 8 + ADED_MAX_NODES * 2) + 15) & ~(size_t)15;
 }
 
 __global__ void __launch_bounds__(32)
@@ -503,11 +503,10 @@ k_mcts_draft(TgView t, const __grid_constant__ McParams p, const int32_t* __rest
     extern __shared__ __align__(16) uint8_t mc_smem[];
     // 8-byte, then 4-byte, then 2-byte, then 1-byte arrays, so that each starts aligned
     double* s_score = reinterpret_cast<double*>(mc_smem);                 // [MC_MAX_NODES] sum of scores
-    int32_t* s_tok = reinterpret_cast<int32_t*>(s_score + MC_MAX_NODES);  // token
+    double* s_prior = s_score + MC_MAX_NODES;                             // Eq. 1 probability of the node's token in its parent's context
+    int32_t* s_tok = reinterpret_cast<int32_t*>(s_prior + MC_MAX_NODES);  // token
     int32_t* s_visits = s_tok + MC_MAX_NODES;
-    uint32_t* s_cnt = reinterpret_cast<uint32_t*>(s_visits + MC_MAX_NODES);   // count of the node's token in its parent's context
-    uint32_t* s_ctxtot = s_cnt + MC_MAX_NODES;                            // expanded nodes: total of their own context
-    int32_t* s_ltok = reinterpret_cast<int32_t*>(s_ctxtot + MC_MAX_NODES);    // lookup scratch
+    int32_t* s_ltok = s_visits + MC_MAX_NODES;                            // lookup scratch
     uint32_t* s_lcnt = reinterpret_cast<uint32_t*>(s_ltok + MC_CHAIN);
     int16_t* s_par = reinterpret_cast<int16_t*>(s_lcnt + MC_CHAIN);
     int16_t* s_first = s_par + MC_MAX_NODES;                              // first child (children are consecutive)
@@ -525,7 +524,7 @@ k_mcts_draft(TgView t, const __grid_constant__ McParams p, const int32_t* __rest
     int n_nodes = 1;
     if (lane == 0) {
         s_tok[0] = root_token; s_par[0] = -1; s_first[0] = 0; s_nkid[0] = 0; s_flag[0] = 0;
-        s_visits[0] = 0; s_score[0] = 0.0; s_cnt[0] = 0; s_ctxtot[0] = 0;
+        s_visits[0] = 0; s_score[0] = 0.0; s_prior[0] = 0.0;
     }
     __syncwarp();
     McLookup lk;
@@ -544,9 +543,9 @@ k_mcts_draft(TgView t, const __grid_constant__ McParams p, const int32_t* __rest
             const int nv = mine ? s_visits[c] : 0;
             int n_sum = nv;
             for (int o = 16; o > 0; o >>= 1) n_sum += __shfl_xor_sync(0xffffffffu, n_sum, o);
-            const double e = p.e_table[n_sum], root_n = sqrt((double)n_sum), tot = (double)s_ctxtot[node];
+            const double e = p.e_table[n_sum], root_n = sqrt((double)n_sum);
             const double q = nv ? __ddiv_rn(s_score[c], (double)nv) : 0.0;
-            const double pr = __ddiv_rn((double)s_cnt[c], tot);
+            const double pr = s_prior[c];
             double best_s = __dadd_rn(q, __ddiv_rn(__dmul_rn(__dmul_rn(e, pr), root_n), __dadd_rn(1.0, (double)nv)));
             double best_p = pr;
             int best = mine ? c : -1;
@@ -567,21 +566,21 @@ k_mcts_draft(TgView t, const __grid_constant__ McParams p, const int32_t* __rest
             mc_lookup_cached(t, a, b, p.k, lane, s_ltok, s_lcnt, s_ckey, s_cval, lk);
             if (lane == 0) {
                 s_flag[node] |= 1;
-                s_ctxtot[node] = lk.total;
                 s_first[node] = (int16_t)n_nodes;
                 s_nkid[node] = (uint8_t)lk.n;
-                for (int j = 0; j < lk.n; ++j) {
-                    const int c = n_nodes + j;
-                    s_tok[c] = lk.word[j]; s_par[c] = (int16_t)node; s_first[c] = 0; s_nkid[c] = 0; s_flag[c] = 0;
-                    s_visits[c] = 0; s_score[c] = 0.0; s_cnt[c] = lk.count[j]; s_ctxtot[c] = 0;
-                }
+            }
+            if (lane < lk.n) {                            // one lane per child: the divisions run side by side
+                const int c = n_nodes + lane;
+                s_tok[c] = lk.word[lane]; s_par[c] = (int16_t)node; s_first[c] = 0; s_nkid[c] = 0; s_flag[c] = 0;
+                s_visits[c] = 0; s_score[c] = 0.0;
+                s_prior[c] = __ddiv_rn((double)lk.count[lane], (double)lk.total);
             }
             __syncwarp();
             if (lk.n > 0) {
                 n_nodes += lk.n;
                 node = n_nodes - 1;                       // the last child created
                 state[len] = s_tok[node];
-                sp[len] = __ddiv_rn((double)s_cnt[node], (double)lk.total);
+                sp[len] = s_prior[node];
                 ++len;
             }
         }
