@@ -145,9 +145,10 @@ __global__ void __launch_bounds__(NW * 32) k_tree_attn_mma(AttnArgs a) {
     bf16* sv = sk + TA_STAGES * TA_BLK * HD;                      // [TA_STAGES][TA_BLK][HD]
     // Before waiting for the previous kernel (which writes the tree's own K/V rows and q): start
     // fetching this CTA's first key blocks if they lie entirely in the committed part of the cache,
-    // which no kernel of this pass writes.  The committed length and the tree size are read here on
-    // trust -- nothing orders this read after the kernels that wrote them -- and read again after the
-    // wait: the early blocks are used only if both reads agree, otherwise they are fetched again.
+    // which no kernel of this pass writes.  The committed length and the tree size were written before
+    // this pass began (a pass opens with a copy on the stream, which no kernel of the pass overtakes),
+    // but this kernel does not rely on that: both are read again after the wait and the early blocks
+    // are used only if the two reads agree, otherwise they are fetched again.
     // The cache block's address and capacity never change after the cache was created.
     const int pre_hh = blockIdx.x, pre_b = blockIdx.z / a.row_blocks;
     const size_t pre_cp = a.cap[pre_b];
