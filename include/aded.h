@@ -334,12 +334,24 @@ aded_status aded_draft_tree(const aded_trigram* t, const int32_t* context_dev, i
  * ties); the best n_candidates (the paper: 24; n_candidates * length + 1 <= ADED_MAX_NODES) are
  * written as sentence_tokens_dev[r][length] (-1 padded) with sentence_scores_dev[r], and merged
  * into one prefix tree tree_tokens_dev / tree_parents_dev (breadth-first, *n_nodes_dev nodes, node 0
- * the last token of the text) ready for aded_verify.  All scores are IEEE doubles computed one
- * rounded operation at a time.  One warp; asynchronous on `stream`. */
+ * the last token of the text) ready for aded_verify.  With n_nodes_target > 0 the prefix tree is then
+ * completed to exactly that many nodes from filler_dev[0 .. n_filler) by the rule of aded_draft_tree
+ * (depth limit `length`, at most k children), so that verification steps keep one shape; a filler
+ * that runs out is reported as there.  All scores are IEEE doubles computed one rounded operation
+ * at a time.  One warp; asynchronous on `stream`. */
 aded_status aded_mcts_draft(const aded_trigram* t, const int32_t* context_dev, int32_t iterations, int32_t length,
                             int32_t n_candidates, int32_t k, float c1, float c2, const float* u_dev, int32_t* tree_tokens_dev,
                             int32_t* tree_parents_dev, int32_t* n_nodes_dev, int32_t* sentence_tokens_dev,
-                            double* sentence_scores_dev, int32_t* n_sentences_dev, void* stream);
+                            double* sentence_scores_dev, int32_t* n_sentences_dev, int32_t n_nodes_target,
+                            const int32_t* filler_dev, int32_t n_filler, void* stream);
+
+/* aded_decode_step with the draft tree made by aded_mcts_draft (the paper's own loop: tree search over
+ * the tri-gram statistics, tree verification, feedback of the output into the statistics), completed
+ * to n_nodes nodes with the filler.  u_dev holds iterations * length uniform numbers for this step. */
+aded_status aded_decode_step_mcts(aded_model* m, aded_kv* kv, aded_trigram* t, int32_t* context_dev, int32_t n_nodes,
+                                  int32_t iterations, int32_t length, int32_t n_candidates, int32_t k, float c1, float c2,
+                                  const float* u_dev, const int32_t* filler_dev, int32_t n_filler, int32_t* out_tokens_dev,
+                                  int32_t* out_accept_len_dev, void* stream);
 
 /* One decoding step, all on the device and asynchronous on `stream`:
  *   aded_draft_tree from context_dev  ->  aded_verify (out_tokens_dev[n_nodes], out_accept_len_dev[1])

@@ -53,28 +53,43 @@ def draft_tree(store: TrigramStore, prev_token: int, root_token: int, n_nodes: i
                 depth.append(depth[head] + 1)
         head += 1
     from_table = len(tokens)
-    if filler is not None and len(tokens) < n_nodes:
-        pos = 0
-        p = 0
-        idle = 0
-        while len(tokens) < n_nodes:
-            kids = [tokens[i] for i in range(1, len(tokens)) if parents[i] == p]
-            if depth[p] < max_depth and len(kids) < k:
-                while pos < len(filler) and int(filler[pos]) in kids:
-                    pos += 1
-                if pos >= len(filler):
-                    raise ValueError("filler exhausted")
-                tokens.append(int(filler[pos]))
-                pos += 1
-                parents.append(p)
-                depth.append(depth[p] + 1)
-                idle = 0
-            else:
-                idle += 1
-                if idle > len(tokens):
-                    raise ValueError("no node has room for a filler child")
-            p = (p + 1) % len(tokens)
+    if filler is not None:
+        tokens, parents = fill_tree(tokens, parents, n_nodes, max_depth, k, filler)
     return tokens, parents, from_table
+
+
+def fill_tree(tokens: Sequence[int], parents: Sequence[int], n_nodes: int, max_depth: int, k: int,
+              filler: Sequence[int]) -> Tuple[List[int], List[int]]:
+    """Completes a draft tree (parents[i] < i) to exactly n_nodes nodes with caller-supplied tokens, by the
+    rule of draft_tree's docstring: nodes are visited round-robin; a visited node with depth < max_depth
+    and fewer than k children gets the next filler token that none of its children holds.  A tree that
+    already has n_nodes nodes or more is returned unchanged."""
+    tokens = [int(t) for t in tokens]
+    parents = [int(p) for p in parents]
+    depth = [0] * len(tokens)
+    for i in range(1, len(tokens)):
+        depth[i] = depth[parents[i]] + 1
+    pos = 0
+    p = 0
+    idle = 0
+    while len(tokens) < n_nodes:
+        kids = [tokens[i] for i in range(1, len(tokens)) if parents[i] == p]
+        if depth[p] < max_depth and len(kids) < k:
+            while pos < len(filler) and int(filler[pos]) in kids:
+                pos += 1
+            if pos >= len(filler):
+                raise ValueError("filler exhausted")
+            tokens.append(int(filler[pos]))
+            pos += 1
+            parents.append(p)
+            depth.append(depth[p] + 1)
+            idle = 0
+        else:
+            idle += 1
+            if idle > len(tokens):
+                raise ValueError("no node has room for a filler child")
+        p = (p + 1) % len(tokens)
+    return tokens, parents
 
 
 def decode_context(prev_token: int, root_token: int, accepted: Sequence[int]) -> Tuple[int, int]:

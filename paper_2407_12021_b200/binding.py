@@ -29,7 +29,7 @@ EXPORTS = [
     "aded_trigram_update", "aded_trigram_update_host", "aded_trigram_topk", "aded_trigram_topk_host",
     "aded_trigram_get", "aded_trigram_stats", "aded_trigram_poll_status", "aded_draft_tree", "aded_decode_step",
     "aded_decode_step_host", "aded_verify_sampled", "aded_sample_tokens", "aded_trigram_export",
-    "aded_trigram_import", "aded_mcts_draft", "aded_trigram_clear", "aded_trigram_prune", "aded_trigram_save", "aded_trigram_load", "aded_status_string",
+    "aded_trigram_import", "aded_mcts_draft", "aded_decode_step_mcts", "aded_trigram_clear", "aded_trigram_prune", "aded_trigram_save", "aded_trigram_load", "aded_status_string",
 ]
 
 
@@ -500,9 +500,15 @@ def aded_trigram_load(t: Trigram, path: str) -> None:
 
 
 def aded_mcts_draft(t: Trigram, context_dev: torch.Tensor, iterations: int, length: int, n_candidates: int, k: int,
-                    u: torch.Tensor, c1: float = 32.0, c2: float = 8.0):
+                    u: torch.Tensor, c1: float = 32.0, c2: float = 8.0, n_nodes_target: int = 0,
+                    filler_dev: Optional[torch.Tensor] = None):
     """Runs the tree search; returns (tokens, parents, sentences) as Python lists after synchronising:
-    the merged prefix tree and the ranked sentences [(tokens after the root, mean score)]."""
+    the merged prefix tree (completed to n_nodes_target nodes from filler_dev when given) and the ranked
+    sentences [(tokens after the root, mean score)]."""
+    nf = 0
+    if filler_dev is not None:
+        _dev_i32(filler_dev, "filler")
+        nf = filler_dev.numel()
     _dev_i32(context_dev, "context"), _dev_f32(u, "u")
     if u.numel() < iterations * length:
         raise ValueError("u must hold iterations * length numbers")
@@ -513,11 +519,26 @@ def aded_mcts_draft(t: Trigram, context_dev: torch.Tensor, iterations: int, leng
     sc = torch.zeros(n_candidates, dtype=torch.float64, device="cuda")
     _check(_lib.aded_mcts_draft(t.handle, _ptr(context_dev), c_int32(iterations), c_int32(length), c_int32(n_candidates),
                                 c_int32(k), c_float(c1), c_float(c2), _ptr(u), _ptr(tok), _ptr(par), c_void_p(n.data_ptr()),
-                                _ptr(st), _ptr(sc), c_void_p(n.data_ptr() + 4), _stream()), "aded_mcts_draft")
+                                _ptr(st), _ptr(sc), c_void_p(n.data_ptr() + 4), c_int32(n_nodes_target), _ptr(filler_dev), c_int32(nf),
+                                _stream()), "aded_mcts_draft")
     torch.cuda.synchronize()
     nn, ns = int(n[0]), int(n[1])
     sentences = [([x for x in st[r].tolist() if x >= 0], float(sc[r])) for r in range(ns)]
     return tok[:nn].tolist(), par[:nn].tolist(), sentences
+
+
+def aded_decode_step_mcts(model: Model, kv: KV, t: Trigram, context_dev: torch.Tensor, n_nodes: int, iterations: int, length: int,
+                          n_candidates: int, k: int, u: torch.Tensor, filler_dev: torch.Tensor, out_tokens: torch.Tensor,
+                          out_accept_len: torch.Tensor, c1: float = 32.0, c2: float = 8.0) -> None:
+    """One decoding step whose draft tree comes from the tree search; context_dev [2] is read and advanced."""
+    _dev_i32(context_dev, "context"), _dev_f32(u, "u"), _dev_i32(filler_dev, "filler")
+    _dev_i32(out_tokens, "out_tokens"), _dev_i32(out_accept_len, "out_accept_len")
+    if u.numel() < iterations * length or out_tokens.numel() < n_nodes or out_accept_len.numel() < 1:
+        raise ValueError("arrays are too short")
+    _check(_lib.aded_decode_step_mcts(model.handle, kv.handle, t.handle, _ptr(context_dev), c_int32(n_nodes), c_int32(iterations),
+                                      c_int32(length), c_int32(n_candidates), c_int32(k), c_float(c1), c_float(c2), _ptr(u),
+                                      _ptr(filler_dev), c_int32(filler_dev.numel()), _ptr(out_tokens), _ptr(out_accept_len),
+                                      _stream()), "aded_decode_step_mcts")
 
 
 def aded_status_string(status: int) -> str:

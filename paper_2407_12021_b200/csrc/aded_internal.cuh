@@ -140,6 +140,8 @@ struct aded_model {
     float samp_temp, samp_top_p;
     const float* samp_u;        // caller's [rows] uniform numbers (device)
 
+    void* step_mcts;            // scratch of aded_decode_step_mcts (allocated on first use)
+
     float* dbg_logits;
     int32_t* dbg_best;
     void* dbg_hidden;   // [n_layers + 1][rows][d] copies of the residual stream (debug capture)

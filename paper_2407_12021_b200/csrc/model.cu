@@ -435,6 +435,7 @@ aded_status aded_model_create(const aded_model_config* cfg, const aded_weights* 
     m->dbg_logits = nullptr;
     m->dbg_best = nullptr;
     m->dbg_hidden = nullptr;
+    m->step_mcts = nullptr;
     m->samp_on = false;
     m->samp_temp = 1.f;
     m->samp_top_p = 1.f;

@@ -247,6 +247,42 @@ __global__ void k_tg_topk(TgView t, const int32_t* __restrict__ ctx, int q, int 
 // supplied tokens under nodes with room, round-robin, until the tree is full.
 constexpr int DRAFT_MAX_FILLER = 4 * ADED_MAX_NODES;
 
+// Filler pass of one thread over a tree held in shared memory (tok, par, dep; kid[p][0 .. nkid[p]) the
+// child tokens of node p): nodes are visited round-robin, a visited node with depth < max_depth and
+// fewer than k children gets the next filler token none of its children holds.  Returns the new node
+// count; *fail when the filler runs out, holds a token outside the vocabulary, or no node has room.
+__device__ __forceinline__ int draft_fill(int32_t* tok, int32_t* par, int32_t* dep, int32_t* nkid, int32_t* kid, int n, int n_nodes,
+                                          int max_depth, int k, const int32_t* fill, int n_filler, int vocab, bool* fail) {
+    int pos = 0, p = 0, idle = 0;
+    while (n < n_nodes) {
+        const int nk = nkid[p];
+        if (dep[p] < max_depth && nk < k) {
+            int32_t f = -1;
+            for (; pos < n_filler; ++pos) {
+                f = fill[pos];
+                bool clash = false;
+                for (int j = 0; j < nk; ++j) clash |= kid[p * ADED_DRAFT_MAX_K + j] == f;
+                if (!clash) break;
+            }
+            if (pos >= n_filler || f < 0 || f >= vocab) { *fail = true; break; }
+            ++pos;
+            kid[p * ADED_DRAFT_MAX_K + nk] = f;
+            nkid[p] = nk + 1;
+            tok[n] = f;
+            par[n] = p;
+            dep[n] = dep[p] + 1;
+            nkid[n] = 0;
+            ++n;
+            idle = 0;
+        } else if (++idle > n) {
+            *fail = true;
+            break;
+        }
+        p = (p + 1) % n;
+    }
+    return n;
+}
+
 __global__ void __launch_bounds__(1024)
 k_draft_tree(TgView t, const int32_t* __restrict__ ctx, int n_nodes, int max_depth, int k,
              const int32_t* __restrict__ filler, int n_filler, int32_t* __restrict__ out_tok,
@@ -307,33 +343,9 @@ k_draft_tree(TgView t, const int32_t* __restrict__ ctx, int n_nodes, int max_dep
         int n = s_n;
         if (out_real) *out_real = n;
         if (filler && n < n_nodes) {
-            int pos = 0, p = 0, idle = 0;
-            while (n < n_nodes) {
-                const int nk = s_nkid[p];
-                if (s_dep[p] < max_depth && nk < k) {
-                    int32_t f = -1;
-                    for (; pos < n_filler; ++pos) {
-                        f = s_fill[pos];
-                        bool clash = false;
-                        for (int j = 0; j < nk; ++j) clash |= s_cand[p * ADED_DRAFT_MAX_K + j] == f;
-                        if (!clash) break;
-                    }
-                    if (pos >= n_filler || f < 0 || f >= t.vocab) { s_fail = 1; break; }
-                    ++pos;
-                    s_cand[p * ADED_DRAFT_MAX_K + nk] = f;
-                    s_nkid[p] = nk + 1;
-                    s_tok[n] = f;
-                    s_par[n] = p;
-                    s_dep[n] = s_dep[p] + 1;
-                    s_nkid[n] = 0;
-                    ++n;
-                    idle = 0;
-                } else if (++idle > n) {
-                    s_fail = 1;
-                    break;
-                }
-                p = (p + 1) % n;
-            }
+            bool fail = false;
+            n = draft_fill(s_tok, s_par, s_dep, s_nkid, s_cand, n, n_nodes, max_depth, k, s_fill, n_filler, t.vocab, &fail);
+            if (fail) s_fail = 1;
             s_n = n;
         }
         if (s_fail) atomicCAS(t.status, 0, (int)ADED_ERR_INVALID_ARG);
@@ -496,10 +508,15 @@ __host__ __device__ constexpr size_t mc_cache_offset() {
     return (((size_t)MC_MAX_NODES * (2 * 8 + 2 * 4 + 2 * 2 + 2 * 1) + (size_t)MC_CHAIN * 8 + ADED_MAX_NODES * 2) + 15) & ~(size_t)15;
 }
 
+__host__ __device__ constexpr size_t mc_fill_offset() {
+    return (mc_cache_offset() + (size_t)MC_CACHE * (8 + sizeof(McLookup)) + (size_t)MC_MAX_ITER * MC_MAX_LEN * sizeof(float) + 15) & ~(size_t)15;
+}
+
 __global__ void __launch_bounds__(32)
 k_mcts_draft(TgView t, const __grid_constant__ McParams p, const int32_t* __restrict__ ctx, const float* __restrict__ u,
              int32_t* __restrict__ out_tok, int32_t* __restrict__ out_par, int32_t* __restrict__ out_n,
-             int32_t* __restrict__ sent_tok, double* __restrict__ sent_score, int32_t* __restrict__ out_n_sent) {
+             int32_t* __restrict__ sent_tok, double* __restrict__ sent_score, int32_t* __restrict__ out_n_sent,
+             int n_target, const int32_t* __restrict__ filler, int n_filler) {
     extern __shared__ __align__(16) uint8_t mc_smem[];
     // 8-byte, then 4-byte, then 2-byte, then 1-byte arrays, so that each starts aligned
     double* s_score = reinterpret_cast<double*>(mc_smem);                 // [MC_MAX_NODES] sum of scores
@@ -644,6 +661,11 @@ k_mcts_draft(TgView t, const __grid_constant__ McParams p, const int32_t* __rest
         __syncwarp();
         ++n_sent;
     }
+    if (n_target > 0 && filler) {
+        int32_t* f_fill = reinterpret_cast<int32_t*>(mc_smem + mc_fill_offset()) + ADED_MAX_NODES * (4 + ADED_DRAFT_MAX_K);
+        for (int i = lane; i < n_filler; i += 32) f_fill[i] = filler[i];
+        __syncwarp();
+    }
     // prefix tree of the chosen sentences, breadth first, children in creation order
     if (lane == 0) {
         int count = 1;
@@ -660,13 +682,34 @@ k_mcts_draft(TgView t, const __grid_constant__ McParams p, const int32_t* __rest
                 ++count;
             }
         }
+        if (n_target > count && filler) {
+            // complete the prefix tree to a fixed number of nodes, by the rule of the draft-tree kernel
+            int32_t* f_tok = reinterpret_cast<int32_t*>(mc_smem + mc_fill_offset());       // [ADED_MAX_NODES] each
+            int32_t* f_par = f_tok + ADED_MAX_NODES;
+            int32_t* f_dep = f_par + ADED_MAX_NODES;
+            int32_t* f_nkid = f_dep + ADED_MAX_NODES;
+            int32_t* f_kid = f_nkid + ADED_MAX_NODES;                                      // [ADED_MAX_NODES][ADED_DRAFT_MAX_K]
+            int32_t* f_fill = f_kid + ADED_MAX_NODES * ADED_DRAFT_MAX_K;                   // [DRAFT_MAX_FILLER], staged above by the whole warp
+            for (int i = 0; i < count; ++i) { f_nkid[i] = 0; }
+            for (int i = 0; i < count; ++i) {
+                f_tok[i] = out_tok[i];
+                f_par[i] = out_par[i];
+                f_dep[i] = i == 0 ? 0 : f_dep[f_par[i]] + 1;
+                if (i > 0) { const int pp = f_par[i]; f_kid[pp * ADED_DRAFT_MAX_K + f_nkid[pp]] = f_tok[i]; f_nkid[pp] += 1; }
+            }
+            bool fail = false;
+            const int n2 = draft_fill(f_tok, f_par, f_dep, f_nkid, f_kid, count, n_target, p.length, p.k, f_fill, n_filler, t.vocab, &fail);
+            for (int i = count; i < n2; ++i) { out_tok[i] = f_tok[i]; out_par[i] = f_par[i]; }
+            count = n2;
+            if (fail) { atomicCAS(t.status, 0, (int)ADED_ERR_INVALID_ARG); out_tok[0] = -1; }
+        }
         *out_n = count;
         *out_n_sent = n_sent;
     }
 }
 
 static size_t mc_smem_bytes() {
-    return mc_cache_offset() + (size_t)MC_CACHE * (8 + sizeof(McLookup)) + (size_t)MC_MAX_ITER * MC_MAX_LEN * sizeof(float);
+    return mc_fill_offset() + (size_t)ADED_MAX_NODES * 4 * (4 + ADED_DRAFT_MAX_K) + (size_t)DRAFT_MAX_FILLER * 4 + 64;
 }
 
 }  // namespace aded
@@ -833,9 +876,13 @@ aded_status aded_draft_tree(const aded_trigram* t, const int32_t* context_dev, i
 aded_status aded_mcts_draft(const aded_trigram* t, const int32_t* context_dev, int32_t iterations, int32_t length,
                             int32_t n_candidates, int32_t k, float c1, float c2, const float* u_dev, int32_t* tree_tokens_dev,
                             int32_t* tree_parents_dev, int32_t* n_nodes_dev, int32_t* sentence_tokens_dev,
-                            double* sentence_scores_dev, int32_t* n_sentences_dev, void* stream) {
+                            double* sentence_scores_dev, int32_t* n_sentences_dev, int32_t n_nodes_target,
+                            const int32_t* filler_dev, int32_t n_filler, void* stream) {
     if (!t || !context_dev || !u_dev || !tree_tokens_dev || !tree_parents_dev || !n_nodes_dev || !sentence_tokens_dev ||
         !sentence_scores_dev || !n_sentences_dev)
+        return ADED_ERR_INVALID_ARG;
+    if (n_nodes_target < 0 || n_nodes_target > ADED_MAX_NODES || n_filler < 0 || n_filler > DRAFT_MAX_FILLER ||
+        (n_nodes_target > 0 && (!filler_dev || n_filler < 1)))
         return ADED_ERR_INVALID_ARG;
     if (iterations < 1 || iterations > MC_MAX_ITER || length < 1 || length > MC_MAX_LEN || k < 1 || k > MC_MAX_K ||
         n_candidates < 1 || n_candidates * length + 1 > ADED_MAX_NODES || !(c2 > 0.f))
@@ -854,7 +901,8 @@ aded_status aded_mcts_draft(const aded_trigram* t, const int32_t* context_dev, i
     note_launch();
     k_mcts_draft<<<1, 32, mc_smem_bytes(), static_cast<cudaStream_t>(stream)>>>(t->view, p, context_dev, u_dev, tree_tokens_dev,
                                                                                tree_parents_dev, n_nodes_dev, sentence_tokens_dev,
-                                                                               sentence_scores_dev, n_sentences_dev);
+                                                                               sentence_scores_dev, n_sentences_dev, n_nodes_target,
+                                                                               n_nodes_target > 0 ? filler_dev : nullptr, n_filler);
     ADED_CUDA_TRY(cudaGetLastError());
     return ADED_OK;
 }
@@ -868,6 +916,36 @@ aded_status aded_decode_step(aded_model* m, aded_kv* kv, aded_trigram* t, int32_
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     aded_status s = aded_draft_tree(t, context_dev, n_nodes, max_depth, k, filler_dev, n_filler, m->tokens, m->parents,
                                     n_from_table_dev ? n_from_table_dev : t->step_i + STEP_REAL, stream);
+    if (s != ADED_OK) return s;
+    s = aded_verify(m, kv, m->tokens, m->parents, n_nodes, out_tokens_dev, out_accept_len_dev, stream);
+    if (s != ADED_OK) return s;
+    note_launch(2);
+    k_decode_advance<<<1, 160, 0, st>>>(out_tokens_dev, out_accept_len_dev, context_dev, t->step_i + STEP_SPAN,
+                                        t->step_i + STEP_LEN, n_nodes);
+    k_tg_update<<<(ADED_MAX_NODES + 255) / 256, 256, 0, st>>>(t->view, t->step_i + STEP_SPAN, n_nodes + 2,
+                                                              t->step_i + STEP_LEN);
+    ADED_CUDA_TRY(cudaGetLastError());
+    return ADED_OK;
+}
+
+aded_status aded_decode_step_mcts(aded_model* m, aded_kv* kv, aded_trigram* t, int32_t* context_dev, int32_t n_nodes,
+                                  int32_t iterations, int32_t length, int32_t n_candidates, int32_t k, float c1, float c2,
+                                  const float* u_dev, const int32_t* filler_dev, int32_t n_filler, int32_t* out_tokens_dev,
+                                  int32_t* out_accept_len_dev, void* stream) {
+    if (!m || !kv || !t || !context_dev || !out_tokens_dev || !out_accept_len_dev) return ADED_ERR_INVALID_ARG;
+    if (n_nodes < 1 || n_nodes > ADED_MAX_NODES || n_nodes > m->cfg.max_rows) return ADED_ERR_INVALID_ARG;
+    if (!m->step_mcts) {      // sentences and counts of the search, which a decoding step does not hand out
+        void* p = nullptr;
+        ADED_CUDA_TRY(cudaMalloc(&p, (size_t)ADED_MAX_NODES * (sizeof(int32_t) + sizeof(double)) + 64));
+        m->step_mcts = p;
+        m->owned.push_back(p);
+    }
+    double* scores = reinterpret_cast<double*>(m->step_mcts);
+    int32_t* sent = reinterpret_cast<int32_t*>(scores + ADED_MAX_NODES);
+    int32_t* counts = t->step_i + STEP_REAL;          // found nodes; the sentence count goes to the span-length word, rewritten below
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    aded_status s = aded_mcts_draft(t, context_dev, iterations, length, n_candidates, k, c1, c2, u_dev, m->tokens, m->parents, counts,
+                                    sent, scores, t->step_i + STEP_LEN, n_nodes, filler_dev, n_filler, stream);
     if (s != ADED_OK) return s;
     s = aded_verify(m, kv, m->tokens, m->parents, n_nodes, out_tokens_dev, out_accept_len_dev, stream);
     if (s != ADED_OK) return s;

@@ -92,3 +92,61 @@ def test_drafts_feed_the_verification_step(cuda_device):
     cpu = ov.verify(arch, ow, cache, tok, par)
     gpu = sess.verify(tok, par)
     H.compare_step(shape, gpu, cpu, tok, par, "mcts tree")
+
+
+def _mcts_tree_cpu(st, prev, root, n_nodes, iters, length, n, k, u, filler):
+    from oracle import draft as od
+    tok, par, _ = om.mcts_draft(st, prev, root, iters, length, n, k, u.reshape(iters, length).tolist())
+    tok, par = tok[:n_nodes], par[:n_nodes]          # breadth-first numbering: a prefix is a tree
+    return od.fill_tree(tok, par, n_nodes, length, k, filler)
+
+
+def test_completed_tree_and_decode_steps(cuda_device):
+    """The paper's loop on the device: tree search over the table -> prefix tree completed to a fixed
+    shape -> verification -> the emitted tokens raise the table's counts -> next context."""
+    from oracle import draft as od
+    from oracle import verify as ov
+    from paper_2407_12021_b200 import binding as B
+    shape = gen.TINY
+    w = gen.model_weights(shape, 61)
+    sess = H.GpuSession(shape, H.weights_to(w, cuda_device), capacity=400)
+    arch = ov.arch_from_shape(shape)
+    ow = ov.Weights(w, keep=True)
+    prompt = gen.zipf_tokens(96, 24, 61, 50).tolist()          # a small alphabet, so that contexts repeat
+    cache = ov.Cache(arch)
+    ov.append(arch, ow, cache, prompt[:-1])
+    sess.append(prompt[:-1])
+    st = TrigramStore()
+    st.update(prompt)
+    t = B.aded_trigram_create(shape.vocab, log2_buckets=12, overflow_buckets=1024)
+    B.aded_trigram_update(t, H.i32(prompt))
+    iters, length, n, k, n_nodes = 60, 4, 8, 4, 24
+    # the completed tree alone, for a context the table knows
+    u = gen.uniform01(iters * length, 61, 1).numpy().astype(np.float32)
+    filler = gen.zipf_tokens(4 * n_nodes, shape.vocab, 61, 2).tolist()
+    got = B.aded_mcts_draft(t, H.i32(prompt[30:32]), iters, length, n, k, torch.tensor(u, device="cuda"), n_nodes_target=n_nodes,
+                            filler_dev=H.i32(filler))
+    want = _mcts_tree_cpu(st, prompt[30], prompt[31], n_nodes, iters, length, n, k, u, filler)
+    assert (got[0], got[1]) == want and len(got[0]) == n_nodes
+    assert len(om.mcts_draft(st, prompt[30], prompt[31], iters, length, n, k, u.reshape(iters, length).tolist())[0]) > 3
+    # decoding steps
+    ctx = H.i32(prompt[-2:])
+    prev, root = prompt[-2], prompt[-1]
+    out = torch.full((n_nodes,), -7, dtype=torch.int32, device="cuda")
+    alen = torch.full((1,), -7, dtype=torch.int32, device="cuda")
+    for step in range(5):
+        u = gen.uniform01(iters * length, 61, 10 + step).numpy().astype(np.float32)
+        filler = gen.zipf_tokens(4 * n_nodes, shape.vocab, 61, 20 + step).tolist()
+        tokens, parents = _mcts_tree_cpu(st, prev, root, n_nodes, iters, length, n, k, u, filler)
+        cpu = ov.verify(arch, ow, cache, tokens, parents)
+        st.update([prev, root] + cpu["out_tokens"])
+        prev, root = od.decode_context(prev, root, cpu["out_tokens"])
+        B.aded_decode_step_mcts(sess.model, sess.kv, t, ctx, n_nodes, iters, length, n, k, torch.tensor(u, device="cuda"),
+                                H.i32(filler), out, alen)
+        torch.cuda.synchronize()
+        assert B.aded_model_poll_status(sess.model) == 0 and B.aded_trigram_poll_status(t) == 0
+        a = int(alen[0])
+        assert a == cpu["accept_len"] and out[:a].tolist() == cpu["out_tokens"], f"step {step}"
+        assert ctx.tolist() == [prev, root] and sess.length() == cache.length
+    for (a_, b_, c_), cnt in st.entries().items():
+        assert B.aded_trigram_get(t, a_, b_, c_) == cnt
