@@ -129,9 +129,7 @@ __global__ void __launch_bounds__(256) k_swiglu_ws(GemmOut gu, bf16* __restrict_
     const float4 g = gemm_out_at4(gu, tg, r, c & 127);
     const float4 u = gemm_out_at4(gu, tu, r, (F + c) & 127);
     if (pass_status != 0) return;
-    *reinterpret_cast<uint2*>(act + (size_t)r * F + c) =
-        pack4_bf16(g.x / (1.f + expf(-g.x)) * u.x, g.y / (1.f + expf(-g.y)) * u.y,
-                   g.z / (1.f + expf(-g.z)) * u.z, g.w / (1.f + expf(-g.w)) * u.w);
+    *reinterpret_cast<uint2*>(act + (size_t)r * F + c) = swiglu4(g, u);
 }
 
 // Rotary embedding + K/V write (see k_rope_kv): block = (row, head), hd/8 threads, each owning four
@@ -153,18 +151,7 @@ __global__ void k_rope_kv_ws(GemmOut qkv, const float* __restrict__ cs, const fl
     const size_t cp = cap[b];
     bf16* kdst = reinterpret_cast<bf16*>(base[b]) + ((((size_t)layer * 2 + 0) * H + hh) * cp + slot) * hd;
     bf16* vdst = reinterpret_cast<bf16*>(base[b]) + ((((size_t)layer * 2 + 1) * H + hh) * cp + slot) * hd;
-    const float4 q0 = gemm_out_at4(qkv, tq, r, (cq + i) & 127), q1 = gemm_out_at4(qkv, tq, r, (cq + i + half) & 127);
-    const float4 k0 = gemm_out_at4(qkv, tk, r, (ck + i) & 127), k1 = gemm_out_at4(qkv, tk, r, (ck + i + half) & 127);
-    const float4 v0 = gemm_out_at4(qkv, tv, r, (cv + i) & 127), v1 = gemm_out_at4(qkv, tv, r, (cv + i + half) & 127);
-    const float4 c = *reinterpret_cast<const float4*>(cs + r * half + i), s = *reinterpret_cast<const float4*>(sn + r * half + i);
-    if (pass_status != 0) return;
-    bf16* qd = q + (size_t)r * d + hh * hd;
-    *reinterpret_cast<uint2*>(qd + i) = pack4_bf16(q0.x * c.x - q1.x * s.x, q0.y * c.y - q1.y * s.y, q0.z * c.z - q1.z * s.z, q0.w * c.w - q1.w * s.w);
-    *reinterpret_cast<uint2*>(qd + i + half) = pack4_bf16(q1.x * c.x + q0.x * s.x, q1.y * c.y + q0.y * s.y, q1.z * c.z + q0.z * s.z, q1.w * c.w + q0.w * s.w);
-    *reinterpret_cast<uint2*>(kdst + i) = pack4_bf16(k0.x * c.x - k1.x * s.x, k0.y * c.y - k1.y * s.y, k0.z * c.z - k1.z * s.z, k0.w * c.w - k1.w * s.w);
-    *reinterpret_cast<uint2*>(kdst + i + half) = pack4_bf16(k1.x * c.x + k0.x * s.x, k1.y * c.y + k0.y * s.y, k1.z * c.z + k0.z * s.z, k1.w * c.w + k0.w * s.w);
-    *reinterpret_cast<uint2*>(vdst + i) = pack4_bf16(v0.x, v0.y, v0.z, v0.w);
-    *reinterpret_cast<uint2*>(vdst + i + half) = pack4_bf16(v1.x, v1.y, v1.z, v1.w);
+    rope_kv_item(qkv, tq, tk, tv, r, cq, ck, cv, i, half, cs + r * half, sn + r * half, q + (size_t)r * d + hh * hd, kdst, vdst, pass_status == 0);
 }
 
 // ---- launchers (callers have checked: bf16 model, result in slots) ----------------------------

@@ -115,9 +115,7 @@ __device__ __forceinline__ void post_swiglu(const FwParams& p, const GemmOut& gu
         const TileRef tg = gu.tiles[c >> 7], tu = gu.tiles[(F + c) >> 7];
         const float4 g = gemm_out_at4(gu, tg, r, c & 127);
         const float4 u = gemm_out_at4(gu, tu, r, (F + c) & 127);
-        *reinterpret_cast<uint2*>(p.act + (size_t)r * F + c) =
-            pack4_bf16(g.x / (1.f + expf(-g.x)) * u.x, g.y / (1.f + expf(-g.y)) * u.y,
-                       g.z / (1.f + expf(-g.z)) * u.z, g.w / (1.f + expf(-g.w)) * u.w);
+        *reinterpret_cast<uint2*>(p.act + (size_t)r * F + c) = swiglu4(g, u);
     }
 }
 
@@ -135,18 +133,7 @@ __device__ __forceinline__ void post_rope_kv(const FwParams& p, const GemmOut& q
         const size_t cp = p.kv_cap[b];
         bf16* kdst = reinterpret_cast<bf16*>(p.kv_base[b]) + ((((size_t)layer * 2 + 0) * H + hh) * cp + slot) * hd;
         bf16* vdst = reinterpret_cast<bf16*>(p.kv_base[b]) + ((((size_t)layer * 2 + 1) * H + hh) * cp + slot) * hd;
-        const float4 q0 = gemm_out_at4(qkv, tq, r, (cq + i) & 127), q1 = gemm_out_at4(qkv, tq, r, (cq + i + half) & 127);
-        const float4 k0 = gemm_out_at4(qkv, tk, r, (ck + i) & 127), k1 = gemm_out_at4(qkv, tk, r, (ck + i + half) & 127);
-        const float4 v0 = gemm_out_at4(qkv, tv, r, (cv + i) & 127), v1 = gemm_out_at4(qkv, tv, r, (cv + i + half) & 127);
-        const float4 c = *reinterpret_cast<const float4*>(p.rope_cos + r * half + i);
-        const float4 s = *reinterpret_cast<const float4*>(p.rope_sin + r * half + i);
-        bf16* qd = p.q + (size_t)r * d + hh * hd;
-        *reinterpret_cast<uint2*>(qd + i) = pack4_bf16(q0.x * c.x - q1.x * s.x, q0.y * c.y - q1.y * s.y, q0.z * c.z - q1.z * s.z, q0.w * c.w - q1.w * s.w);
-        *reinterpret_cast<uint2*>(qd + i + half) = pack4_bf16(q1.x * c.x + q0.x * s.x, q1.y * c.y + q0.y * s.y, q1.z * c.z + q0.z * s.z, q1.w * c.w + q0.w * s.w);
-        *reinterpret_cast<uint2*>(kdst + i) = pack4_bf16(k0.x * c.x - k1.x * s.x, k0.y * c.y - k1.y * s.y, k0.z * c.z - k1.z * s.z, k0.w * c.w - k1.w * s.w);
-        *reinterpret_cast<uint2*>(kdst + i + half) = pack4_bf16(k1.x * c.x + k0.x * s.x, k1.y * c.y + k0.y * s.y, k1.z * c.z + k0.z * s.z, k1.w * c.w + k0.w * s.w);
-        *reinterpret_cast<uint2*>(vdst + i) = pack4_bf16(v0.x, v0.y, v0.z, v0.w);
-        *reinterpret_cast<uint2*>(vdst + i + half) = pack4_bf16(v1.x, v1.y, v1.z, v1.w);
+        rope_kv_item(qkv, tq, tk, tv, r, cq, ck, cv, i, half, p.rope_cos + r * half, p.rope_sin + r * half, p.q + (size_t)r * d + hh * hd, kdst, vdst, true);
     }
 }
 

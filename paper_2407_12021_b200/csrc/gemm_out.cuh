@@ -122,6 +122,32 @@ __device__ __forceinline__ float4 unpack4_bf16(uint2 u) {
     return make_float4(__low2float(lo), __high2float(lo), __low2float(hi), __high2float(hi));
 }
 
+
+// act = round(silu(gate) * up) for four adjacent columns.
+__device__ __forceinline__ uint2 swiglu4(float4 g, float4 u) {
+    return pack4_bf16(g.x / (1.f + expf(-g.x)) * u.x, g.y / (1.f + expf(-g.y)) * u.y,
+                      g.z / (1.f + expf(-g.z)) * u.z, g.w / (1.f + expf(-g.w)) * u.w);
+}
+
+// Rotary embedding of four adjacent pairs (i .. i+3 with i+half .. i+half+3) of one head's q and k of
+// row r, and the copy of v: gathers the QKV projection's partial tiles, rotates with the row's
+// cos/sin, rounds to bf16 and (when `store`) writes q to qd and K/V to the cache rows kdst / vdst.
+__device__ __forceinline__ void rope_kv_item(const GemmOut& qkv, const TileRef& tq, const TileRef& tk, const TileRef& tv, int r,
+                                             int cq, int ck, int cv, int i, int half, const float* __restrict__ cs_row,
+                                             const float* __restrict__ sn_row, __nv_bfloat16* qd, __nv_bfloat16* kdst,
+                                             __nv_bfloat16* vdst, bool store) {
+    const float4 q0 = gemm_out_at4(qkv, tq, r, (cq + i) & 127), q1 = gemm_out_at4(qkv, tq, r, (cq + i + half) & 127);
+    const float4 k0 = gemm_out_at4(qkv, tk, r, (ck + i) & 127), k1 = gemm_out_at4(qkv, tk, r, (ck + i + half) & 127);
+    const float4 v0 = gemm_out_at4(qkv, tv, r, (cv + i) & 127), v1 = gemm_out_at4(qkv, tv, r, (cv + i + half) & 127);
+    const float4 c = *reinterpret_cast<const float4*>(cs_row + i), s = *reinterpret_cast<const float4*>(sn_row + i);
+    if (!store) return;
+    *reinterpret_cast<uint2*>(qd + i) = pack4_bf16(q0.x * c.x - q1.x * s.x, q0.y * c.y - q1.y * s.y, q0.z * c.z - q1.z * s.z, q0.w * c.w - q1.w * s.w);
+    *reinterpret_cast<uint2*>(qd + i + half) = pack4_bf16(q1.x * c.x + q0.x * s.x, q1.y * c.y + q0.y * s.y, q1.z * c.z + q0.z * s.z, q1.w * c.w + q0.w * s.w);
+    *reinterpret_cast<uint2*>(kdst + i) = pack4_bf16(k0.x * c.x - k1.x * s.x, k0.y * c.y - k1.y * s.y, k0.z * c.z - k1.z * s.z, k0.w * c.w - k1.w * s.w);
+    *reinterpret_cast<uint2*>(kdst + i + half) = pack4_bf16(k1.x * c.x + k0.x * s.x, k1.y * c.y + k0.y * s.y, k1.z * c.z + k0.z * s.z, k1.w * c.w + k0.w * s.w);
+    *reinterpret_cast<uint2*>(vdst + i) = pack4_bf16(v0.x, v0.y, v0.z, v0.w);
+    *reinterpret_cast<uint2*>(vdst + i + half) = pack4_bf16(v1.x, v1.y, v1.z, v1.w);
+}
 #endif
 
 }  // namespace aded
