@@ -105,6 +105,7 @@ struct aded_kv {
     char** base_dev;              // [B] device array of the same pointers
     int32_t* cap_dev;             // [B]
     int32_t* len_dev;             // [B] committed lengths
+    CUtensorMap* maps_dev;        // [B] TMA descriptors of the blocks (tensor-core attention), or NULL
 };
 
 struct aded_model {
@@ -147,6 +148,8 @@ struct aded_model {
     void* dbg_hidden;   // [n_layers + 1][rows][d] copies of the residual stream (debug capture)
 
     bool att_mma;       // bf16 models: tensor-core split-KV attention kernel
+    bool att_tc;        // bf16 models with head_dim 128: the tcgen05 attention kernel (tree_attention_tc.cu)
+    CUtensorMap att_q_map;   // TMA descriptor of q for it
 
     // tensor-core GEMM path (bf16 models): TMA descriptors and split-tile scratch
     bool ws_ready;
@@ -236,6 +239,12 @@ cudaError_t fw_launch(aded_model* m, aded_kv* kv, const FwPair* pairs, int n_pai
 bool sample_supported(int vocab);
 cudaError_t launch_sample_rows(const float* logits, int rows, int vocab, int ld, float temperature, float top_p, const float* u,
                                int32_t* out, const int32_t* status, cudaStream_t st);
+
+// tree_attention_tc.cu
+bool attn_tc_supported(const aded_model_config& c);
+bool attn_tc_prepare();
+bool attn_tc_make_kv_map(CUtensorMap* map, const void* block, uint64_t capacity, uint64_t planes);
+void launch_tree_attention_tc(aded_model* m, aded_kv* kv, int layer, int batch, int max_tree, cudaStream_t st);
 
 // tree_attention.cu
 // max_tree: most nodes any sequence's tree has in this call

@@ -109,6 +109,9 @@ static aded_status alloc_model(aded_model* m) {
     ADED_CUDA_TRY(cudaMemset(m->act, 0, R * F * m->elem));
 
     m->att_mma = c.dtype == ADED_BF16 && !getenv("ADED_PLAIN_ATTN") && attn_prepare();
+    // head_dim 128: the tcgen05 kernel (opt-in while it is being measured against the mma.sync kernel)
+    m->att_tc = m->att_mma && attn_tc_supported(c) && getenv("ADED_ATTN_TC") && attn_tc_prepare() &&
+                ws_make_map(&m->att_q_map, m->q, R, d, 64);
 
     // tensor-core GEMM path: bf16 models whose every matrix tiles into 128-row x 64-column blocks
     m->ws_ready = false;
@@ -489,6 +492,7 @@ aded_status aded_kv_create(const aded_model* m, int32_t batch, const int32_t* ca
     kv->base_dev = nullptr;
     kv->cap_dev = nullptr;
     kv->len_dev = nullptr;
+    kv->maps_dev = nullptr;
     const aded_model_config& c = m->cfg;
     aded_status s = ADED_OK;
     for (int b = 0; b < batch && s == ADED_OK; ++b) {
@@ -501,6 +505,17 @@ aded_status aded_kv_create(const aded_model* m, int32_t batch, const int32_t* ca
             break;
         }
         kv->base.push_back(static_cast<char*>(p));
+        // Zero-filled: rows past the last key are read (with probability exactly zero) by the attention
+        // kernel's last key block and must hold finite values.
+        if (cudaMemset(p, 0, bytes) != cudaSuccess) s = ADED_ERR_CUDA;
+    }
+    if (s == ADED_OK && m->att_tc) {
+        std::vector<CUtensorMap> maps(batch);
+        for (int b = 0; b < batch && s == ADED_OK; ++b)
+            if (!aded::attn_tc_make_kv_map(&maps[b], kv->base[b], (uint64_t)kv->cap[b], (uint64_t)c.n_layers * 2 * c.n_heads)) s = ADED_ERR_CUDA;
+        if (s == ADED_OK && (cudaMalloc((void**)&kv->maps_dev, batch * sizeof(CUtensorMap)) != cudaSuccess ||
+                             cudaMemcpy(kv->maps_dev, maps.data(), batch * sizeof(CUtensorMap), cudaMemcpyHostToDevice) != cudaSuccess))
+            s = ADED_ERR_CUDA;
     }
     if (s == ADED_OK && (cudaMalloc((void**)&kv->base_dev, batch * sizeof(char*)) != cudaSuccess ||
                          cudaMalloc((void**)&kv->cap_dev, batch * sizeof(int32_t)) != cudaSuccess ||
@@ -525,6 +540,7 @@ aded_status aded_kv_destroy(aded_kv* kv) {
     if (kv->base_dev) cudaFree(kv->base_dev);
     if (kv->cap_dev) cudaFree(kv->cap_dev);
     if (kv->len_dev) cudaFree(kv->len_dev);
+    if (kv->maps_dev) cudaFree(kv->maps_dev);
     delete kv;
     return ADED_OK;
 }

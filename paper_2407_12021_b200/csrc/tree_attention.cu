@@ -514,6 +514,10 @@ bool attn_prepare() {
 
 void launch_tree_attention(aded_model* m, aded_kv* kv, int layer, int batch, int rows, int max_tree, cudaStream_t st) {
     const int H = m->cfg.n_heads, hd = m->cfg.head_dim;
+    if (m->att_tc && kv->maps_dev) {
+        launch_tree_attention_tc(m, kv, layer, batch, max_tree, st);
+        return;
+    }
     if (m->cfg.dtype == ADED_BF16 && m->att_mma) {
         if (hd == 128) launch_mma<128>(m, kv, layer, batch, rows, max_tree, st);
         else launch_mma<64>(m, kv, layer, batch, rows, max_tree, st);
