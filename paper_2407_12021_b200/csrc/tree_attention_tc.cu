@@ -39,6 +39,7 @@ constexpr int AT_STAGES = 2;      // K and V blocks in flight
 constexpr int AT_THREADS = 192;
 constexpr int AT_TMEM_COLS = 128; // S: 2 x 32, O: 64
 constexpr uint32_t AT_S_COL = 0, AT_O_COL = 64;
+constexpr float AT_SLACK = 8.f;   // how far a row's maximum may exceed its reference (log2 domain) before O is rescaled
 constexpr uint32_t AT_SUB = 64 * 128;            // bytes of a 64-row x 128-byte sub-tile
 // shared-memory map (from a 1024-byte aligned base)
 constexpr uint32_t AT_OFF_Q = 0;                                   // 2 sub-tiles (head_dim halves)
@@ -66,6 +67,30 @@ __device__ __forceinline__ void tma_load_3d(const CUtensorMap* map, uint64_t* ba
     asm volatile(
         "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
         ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2) : "memory");
+}
+
+__device__ __forceinline__ void tma_prefetch_3d(const CUtensorMap* map, int c0, int c1, int c2) {
+    asm volatile("cp.async.bulk.prefetch.tensor.3d.L2.global.tile [%0, {%1, %2, %3}];" ::"l"(map), "r"(c0), "r"(c1), "r"(c2) : "memory");
+}
+
+// tcgen05.mma / commit issued by one elected lane of a converged warp.  The whole warp runs the issuing
+// code, so addresses and descriptors stay warp-uniform; measured on B200, an instruction issued from a
+// single-lane branch costs the issuing thread about 150 cycles, an elected one 27 to 64 (the tensor
+// core's own time for these shapes).  The same lane is elected every time, as commit requires.
+__device__ __forceinline__ void tc_mma_bf16_elect(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t"
+        "elect.sync _|q, 0xffffffff;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void tc_commit_elect(uint64_t* bar) {
+    asm volatile(
+        "{\n\t.reg .pred q;\n\t"
+        "elect.sync _|q, 0xffffffff;\n\t"
+        "@q tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n\t}"
+        ::"r"(smem_u32(bar)) : "memory");
 }
 
 // 32 consecutive fp32 columns of this warp's 32 TMEM lanes.
@@ -146,6 +171,7 @@ k_tree_attn_tc(const __grid_constant__ CUtensorMap map_q, AttnTcArgs a) {
     uint64_t* p_empty = bars + 15;
     uint32_t* s_tmem = (uint32_t*)(bars + 17);
     volatile int* s_flag = (volatile int*)(s_tmem + 2);     // [0] abort
+    volatile int* s_off = s_flag + 2;                       // [stage] 1: the stage's full barriers are one phase ahead
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (threadIdx.x == 0) {
@@ -157,6 +183,8 @@ k_tree_attn_tc(const __grid_constant__ CUtensorMap map_q, AttnTcArgs a) {
             mbar_init(&p_full[i], 4); mbar_init(&p_empty[i], 1);
         }
         s_flag[0] = 0;
+        s_off[0] = 0;
+        s_off[1] = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
@@ -171,6 +199,46 @@ k_tree_attn_tc(const __grid_constant__ CUtensorMap map_q, AttnTcArgs a) {
     // Only now may the next kernel's blocks appear: every block of this kernel holds its tensor memory,
     // so a later kernel's allocation can make none of them wait.
     pdl_launch_dependents();
+    // While the previous kernel (which writes q and the tree's own K/V rows) is still running, the
+    // producer already fetches this CTA's first two key blocks into their stages, if they lie entirely in
+    // the committed part of the cache (which no kernel of the pass writes), and asks L2 for the others.
+    // The committed length and the tree size are read on trust here; both are read again after the wait
+    // and the early blocks are used only if the two reads agree, otherwise they are fetched again.
+    int n_pre = 0, pre_L = -1, pre_T = -1;
+    if (warp == 0 && lane == 0) {
+        const int pb = blockIdx.z / a.row_blocks;
+        const CUtensorMap* kvm = a.kv_maps + pb;
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&map_q) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(kvm) : "memory");
+        pre_L = __ldcg(a.len + pb);
+        pre_T = __ldcg(a.row_off + pb + 1) - __ldcg(a.row_off + pb);
+        if (pre_L >= 0 && pre_T >= 1 && pre_T <= ADED_MAX_NODES && pre_L < (1 << 28)) {
+            const int pnb = (pre_L + pre_T + AT_BLK - 1) / AT_BLK;
+            const int b0 = (int)((long long)blockIdx.y * pnb / a.n_splits);
+            int b1 = (int)((long long)(blockIdx.y + 1) * pnb / a.n_splits);
+            if (b1 > b0 + 32) b1 = b0 + 32;
+            const int plane_k = (a.layer * 2 + 0) * a.H + blockIdx.x, plane_v = (a.layer * 2 + 1) * a.H + blockIdx.x;
+            for (int blk = b0; blk < b1; ++blk) {
+                const int j = blk - b0, key0 = blk * AT_BLK;
+                if (j < AT_STAGES && n_pre == j && key0 + AT_BLK <= pre_L) {
+                    uint8_t* dk = base + AT_OFF_K + (uint32_t)j * 2 * AT_SUB;
+                    uint8_t* dv = base + AT_OFF_V + (uint32_t)j * 2 * AT_SUB;
+                    mbar_expect_tx(&k_full[j], 2 * AT_SUB);
+                    tma_load_3d(kvm, &k_full[j], dk, 0, key0, plane_k);
+                    tma_load_3d(kvm, &k_full[j], dk + AT_SUB, 64, key0, plane_k);
+                    mbar_expect_tx(&v_full[j], 2 * AT_SUB);
+                    tma_load_3d(kvm, &v_full[j], dv, 0, key0, plane_v);
+                    tma_load_3d(kvm, &v_full[j], dv + AT_SUB, 64, key0, plane_v);
+                    ++n_pre;
+                } else {
+                    tma_prefetch_3d(kvm, 0, key0, plane_k);
+                    tma_prefetch_3d(kvm, 64, key0, plane_k);
+                    tma_prefetch_3d(kvm, 0, key0, plane_v);
+                    tma_prefetch_3d(kvm, 64, key0, plane_v);
+                }
+            }
+        }
+    }
     pdl_wait();
     const int pass_status = *a.status;
 
@@ -188,80 +256,117 @@ k_tree_attn_tc(const __grid_constant__ CUtensorMap map_q, AttnTcArgs a) {
 
     if (warp == 0) {
         // ---------------- TMA producer ----------------
-        if (lane == 0 && nblk > 0) {
-            const CUtensorMap* kvm = a.kv_maps + b;
-            asm volatile("prefetch.tensormap [%0];" ::"l"(&map_q) : "memory");
-            asm volatile("prefetch.tensormap [%0];" ::"l"(kvm) : "memory");
-            const int plane_k = (a.layer * 2 + 0) * a.H + hh, plane_v = (a.layer * 2 + 1) * a.H + hh;
-            mbar_expect_tx(q_full, 2 * AT_SUB);
-            tma_load_2d(&map_q, q_full, base + AT_OFF_Q, hh * AT_HD, off + row_base);
-            tma_load_2d(&map_q, q_full, base + AT_OFF_Q + AT_SUB, hh * AT_HD + 64, off + row_base);
-            for (int j = 0; j < nblk; ++j) {
-                const int s = j & 1, u = j >> 1, key0 = (blk0 + j) * AT_BLK;
-                if (j >= 2 && !at_wait(&k_empty[s], (uint32_t)(u - 1) & 1, s_flag)) { s_flag[0] = 1; atomicCAS(a.status, 0, (int)ADED_ERR_TIMEOUT); break; }
-                uint8_t* dk = base + AT_OFF_K + (uint32_t)s * 2 * AT_SUB;
-                mbar_expect_tx(&k_full[s], 2 * AT_SUB);
-                tma_load_3d(kvm, &k_full[s], dk, 0, key0, plane_k);
-                tma_load_3d(kvm, &k_full[s], dk + AT_SUB, 64, key0, plane_k);
-                if (j >= 2 && !at_wait(&v_empty[s], (uint32_t)(u - 1) & 1, s_flag)) { s_flag[0] = 1; atomicCAS(a.status, 0, (int)ADED_ERR_TIMEOUT); break; }
-                uint8_t* dv = base + AT_OFF_V + (uint32_t)s * 2 * AT_SUB;
-                mbar_expect_tx(&v_full[s], 2 * AT_SUB);
-                tma_load_3d(kvm, &v_full[s], dv, 0, key0, plane_v);
-                tma_load_3d(kvm, &v_full[s], dv + AT_SUB, 64, key0, plane_v);
+        if (lane == 0) {
+            bool ok = true;
+            if (n_pre > 0 && (L != pre_L || T != pre_T || nblk < n_pre)) {
+                // The early reads were stale (or the pass has failed): let the early copies land; the stages
+                // are then filled again, in the next phase of their barriers (s_off tells the consumers).
+                for (int j = 0; j < n_pre; ++j) {
+                    ok = ok && at_wait(&k_full[j], 0, s_flag) && at_wait(&v_full[j], 0, s_flag);
+                    s_off[j] = 1;
+                }
+                n_pre = 0;
             }
+            if (ok && nblk > 0) {
+                const CUtensorMap* kvm = a.kv_maps + b;
+                const int plane_k = (a.layer * 2 + 0) * a.H + hh, plane_v = (a.layer * 2 + 1) * a.H + hh;
+                mbar_expect_tx(q_full, 2 * AT_SUB);      // (its release also publishes s_off)
+                tma_load_2d(&map_q, q_full, base + AT_OFF_Q, hh * AT_HD, off + row_base);
+                tma_load_2d(&map_q, q_full, base + AT_OFF_Q + AT_SUB, hh * AT_HD + 64, off + row_base);
+                // K stage j & 1 is free once the scores of block j - 2 are done, V stage once its P V is.
+                auto load_k = [&](int j) -> bool {
+                    if (j >= 2 && !at_wait(&k_empty[j & 1], (uint32_t)((j >> 1) - 1) & 1, s_flag)) return false;
+                    uint8_t* dk = base + AT_OFF_K + (uint32_t)(j & 1) * 2 * AT_SUB;
+                    const int key0 = (blk0 + j) * AT_BLK;
+                    mbar_expect_tx(&k_full[j & 1], 2 * AT_SUB);
+                    tma_load_3d(kvm, &k_full[j & 1], dk, 0, key0, plane_k);
+                    tma_load_3d(kvm, &k_full[j & 1], dk + AT_SUB, 64, key0, plane_k);
+                    return true;
+                };
+                auto load_v = [&](int j) -> bool {
+                    if (j >= 2 && !at_wait(&v_empty[j & 1], (uint32_t)((j >> 1) - 1) & 1, s_flag)) return false;
+                    uint8_t* dv = base + AT_OFF_V + (uint32_t)(j & 1) * 2 * AT_SUB;
+                    const int key0 = (blk0 + j) * AT_BLK;
+                    mbar_expect_tx(&v_full[j & 1], 2 * AT_SUB);
+                    tma_load_3d(kvm, &v_full[j & 1], dv, 0, key0, plane_v);
+                    tma_load_3d(kvm, &v_full[j & 1], dv + AT_SUB, 64, key0, plane_v);
+                    return true;
+                };
+                // Requests follow the order in which the tensor core hands stages back
+                // (S0 S1 PV0 S2 PV1 S3 ...): K0 V0 K1 V1 K2 K3 V2 K4 V3 K5 ...
+                for (int j = n_pre; ok && j < 2 && j < nblk; ++j) ok = load_k(j) && load_v(j);
+                for (int j = 2; ok && j < 4 && j < nblk; ++j) ok = load_k(j);
+                for (int j = 2; ok && j < nblk; ++j) {
+                    ok = load_v(j);
+                    if (ok && j + 2 < nblk) ok = load_k(j + 2);
+                }
+            }
+            if (!ok) { s_flag[0] = 1; atomicCAS(a.status, 0, (int)ADED_ERR_TIMEOUT); }
         }
     } else if (warp == 1) {
-        // ---------------- MMA issuer ----------------
-        if (lane == 0 && nblk > 0) {
+        // ---------------- MMA issuer (the whole warp runs this; one elected lane issues) ----------------
+        if (nblk > 0) {
             // fp32 accumulate, bf16 operands; S: M 64 x N 32, both operands K-major; O: M 64 x N 64, B MN-major
             const uint32_t idesc_s = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(32 >> 3) << 17) | ((uint32_t)(64 >> 4) << 24);
             const uint32_t idesc_o = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((uint32_t)(64 >> 3) << 17) | ((uint32_t)(64 >> 4) << 24);
-            const uint32_t q_addr = smem_u32(base + AT_OFF_Q), k_addr = smem_u32(base + AT_OFF_K), v_addr = smem_u32(base + AT_OFF_V),
-                           p_addr = smem_u32(base + AT_OFF_P);
+            const uint64_t q_desc = smem_desc_sw128(smem_u32(base + AT_OFF_Q)), k_desc = smem_desc_sw128(smem_u32(base + AT_OFF_K));
+            const uint64_t p_desc = smem_desc_sw128(smem_u32(base + AT_OFF_P)), v_desc = smem_desc_mn_sw128(smem_u32(base + AT_OFF_V), AT_SUB);
             bool ok = at_wait(q_full, 0, s_flag);
-            // scores of block j: key half kh goes to lanes 16 * kh .. 16 * kh + 15 of every lane quarter
+            __syncwarp();
+            const uint32_t off0 = (uint32_t)s_off[0], off1 = (uint32_t)s_off[1];    // published by the producer before q
+            // Scores of block j: key half kh goes to lanes 16 * kh .. 16 * kh + 15 of every lane quarter.  The
+            // two halves accumulate into different lanes and alternate, so that consecutive instructions do
+            // not depend on each other.  (Descriptor addresses are in 16-byte units.)
             auto issue_s = [&](int j) -> bool {
                 const int s = j & 1;
-                if (!at_wait(&k_full[s], (uint32_t)(j >> 1) & 1, s_flag)) return false;
-                if (j >= 2 && !at_wait(&s_empty[s], (uint32_t)((j >> 1) - 1) & 1, s_flag)) return false;
+                bool w = at_wait(&k_full[s], ((uint32_t)(j >> 1) + (s ? off1 : off0)) & 1, s_flag);
+                if (j >= 2) w = w && at_wait(&s_empty[s], (uint32_t)((j >> 1) - 1) & 1, s_flag);
+                if (!__all_sync(0xffffffffu, w)) return false;
                 tc_fence_after();
+                const uint64_t kd = k_desc + (uint64_t)((uint32_t)s * 2 * AT_SUB >> 4);
 #pragma unroll
-                for (int kh = 0; kh < 2; ++kh) {
-                    const uint32_t d = tmem_base + ((uint32_t)(kh * 16) << 16) + AT_S_COL + (uint32_t)s * 32;
+                for (int h = 0; h < 2; ++h) {
 #pragma unroll
-                    for (int h = 0; h < 2; ++h) {
+                    for (int kk = 0; kk < 4; ++kk) {
 #pragma unroll
-                        for (int kk = 0; kk < 4; ++kk) {
-                            const uint64_t da = smem_desc_sw128(q_addr + (uint32_t)h * AT_SUB + (uint32_t)kk * 32);
-                            const uint64_t db = smem_desc_sw128(k_addr + (uint32_t)(s * 2 + h) * AT_SUB + (uint32_t)kh * 4096 + (uint32_t)kk * 32);
-                            tc_mma_bf16(d, da, db, idesc_s, (h | kk) ? 1u : 0u);
+                        for (int kh = 0; kh < 2; ++kh) {
+                            const uint32_t d = tmem_base + ((uint32_t)(kh * 16) << 16) + AT_S_COL + (uint32_t)s * 32;
+                            tc_mma_bf16_elect(d, q_desc + (uint64_t)((h * AT_SUB + kk * 32) >> 4),
+                                              kd + (uint64_t)((h * AT_SUB + kh * 4096 + kk * 32) >> 4), idesc_s, (h | kk) ? 1u : 0u);
                         }
                     }
                 }
-                tc_commit(&k_empty[s]);
-                tc_commit(&s_full[s]);
+                tc_commit_elect(&k_empty[s]);
+                tc_commit_elect(&s_full[s]);
                 return true;
             };
-            ok = ok && issue_s(0);
-            for (int j = 0; ok && j < nblk; ++j) {
+            auto issue_pv = [&](int j) -> bool {
                 const int s = j & 1;
-                if (j + 1 < nblk && !issue_s(j + 1)) { ok = false; break; }
-                if (!at_wait(&p_full[s], (uint32_t)(j >> 1) & 1, s_flag) || !at_wait(&v_full[s], (uint32_t)(j >> 1) & 1, s_flag)) { ok = false; break; }
+                const bool w = at_wait(&p_full[s], (uint32_t)(j >> 1) & 1, s_flag) &&
+                               at_wait(&v_full[s], ((uint32_t)(j >> 1) + (s ? off1 : off0)) & 1, s_flag);
+                if (!__all_sync(0xffffffffu, w)) return false;
                 tc_fence_after();
+                const uint64_t pd = p_desc + (uint64_t)((uint32_t)s * AT_SUB >> 4), vd = v_desc + (uint64_t)((uint32_t)s * 2 * AT_SUB >> 4);
 #pragma unroll
-                for (int h = 0; h < 2; ++h) {
-                    const uint32_t d = tmem_base + ((uint32_t)(h * 16) << 16) + AT_O_COL;
+                for (int kk = 0; kk < 4; ++kk) {
 #pragma unroll
-                    for (int kk = 0; kk < 4; ++kk) {
-                        const uint64_t da = smem_desc_sw128(p_addr + (uint32_t)s * AT_SUB + (uint32_t)kk * 32);
-                        const uint64_t db = smem_desc_mn_sw128(v_addr + (uint32_t)(s * 2 + h) * AT_SUB + (uint32_t)kk * 2048, AT_SUB);
-                        tc_mma_bf16(d, da, db, idesc_o, (j | kk) ? 1u : 0u);
+                    for (int h = 0; h < 2; ++h) {
+                        const uint32_t d = tmem_base + ((uint32_t)(h * 16) << 16) + AT_O_COL;
+                        tc_mma_bf16_elect(d, pd + (uint64_t)((kk * 32) >> 4), vd + (uint64_t)((h * AT_SUB + kk * 2048) >> 4), idesc_o, (j | kk) ? 1u : 0u);
                     }
                 }
-                tc_commit(&v_empty[s]);
-                tc_commit(&p_empty[s]);
+                tc_commit_elect(&v_empty[s]);
+                tc_commit_elect(&p_empty[s]);
+                return true;
+            };
+            // Scores run two blocks ahead of the softmax (two S buffers), so a K stage is handed back early.
+            ok = __all_sync(0xffffffffu, ok) && issue_s(0);
+            if (ok && nblk > 1) ok = issue_s(1);
+            for (int j = 0; ok && j < nblk; ++j) {
+                ok = issue_pv(j);
+                if (ok && j + 2 < nblk) ok = issue_s(j + 2);
             }
-            if (!ok) { s_flag[0] = 1; atomicCAS(a.status, 0, (int)ADED_ERR_TIMEOUT); }
+            if (!ok && lane == 0) { s_flag[0] = 1; atomicCAS(a.status, 0, (int)ADED_ERR_TIMEOUT); }
         }
     } else {
         // ---------------- softmax: warps 2..5, TMEM lane quarter = warp % 4 ----------------
@@ -293,12 +398,17 @@ k_tree_attn_tc(const __grid_constant__ CUtensorMap map_q, AttnTcArgs a) {
                     if (!keep) sr[c] = 0xff800000u;     // -inf
                 }
             }
-            float bm = -INFINITY;
+            float bm4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-            for (int c = 0; c < 32; ++c) bm = fmaxf(bm, __uint_as_float(sr[c]));
+            for (int c = 0; c < 32; ++c) bm4[c & 3] = fmaxf(bm4[c & 3], __uint_as_float(sr[c]));
+            float bm = fmaxf(fmaxf(bm4[0], bm4[1]), fmaxf(bm4[2], bm4[3]));
             bm = fmaxf(bm, __shfl_xor_sync(0xffffffffu, bm, 16));
-            // integer reference (scores in the log2 domain), as in k_tree_attn_mma
-            const float nm = fmaxf(mrow, ceilf(bm * a.scale_log2));
+            // Integer reference (scores in the log2 domain), as in k_tree_attn_mma, but kept while a new
+            // maximum exceeds it by at most AT_SLACK: numerators then reach 2^AT_SLACK instead of 1, which
+            // changes nothing (scaling by a power of two commutes with the bf16 rounding and with the fp32
+            // sums), and the costly rescaling of O in tensor memory becomes rare.
+            const float cand = ceilf(bm * a.scale_log2);
+            const float nm = mrow == -INFINITY ? cand : (cand > mrow + AT_SLACK ? cand : mrow);
             const float use = nm == -INFINITY ? 0.f : nm;
             const bool moved = mrow != nm && mrow != -INFINITY;
             if (__any_sync(0xffffffffu, moved)) {
@@ -319,16 +429,16 @@ k_tree_attn_tc(const __grid_constant__ CUtensorMap map_q, AttnTcArgs a) {
                 lsum *= corr;
             }
             mrow = nm;
-            float ps = 0.f;
+            float ps4[4] = {0.f, 0.f, 0.f, 0.f};
             uint32_t pk[16];
 #pragma unroll
             for (int c = 0; c < 32; c += 2) {
                 const float e0 = at_ex2(fmaf(__uint_as_float(sr[c]), a.scale_log2, -use));
                 const float e1 = at_ex2(fmaf(__uint_as_float(sr[c + 1]), a.scale_log2, -use));
-                ps += e0 + e1;
+                ps4[(c >> 1) & 3] += e0 + e1;
                 pk[c >> 1] = at_pack(e0, e1);
             }
-            lsum += ps;
+            lsum += (ps4[0] + ps4[1]) + (ps4[2] + ps4[3]);
             if (j >= 2 && !__all_sync(0xffffffffu, at_wait(&p_empty[s], (uint32_t)((j >> 1) - 1) & 1, s_flag))) { ok = false; break; }
             uint8_t* prow = base + AT_OFF_P + (uint32_t)s * AT_SUB + (uint32_t)row * 128;
 #pragma unroll
