@@ -125,39 +125,45 @@ k_gemm_ws(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUt
         }
     } else if (warp == 1) {
         // ---------------- MMA issuer ----------------
-        if (lane == 0 && live) {
+        // The whole warp runs the loop and one elected lane issues: operands then stay warp-uniform.  An
+        // instruction issued from a single-lane branch costs the issuing thread about 150 cycles on B200, an
+        // elected one 30 to 60, and that time sits between a stage's arrival and its release.
+        if (live) {
             const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(p.rb >> 3) << 17) | ((uint32_t)(WS_BM >> 4) << 24);
+            const uint64_t desc0 = smem_desc_sw128(smem_u32(base));
             int s = 0;
             uint32_t ph = 0;
             int seg = 0;
             long long u = u0;
-            while (u < u1 && !s_flag[0]) {
+            bool ok = true;
+            // (every exit from these loops is taken by the whole warp: the elected issue needs all 32 lanes)
+            while (ok && u < u1 && !__any_sync(0xffffffffu, s_flag[0] != 0)) {
                 const int kb0 = (int)(u % p.kb);
                 long long ue = u + (p.kb - kb0);
                 if (ue > u1) ue = u1;
                 const int a = seg & 1;
                 const uint32_t aph = (uint32_t)(seg >> 1) & 1;
-                if (!mbar_wait(&acc_empty[a], aph ^ 1)) { s_flag[0] = 1; atomicCAS(p.status, 0, (int)ADED_ERR_TIMEOUT); break; }
+                if (!__all_sync(0xffffffffu, mbar_wait(&acc_empty[a], aph ^ 1))) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(a * p.rb);
                 bool first = true;
                 for (; u < ue; ++u) {
-                    if (!mbar_wait(&full[s], ph)) { s_flag[0] = 1; atomicCAS(p.status, 0, (int)ADED_ERR_TIMEOUT); break; }
+                    if (!__all_sync(0xffffffffu, mbar_wait(&full[s], ph))) { ok = false; break; }
                     tc_fence_after();
-                    const uint32_t sa = smem_u32(base + (size_t)s * stage_bytes);
-                    const uint64_t da = smem_desc_sw128(sa), db = smem_desc_sw128(sa + a_bytes);
+                    const uint64_t da = desc0 + (uint64_t)(((uint32_t)s * stage_bytes) >> 4), db = da + (uint64_t)(a_bytes >> 4);
 #pragma unroll
                     for (int kk = 0; kk < WS_BK / 16; ++kk) {
-                        tc_mma_bf16(d_tmem, da + (uint64_t)(kk * 2), db + (uint64_t)(kk * 2), idesc, first && kk == 0 ? 0u : 1u);
+                        tc_mma_bf16_elect(d_tmem, da + (uint64_t)(kk * 2), db + (uint64_t)(kk * 2), idesc, first && kk == 0 ? 0u : 1u);
                     }
                     first = false;
-                    tc_commit(&empty[s]);      // stage reusable once these MMAs have read it
+                    tc_commit_elect(&empty[s]);      // stage reusable once these MMAs have read it
                     if (++s == p.stages) { s = 0; ph ^= 1; }
                 }
-                if (s_flag[0]) break;
-                tc_commit(&acc_full[a]);       // accumulator complete
+                if (!ok) break;
+                tc_commit_elect(&acc_full[a]);       // accumulator complete
                 ++seg;
             }
+            if (!ok && lane == 0) { s_flag[0] = 1; atomicCAS(p.status, 0, (int)ADED_ERR_TIMEOUT); }
         }
     } else {
         // ---------------- epilogue: warps 2..5, TMEM lane quarter = warp % 4 ----------------

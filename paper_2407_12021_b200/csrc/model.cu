@@ -109,8 +109,8 @@ static aded_status alloc_model(aded_model* m) {
     ADED_CUDA_TRY(cudaMemset(m->act, 0, R * F * m->elem));
 
     m->att_mma = c.dtype == ADED_BF16 && !getenv("ADED_PLAIN_ATTN") && attn_prepare();
-    // head_dim 128: the tcgen05 kernel (opt-in while it is being measured against the mma.sync kernel)
-    m->att_tc = m->att_mma && attn_tc_supported(c) && getenv("ADED_ATTN_TC") && attn_tc_prepare() &&
+    // head_dim 128: the tcgen05 kernel (ADED_ATTN_MMA=1 keeps the mma.sync kernel, for comparisons)
+    m->att_tc = m->att_mma && attn_tc_supported(c) && !getenv("ADED_ATTN_MMA") && attn_tc_prepare() &&
                 ws_make_map(&m->att_q_map, m->q, R, d, 64);
 
     // tensor-core GEMM path: bf16 models whose every matrix tiles into 128-row x 64-column blocks
