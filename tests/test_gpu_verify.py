@@ -254,6 +254,39 @@ def test_c2_one_7b_layer_bf16(cuda_device):
     assert cpu2["accept_len"] >= 2
 
 
+@pytest.mark.parametrize("nodes,ctx,depth", [(100, 300, 6), (64, 2047, 6), (5, 1, 2)])
+def test_attention_kernels_agree(cuda_device, monkeypatch, nodes, ctx, depth):
+    """head_dim 128 has two attention kernels: tcgen05 (the default) and mma.sync (ADED_ATTN_MMA set when the
+    model is created).  Same rounding points (integer reference in the log2 domain, numerators rounded to
+    bf16, unrounded row sums); the fp32 sums run in another order, so outputs agree to a few bf16 ulps."""
+    from paper_2407_12021_b200 import binding as B
+    shape = gen.ModelShape("bf16-4x128", 2, 512, 4, 128, 1024, 1024, "bf16")
+    w = H.weights_to(gen.model_weights(shape, 31), cuda_device)
+    tokens, parents = gen.make_tree(nodes, depth, 4, shape.vocab, 32)
+    results = []
+    for mma in (False, True):
+        if mma:
+            monkeypatch.setenv("ADED_ATTN_MMA", "1")
+        else:
+            monkeypatch.delenv("ADED_ATTN_MMA", raising=False)
+        m = B.aded_model_create(shape, w, max_rows=128, max_batch=1)
+        kv = B.aded_kv_create(m, [ctx + 256])
+        for l in range(shape.n_layers):
+            k, v = gen.kv_normal(shape, ctx, 33, l, device=cuda_device)
+            B.aded_kv_load(kv, 0, l, k, v)
+        out = torch.full((nodes,), -7, dtype=torch.int32, device="cuda")
+        alen = torch.full((1,), -7, dtype=torch.int32, device="cuda")
+        B.aded_verify(m, kv, H.i32(tokens), H.i32(parents), out, alen)
+        torch.cuda.synchronize()
+        assert B.aded_model_poll_status(m) == 0
+        results.append((B.aded_debug_read_buffer(m, 3, nodes).float().clone(), B.aded_debug_read_buffer(m, 0, nodes).float().clone()))
+    monkeypatch.delenv("ADED_ATTN_MMA", raising=False)
+    (att0, h0), (att1, h1) = results
+    assert (att0 - att1).abs().max() <= 2e-2 * att0.abs().max()
+    assert (h0 - h1).abs().max() <= 2e-2 * h0.abs().max()
+    assert att0.abs().max() > 0
+
+
 @pytest.mark.parametrize("heads,hd,nodes,depth,ctx", [(4, 64, 128, 8, 100), (2, 128, 37, 5, 191), (2, 128, 128, 8, 70),
                                                      (4, 64, 16, 3, 64), (2, 128, 1, 0, 129)])
 def test_bf16_small_models_tree_shapes(cuda_device, heads, hd, nodes, depth, ctx):
