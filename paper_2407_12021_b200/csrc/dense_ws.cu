@@ -126,8 +126,18 @@ __global__ void __launch_bounds__(256) k_swiglu_ws(GemmOut gu, bf16* __restrict_
     pdl_wait();
     if (c >= F) return;
     const int pass_status = *status;     // checked before the store, not before the loads
-    const float4 g = gemm_out_at4(gu, tg, r, c & 127);
-    const float4 u = gemm_out_at4(gu, tu, r, (F + c) & 127);
+    float4 g, u;
+    constexpr int SB = 4;      // gate/up tiles have two or three contributors at the 7B and 13B widths
+    if (tg.count <= SB && tu.count <= SB) {
+        float4 fg[SB], fu[SB];
+        gemm_out_fetch4<SB>(gu, tg, r, c & 127, fg);
+        gemm_out_fetch4<SB>(gu, tu, r, (F + c) & 127, fu);
+        g = gemm_out_sum4<SB>(fg, tg);
+        u = gemm_out_sum4<SB>(fu, tu);
+    } else {
+        g = gemm_out_at4(gu, tg, r, c & 127);
+        u = gemm_out_at4(gu, tu, r, (F + c) & 127);
+    }
     if (pass_status != 0) return;
     *reinterpret_cast<uint2*>(act + (size_t)r * F + c) = swiglu4(g, u);
 }

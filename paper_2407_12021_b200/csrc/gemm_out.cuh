@@ -110,6 +110,30 @@ __device__ __forceinline__ float4 gemm_out_at4(const GemmOut& o, const TileRef& 
     return sum;
 }
 
+// The same gather in two steps, for kernels that need several tiles' values at once: first the loads of up
+// to B contributors (predicated, no use of the values), then the sum in CTA order.  Issuing the loads of
+// all gathers before the first sum puts them in flight together -- one L2 round trip instead of one per
+// gather.  Only for tiles with at most B contributors: callers check t.count <= B and otherwise use
+// gemm_out_at4.
+template <int B>
+__device__ __forceinline__ void gemm_out_fetch4(const GemmOut& o, const TileRef& t, int r, int col, float4 (&v)[B]) {
+    const int rb = gemm_block_rb(o, r);
+    const size_t region = (size_t)(r >> 7) * (size_t)(o.n_tiles + o.g) * 128 * 128;
+    const float* p = o.slots + region + ((size_t)t.first_slot * rb + (r & 127)) * 128 + col;
+    const size_t stride = (size_t)rb * 128;
+#pragma unroll
+    for (int j = 0; j < B; ++j)
+        v[j] = j < t.count ? __ldcg(reinterpret_cast<const float4*>(p + (size_t)j * stride)) : make_float4(0.f, 0.f, 0.f, 0.f);
+}
+template <int B>
+__device__ __forceinline__ float4 gemm_out_sum4(const float4 (&v)[B], const TileRef& t) {
+    float4 sum = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+    for (int j = 0; j < B; ++j)
+        if (j < t.count) sum = f4_add(sum, v[j]);
+    return sum;
+}
+
 __device__ __forceinline__ uint2 pack4_bf16(float a, float b, float c, float d) {
     const __nv_bfloat162 lo = __floats2bfloat162_rn(a, b), hi = __floats2bfloat162_rn(c, d);
     uint2 u;
@@ -136,9 +160,24 @@ __device__ __forceinline__ void rope_kv_item(const GemmOut& qkv, const TileRef& 
                                              int cq, int ck, int cv, int i, int half, const float* __restrict__ cs_row,
                                              const float* __restrict__ sn_row, __nv_bfloat16* qd, __nv_bfloat16* kdst,
                                              __nv_bfloat16* vdst, bool store) {
-    const float4 q0 = gemm_out_at4(qkv, tq, r, (cq + i) & 127), q1 = gemm_out_at4(qkv, tq, r, (cq + i + half) & 127);
-    const float4 k0 = gemm_out_at4(qkv, tk, r, (ck + i) & 127), k1 = gemm_out_at4(qkv, tk, r, (ck + i + half) & 127);
-    const float4 v0 = gemm_out_at4(qkv, tv, r, (cv + i) & 127), v1 = gemm_out_at4(qkv, tv, r, (cv + i + half) & 127);
+    float4 q0, q1, k0, k1, v0, v1;
+    constexpr int RB = 6;      // the QKV projection's tiles have three to five contributors at the 7B and 13B widths
+    if (tq.count <= RB && tk.count <= RB && tv.count <= RB) {
+        float4 fq0[RB], fq1[RB], fk0[RB], fk1[RB], fv0[RB], fv1[RB];
+        gemm_out_fetch4<RB>(qkv, tq, r, (cq + i) & 127, fq0);
+        gemm_out_fetch4<RB>(qkv, tq, r, (cq + i + half) & 127, fq1);
+        gemm_out_fetch4<RB>(qkv, tk, r, (ck + i) & 127, fk0);
+        gemm_out_fetch4<RB>(qkv, tk, r, (ck + i + half) & 127, fk1);
+        gemm_out_fetch4<RB>(qkv, tv, r, (cv + i) & 127, fv0);
+        gemm_out_fetch4<RB>(qkv, tv, r, (cv + i + half) & 127, fv1);
+        q0 = gemm_out_sum4<RB>(fq0, tq); q1 = gemm_out_sum4<RB>(fq1, tq);
+        k0 = gemm_out_sum4<RB>(fk0, tk); k1 = gemm_out_sum4<RB>(fk1, tk);
+        v0 = gemm_out_sum4<RB>(fv0, tv); v1 = gemm_out_sum4<RB>(fv1, tv);
+    } else {
+        q0 = gemm_out_at4(qkv, tq, r, (cq + i) & 127); q1 = gemm_out_at4(qkv, tq, r, (cq + i + half) & 127);
+        k0 = gemm_out_at4(qkv, tk, r, (ck + i) & 127); k1 = gemm_out_at4(qkv, tk, r, (ck + i + half) & 127);
+        v0 = gemm_out_at4(qkv, tv, r, (cv + i) & 127); v1 = gemm_out_at4(qkv, tv, r, (cv + i + half) & 127);
+    }
     const float4 c = *reinterpret_cast<const float4*>(cs_row + i), s = *reinterpret_cast<const float4*>(sn_row + i);
     if (!store) return;
     *reinterpret_cast<uint2*>(qd + i) = pack4_bf16(q0.x * c.x - q1.x * s.x, q0.y * c.y - q1.y * s.y, q0.z * c.z - q1.z * s.z, q0.w * c.w - q1.w * s.w);
