@@ -142,19 +142,26 @@ __global__ void __launch_bounds__(256) k_swiglu_ws(GemmOut gu, bf16* __restrict_
     *reinterpret_cast<uint2*>(act + (size_t)r * F + c) = swiglu4(g, u);
 }
 
-// Rotary embedding + K/V write (see k_rope_kv): block = (row, head), hd/8 threads, each owning four
-// adjacent rotary pairs (i .. i+3, i+half .. i+half+3).
-__global__ void k_rope_kv_ws(GemmOut qkv, const float* __restrict__ cs, const float* __restrict__ sn,
-                             bf16* __restrict__ q, char* const* __restrict__ base, const int32_t* __restrict__ cap,
-                             const int32_t* __restrict__ len, const int32_t* __restrict__ row_seq,
-                             const int32_t* __restrict__ row_local, int layer, int H, int hd, const int32_t* status) {
+// Rotary embedding + K/V write (see k_rope_kv): hd/8 threads per (row, head), each owning four adjacent
+// rotary pairs (i .. i+3, i+half .. i+half+3); a block of ROPE_WS_THREADS threads takes consecutive heads
+// of one row, so its warps are full and a pass is a few hundred blocks instead of rows x heads tiny ones.
+constexpr int ROPE_WS_THREADS = 128;
+__global__ void __launch_bounds__(ROPE_WS_THREADS)
+k_rope_kv_ws(GemmOut qkv, const float* __restrict__ cs, const float* __restrict__ sn,
+             bf16* __restrict__ q, char* const* __restrict__ base, const int32_t* __restrict__ cap,
+             const int32_t* __restrict__ len, const int32_t* __restrict__ row_seq,
+             const int32_t* __restrict__ row_local, int layer, int H, int hd, const int32_t* status) {
     pdl_launch_dependents();
-    const int r = blockIdx.x, hh = blockIdx.y, half = hd >> 1, d = H * hd;
-    const int i = threadIdx.x * 4;
-    const int cq = hh * hd, ck = d + hh * hd, cv = 2 * d + hh * hd;
+    const int tph = hd >> 3;                                   // threads per head
+    const int r = blockIdx.x, half = hd >> 1, d = H * hd;
+    const int hh = blockIdx.y * (ROPE_WS_THREADS / tph) + threadIdx.x / tph;
+    const int i = (threadIdx.x % tph) * 4;
+    const bool mine = hh < H;
+    const int hc = mine ? hh : 0;
+    const int cq = hc * hd, ck = d + hc * hd, cv = 2 * d + hc * hd;
     const TileRef tq = qkv.tiles[cq >> 7], tk = qkv.tiles[ck >> 7], tv = qkv.tiles[cv >> 7];   // constant table
     pdl_wait();
-    if (i >= half) return;
+    if (!mine) return;
     const int pass_status = *status;     // checked before the stores, not before the loads
     const int b = row_seq[r];
     const size_t slot = (size_t)len[b] + row_local[r];
@@ -187,8 +194,9 @@ void launch_swiglu_ws(aded_model* m, const GemmOut& gu, int rows, cudaStream_t s
 }
 
 void launch_rope_kv_ws(aded_model* m, aded_kv* kv, const GemmOut& qkv, int layer, int rows, cudaStream_t st) {
-    dim3 grid(rows, m->cfg.n_heads);
-    launch_k(k_rope_kv_ws, grid, dim3(32), 0, st, qkv, (const float*)m->rope_cos, (const float*)m->rope_sin, (bf16*)m->q,
+    const int heads_per_block = ROPE_WS_THREADS / (m->cfg.head_dim / 8);
+    dim3 grid(rows, (m->cfg.n_heads + heads_per_block - 1) / heads_per_block);
+    launch_k(k_rope_kv_ws, grid, dim3(ROPE_WS_THREADS), 0, st, qkv, (const float*)m->rope_cos, (const float*)m->rope_sin, (bf16*)m->q,
              (char* const*)kv->base_dev, (const int32_t*)kv->cap_dev, (const int32_t*)kv->len_dev,
              (const int32_t*)m->rows.seq, (const int32_t*)m->rows.local, layer, m->cfg.n_heads, m->cfg.head_dim,
              (const int32_t*)m->status);
