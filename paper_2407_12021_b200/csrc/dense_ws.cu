@@ -23,7 +23,8 @@ __device__ __forceinline__ float warp_sum_f(float v) {
 // The next kernel (a projection) is released right after the wait, not at the top of the kernel.  Measured on
 // a 32-layer step: released at the top (its blocks can then appear while the previous projection is still
 // running) the step is 1.3 % slower; released after the gather or at exit (its weight prefetch no longer
-// runs under this kernel) 4 % slower.  The SwiGLU and rotary kernels below do the same.
+// runs under this kernel) 4 % slower.  The SwiGLU and rotary kernels below do the same (for them the top of
+// the kernel measures the same; the difference comes from this kernel, whose blocks each take a whole SM's registers).
 __global__ void __launch_bounds__(1024) k_add_rmsnorm_ws(bf16* __restrict__ h, GemmOut y, const bf16* __restrict__ gain,
                                                          bf16* __restrict__ x, int d, float eps, const int32_t* status) {
     __shared__ float red[32];
