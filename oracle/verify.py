@@ -202,7 +202,7 @@ def decoder_layer(arch: Arch, p: Dict[str, np.ndarray], cache_k: np.ndarray, cac
     H, hd, d, F = arch.n_heads, arch.head_dim, arch.d_model, arch.d_ffn
     scale = 1.0 / np.sqrt(hd)
     wq, wk, wv = p["wqkv"][:d], p["wqkv"][d:2 * d], p["wqkv"][2 * d:]
-    x = r(rmsnorm(h, p["norm1"], arch.rms_eps))
+    x1 = x = r(rmsnorm(h, p["norm1"], arch.rms_eps))
     q = r(rope((x @ wq.T).reshape(T, H, hd), pos, arch.rope_theta))
     k = r(rope((x @ wk.T).reshape(T, H, hd), pos, arch.rope_theta))
     v = r((x @ wv.T).reshape(T, H, hd))
@@ -214,13 +214,13 @@ def decoder_layer(arch: Arch, p: Dict[str, np.ndarray], cache_k: np.ndarray, cac
         s = np.einsum("hd,hnd->hn", q[i], keys) * scale
         o[i] = np.einsum("hn,hnd->hd", attention_weights(s, arch.bf16), vals)
     o = r(o).reshape(T, d)
-    h = r(h + o @ p["wo"].T)
+    h_mid = h = r(h + o @ p["wo"].T)
     x = r(rmsnorm(h, p["norm2"], arch.rms_eps))
     gate, up = x @ p["wgu"][:F].T, x @ p["wgu"][F:].T
     a = r(silu(gate) * up)
     h = r(h + a @ p["wd"].T)
     if trace is not None:      # intermediates, for stage-by-stage comparisons
-        trace.update(q=q.reshape(T, d), attn=o, act=a, h=h)
+        trace.update(x1=x1, q=q.reshape(T, d), attn=o, h_mid=h_mid, x2=x, act=a, h=h)
     return h, k, v
 
 

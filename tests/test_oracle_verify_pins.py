@@ -335,3 +335,122 @@ def test_bf16_attention_weights_are_softmax_with_rounded_numerators():
     merged = np.concatenate([n * np.exp2(r - top) for n, r in zip(nums, refs)], axis=-1)
     den = sum(d * np.exp2(r - top) for d, r in zip(dens, refs))
     assert np.allclose(merged / den, w, rtol=1e-13, atol=0)
+
+
+# ----------------------------------------------------------------------------- where bf16 models round
+def _on_bf16_grid(a: np.ndarray) -> bool:
+    """Every value survives a round trip through torch's bfloat16 (a library cast, not the checker's)."""
+    t = torch.from_numpy(np.ascontiguousarray(a, dtype=np.float64))
+    return bool(torch.equal(t.to(torch.bfloat16).to(torch.float64), t))
+
+
+class _SkipNthRounding:
+    """Stand-in for the checker's rounding routine that leaves its n-th call (0-based) unrounded:
+    a planted mistake, on the CPU, in the checker."""
+
+    def __init__(self, real, skip):
+        self.real, self.skip, self.calls = real, skip, 0
+
+    def __call__(self, a):
+        i = self.calls
+        self.calls += 1
+        return np.asarray(a, dtype=np.float64) if i == self.skip else self.real(a)
+
+
+def _bf16_layer_case():
+    shape = gen.ModelShape("pin16", 1, 64, 4, 16, 96, 128, "bf16")
+    w = gen.model_weights(shape, 19)
+    p = w["layers"][0]
+    for k in ("wqkv", "wo", "wgu", "wd"):
+        p[k] = (p[k].float() * 6).to(torch.bfloat16)
+    w["lm_head"] = (w["lm_head"].float() * 6).to(torch.bfloat16)
+    arch = ov.arch_from_shape(shape)
+    ow = ov.Weights(w, keep=True)
+    T, L = 6, 5
+    parents = [-1, 0, 0, 1, 1, 3]
+    paths, depth = ov.paths_and_depths(parents)
+    rng = np.random.default_rng(23)
+    as_bf16 = lambda a: torch.from_numpy(a).to(torch.bfloat16).to(torch.float64).numpy()
+    h = as_bf16(rng.normal(size=(T, shape.d_model)))
+    ck = as_bf16(rng.normal(size=(shape.n_heads, L, shape.head_dim)))
+    cv = as_bf16(rng.normal(size=(shape.n_heads, L, shape.head_dim)))
+    return arch, ow, h, ck, cv, paths, L + np.asarray(depth), T
+
+
+def test_every_bf16_rounding_site_of_a_layer_is_needed_and_lands_on_the_grid(monkeypatch):
+    """The rounding contract of bf16 models names nine stores in a decoder layer (first norm, q, k, v,
+    attention output, residual stream after attention, second norm, SwiGLU product, residual stream after
+    the FFN) plus the softmax numerators.  With all of them in place every one of those intermediates
+    is a bfloat16 number (checked with torch's cast).  Leaving any single one unrounded (a) takes exactly
+    that intermediate off the grid and (b) changes the layer's output -- so a checker that dropped a
+    site would fail here."""
+    arch, ow, h, ck, cv, paths, pos, T = _bf16_layer_case()
+    p = ow.layer(0)
+    base = {}
+    h_out, k, v = ov.decoder_layer(arch, p, ck, cv, h, paths, pos, base)
+    base.update(k=k, v=v)
+    stores = ["x1", "q", "k", "v", "attn", "h_mid", "x2", "act", "h"]
+    for name in stores:
+        assert _on_bf16_grid(base[name]), name
+    assert np.array_equal(base["h"], h_out)
+    # call order of the rounding routine inside decoder_layer: x1 q k v, one call per node for the
+    # softmax numerators, then attn h_mid x2 act h
+    real = ov.round_bf16
+    counter = _SkipNthRounding(real, -1)
+    monkeypatch.setattr(ov, "round_bf16", counter)
+    ov.decoder_layer(arch, p, ck, cv, h, paths, pos, {})
+    assert counter.calls == 9 + T
+    site_of_call = {0: "x1", 1: "q", 2: "k", 3: "v", 4 + T: "attn", 5 + T: "h_mid", 6 + T: "x2", 7 + T: "act", 8 + T: "h"}
+    for call, name in site_of_call.items():
+        monkeypatch.setattr(ov, "round_bf16", _SkipNthRounding(real, call))
+        tr = {}
+        h2, k2, v2 = ov.decoder_layer(arch, p, ck, cv, h, paths, pos, tr)
+        tr.update(k=k2, v=v2)
+        assert not _on_bf16_grid(tr[name]), f"skipping call {call} should leave {name} unrounded"
+        for other in stores[:stores.index(name)]:
+            assert np.array_equal(tr[other], base[other]), (name, other)     # nothing upstream moves
+        assert not np.array_equal(h2, h_out), name                         # and the layer's output does
+    # the softmax numerators of one node: the attention output of that node alone moves
+    for node in (0, T - 1):
+        monkeypatch.setattr(ov, "round_bf16", _SkipNthRounding(real, 4 + node))
+        tr = {}
+        ov.decoder_layer(arch, p, ck, cv, h, paths, pos, tr)
+        moved = np.any(tr["attn"] != base["attn"], axis=1)
+        assert moved[node] and not np.any(np.delete(moved, node)), (node, moved)
+
+
+def test_lm_head_rounds_the_normalised_hidden_state_and_nothing_else(monkeypatch):
+    """Logits of a bf16 model = (final RMSNorm output stored as bf16) x head weights, unrounded: equal to the
+    same steps done with torch's own routines (rms_norm, bfloat16 cast, float64 matmul), and different as
+    soon as the one rounding is skipped."""
+    arch, ow, h, *_ = _bf16_layer_case()
+    got = ov.lm_head(arch, ow, h)
+    g = torch.from_numpy(ow.top("final_norm"))
+    x = torch.nn.functional.rms_norm(torch.from_numpy(h), (h.shape[1],), g, arch.rms_eps)
+    want = (x.to(torch.bfloat16).to(torch.float64) @ torch.from_numpy(ow.top("lm_head")).T).numpy()
+    assert np.allclose(got, want, rtol=1e-12, atol=1e-12)
+    assert not _on_bf16_grid(got)
+    real = ov.round_bf16
+    counter = _SkipNthRounding(real, 0)
+    monkeypatch.setattr(ov, "round_bf16", counter)
+    skipped = ov.lm_head(arch, ow, h)
+    assert counter.calls == 1
+    assert np.max(np.abs(skipped - want)) > 1e-6
+
+
+def test_top2_margin_against_a_full_sort():
+    rng = np.random.default_rng(31)
+    logits = rng.normal(size=(40, 257))
+    logits[3, 10] = logits[3, 200] = logits[3].max() + 1.0        # an exact tie at the top: margin 0
+    logits[4] = -np.abs(logits[4])                                # all negative
+    logits[5, :] = 0.25                                           # a constant row
+    s = np.sort(logits, axis=-1)
+    want = s[:, -1] - s[:, -2]
+    got = ov.top2_margin(logits)
+    assert np.array_equal(got, want)
+    assert got[3] == 0.0 and got[5] == 0.0 and np.all(got >= 0)
+    # the margin is what decides an exemption: the greedy token is the largest entry, the runner-up is `margin` below
+    best = ov.greedy(logits)
+    for r in (0, 7, 21):
+        rest = np.delete(logits[r], best[r])
+        assert got[r] == logits[r, best[r]] - rest.max()
