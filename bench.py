@@ -1,6 +1,6 @@
 """Benchmark of the verification step: accepted tokens/s and verify-step latency on one B200.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c3|c2|c4] [--impl ours|reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c3|c2|c4|c5|tg] [--impl ours|reference]
 
 A step is one decode step of the loop: the 64-node draft tree retrieved from the tri-gram table
 with the last two tokens of the text, its verification (all layers, LM head, greedy choice,
@@ -11,6 +11,9 @@ context -- one library call, every stage on the device.  Two passes over the sam
   * device resident: the cache and the table are rolled back and the same steps run through
     `aded_decode_step` from device memory only.  The emitted tokens must equal the first pass's.
 With --gpus N every rank runs an independent replica (nothing in the step is exchanged).
+Two more workloads, not part of the default run: `--workload tg` times the tri-gram store alone (bulk update
+and top-4 queries on 10^6- and 5 x 10^7-token Zipf corpora, the CPU checker's store beside it), `--workload c5`
+the ragged batches of 1, 4 and 16 sequences at the 7B model's full depth.
 """
 from __future__ import annotations
 
@@ -41,7 +44,7 @@ def parse_args():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=256)
     ap.add_argument("--warmup", type=int, default=4)
-    ap.add_argument("--workload", default="c3", choices=["c2", "c3", "c4"])
+    ap.add_argument("--workload", default="c3", choices=["c2", "c3", "c4", "c5", "tg"])
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--layers", type=int, default=0, help="override the layer count (debugging only)")
     ap.add_argument("--context", type=int, default=0, help="override the prompt length (debugging only)")
@@ -211,11 +214,17 @@ def run_ours(args, rank, world):
         return step_ev[0].elapsed_time(step_ev[-1]), per_step, launches, sum(lens[warm:]), prof
 
     sampler.start()
+    B.aded_trace_begin(model)      # one timestamp per kernel, taken by one thread: the timed pass is the traced pass
     dev_ms, per_step, launches, accepted, _ = replay(profile=False)
+    marks = B.aded_trace_end(model)
     clocks = sampler.stop()
+    in_step = stage_times(marks, shape.n_layers)
     assert accepted == accepted_e2e
     final_len = B.aded_kv_len(kv, 0)
     _, _, _, _, (prof_ms, prof_n) = replay(profile=True)
+
+    # ---------------- planted arm: the same decode with a table that knows part of the model's own text ----
+    planted = planted_arm(B, model, kv, fresh_table, ctx, ctx0, base_len, fill_d, wl, shape, steps, warm, dev, world, rank)
 
     # ---------------- roofline of the dominant kernel (the weight-streaming GEMMs) ------------------------
     pk = peaks()
@@ -234,14 +243,295 @@ def run_ours(args, rank, world):
                      "frac": round(achieved / pk["hbm_gbs"], 4), "traffic": gemm_traffic_per_launch(shape),
                      "algorithmic_bytes_per_launch": gemm_bytes_step // gemm_launches_step,
                      "avg_launch_us": round(gemm_ms_launch * 1e3, 2),
-                     "time_share": {k: round(v / max(sum(prof_ms.values()), 1e-9), 4) for k, v in prof_ms.items()},
+                     "serialised_time_share": {k: round(v / max(sum(prof_ms.values()), 1e-9), 4) for k, v in prof_ms.items()},
+                     "in_step": in_step,
                      "whole_step": {"bytes": int(step_bytes), "achieved_gbs": round(whole, 1),
                                     "frac_of_measured_peak": round(whole / pk["hbm_gbs"], 4),
                                     "frac_of_8tbs": round(whole / 8000.0, 4)}},
         "shape": shape, "wl": wl, "context": context, "from_topk": float(d_real[warm:].float().mean()),
-        "weights": w, "prompt": prompt,
+        "weights": w, "prompt": prompt, "planted": planted,
     }
     return result
+
+
+PLANT_KEEP = 0.6        # share of the model's own tri-grams the planted table knows
+PLANT_COUNT = 1 << 20   # their count: above anything the prompt put into the table
+
+
+def planted_arm(B, model, kv, fresh_table, ctx, ctx0, base_len, fill_d, wl, shape, steps, warm, dev, world, rank):
+    """A second timed decode in which drafts are approved.  With random-init weights the model's greedy text is
+    unrelated to the Zipf prompt, so a table built from the prompt alone never predicts it (accept length 1).  Here
+    the table is told, before decoding starts, a seeded PLANT_KEEP share of the tri-grams of the model's OWN
+    greedy continuation (recorded first, by ordinary decode steps from the same prompt) -- the state the paper's
+    adaptive table reaches on text it has seen before.  Draft trees then come from top-k lists that hold the
+    model's path, accept lengths spread over 1 .. depth + 1 (mean about 1 / (1 - keep)), and the approved K/V rows
+    are compacted inside the timed region.  Same model, cache, prompt and filler as the main arm."""
+    n, total = wl.tree_nodes, steps + warm
+    n_rec = int(total / (1.0 - PLANT_KEEP)) + 32                 # decode steps to record: one token each
+    rec_out = torch.zeros((n_rec, n), dtype=torch.int32, device=dev)
+    rec_len = torch.zeros((n_rec, 1), dtype=torch.int32, device=dev)
+    B.aded_kv_set_len(kv, 0, base_len)
+    table = fresh_table()
+    ctx.copy_(ctx0)
+    for s in range(n_rec):
+        B.aded_decode_step(model, kv, table, ctx, n, wl.tree_depth, wl.topk, fill_d[s % total], rec_out[s], rec_len[s], None)
+    torch.cuda.synchronize()
+    lens = rec_len[:, 0].tolist()
+    text = ctx0.tolist() + [t for s in range(n_rec) for t in rec_out[s, :lens[s]].tolist()]
+    keep = (gen.uniform01(len(text) - 2, SEED + rank, 7777) < PLANT_KEEP).tolist()
+    keys = [text[i:i + 3] for i in range(len(text) - 2) if keep[i]]
+    table = fresh_table()
+    B.aded_trigram_import(table, torch.tensor(keys, dtype=torch.int32, device=dev).contiguous(),
+                          torch.full((len(keys),), PLANT_COUNT, dtype=torch.int32, device=dev))
+    B.aded_kv_set_len(kv, 0, base_len)
+    ctx.copy_(ctx0)
+    p_out = torch.zeros((total, n), dtype=torch.int32, device=dev)
+    p_len = torch.zeros((total, 1), dtype=torch.int32, device=dev)
+    p_real = torch.zeros((total, 1), dtype=torch.int32, device=dev)
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+    torch.cuda.synchronize()
+    for step in range(total):
+        if step == warm:
+            if world > 1:
+                torch.distributed.barrier()
+            torch.cuda.synchronize()
+            ev[0].record()
+        B.aded_decode_step(model, kv, table, ctx, n, wl.tree_depth, wl.topk, fill_d[step], p_out[step], p_len[step], p_real[step])
+    ev[1].record()
+    torch.cuda.synchronize()
+    assert B.aded_model_poll_status(model) == 0 and B.aded_trigram_poll_status(table) == 0
+    ms = ev[0].elapsed_time(ev[1])
+    plens = p_len[:, 0].tolist()
+    emitted = [t for s in range(total) for t in p_out[s, :plens[s]].tolist()]
+    accepted = sum(plens[warm:])
+    hist = {}
+    for a in plens[warm:]:
+        hist[a] = hist.get(a, 0) + 1
+    # verification equals plain decoding: the text must be the recorded one (a near-tie may legitimately move a token)
+    m = min(len(emitted), len(text) - 2)
+    same = emitted[:m] == text[2:2 + m]
+    first_diff = next((i for i in range(m) if emitted[i] != text[2 + i]), None)
+    return {"ms": ms, "accepted": accepted, "ms_per_step": ms / steps, "accept_len_mean": accepted / steps,
+            "accept_len_histogram": {str(k): hist[k] for k in sorted(hist)},
+            "tree_nodes_from_table_mean": float(p_real[warm:].float().mean()),
+            "table": f"prompt tri-grams + a seeded {PLANT_KEEP:.0%} of the tri-grams of the model's own greedy continuation "
+                     f"({len(keys)} of {len(text) - 2}, count {PLANT_COUNT})",
+            "text_equals_recorded_decode": same, "first_difference_at_token": first_diff, "tokens_compared": m}
+
+
+def stage_times(marks, n_layers):
+    """Per-stage times of the timed pass from the device-side trace: every kernel of a pass records when its
+    wait for the previous kernel ended; the gap to the next mark is what that kernel added to the pass,
+    overlap under programmatic dependent launch included.  Returns microseconds per layer for the per-layer
+    stages and per step for the rest, averaged over the whole steps the trace holds."""
+    from paper_2407_12021_b200.binding import TRACE_KINDS
+    ts, kinds = marks
+    ends = [i for i, k in enumerate(kinds) if k == 11]          # a commit ends a pass
+    if len(ends) < 2:
+        return None
+    first, last = ends[0], ends[-1]
+    n_steps = len(ends) - 1
+    tot = {}
+    for i in range(first, last):
+        name = "between_passes" if kinds[i] == 11 else TRACE_KINDS.get(kinds[i], str(kinds[i]))
+        tot[name] = tot.get(name, 0.0) + (ts[i + 1] - ts[i]) * 1e-3
+    per_layer = {k: round(tot.get(k, 0.0) / n_steps / n_layers, 2) for k in
+                 ("gemm_qkv", "attention", "gemm_o", "rmsnorm", "gemm_gate_up", "gemm_down", "rotary_kv", "swiglu") if k in tot}
+    per_step = {k: round(tot.get(k, 0.0) / n_steps, 1) for k in ("gemm_lm_head", "pick_accept", "other", "between_passes") if k in tot}
+    proj = sum(per_layer.get(k, 0.0) for k in ("gemm_qkv", "gemm_o", "gemm_gate_up", "gemm_down"))
+    return {"steps_traced": n_steps, "us_per_layer": per_layer, "us_per_step": per_step,
+            "us_per_layer_projections": round(proj, 2), "us_per_layer_total": round(sum(per_layer.values()), 2),
+            "note": "device timestamps at the end of each kernel's dependency wait, in the timed pass; 'between_passes' is the "
+                    "commit, the table update, the next context and the next draft tree"}
+
+
+def zipf_tokens_on(dev, n, vocab, seed, stream):
+    """gen.zipf_tokens computed on the device (the same inverse-CDF arithmetic on the same uniform numbers)."""
+    out = torch.empty(n, dtype=torch.int32, device=dev)
+    cdf = gen.zipf_cdf(vocab).to(dev)
+    for s0 in range(0, n, 1 << 24):
+        m = min(1 << 24, n - s0)
+        u = gen.uniform01(m, seed, stream, device=dev, offset=s0)
+        out[s0:s0 + m] = torch.searchsorted(cdf, u).clamp_(max=vocab - 1).to(torch.int32)
+    return out
+
+
+def run_tg(args, rank, world):
+    """The tri-gram store alone: Algorithm 2 over a whole corpus in one call, then top-4 lookups (Eq. 1 ranking)
+    for contexts drawn from the corpus.  One JSON line per corpus size is printed; the last one is the line of
+    the larger corpus (the table then is in the hundreds-of-MB regime the paper reports for its corpora)."""
+    from paper_2407_12021_b200 import build as libbuild
+    libbuild.build()
+    from paper_2407_12021_b200 import binding as B
+    from oracle.trigram import TrigramStore
+    dev = torch.device("cuda", int(os.environ.get("LOCAL_RANK", 0)))
+    torch.cuda.set_device(dev)
+    vocab, k, n_q = 32000, 4, 1 << 20
+    pk = peaks()
+    reps = max(args.steps if args.steps != 256 else 5, 3)
+    lines = []
+    for n_tok, log2b, overflow in ((1_000_000, 21, 1 << 19), (50_000_000, 26, 1 << 23)):
+        toks = zipf_tokens_on(dev, n_tok, vocab, SEED + rank, 60)
+        qi = (gen.uniform01(n_q, SEED + rank, 61, device=dev) * (n_tok - 2)).long()
+        ctxs = torch.stack([toks[qi], toks[qi + 1]], dim=1).contiguous()
+        out_t = torch.empty((n_q, k), dtype=torch.int32, device=dev)
+        out_c = torch.empty((n_q, k), dtype=torch.int32, device=dev)
+        upd_ms, top_ms = [], []
+        for r in range(reps + 1):                      # first repetition is the warm-up
+            t = B.aded_trigram_create(vocab, log2_buckets=log2b, overflow_buckets=overflow)
+            torch.cuda.synchronize()
+            e = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
+            e[0].record()
+            B.aded_trigram_update(t, toks)
+            e[1].record()
+            B.aded_trigram_topk(t, ctxs, k, out_t, out_c)      # first pass over the queries: table lines come from HBM
+            e[2].record()
+            torch.cuda.synchronize()
+            assert B.aded_trigram_poll_status(t) == 0
+            if r:
+                upd_ms.append(e[0].elapsed_time(e[1]))
+                top_ms.append(e[1].elapsed_time(e[2]))
+            entries, buckets = B.aded_trigram_stats(t)
+            if r < reps:
+                del t
+        upd, top = statistics.median(upd_ms), statistics.median(top_ms)
+        windows = n_tok - 2
+        # algorithmic traffic: one 64-byte bucket read + one 4-byte count written back per window; one bucket per query
+        upd_gbs = windows * 68 / (upd * 1e-3) / 1e9
+        top_gbs = n_q * 64 / (top * 1e-3) / 1e9
+        # the checker's dictionary store on a bounded sample of the same corpus and queries
+        sample_tok, sample_q = min(n_tok, 300_000), 20_000
+        st = TrigramStore()
+        host = toks[:sample_tok].cpu().tolist()
+        t0 = time.perf_counter(); st.update(host); cpu_upd = time.perf_counter() - t0
+        hq = ctxs[:sample_q].cpu().tolist()
+        t0 = time.perf_counter()
+        for a, b in hq:
+            st.topk(a, b, k)
+        cpu_top = time.perf_counter() - t0
+        if n_tok == sample_tok:                        # the small corpus is checked in full: lists equal the checker's
+            got_t, got_c = out_t[:sample_q].cpu().tolist(), out_c[:sample_q].cpu().tolist()
+            for i, (a, b) in enumerate(hq[:2000]):
+                assert (got_t[i], got_c[i]) == st.topk(a, b, k), (a, b)
+        lines.append({
+            "metric": "trigram_update_windows_per_s", "value": windows / (upd * 1e-3), "unit": "windows/s", "n_gpus": 1,
+            "steps": reps, "warmup": 1, "ms_per_step": upd, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "u32", "data": "synthetic",
+            "config": {"workload": f"tg: Zipf(1.1) corpus of {n_tok} tokens over {vocab} ids, one bulk update, then {n_q} top-{k} queries for contexts drawn from the corpus",
+                       "l2": "table larger than L2" if buckets * 64 > 126e6 else "table fits L2 (the update of the small corpus is L2 traffic)",
+                       "table_mb": round(buckets * 64 / 1e6, 1), "entries": entries, "buckets_in_use": buckets},
+            "topk": {"queries_per_s": n_q / (top * 1e-3), "ms": top, "bytes_per_query": 64, "achieved_gbs": round(top_gbs, 1),
+                     "frac_of_hbm_peak": round(top_gbs / pk["hbm_gbs"], 4)},
+            "roofline": {"bound": "hbm", "kernel": "k_tg_update", "achieved": round(upd_gbs, 1), "peak": pk["hbm_gbs"],
+                         "peak_source": pk["source"], "unit": "GB/s", "frac": round(upd_gbs / pk["hbm_gbs"], 4), "traffic": None,
+                         "algorithmic_bytes_per_window": 68,
+                         "note": "random 64-byte buckets: a DRAM sector access is 32-64 bytes of a 64-byte burst, and every window is an atomic read-modify-write"},
+            "gpu_launches": 2,
+            "cpu_baseline": {"value": (sample_tok - 2) / cpu_upd, "unit": "windows/s", "cores": 1, "kind": "oracle",
+                             "sample": f"dictionary store: first {sample_tok} tokens of the corpus ({cpu_upd:.2f} s), {sample_q} of the queries ({cpu_top:.2f} s)",
+                             "topk_queries_per_s": sample_q / cpu_top},
+            "e2e": None,
+        })
+        del t, toks
+    for line in lines:
+        print(json.dumps(line))
+
+
+def run_c5(args, rank, world):
+    """Ragged batches of 1, 4 and 16 sequences at the 7B model's full depth: contexts from U[512, 8192], trees of
+    32..128 nodes, caches pre-filled with N(0,1) keys/values; one aded_verify_batch call per step."""
+    from paper_2407_12021_b200 import build as libbuild
+    libbuild.build()
+    from paper_2407_12021_b200 import binding as B
+    dev = torch.device("cuda", int(os.environ.get("LOCAL_RANK", 0)))
+    torch.cuda.set_device(dev)
+    shape = gen.LLAMA7B if not args.layers else gen.LLAMA7B.with_layers(args.layers)
+    w = gen.model_weights(shape, SEED + rank, device=dev)
+    pk = peaks()
+    bf16_peak = 1388.9
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            bf16_peak = float(json.load(f).get("bf16_tflops_sustained", bf16_peak))
+    steps, warm = (args.steps if args.steps != 256 else 10), max(args.warmup, 3)
+    batches = {}
+    for batch in (1, 4, 16):
+        ctx_len = [512 + v for v in gen.randint(batch, 8192 - 512 + 1, SEED + batch, 1)]
+        n_nodes = [32 + v for v in gen.randint(batch, 128 - 32 + 1, SEED + batch, 2)]
+        depth = [3 + v for v in gen.randint(batch, 6, SEED + batch, 3)]
+        rows = sum(n_nodes)
+        model = B.aded_model_create(shape, w, max_rows=rows, max_batch=batch)
+        kv = B.aded_kv_create(model, [c + 128 for c in ctx_len])
+        for b in range(batch):
+            for l in range(shape.n_layers):
+                kk, vv = gen.kv_normal(shape, ctx_len[b], SEED + 100 + b, l, device=dev)
+                B.aded_kv_load(kv, b, l, kk, vv)
+        trees = [gen.make_tree(n_nodes[b], depth[b], 6, shape.vocab, SEED + 200 + b) for b in range(batch)]
+        offsets = [0]
+        for b in range(batch):
+            offsets.append(offsets[-1] + n_nodes[b])
+        tok = torch.tensor([t for tr in trees for t in tr[0]], dtype=torch.int32, device=dev)
+        par = torch.tensor([p for tr in trees for p in tr[1]], dtype=torch.int32, device=dev)
+        out = torch.zeros((batch, 128), dtype=torch.int32, device=dev)
+        out_len = torch.zeros((batch,), dtype=torch.int32, device=dev)
+        times = []
+        for step in range(warm + steps):
+            for b in range(batch):
+                B.aded_kv_set_len(kv, b, ctx_len[b])           # every step verifies from the same committed lengths
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            B.aded_verify_batch(model, kv, offsets, tok, par, out, out_len)
+            e1.record()
+            torch.cuda.synchronize()
+            if step >= warm:
+                times.append(e0.elapsed_time(e1))
+        assert B.aded_model_poll_status(model) == 0
+        B.aded_trace_begin(model)
+        for b in range(batch):
+            B.aded_kv_set_len(kv, b, ctx_len[b])
+        B.aded_verify_batch(model, kv, offsets, tok, par, out, out_len)
+        B.aded_verify_batch(model, kv, offsets, tok, par, out, out_len)      # (a second pass so that the trace holds a whole one)
+        ts, kinds = B.aded_trace_end(model)
+        ends = [i for i, kd in enumerate(kinds) if kd == 11]
+        gemm_us = attn_us = 0.0
+        if len(ends) >= 2:
+            for i in range(ends[-2], ends[-1]):
+                dt = (ts[i + 1] - ts[i]) * 1e-3
+                if kinds[i] in (1, 2, 3, 4, 5):
+                    gemm_us += dt
+                elif kinds[i] == 6:
+                    attn_us += dt
+        ms = statistics.median(times)
+        kv_bytes = shape.kv_bytes_per_position() * sum(ctx_len)
+        flops = 2.0 * (shape.weight_bytes_per_step / 2) * rows
+        passes = (rows + 127) // 128
+        batches[str(batch)] = {
+            "rows": rows, "contexts": ctx_len, "tree_nodes": n_nodes, "ms_per_call": round(ms, 3),
+            "accepted_tokens_per_s": float(out_len.sum()) / (ms * 1e-3),
+            "algorithmic_bytes": int(shape.weight_bytes_per_step + kv_bytes),
+            "hbm_frac_whole_call": round((shape.weight_bytes_per_step + kv_bytes) / (ms * 1e-3) / 1e9 / pk["hbm_gbs"], 4),
+            "attention_us": round(attn_us, 1), "attention_hbm_frac": round(kv_bytes / max(attn_us, 1e-9) / 1e3 / pk["hbm_gbs"], 4),
+            "gemm_us": round(gemm_us, 1), "gemm_tensor_frac": round(flops / max(gemm_us, 1e-9) / 1e6 / bf16_peak, 4),
+            "gemm_weight_passes": passes,
+            "gemm_hbm_frac_of_streamed_weights": round(passes * shape.weight_bytes_per_step / max(gemm_us, 1e-9) / 1e3 / pk["hbm_gbs"], 4),
+        }
+        del kv, model
+        torch.cuda.empty_cache()
+    b16 = batches["16"]
+    line = {"metric": "verify_batch_ms", "value": b16["ms_per_call"], "unit": "ms", "n_gpus": 1, "steps": steps, "warmup": warm,
+            "ms_per_step": b16["ms_per_call"], "higher_is_better": False, "scaling": "weak", "vs_baseline": None, "dtype": shape.dtype,
+            "data": "synthetic",
+            "config": {"workload": f"c5: {shape.name} ({shape.n_layers} layers), ragged batches 1 / 4 / 16, contexts U[512, 8192], trees of 32..128 nodes, "
+                                   "pre-filled N(0,1) caches, one aded_verify_batch call per step; value = batch 16",
+                       "l2": "inputs larger than L2"},
+            "batches": batches, "gpu_launches": None, "e2e": None,
+            "roofline": {"bound": "tensor" if b16["gemm_tensor_frac"] > b16["hbm_frac_whole_call"] else "hbm",
+                         "achieved": round(b16["gemm_tensor_frac"] * bf16_peak, 1), "peak": bf16_peak, "unit": "TFLOP/s",
+                         "frac": b16["gemm_tensor_frac"], "traffic": None,
+                         "note": "batch 16, projections only; peak = measured sustained bf16 matmul; the tensor-core GEMM makes one pass over the "
+                                 "weights per 128 rows (gemm_weight_passes), so its HBM traffic is that many times the weight bytes"}}
+    print(json.dumps(line))
 
 
 def cpu_oracle_sample(shape, wl, weights, context, layers_timed=6, threads=None):
@@ -310,41 +600,56 @@ def main():
     args = parse_args()
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
-    wl = gen.WORKLOADS[args.workload]
+    wl = gen.WORKLOADS.get(args.workload, gen.WORKLOADS["c3"])
 
     if args.impl == "reference":
-        # the CPU checker as it stands, rank 0 only
+        # The CPU checker as it stands, on the host cores, rank 0 only.  A full 32-layer step takes it about a minute
+        # and a half, so a "step" of this arm is a bounded sample of one verification step of the same workload:
+        # LAYERS_TIMED decoder layers over the workload's tree and context plus the LM head.  `ms_per_step` is what
+        # a step of this arm really took; `value` scales the layer part to the model's depth (stated in the line).
         if rank != 0:
             return
         shape = wl.shape if not args.layers else wl.shape.with_layers(args.layers)
         context = args.context or wl.context
-        sub = shape.with_layers(min(2, shape.n_layers))
-        w = gen.model_weights(sub, SEED)
-        w_full = dict(w)
-        times = []
+        layers_timed = min(2, shape.n_layers)
+        w = gen.model_weights(shape.with_layers(layers_timed), SEED)
+        scaled, measured = [], []
         for _ in range(max(args.warmup, 0) + args.steps):
-            s, sample = cpu_oracle_sample(shape, wl, w_full, context, layers_timed=sub.n_layers)
-            times.append(s)
-        times = times[max(args.warmup, 0):]
-        step_s = statistics.mean(times)
+            t0 = time.perf_counter()
+            step_s, sample = cpu_oracle_sample(shape, wl, dict(w), context, layers_timed=layers_timed)
+            measured.append(time.perf_counter() - t0)
+            scaled.append(step_s)
+        scaled, measured = scaled[max(args.warmup, 0):], measured[max(args.warmup, 0):]
+        step_s = statistics.mean(scaled)
         val = 1.0 / step_s     # one token per step: random-init drafts are accepted at the floor rate
         line = {"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
-                "warmup": args.warmup, "ms_per_step": step_s * 1e3, "higher_is_better": True, "scaling": "weak",
-                "vs_baseline": None, "dtype": shape.dtype, "data": "synthetic",
+                "warmup": args.warmup, "ms_per_step": statistics.mean(measured) * 1e3, "higher_is_better": True, "scaling": "weak",
+                "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+                "layers_timed": layers_timed, "layers_total": shape.n_layers,
+                "ms_per_full_step_scaled": step_s * 1e3,
                 "config": {"workload": f"{args.workload}: {shape.name}, context {context}, {wl.tree_nodes}-node trees",
-                           "note": "accept length taken as 1 token per step"},
+                           "note": f"each step of this arm runs {layers_timed} of {shape.n_layers} layers + the LM head of one verification step "
+                                   "(ms_per_step); value = 1 token / (layer time x layers_total / layers_timed + head time): "
+                                   "accept length taken as 1 token per step"},
                 "cpu_baseline": {"value": val, "unit": UNIT, "cores": torch.get_num_threads(), "kind": "oracle",
                                  "sample": sample},
                 "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
         print(json.dumps(line))
         return
 
+    if args.workload in ("tg", "c5"):
+        # secondary workloads: single GPU, rank 0 (replicas would only repeat them)
+        if rank == 0:
+            (run_tg if args.workload == "tg" else run_c5)(args, rank, world)
+        return
     if world > 1:
         torch.distributed.init_process_group("nccl", device_id=torch.device("cuda", int(os.environ.get("LOCAL_RANK", 0))))
     res = run_ours(args, rank, world)
     acc = res["accepted"]
-    ms, e2e_ms, acc_total = aggregate_over_ranks(res["ms"], res["e2e_ms"], acc, world,
-                                                 torch.device("cuda", int(os.environ.get("LOCAL_RANK", 0))))
+    here = torch.device("cuda", int(os.environ.get("LOCAL_RANK", 0)))
+    ms, e2e_ms, acc_total = aggregate_over_ranks(res["ms"], res["e2e_ms"], acc, world, here)
+    pl = res["planted"]
+    pl_ms, _, pl_acc = aggregate_over_ranks(pl["ms"], pl["ms"], pl["accepted"], world, here)
     if rank != 0:
         torch.distributed.destroy_process_group()
         return
@@ -363,6 +668,8 @@ def main():
                 "h2d_bytes_per_step": res["h2d"], "d2h_bytes_per_step": res["d2h"]},
         "gpu_launches": res["launches"], "clocks": res["clocks"], "roofline": res["roofline"],
     }
+    line["planted"] = {"metric": METRIC, "value": pl_acc / (pl_ms * 1e-3), "unit": UNIT, "ms_per_step": pl_ms / steps,
+                       **{k: v for k, v in pl.items() if k not in ("ms", "accepted", "ms_per_step")}}
     if not args.no_cpu_baseline:
         cores = os.cpu_count() or 1
         step_s, sample = cpu_oracle_sample(shape, wl, res["weights"], res["context"], threads=cores)

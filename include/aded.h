@@ -16,9 +16,16 @@
  *    was created; pointers named *_host are HOST pointers.  The caller owns both and keeps
  *    them alive until the work has finished on the stream.
  *  - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).  Calls
- *    taking device pointers only enqueue work and never synchronise.  Calls with a _host
- *    suffix copy their arguments in and their results out and return after the stream has
- *    drained.
+ *    taking device pointers only enqueue work and never synchronise -- except those whose
+ *    comment says "synchronises" (aded_kv_len, aded_kv_load, aded_kv_set_len, the poll_status
+ *    calls, aded_trigram_get/stats/export/prune/save/load, aded_profile_end, aded_trace_begin/end):
+ *    they hand a host value to or from the device and return after the stream has drained.
+ *    Calls with a _host suffix copy their arguments in and their results out and likewise
+ *    return after the stream has drained.
+ *  - Device memory: handles allocate their workspace, cache blocks and tables with cudaMalloc
+ *    when they are created (and aded_trigram_prune / aded_decode_step_mcts once more on first
+ *    use) and free it when they are destroyed; the weights stay the caller's.  Nothing is
+ *    allocated by the calls of a decoding step.
  *  - Errors the host can see (NULL handles, sizes out of range) are returned at once and
  *    nothing is launched.  Errors only the device can see (malformed parent array, cache
  *    capacity, hash table full, a bounded wait that ran out) are recorded in a device status
@@ -82,7 +89,7 @@ typedef struct aded_trigram_config {
     int32_t vocab;            /* token ids are 0 .. vocab-1 */
     int32_t log2_buckets;     /* 2^log2_buckets home buckets (one per two-token context), 4..28 */
     int32_t overflow_buckets; /* extra buckets for contexts with more than 6 continuations */
-    uint32_t cap;             /* counts saturate here (Algorithm 2's maximum); 0 = 2^31 - 1 */
+    uint32_t cap;             /* counts saturate here (Algorithm 2's maximum); 0 = 2^31 - 1, which is also the largest allowed */
     uint32_t min_count;       /* top-k skips entries below this count; 0 = off */
 } aded_trigram_config;
 
@@ -108,12 +115,12 @@ aded_status aded_kv_destroy(aded_kv* kv);
 aded_status aded_kv_len(const aded_kv* kv, int32_t seq, int32_t* out_len_host, void* stream);
 /* Overwrite positions [0, n_pos) of layer `layer` of sequence `seq` with given keys/values
  * (device pointers, [head][n_pos][head_dim], model dtype) and set the committed length to
- * n_pos.  For workloads that start from a pre-filled cache. */
+ * n_pos.  For workloads that start from a pre-filled cache.  Synchronises `stream`. */
 aded_status aded_kv_load(aded_kv* kv, int32_t seq, int32_t layer, const void* k_dev, const void* v_dev,
                          int32_t n_pos, void* stream);
 /* Set the committed length of sequence `seq` to new_len (0 <= new_len <= capacity): roll a
  * sequence back to an earlier point, e.g. to the end of its prompt.  Rows past new_len stay in
- * memory and are overwritten by later calls. */
+ * memory and are overwritten by later calls.  Synchronises `stream`. */
 aded_status aded_kv_set_len(aded_kv* kv, int32_t seq, int32_t new_len, void* stream);
 /* Copy out positions [pos0, pos0 + n_pos) of one layer: k_dev / v_dev receive
  * [head][n_pos][head_dim].  For tests. */
@@ -202,10 +209,38 @@ aded_status aded_profile_end(aded_model* m, float* out_ms_host, int32_t* out_lau
 /* Kernels launched by this library in this process so far (all handles). */
 uint64_t aded_launch_count(void);
 
+/* Stage trace of the verification step as it really runs, kernels overlapping under programmatic
+ * dependent launch (not part of the paper's method; the per-launch events of aded_profile_begin serialise
+ * the kernels, this does not).  Between begin and end every kernel of a pass records, from one thread,
+ * the device's global-timer value (ns) at the moment its wait for the previous kernel ended, with a
+ * kind: 0 other, 1..5 the QKV / O / gate-up / down / LM-head projection, 6 tree attention, 7 RMSNorm,
+ * 8 rotary + K/V write, 9 SwiGLU (8 and 9 only where they are kernels of their own: fp32 models),
+ * 10 greedy choice and approval, 11 the commit that ends a pass.  The difference between two
+ * consecutive marks is the time the earlier kernel added to the pass.  The device keeps the last 16384
+ * marks.  end() stops recording, synchronises `stream` and writes the last min(max_marks, kept)
+ * marks, oldest first, to out_ns_host / out_kind_host and their number to out_n_host. */
+aded_status aded_trace_begin(aded_model* m, void* stream);
+aded_status aded_trace_end(aded_model* m, uint64_t* out_ns_host, int32_t* out_kind_host, int32_t max_marks,
+                           int32_t* out_n_host, void* stream);
+
 /* Ask the next verify call to also store the residual stream before the first layer and after
  * every layer: hidden_dev receives [n_layers + 1][rows][d_model] in the model dtype.  Lets a checker
  * re-run any single layer from the inputs the device actually had.  Parity checks only. */
 aded_status aded_debug_capture_hidden(aded_model* m, void* hidden_dev);
+
+/* Failure-path check ("every device-side wait is bounded", see Conventions): runs one of the library's two
+ * kinds of device-side wait -- which = 0: the mbarrier wait of the tensor-core kernels, 1: the wait at an
+ * arrival counter of the LM head's tail -- on something that never happens, with a limit of limit_cycles
+ * SM clock cycles (1 .. 2^32; about 2 x 10^6 per millisecond).  The wait runs out, the kernel returns, and
+ * the model's status word becomes ADED_ERR_TIMEOUT exactly as after a real time-out: later calls do nothing
+ * until aded_model_poll_status has read and cleared it.  Nothing faults or hangs.  Asynchronous. */
+aded_status aded_debug_wait_timeout(aded_model* m, int32_t which, uint64_t limit_cycles, void* stream);
+
+/* head_dim-128 bf16 models have two tree-attention kernels that compute the same thing with the same
+ * rounding points: tcgen05 (which = 0, the default) and mma.sync (which = 1; the kernel head_dim 64
+ * always uses).  Selects the one later calls on this model use, so that a test can compare them.
+ * ADED_ERR_UNSUPPORTED for models without a tensor-core attention kernel (fp32). */
+aded_status aded_debug_attention_kernel(aded_model* m, int32_t which);
 
 /* Copy out one of the model's activation buffers as the last verify/append call left it (after
  * its last layer): which = 0 residual stream h [rows, d], 1 normalised input x [rows, d], 2 rotated
@@ -228,8 +263,11 @@ aded_status aded_debug_read_buffer(aded_model* m, int32_t which, int32_t rows, v
  * intermediate results live in a fixed 16 KiB array inside the library's device image (every
  * device that loads the library holds it until the process exits), which bounds the size:
  * rows <= ADED_NOALLOC_MAX_ROWS, otherwise ADED_ERR_INVALID_ARG and nothing is launched.
- * The first call on each device looks up the array's device address (with that device current);
- * make that first call outside any stream capture.  All calls share the one array: it keeps the
+ * The first call on each device looks up the array's device address (with that device current)
+ * and keeps it for the life of the process; make that first call outside any stream capture.  The
+ * kept address does not survive cudaDeviceReset or the teardown of the device's primary context --
+ * do not call this entry point again in a process that has done either -- and only device ordinals
+ * 0..63 are served (ADED_ERR_UNSUPPORTED beyond).  All calls share the one array: it keeps the
  * previous call's contents, which is harmless because every entry is rewritten before it is read,
  * but two calls whose kernels overlap on the GPU (different streams, no dependency) race on it --
  * keep calls on one stream or order them with events.  Work is enqueued on `stream`; the call does

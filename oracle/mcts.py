@@ -27,6 +27,14 @@ these readings where the listing or the text leave a choice:
     leaves first on ties; the best `n_candidates` are merged into one prefix tree, numbered breadth
     first, children in creation (rank) order.
 All floating-point work is IEEE double, one rounded operation at a time, in the order written.
+
+What is the algorithm's and what is this module's: the order of the four phases inside an iteration, the
+rule that expansion creates every candidate at once and goes on with the last one, the score of 1.0 plus
+tri-gram probabilities, and back propagation to every ancestor are Algorithm 1's definition of the search --
+an iteration reads the visit counts and scores the previous one left, so any other order is a different
+search and a different draft.  They are restated here from that definition.  The data structures (parallel
+lists indexed by node number, contexts kept per node), the selection rule's tie break, the integer inverse
+CDF of the simulation, the ranking and the prefix-tree merge are this module's own, as listed above.
 """
 from __future__ import annotations
 

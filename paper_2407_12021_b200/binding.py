@@ -25,7 +25,7 @@ STATUS_NAMES = {0: "ADED_OK", 1: "ADED_ERR_INVALID_ARG", 2: "ADED_ERR_BAD_TREE",
 EXPORTS = [
     "aded_model_create", "aded_model_destroy", "aded_kv_create", "aded_kv_destroy", "aded_kv_len",
     "aded_kv_load", "aded_kv_set_len", "aded_kv_read", "aded_append", "aded_verify", "aded_verify_batch", "aded_verify_host",
-    "aded_debug_capture", "aded_debug_capture_hidden", "aded_debug_gemm", "aded_debug_read_buffer", "aded_greedy_noalloc", "aded_profile_begin", "aded_profile_end", "aded_launch_count", "aded_model_poll_status", "aded_trigram_create", "aded_trigram_destroy",
+    "aded_debug_capture", "aded_debug_capture_hidden", "aded_debug_gemm", "aded_debug_read_buffer", "aded_greedy_noalloc", "aded_profile_begin", "aded_profile_end", "aded_trace_begin", "aded_trace_end", "aded_debug_attention_kernel", "aded_debug_wait_timeout", "aded_launch_count", "aded_model_poll_status", "aded_trigram_create", "aded_trigram_destroy",
     "aded_trigram_update", "aded_trigram_update_host", "aded_trigram_topk", "aded_trigram_topk_host",
     "aded_trigram_get", "aded_trigram_stats", "aded_trigram_poll_status", "aded_draft_tree", "aded_decode_step",
     "aded_decode_step_host", "aded_verify_sampled", "aded_sample_tokens", "aded_trigram_export",
@@ -303,6 +303,31 @@ def aded_profile_end(model: Model):
     _check(_lib.aded_profile_end(model.handle, ms, n, _stream()), "aded_profile_end")
     names = ("gemm", "attention", "other")
     return dict(zip(names, [float(v) for v in ms])), dict(zip(names, [int(v) for v in n]))
+
+
+TRACE_KINDS = {0: "other", 1: "gemm_qkv", 2: "gemm_o", 3: "gemm_gate_up", 4: "gemm_down", 5: "gemm_lm_head", 6: "attention",
+               7: "rmsnorm", 8: "rotary_kv", 9: "swiglu", 10: "pick_accept", 11: "commit"}
+
+
+def aded_trace_begin(model: Model) -> None:
+    _check(_lib.aded_trace_begin(model.handle, _stream()), "aded_trace_begin")
+
+
+def aded_trace_end(model: Model, max_marks: int = 16384):
+    """Returns (times in ns, kinds) of the last marks, oldest first, as two python lists."""
+    ts = (c_uint64 * max_marks)()
+    kinds = (c_int32 * max_marks)()
+    n = c_int32(0)
+    _check(_lib.aded_trace_end(model.handle, ts, kinds, c_int32(max_marks), ctypes.byref(n), _stream()), "aded_trace_end")
+    return list(ts[:n.value]), list(kinds[:n.value])
+
+
+def aded_debug_wait_timeout(model: Model, which: int, limit_cycles: int) -> None:
+    _check(_lib.aded_debug_wait_timeout(model.handle, c_int32(which), c_uint64(limit_cycles), _stream()), "aded_debug_wait_timeout")
+
+
+def aded_debug_attention_kernel(model: Model, which: int) -> None:
+    _check(_lib.aded_debug_attention_kernel(model.handle, c_int32(which)), "aded_debug_attention_kernel")
 
 
 def aded_launch_count() -> int:

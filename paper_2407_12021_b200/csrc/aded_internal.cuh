@@ -9,7 +9,6 @@
 #include <vector>
 
 #include "aded.h"
-#include "fused_ws.cuh"
 #include "gemm_out.cuh"
 
 #define ADED_CUDA_TRY(expr)                      \
@@ -50,7 +49,30 @@ __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepc
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void pdl_enter() { pdl_launch_dependents(); pdl_wait(); }
 
-bool pdl_enabled();
+// ---- stage trace ---------------------------------------------------------------------------------
+// The status word of a model is the first of a small block of device memory:
+//   int32 [0] status, [1] trace switch, [2] marks taken, [3] unused; then TRACE_CAP 64-bit times (ns of
+//   the global timer) and TRACE_CAP int32 kinds.
+// While the switch is on, every kernel of a pass records, from one thread of its first block, the time at
+// which its wait for the previous kernel ended.  The difference between two consecutive marks is the
+// time the earlier kernel added to the pass (its overlap with its neighbours included), which is what
+// a roofline report of a step chained by programmatic dependent launch needs; event pairs around
+// launches would serialise the kernels.
+enum { TRACE_CAP = 16384, STATUS_WORDS = 4 + 3 * TRACE_CAP };
+enum { TK_OTHER = 0, TK_GEMM_QKV = 1, TK_GEMM_O = 2, TK_GEMM_GU = 3, TK_GEMM_DOWN = 4, TK_GEMM_HEAD = 5, TK_ATTN = 6,
+       TK_NORM = 7, TK_ROPE = 8, TK_SWIGLU = 9, TK_PICK = 10, TK_STEP_END = 11 };
+__device__ __forceinline__ void trace_mark(const int32_t* status, int kind) {
+    int32_t* s = const_cast<int32_t*>(status);
+    if (__ldcg(s + 1) == 0) return;
+    const int i = atomicAdd(s + 2, 1) & (TRACE_CAP - 1);
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    reinterpret_cast<unsigned long long*>(s + 4)[i] = t;
+    (s + 4 + 2 * TRACE_CAP)[i] = kind;
+}
+__device__ __forceinline__ bool first_thread_of_grid() {
+    return threadIdx.x == 0 && blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0;
+}
 
 template <typename... KArgs, typename... Args>
 inline cudaError_t launch_k(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args... args) {
@@ -63,7 +85,7 @@ inline cudaError_t launch_k(void (*kernel)(KArgs...), dim3 grid, dim3 block, siz
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = pdl_enabled() ? 1 : 0;
+    cfg.numAttrs = 1;
     return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
 }
 
@@ -87,12 +109,60 @@ struct CallPtrs {
     int32_t out_stride;
 };
 
+// Draft approval of one sequence, by one thread (a tree has at most ADED_MAX_NODES nodes; arrays in shared
+// memory).  A node is approved when its parent is approved and its token equals the model's token at the
+// parent; the deepest approved node (lowest index among equals) ends the accepted path.  Emits the
+// model's token of every path node: the approved drafts' successors, ending with the model's own next
+// token.  A failed pass emits nothing and keeps the committed length.
+__device__ __forceinline__ void approval_walk(const int32_t* s_par, const int32_t* s_tok, const int32_t* s_best,
+                                              const int32_t* s_dep, int T, int pass_status, int committed,
+                                              int32_t* out_tokens, int32_t* out_len, int32_t* path, int32_t* new_len) {
+    if (pass_status != 0) {
+        *out_len = 0;
+        *new_len = committed;
+        return;
+    }
+    uint64_t ok_lo = 1ull, ok_hi = 0ull;   // approved set; the root always is
+    int deepest = 0, deepest_depth = 0;
+    for (int i = 1; i < T; ++i) {
+        const int p = s_par[i];
+        const bool p_ok = p < 64 ? (ok_lo >> p) & 1 : (ok_hi >> (p - 64)) & 1;
+        if (p_ok && s_tok[i] == s_best[p]) {
+            if (i < 64) ok_lo |= 1ull << i; else ok_hi |= 1ull << (i - 64);
+            const int d = s_dep[i];
+            if (d > deepest_depth) { deepest_depth = d; deepest = i; }
+        }
+    }
+    // path[j] for j = depth .. 0 by climbing; the node at depth j is path element j
+    int cur = deepest;
+    for (int j = deepest_depth; j >= 0; --j) {
+        path[j] = cur;
+        out_tokens[j] = s_best[cur];
+        cur = s_par[cur];
+    }
+    *out_len = deepest_depth + 1;
+    *new_len = committed + deepest_depth + 1;
+}
+
 struct SeqMeta {
     int32_t* row_off;  // [B+1] first row of each sequence
     int32_t* path;     // [B][ADED_MAX_NODES] accepted path (local node indices), root first
     int32_t* new_len;  // [B] committed length after this call
 };
 
+}  // namespace aded
+
+namespace aded {
+// What the weight-streaming GEMM leaves behind (gemm_ws.cu): the partial tiles alone, or also -- the LM
+// head -- per-row greedy candidates of every tile, reduced in the kernel's tail.
+enum { WS_EPI_SLOTS = 0, WS_EPI_ARGMAX = 1 };
+struct WsEpilogue {
+    int mode;
+    const TileRef* tiles;        // contributors of every tile
+    uint32_t* counters;          // one arrival counter per tile; never reset: the epoch-th launch waits for
+    uint32_t epoch;              //   n x epoch arrivals (modulo 2^32)
+    float* cand_val; int32_t* cand_idx;   // best logit and its column per (row, tile): [R][n_tiles]
+};
 }  // namespace aded
 
 struct aded_kv {
@@ -149,6 +219,7 @@ struct aded_model {
 
     bool att_mma;       // bf16 models: tensor-core split-KV attention kernel
     bool att_tc;        // bf16 models with head_dim 128: the tcgen05 attention kernel (tree_attention_tc.cu)
+    bool att_tc_ok;     // the tcgen05 kernel can be used (aded_debug_attention_kernel switches between the two)
     CUtensorMap att_q_map;   // TMA descriptor of q for it
 
     // tensor-core GEMM path (bf16 models): TMA descriptors and split-tile scratch
@@ -156,32 +227,17 @@ struct aded_model {
     std::vector<CUtensorMap> ws_maps;   // per layer: wqkv, wo, wgu, wd; then lm_head; then x, attn, act
     float* ws_slots;                    // partial result tiles (see gemm_out.cuh)
     aded::TileRef* ws_tiles[5];         // contributor tables of the wqkv, wo, wgu, wd and LM-head results
-
-    // persistent projection kernel (fused_ws.cu): passes of at most 128 rows
-    bool fw_ready;
-    CUtensorMap* fw_maps;               // device copy of ws_maps
-    uint32_t* fw_counters;              // [FW_COUNTERS] grid-barrier counters, zeroed at the start of a pass
+    uint32_t* ws_counters;              // arrival counters of the LM head's tail, one per tile
+    uint32_t ws_epoch;                  // LM-head launches with a tail so far (host side of the counters)
+    float* cand_val;                    // [R][vocab / 128] per-tile greedy candidates of the LM head
+    int32_t* cand_idx;
 
     float* norm_ssq;        // [R][32] per-chunk sums of squares of the RMSNorm kernel
     int32_t* norm_count;    // [R] chunk arrival counters, zero between launches
     float* argmax_val;      // [R][ARGMAX_CHUNKS] best logit of each column chunk
     int32_t* argmax_idx;
 
-    // captured launch sequences, one per call shape (see model.cu)
-    struct GraphEntry {
-        std::vector<int64_t> key;
-        cudaGraphExec_t exec;
-        int32_t* offsets_pin;     // pinned copy of the row offsets the graph uploads
-        uint64_t last_use;
-        std::vector<aded::ProfSpan> spans;   // event pairs recorded by the graph (profiling variant only)
-    };
-    std::vector<GraphEntry> graphs;
-    uint64_t graph_clock;
-    bool graphs_on;
-
     bool prof_on;
-    std::vector<aded::ProfSpan>* capture_spans;   // while a profiling graph is being captured: where its spans go
-    int prof_pending;                             // index of the graph whose last replay's events are unread, or -1
     float prof_ms[aded::PROF_GROUPS];             // harvested so far
     int32_t prof_n[aded::PROF_GROUPS];
     std::vector<aded::ProfSpan> prof_spans;   // spans recorded by direct launches since aded_profile_begin
@@ -203,8 +259,9 @@ void launch_rope_table(aded_model* m, int rows, cudaStream_t st);
 void launch_add_rmsnorm(aded_model* m, const GemmOut* y, const void* gain, int rows, cudaStream_t st);
 // w_map / x_map: indices into m->ws_maps of the operands' TMA descriptors (-1: none, plain kernel).
 // `y` is the fp32 buffer the plain kernel writes; the returned descriptor says where the result is.
+// `epi_mode` (WS_EPI_*): whether the tensor-core kernel's tail also leaves per-tile greedy candidates (LM head).
 GemmOut launch_gemm(aded_model* m, int w_map, int x_map, const void* x, const void* w, float* y, int rows, int n, int k,
-                    cudaStream_t st);
+                    int epi_mode, int trace_kind, cudaStream_t st);
 void launch_rope_kv(aded_model* m, aded_kv* kv, const GemmOut& qkv, int layer, int rows, cudaStream_t st);
 void launch_swiglu(aded_model* m, const GemmOut& gu, int rows, cudaStream_t st);
 void launch_argmax(aded_model* m, const GemmOut& logits, int rows, cudaStream_t st);
@@ -214,10 +271,12 @@ void launch_materialize(aded_model* m, const GemmOut& src, float* dst, int rows,
 // dense_ws.cu: bf16 consumers of slot-resident projection results
 void launch_add_rmsnorm_ws(aded_model* m, const GemmOut& y, const void* gain, int rows, cudaStream_t st);
 void launch_swiglu_ws(aded_model* m, const GemmOut& gu, int rows, cudaStream_t st);
+void launch_rope_kv_ws(aded_model* m, aded_kv* kv, const GemmOut& qkv, int layer, int rows, cudaStream_t st);
 bool embed_norm_ws_supported(const aded_model* m);
 // embedding lookup and the first RMSNorm in one kernel
 void launch_embed_norm_ws(aded_model* m, const void* gain, int rows, cudaStream_t st);
-void launch_rope_kv_ws(aded_model* m, aded_kv* kv, const GemmOut& qkv, int layer, int rows, cudaStream_t st);
+// greedy token per row from the LM head's per-tile candidates, then the approval walk (one launch)
+void launch_pick_accept(aded_model* m, aded_kv* kv, int batch, int n_tiles, cudaStream_t st);
 
 // gemm_ws.cu
 bool ws_make_map(CUtensorMap* map, const void* ptr, uint64_t rows, uint64_t cols, uint32_t box_rows);
@@ -228,12 +287,9 @@ int ws_grid_limit(int device);
 int ws_grid(int device, int n, int k);
 size_t ws_slot_floats(int device, int max_n, int max_rows);
 cudaError_t ws_launch(const CUtensorMap& map_w, const CUtensorMap& map_x, int rows, int row0, int n, int k,
-                      float* slots, int32_t* status, int device, cudaStream_t st);
+                      float* slots, int32_t* status, const WsEpilogue& epi, int trace_kind, int device, cudaStream_t st);
 enum { WS_MAP_QKV = 0, WS_MAP_O = 1, WS_MAP_GU = 2, WS_MAP_D = 3 };   // per-layer map order
-
-// fused_ws.cu
-bool fw_prepare(int device);
-cudaError_t fw_launch(aded_model* m, aded_kv* kv, const FwPair* pairs, int n_pairs, int rows, int launch_index, cudaStream_t st);
+cudaError_t ws_wait_probe(int which, long long limit_cycles, const uint32_t* never_raised, int32_t* status, cudaStream_t st);
 
 // sample.cu
 bool sample_supported(int vocab);

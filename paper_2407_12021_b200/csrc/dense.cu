@@ -5,6 +5,8 @@
 // Rounding: activations are stored in the model dtype (bf16 models round to nearest even at
 // every store below); all sums are fp32.  Kernels that consume a projection read it through
 // GemmOut (gemm_out.cuh): either a plain fp32 matrix or per-CTA partial tiles added in CTA order.
+// These are the kernels of fp32 models; bf16 models on the tensor-core path use the four-columns-per-thread
+// versions in dense_ws.cu.
 #include "aded_internal.cuh"
 
 namespace aded {
@@ -30,6 +32,7 @@ template <typename T>
 __global__ void k_embed(const T* __restrict__ table, const CallPtrs* __restrict__ call, T* __restrict__ h,
                         int d, const int32_t* status) {
     pdl_enter();
+    if (first_thread_of_grid()) trace_mark(status, TK_OTHER);
     if (*status != 0) return;
     const int32_t* __restrict__ tokens = call->tokens;
     const int r = blockIdx.x;
@@ -42,6 +45,7 @@ __global__ void k_embed(const T* __restrict__ table, const CallPtrs* __restrict_
 __global__ void k_rope_table(const int32_t* __restrict__ pos, float* __restrict__ cs, float* __restrict__ sn,
                              int half, double theta, const int32_t* status) {
     pdl_enter();
+    if (first_thread_of_grid()) trace_mark(status, TK_OTHER);
     if (*status != 0) return;
     const int r = blockIdx.x;
     for (int i = threadIdx.x; i < half; i += blockDim.x) {
@@ -63,6 +67,7 @@ __global__ void __launch_bounds__(256) k_add_rmsnorm(T* __restrict__ h, GemmOut 
                                                      T* __restrict__ x, int d, float eps, float* __restrict__ ssq,
                                                      int32_t* __restrict__ row_count, const int32_t* status) {
     pdl_enter();
+    if (first_thread_of_grid()) trace_mark(status, TK_NORM);
     if (*status != 0) return;
     __shared__ float red[32];
     __shared__ int s_last;
@@ -117,8 +122,9 @@ __global__ void __launch_bounds__(256) k_add_rmsnorm(T* __restrict__ h, GemmOut 
 template <typename T>
 __global__ void __launch_bounds__(256) k_gemm_plain(const T* __restrict__ x, const T* __restrict__ w,
                                                     float* __restrict__ y, int rows, int n, int k,
-                                                    const int32_t* status) {
+                                                    const int32_t* status, int trace_kind) {
     pdl_enter();
+    if (first_thread_of_grid()) trace_mark(status, trace_kind);
     if (*status != 0) return;
     __shared__ float sx[16][64 + 4];
     __shared__ float sw[16][64 + 4];
@@ -162,6 +168,7 @@ __global__ void k_rope_kv(GemmOut qkv, const float* __restrict__ cs, const float
                           const int32_t* __restrict__ len, const int32_t* __restrict__ row_seq,
                           const int32_t* __restrict__ row_local, int layer, int H, int hd, const int32_t* status) {
     pdl_enter();
+    if (first_thread_of_grid()) trace_mark(status, TK_ROPE);
     if (*status != 0) return;
     const int r = blockIdx.x, hh = blockIdx.y, half = hd >> 1, d = H * hd;
     const int b = row_seq[r];
@@ -193,6 +200,7 @@ __global__ void k_rope_kv(GemmOut qkv, const float* __restrict__ cs, const float
 template <typename T>
 __global__ void k_swiglu(GemmOut gu, T* __restrict__ act, int F, const int32_t* status) {
     pdl_enter();
+    if (first_thread_of_grid()) trace_mark(status, TK_SWIGLU);
     if (*status != 0) return;
     const int r = blockIdx.y;
     const int c = blockIdx.x * blockDim.x + threadIdx.x;
@@ -207,6 +215,7 @@ __global__ void k_swiglu(GemmOut gu, T* __restrict__ act, int F, const int32_t* 
 __global__ void __launch_bounds__(256) k_argmax_chunks(GemmOut logits, float* __restrict__ pv, int32_t* __restrict__ pi,
                                                        int V, int chunk, const int32_t* status) {
     pdl_enter();
+    if (first_thread_of_grid()) trace_mark(status, TK_PICK);
     if (*status != 0) return;
     __shared__ float sv[8];
     __shared__ int si[8];
@@ -248,6 +257,7 @@ __global__ void __launch_bounds__(256) k_argmax_chunks(GemmOut logits, float* __
 __global__ void k_argmax_final(const float* __restrict__ pv, const int32_t* __restrict__ pi, int32_t* __restrict__ best,
                                int chunks, int rows, const int32_t* status) {
     pdl_enter();
+    if (first_thread_of_grid()) trace_mark(status, TK_PICK);
     if (*status != 0) return;
     const int r = blockIdx.x * blockDim.x + threadIdx.x;
     if (r >= rows) return;
@@ -263,6 +273,7 @@ __global__ void k_argmax_final(const float* __restrict__ pv, const int32_t* __re
 
 __global__ void k_materialize(GemmOut src, float* __restrict__ dst, int n, const int32_t* status) {
     pdl_enter();
+    if (first_thread_of_grid()) trace_mark(status, TK_OTHER);
     if (*status != 0) return;
     const int r = blockIdx.y;
     const int c = blockIdx.x * blockDim.x + threadIdx.x;
@@ -295,32 +306,41 @@ void launch_add_rmsnorm(aded_model* m, const GemmOut* y, const void* gain, int r
              (launch_k(k_add_rmsnorm<float>, grid, 256, 0, st, (float*)m->h, yy, has, (const float*)gain, (float*)m->x, d, m->cfg.rms_eps, m->norm_ssq, m->norm_count, m->status)));
 }
 
-static void launch_gemm_plain(aded_model* m, const void* x, const void* w, float* y, int rows, int n, int k, cudaStream_t st) {
+static void launch_gemm_plain(aded_model* m, const void* x, const void* w, float* y, int rows, int n, int k, int trace_kind,
+                              cudaStream_t st) {
     dim3 grid((n + 63) / 64, (rows + 63) / 64);
-    BY_DTYPE(m, (launch_k(k_gemm_plain<bf16>, grid, 256, 0, st, (const bf16*)x, (const bf16*)w, y, rows, n, k, m->status)),
-             (launch_k(k_gemm_plain<float>, grid, 256, 0, st, (const float*)x, (const float*)w, y, rows, n, k, m->status)));
+    BY_DTYPE(m, (launch_k(k_gemm_plain<bf16>, grid, 256, 0, st, (const bf16*)x, (const bf16*)w, y, rows, n, k, m->status, trace_kind)),
+             (launch_k(k_gemm_plain<float>, grid, 256, 0, st, (const float*)x, (const float*)w, y, rows, n, k, m->status, trace_kind)));
 }
 
 GemmOut launch_gemm(aded_model* m, int w_map, int x_map, const void* x, const void* w, float* y, int rows, int n, int k,
-                    cudaStream_t st) {
+                    int epi_mode, int trace_kind, cudaStream_t st) {
     GemmOut out = {};
     out.n = n;
     out.rows = rows;
     if (m->ws_ready && w_map >= 0 && x_map >= 0 && ws_supported(n, k)) {
         // tensor-core path, 128 rows of x per pass over the weights; the result stays in slots
+        const int table = w_map < 4 * m->cfg.n_layers ? w_map % 4 : 4;
+        WsEpilogue e = {};
+        e.mode = epi_mode;
+        e.tiles = m->ws_tiles[table];
+        e.counters = m->ws_counters;
+        e.cand_val = m->cand_val;
+        e.cand_idx = m->cand_idx;
         for (int row0 = 0; row0 < rows; row0 += 128) {
             const int part = rows - row0 < 128 ? rows - row0 : 128;
-            ws_launch(m->ws_maps[w_map], m->ws_maps[x_map], part, row0, n, k, m->ws_slots, m->status, m->device, st);
+            if (epi_mode != WS_EPI_SLOTS) e.epoch = ++m->ws_epoch;
+            ws_launch(m->ws_maps[w_map], m->ws_maps[x_map], part, row0, n, k, m->ws_slots, m->status, e, trace_kind, m->device, st);
         }
         out.mode = 1;
         out.slots = m->ws_slots;
         out.n_tiles = n / 128;
         out.kb = k / 64;
         out.g = ws_grid(m->device, n, k);
-        out.tiles = m->ws_tiles[w_map < 4 * m->cfg.n_layers ? w_map % 4 : 4];
+        out.tiles = m->ws_tiles[table];
         return out;
     }
-    launch_gemm_plain(m, x, w, y, rows, n, k, st);
+    launch_gemm_plain(m, x, w, y, rows, n, k, trace_kind, st);
     out.mode = 0;
     out.y = y;
     return out;

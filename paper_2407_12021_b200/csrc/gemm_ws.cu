@@ -1,5 +1,6 @@
 // Weight-streaming bf16 GEMM for the decoder's projections, FFN and LM head on the 5th-generation
-// tensor cores (tcgen05, accumulators in TMEM, operands staged by TMA).
+// tensor cores (tcgen05, accumulators in TMEM, operands staged by TMA), with the step that consumes
+// each projection folded into the kernel's tail.
 //
 //   y[r, n] = sum_k x[r, k] * w[n, k]        r < rows <= 128,  w row-major [N, K], x row-major [R, K]
 //
@@ -11,17 +12,27 @@
 //   * work = (W tile, k block) units, split evenly over all resident CTAs (two per SM), so every CTA
 //     streams the same number of bytes whatever N and K are; a CTA's range covers the tail of one
 //     tile, whole tiles, and the head of another;
-//   * a CTA stores the fp32 partial tile of each of its segments to a slot; the kernel that consumes
-//     the result adds a tile's slots in CTA order -- a fixed order, so results do not depend on
-//     timing, and the GEMM itself ends without counters, fences or dependent reads;
+//   * a CTA stores the fp32 partial tile of each of its segments to a slot (gemm_out.cuh); the kernel
+//     that consumes the result (rotary/K-V write, residual add + RMSNorm, SwiGLU) adds a tile's slots
+//     in CTA order -- a fixed order, so results do not depend on timing -- and the GEMM itself ends
+//     without counters, fences or dependent reads.  The consumers are small kernels of their own on
+//     purpose: while one runs, the next projection's CTAs are already resident and stream their
+//     first W tiles.  (Measured on a 32-layer step: folding the consumers into this kernel's tail,
+//     the contributors of a tile meeting at a counter, made every projection 7-9 us longer for a
+//     consumer kernel of 4-8 us saved, because the next projection then starts cold.)
+//   * the LM head alone has such a tail (template parameter): the CTAs that contributed to a tile meet
+//     at a counter in global memory and each reduces a share of the tile's rows to per-row greedy
+//     candidates (best logit of the tile's 128 columns), so the [rows, vocab] logits are never
+//     gathered by a later kernel.  All CTAs of a launch are resident at once (at most two per SM
+//     are launched), so the meeting cannot deadlock; the wait is bounded all the same.  The counters
+//     are never reset: launch number e waits for n x e arrivals (arithmetic modulo 2^32);
 //   * the kernel is launched with programmatic dependent launch: its blocks become resident while
 //     the previous kernel drains, set up barriers and TMEM, and already stream their first W tiles;
-//     only the loads of x wait for the previous kernel.  (Also tried: TMA L2 prefetches of the next
-//     projection's first tiles at the end of the kernel -- no measurable gain, removed.)
-//   * warp 0 issues TMA loads, warp 1 issues MMAs, warps 2..5 drain TMEM and run the epilogue; two
-//     TMEM accumulators let the MMAs of the next segment run under the epilogue of the last.
-// Every mbarrier wait is bounded; a wait that runs out raises ADED_ERR_TIMEOUT in the status word
-// and the CTA unwinds (drains its own copies, frees TMEM).
+//     only the loads of x wait for the previous kernel;
+//   * warp 0 issues TMA loads, warp 1 issues MMAs, warps 2..5 drain TMEM; two TMEM accumulators let
+//     the MMAs of the next segment run under the drain of the last; all six warps run the LM head's tail.
+// Every wait is bounded; a wait that runs out raises ADED_ERR_TIMEOUT in the status word and the
+// CTA unwinds (drains its own copies, frees TMEM).
 #include <cuda.h>
 
 #include <cstdio>
@@ -35,6 +46,8 @@ namespace aded {
 constexpr int WS_BM = 128;           // W rows per tile (MMA M)
 constexpr int WS_BK = 64;            // k elements per stage (128 bytes of bf16)
 constexpr int WS_THREADS = 192;
+constexpr long long WS_MEET_CYCLES = 400000000ll;   // about 0.2 s of SM clock: limit of the wait at a counter
+constexpr int WS_GMAX = 16;          // tile groups of a CTA handled per round of its tail
 
 struct WsParams {
     int rows;            // valid rows of x
@@ -44,12 +57,79 @@ struct WsParams {
     int n_tiles, kb;     // tiles of 128 W rows, k blocks per tile
     int stages;
     int tmem_cols;       // power of two >= 2 * rb
+    int trace_kind;
+    int narrow;          // units * (CTAs + 1) < 2^31: the work split can be computed in 32-bit arithmetic
     float* slots;        // this row block's slot region: [n_tiles + gridDim.x][rb][128] fp32
     int32_t* status;
+    WsEpilogue epi;
 };
 
+// Waits until the counter has reached `target` (arrivals are counted modulo 2^32 and never reset).
+__device__ __forceinline__ bool ws_poll(const uint32_t* counter, uint32_t target, long long limit = WS_MEET_CYCLES) {
+    const long long t0 = clock64();
+    for (uint32_t spin = 0;; ++spin) {
+        uint32_t v;
+        asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(counter) : "memory");
+        if ((int32_t)(v - target) >= 0) return true;
+        if ((spin & 63) == 63 && clock64() - t0 > limit) return false;
+    }
+}
+__device__ __forceinline__ void ws_arrive(uint32_t* counter) {
+    asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(counter) : "memory");
+}
+// ws_owner (gemm_out.cuh) in 32-bit arithmetic when the products fit.
+__device__ __forceinline__ int ws_owner_dev(long long u, long long units, long long G, bool narrow) {
+    if (!narrow) return ws_owner(u, units, G);
+    const int u32 = (int)u, n32 = (int)units, g32 = (int)G;
+    int c = ((u32 + 1) * g32 - 1) / n32;
+    if (c >= g32) c = g32 - 1;
+    while (c > 0 && c * n32 / g32 > u32) --c;
+    while (c + 1 < g32 && (c + 1) * n32 / g32 <= u32) ++c;
+    return c;
+}
+
+// Sum of a tile's slots (CTA order) for four adjacent columns of local row r.
+__device__ __forceinline__ float4 ws_sum4(const float* slots, const TileRef& t, int rb, int r, int col) {
+    const float* p = slots + ((size_t)t.first_slot * rb + r) * WS_BM + col;
+    const size_t stride = (size_t)rb * WS_BM;
+    float4 sum = make_float4(0.f, 0.f, 0.f, 0.f);
+    constexpr int B = 12;
+    for (int i0 = 0; i0 < t.count; i0 += B) {
+        float4 v[B];
+#pragma unroll
+        for (int j = 0; j < B; ++j)
+            v[j] = i0 + j < t.count ? __ldcg(reinterpret_cast<const float4*>(p + (size_t)(i0 + j) * stride)) : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+        for (int j = 0; j < B; ++j)
+            if (i0 + j < t.count) sum = f4_add(sum, v[j]);
+    }
+    return sum;
+}
+
+// LM head: a warp per row; the best (value, lowest column) of the tile's 128 logits goes to
+// cand_val / cand_idx [row][tile].
+__device__ __forceinline__ void ws_row_argmax(const WsParams& p, const TileRef& t, int vt, int r, int lane, bool store) {
+    const float4 v = ws_sum4(p.slots, t, p.rb, r, lane * 4);
+    float bv = v.x;
+    int bi = vt * WS_BM + lane * 4;
+    if (v.y > bv) { bv = v.y; bi = vt * WS_BM + lane * 4 + 1; }
+    if (v.z > bv) { bv = v.z; bi = vt * WS_BM + lane * 4 + 2; }
+    if (v.w > bv) { bv = v.w; bi = vt * WS_BM + lane * 4 + 3; }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
+        const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+        if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
+    }
+    if (lane == 0 && store) {
+        p.epi.cand_val[(size_t)(p.row0 + r) * p.n_tiles + vt] = bv;
+        p.epi.cand_idx[(size_t)(p.row0 + r) * p.n_tiles + vt] = bi;
+    }
+}
+
+template <bool TAIL>
 __global__ void __launch_bounds__(WS_THREADS, 2)
-k_gemm_ws(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_x, WsParams p) {
+k_gemm_ws(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_x, const __grid_constant__ WsParams p) {
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     // carve: stages x (W tile 16 KB | x tile rb*128 B), then barriers
     uint8_t* base = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
@@ -60,7 +140,7 @@ k_gemm_ws(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUt
     uint64_t* acc_full = bars + 2 * p.stages;
     uint64_t* acc_empty = acc_full + 2;
     uint32_t* s_tmem = (uint32_t*)(acc_empty + 2);
-    volatile int* s_flag = (volatile int*)(s_tmem + 1);   // [0] abort, [2] live
+    volatile int* s_flag = (volatile int*)(s_tmem + 1);   // [0] abort, [2] live, [3] meeting result
 
     pdl_launch_dependents();   // the next kernel may start its preamble; it waits for this one's results itself
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -74,6 +154,7 @@ k_gemm_ws(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUt
         s_flag[0] = 0;
         s_flag[1] = 0;
         s_flag[2] = *p.status == 0;
+        s_flag[3] = 1;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
@@ -105,6 +186,7 @@ k_gemm_ws(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUt
                 tma_load_2d_hint(&map_w, &full[i], base + (size_t)i * stage_bytes, kb * WS_BK, tile * WS_BM, pol_stream);
             }
             pdl_wait();
+            if (blockIdx.x == 0) trace_mark(p.status, p.trace_kind);
             for (int i = 0; i < ahead; ++i) {
                 const int kb = (int)((u0 + i) % p.kb);
                 uint8_t* sb = base + (size_t)i * stage_bytes + a_bytes;
@@ -166,9 +248,8 @@ k_gemm_ws(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUt
             if (!ok && lane == 0) { s_flag[0] = 1; atomicCAS(p.status, 0, (int)ADED_ERR_TIMEOUT); }
         }
     } else {
-        // ---------------- epilogue: warps 2..5, TMEM lane quarter = warp % 4 ----------------
-        // Every segment's partial tile goes to slot (tile + CTA); the consumer of the result adds a
-        // tile's slots in CTA order (see gemm_out.cuh).
+        // ---------------- drain: warps 2..5, TMEM lane quarter = warp % 4 ----------------
+        // Every segment's partial tile goes to slot (tile + CTA).
         const int quarter = warp & 3;
         const int row_in_tile = quarter * 32 + lane;           // W row inside the tile = TMEM lane
         int seg = 0;
@@ -197,8 +278,66 @@ k_gemm_ws(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUt
         }
     }
 
-    // ---------------- teardown ----------------
+    // ---------------- tail (LM head): per-row greedy candidates of the tiles this CTA contributed to ----------------
+    // A tile's contributors are the consecutive CTAs whose unit ranges meet it.  Each publishes its partial
+    // tiles (fence, then one arrival at every tile's counter), waits until all have arrived at its tiles,
+    // and reduces a contiguous share of each tile's rows, a warp per row.
     tc_fence_before();
+    __syncthreads();
+    if (TAIL && u1 > u0) {
+        // (A CTA that found the pass already failed when it started has computed nothing; it still arrives
+        // at its counters, so that the others do not wait for it and the counts stay whole.)
+        __shared__ int s_r0[WS_GMAX], s_item0[WS_GMAX + 1], s_ok;
+        __shared__ TileRef s_tile[WS_GMAX];
+        pdl_wait();                                  // (satisfied long ago; every thread now sees the previous kernels' writes)
+        const bool store = live && *p.status == 0 && s_flag[0] == 0;
+        const bool narrow = p.narrow != 0;
+        const long long gu = p.kb;                   // units per tile
+        const int g0 = (int)(u0 / gu), g1 = (int)((u1 - 1) / gu);
+        __threadfence();
+        __syncthreads();
+        // arrive at every tile first: a CTA that waited at its first tile before announcing itself at its
+        // second would chain the tiles of the whole launch one behind the other
+        for (int g = g0 + (int)threadIdx.x; g <= g1; g += WS_THREADS)
+            if (ws_owner_dev(g * gu, units, G, narrow) != ws_owner_dev((g + 1) * gu - 1, units, G, narrow)) ws_arrive(p.epi.counters + g);
+        bool all_met = true;
+        for (int gs = g0; gs <= g1 && all_met; gs += WS_GMAX) {
+            const int ng = g1 - gs + 1 < WS_GMAX ? g1 - gs + 1 : WS_GMAX;
+            if (threadIdx.x == 0) s_ok = 1;
+            __syncthreads();
+            if ((int)threadIdx.x < ng) {
+                // one thread per tile: who contributes, this CTA's share of the rows, and the wait
+                const int g = gs + (int)threadIdx.x;
+                const int cf = ws_owner_dev(g * gu, units, G, narrow), cl = ws_owner_dev((g + 1) * gu - 1, units, G, narrow);
+                const int n = cl - cf + 1, rank = (int)blockIdx.x - cf;
+                const int r0 = rank * p.rows / n, r1 = (rank + 1) * p.rows / n;
+                s_r0[threadIdx.x] = r0;
+                s_item0[threadIdx.x + 1] = r1 - r0;
+                s_tile[threadIdx.x] = p.epi.tiles[g];
+                if (n > 1 && live && !ws_poll(p.epi.counters + g, (uint32_t)n * p.epi.epoch)) s_ok = 0;
+            }
+            __syncthreads();
+            if (threadIdx.x == 0) {
+                s_item0[0] = 0;
+                for (int i = 0; i < ng; ++i) s_item0[i + 1] += s_item0[i];
+            }
+            __syncthreads();
+            if (s_ok == 0) {
+                if (threadIdx.x == 0) { s_flag[0] = 1; atomicCAS(p.status, 0, (int)ADED_ERR_TIMEOUT); }
+                all_met = false;
+            } else if (live) {
+                const int total = s_item0[ng];
+                for (int it = warp; it < total; it += WS_THREADS / 32) {
+                    int gi = 0;
+                    while (it >= s_item0[gi + 1]) ++gi;
+                    ws_row_argmax(p, s_tile[gi], gs + gi, s_r0[gi] + it - s_item0[gi], lane, store);
+                }
+            }
+            __syncthreads();
+        }
+    }
+
+    // ---------------- teardown ----------------
     __syncthreads();
     if (warp == 0 && lane == 0 && s_flag[0]) {
         // unwinding after a timeout: give copies that are still in flight time to land (bounded)
@@ -209,6 +348,27 @@ k_gemm_ws(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUt
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)p.tmem_cols) : "memory");
     }
+}
+
+// One warp runs the library's two kinds of bounded device-side wait on something that never happens -- an
+// mbarrier nobody arrives at, an arrival counter nobody raises -- with a caller-chosen limit, and reports
+// the outcome the way the kernels above do: ADED_ERR_TIMEOUT in the status word.  `which`: 0 mbarrier, 1 counter.
+__global__ void k_wait_probe(int which, long long limit_cycles, const uint32_t* never_raised, int32_t* status) {
+    __shared__ uint64_t bar;
+    if (threadIdx.x == 0) {
+        mbar_init(&bar, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncwarp();
+    bool ok;
+    if (which == 0) ok = __all_sync(0xffffffffu, mbar_wait(&bar, 0, limit_cycles));
+    else ok = ws_poll(never_raised, 0x40000000u, limit_cycles);
+    if (!ok && threadIdx.x == 0) atomicCAS(status, 0, (int)ADED_ERR_TIMEOUT);
+}
+
+cudaError_t ws_wait_probe(int which, long long limit_cycles, const uint32_t* never_raised, int32_t* status, cudaStream_t st) {
+    k_wait_probe<<<1, 32, 0, st>>>(which, limit_cycles, never_raised, status);
+    return cudaGetLastError();
 }
 
 // ---- host side --------------------------------------------------------------------------------
@@ -267,16 +427,17 @@ size_t ws_slot_floats(int device, int max_n, int max_rows) {
 
 // Raises the kernel's dynamic shared-memory limit; once per process, before any launch or capture.
 bool ws_prepare() {
-    return cudaFuncSetAttribute(k_gemm_ws, cudaFuncAttributeMaxDynamicSharedMemorySize, 112 * 1024) == cudaSuccess;
+    return cudaFuncSetAttribute(k_gemm_ws<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 112 * 1024) == cudaSuccess &&
+           cudaFuncSetAttribute(k_gemm_ws<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 112 * 1024) == cudaSuccess;
 }
 
 // Shapes the tensor-core path takes.
 bool ws_supported(int n, int k) { return n % WS_BM == 0 && k % WS_BK == 0 && k >= WS_BK; }
 
 // One pass: rows [row0, row0 + rows) of x (rows <= 128) against all of W.  Partial tiles go to the
-// slot region of row block row0 / 128.
+// slot region of row block row0 / 128; `epi` says whether the kernel's tail reduces them to greedy candidates.
 cudaError_t ws_launch(const CUtensorMap& map_w, const CUtensorMap& map_x, int rows, int row0, int n, int k,
-                      float* slots, int32_t* status, int device, cudaStream_t st) {
+                      float* slots, int32_t* status, const WsEpilogue& epi, int trace_kind, int device, cudaStream_t st) {
     WsParams p;
     p.rows = rows;
     p.rb = (rows + 15) / 16 * 16;
@@ -292,11 +453,15 @@ cudaError_t ws_launch(const CUtensorMap& map_w, const CUtensorMap& map_x, int ro
     if (p.stages > 8) p.stages = 8;
     p.tmem_cols = 32;
     while (p.tmem_cols < 2 * p.rb) p.tmem_cols *= 2;
+    p.trace_kind = trace_kind;
     const int grid = ws_grid(device, n, k);
+    p.narrow = (long long)p.n_tiles * p.kb * (grid + 1) < (1ll << 31);
     p.slots = slots + (size_t)(row0 / 128) * (size_t)(p.n_tiles + grid) * 128 * WS_BM;
     p.status = status;
+    p.epi = epi;
     const size_t smem = (size_t)p.stages * stage_bytes + 1024 + 256;
-    return launch_k(k_gemm_ws, dim3(grid), dim3(WS_THREADS), smem, st, map_w, map_x, p);
+    if (epi.mode == WS_EPI_ARGMAX) return launch_k(k_gemm_ws<true>, dim3(grid), dim3(WS_THREADS), smem, st, map_w, map_x, p);
+    return launch_k(k_gemm_ws<false>, dim3(grid), dim3(WS_THREADS), smem, st, map_w, map_x, p);
 }
 
 }  // namespace aded

@@ -102,10 +102,10 @@ extern "C" aded_status aded_greedy_noalloc(const float* logits_dev, int32_t rows
     const aded_status s = na_scratch_address(&scratch);
     if (s != ADED_OK) return s;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    const int chunk = (vocab + NA_CHUNKS - 1) / NA_CHUNKS;
-    note_launch(2);
+    const int chunk = (int)(((long long)vocab + NA_CHUNKS - 1) / NA_CHUNKS);      // (64-bit: vocab may be close to INT_MAX)
     k_na_chunks<<<dim3(NA_CHUNKS, rows), 256, 0, st>>>(logits_dev, scratch, vocab, chunk);
     k_na_final<<<(rows + 127) / 128, 128, 0, st>>>(scratch, out_best_dev, rows);
     ADED_CUDA_TRY(cudaGetLastError());
+    note_launch(2);
     return ADED_OK;
 }

@@ -18,11 +18,6 @@ void note_cuda_error(cudaError_t e, const char* what) {
     cudaGetLastError();
 }
 
-bool pdl_enabled() {
-    static const bool on = getenv("ADED_NO_PDL") == nullptr;
-    return on;
-}
-
 static std::atomic<uint64_t> g_launches{0};
 void note_launch(int n) { g_launches.fetch_add((uint64_t)n, std::memory_order_relaxed); }
 
@@ -41,13 +36,12 @@ struct Span {
             if (!m->prof_pool.empty()) { *e = m->prof_pool.back(); m->prof_pool.pop_back(); }
             else if (cudaEventCreate(e) != cudaSuccess) { on = false; cudaGetLastError(); return; }
         }
-        // inside a capture the record becomes a node of the graph and is timed on every replay
-        cudaEventRecordWithFlags(rec.a, st, m->capture_spans ? cudaEventRecordExternal : cudaEventRecordDefault);
+        cudaEventRecord(rec.a, st);
     }
     ~Span() {
         if (!on) return;
-        cudaEventRecordWithFlags(rec.b, st, m->capture_spans ? cudaEventRecordExternal : cudaEventRecordDefault);
-        (m->capture_spans ? *m->capture_spans : m->prof_spans).push_back(rec);
+        cudaEventRecord(rec.b, st);
+        m->prof_spans.push_back(rec);
     }
 };
 
@@ -86,7 +80,7 @@ static aded_status alloc_model(aded_model* m) {
     TRY(dev_alloc(m, &m->parents, R));
     TRY(dev_alloc(m, &m->out_tokens, R));
     TRY(dev_alloc(m, &m->out_len, B));
-    TRY(dev_alloc(m, &m->status, 1));
+    TRY(dev_alloc(m, &m->status, (size_t)STATUS_WORDS));
     TRY(dev_alloc(m, &m->rows.seq, R));
     TRY(dev_alloc(m, &m->rows.local, R));
     TRY(dev_alloc(m, &m->rows.depth, R));
@@ -102,22 +96,21 @@ static aded_status alloc_model(aded_model* m) {
     TRY(dev_alloc(m, &m->argmax_idx, R * ARGMAX_CHUNKS));
     ADED_CUDA_TRY(cudaMemset(m->norm_count, 0, R * sizeof(int32_t)));
     if (d > 32 * 256) return ADED_ERR_UNSUPPORTED;   // the norm kernel keeps at most 32 column chunks per row
-    ADED_CUDA_TRY(cudaMemset(m->status, 0, sizeof(int32_t)));
+    ADED_CUDA_TRY(cudaMemset(m->status, 0, STATUS_WORDS * sizeof(int32_t)));
     ADED_CUDA_TRY(cudaMemset(m->h, 0, R * d * m->elem));
     ADED_CUDA_TRY(cudaMemset(m->x, 0, R * d * m->elem));
     ADED_CUDA_TRY(cudaMemset(m->attn, 0, R * d * m->elem));
     ADED_CUDA_TRY(cudaMemset(m->act, 0, R * F * m->elem));
 
-    m->att_mma = c.dtype == ADED_BF16 && !getenv("ADED_PLAIN_ATTN") && attn_prepare();
-    // head_dim 128: the tcgen05 kernel (ADED_ATTN_MMA=1 keeps the mma.sync kernel, for comparisons)
-    m->att_tc = m->att_mma && attn_tc_supported(c) && !getenv("ADED_ATTN_MMA") && attn_tc_prepare() &&
-                ws_make_map(&m->att_q_map, m->q, R, d, 64);
+    m->att_mma = c.dtype == ADED_BF16 && attn_prepare();
+    // head_dim 128: the tcgen05 kernel (aded_debug_attention_kernel selects the mma.sync kernel, for comparisons)
+    m->att_tc_ok = m->att_mma && attn_tc_supported(c) && attn_tc_prepare() && ws_make_map(&m->att_q_map, m->q, R, d, 64);
+    m->att_tc = m->att_tc_ok;
 
     // tensor-core GEMM path: bf16 models whose every matrix tiles into 128-row x 64-column blocks
     m->ws_ready = false;
-    m->fw_ready = false;
-    if (c.dtype == ADED_BF16 && !getenv("ADED_PLAIN_GEMM") && ws_supported(3 * (int)d, (int)d) && ws_supported((int)d, (int)d) &&
-        ws_supported(2 * (int)F, (int)d) && ws_supported((int)d, (int)F) && ws_supported((int)V, (int)d)) {
+    if (c.dtype == ADED_BF16 && ws_supported(3 * (int)d, (int)d) && ws_supported((int)d, (int)d) && ws_supported(2 * (int)F, (int)d) &&
+        ws_supported((int)d, (int)F) && ws_supported((int)V, (int)d)) {
         const int L = c.n_layers;
         m->ws_maps.resize(4 * L + 4);
         bool ok = ws_prepare();
@@ -145,50 +138,28 @@ static aded_status alloc_model(aded_model* m) {
                 TRY(dev_alloc(m, &m->ws_tiles[i], (size_t)nt));
                 ADED_CUDA_TRY(cudaMemcpy(m->ws_tiles[i], table.data(), nt * sizeof(TileRef), cudaMemcpyHostToDevice));
             }
+            // the LM head's tail: one arrival counter per tile, per-tile greedy candidates of every row
+            TRY(dev_alloc(m, &m->ws_counters, V / 128));
+            ADED_CUDA_TRY(cudaMemset(m->ws_counters, 0, (V / 128) * sizeof(uint32_t)));
+            m->ws_epoch = 0;
+            TRY(dev_alloc(m, &m->cand_val, R * (V / 128)));
+            TRY(dev_alloc(m, &m->cand_idx, R * (V / 128)));
             m->ws_ready = true;
-            // persistent kernel (opt-in with ADED_FUSED=1 while it is slower than the separate kernels):
-            // device copy of the descriptors, barrier counters
-            if (getenv("ADED_FUSED") && d % 4 == 0 && (c.head_dim / 2) % 4 == 0 && fw_prepare(m->device)) {
-                TRY(dev_alloc(m, &m->fw_maps, m->ws_maps.size()));
-                ADED_CUDA_TRY(cudaMemcpy(m->fw_maps, m->ws_maps.data(), m->ws_maps.size() * sizeof(CUtensorMap), cudaMemcpyHostToDevice));
-                TRY(dev_alloc(m, &m->fw_counters, (size_t)2 * FW_COUNTERS));
-                ADED_CUDA_TRY(cudaMemset(m->fw_counters, 0, 2 * FW_COUNTERS * sizeof(uint32_t)));
-                m->fw_ready = true;
-            }
         }
     }
     return ADED_OK;
 }
 
-// The persistent projection kernel takes passes of at most 128 rows (one row block) with fewer
-// launches than barrier counters; the debug capture of the residual stream needs the layer-by-layer path.
-static bool use_fused(const aded_model* m, int rows) {
-    return m->fw_ready && rows <= 128 && !m->dbg_hidden && m->cfg.n_layers + 1 <= FW_COUNTERS;
-}
-
-// Kernels one pass launches (what enqueue_pass enqueues), for the launch counter of graph replays.
-static int pass_launches(const aded_model* m, int rows, int chain_mode) {
-    const int head = embed_norm_ws_supported(m) ? 3 : 4;
-    if (use_fused(m, rows)) return head + 1 + 2 * m->cfg.n_layers + (chain_mode ? 1 : 5);
-    const int gemm_passes = (rows + 127) / 128;   // the tensor-core GEMM runs once per 128 rows
-    const int per_gemm = m->ws_ready ? gemm_passes : 1;
-    int n = head + m->cfg.n_layers * (4 * per_gemm + 3 + 1);
-    n += chain_mode ? 1 : per_gemm + 5;
-    return n;
-}
-
-// The launch sequence of one pass over `rows` rows.  Everything it touches is owned by the handles
-// (the caller's arrays are reached through m->call_dev), so the sequence can be captured once per
-// call shape and replayed.  chain_mode: the rows form a chain per sequence, every row is accepted
-// and no logits are needed (prefill).
+// The launch sequence of one pass over `rows` rows.  chain_mode: the rows form a chain per sequence,
+// every row is accepted and no logits are needed (prefill).
 static aded_status enqueue_pass(aded_model* m, aded_kv* kv, const int32_t* offsets_src, int batch, int rows,
                                 int max_tree, int chain_mode, cudaStream_t st) {
     const aded_model_config& c = m->cfg;
     const int d = c.d_model, F = c.d_ffn;
     const int xm = 4 * c.n_layers + 1;   // TMA descriptor indices of x, attn, act
+    const bool ws = m->ws_ready;
     ADED_CUDA_TRY(cudaMemcpyAsync(m->seqs.row_off, offsets_src, (batch + 1) * sizeof(int32_t),
                                   cudaMemcpyHostToDevice, st));
-    if (use_fused(m, rows)) ADED_CUDA_TRY(cudaMemsetAsync(m->fw_counters, 0, 2 * FW_COUNTERS * sizeof(uint32_t), st));
     {
         const bool one = embed_norm_ws_supported(m);
         Span sp(m, PROF_OTHER, one ? 3 : 4, st);
@@ -203,90 +174,54 @@ static aded_status enqueue_pass(aded_model* m, aded_kv* kv, const int32_t* offse
     }
     const size_t hid_bytes = (size_t)rows * d * m->elem;
     if (m->dbg_hidden) ADED_CUDA_TRY(cudaMemcpyAsync(m->dbg_hidden, m->h, hid_bytes, cudaMemcpyDeviceToDevice, st));
-    const bool fused = use_fused(m, rows);
-    GemmOut fused_logits = {};
-    if (fused) {
-        // Persistent-kernel path: [QKV_0, rotary] | attention_0 | [O, norm, gate/up, SwiGLU, down, norm,
-        // QKV_1, rotary] | attention_1 | ... | [O, norm, gate/up, SwiGLU, down, final norm, LM head].
-        const int F2 = 2 * F;
-        auto pair = [&](int map_w, int map_x, int n, int k, int table, int post, int layer, const void* gain) {
-            FwPair pr;
-            pr.map_w = map_w;
-            pr.map_x = map_x;
-            pr.n_tiles = n / 128;
-            pr.kb = k / 64;
-            pr.tiles = m->ws_tiles[table];
-            pr.post = post;
-            pr.layer = layer;
-            pr.gain = gain;
-            return pr;
-        };
-        int launch_index = 0;
-        {
-            const FwPair first = pair(WS_MAP_QKV, xm, 3 * d, d, 0, FW_POST_ROPE_KV, 0, nullptr);
-            Span sp(m, PROF_GEMM, 1, st);
-            ADED_CUDA_TRY(fw_launch(m, kv, &first, 1, rows, launch_index++, st));
-            note_launch();
-        }
-        for (int l = 0; l < c.n_layers; ++l) {
-            const aded_layer_weights& w = m->layers[l];
-            { Span sp(m, PROF_ATTN, 1, st); launch_tree_attention(m, kv, l, batch, rows, max_tree, st); }
-            const bool last = l + 1 == c.n_layers;
-            FwPair prs[FW_MAX_PAIRS];
-            int np = 0;
-            prs[np++] = pair(4 * l + WS_MAP_O, xm + 1, d, d, 1, FW_POST_ADD_NORM, 0, w.norm2);
-            prs[np++] = pair(4 * l + WS_MAP_GU, xm, F2, d, 2, FW_POST_SWIGLU, 0, nullptr);
-            prs[np++] = pair(4 * l + WS_MAP_D, xm + 2, d, F, 3, FW_POST_ADD_NORM, 0, last ? m->top.final_norm : m->layers[l + 1].norm1);
-            if (!last) prs[np++] = pair(4 * (l + 1) + WS_MAP_QKV, xm, 3 * d, d, 0, FW_POST_ROPE_KV, l + 1, nullptr);
-            else if (!chain_mode) prs[np++] = pair(4 * c.n_layers, xm, c.vocab, d, 4, FW_POST_NONE, 0, nullptr);
-            Span sp(m, PROF_GEMM, 1, st);
-            ADED_CUDA_TRY(fw_launch(m, kv, prs, np, rows, launch_index++, st));
-            note_launch();
-        }
-        fused_logits.y = nullptr;
-        fused_logits.slots = m->ws_slots;
-        fused_logits.tiles = m->ws_tiles[4];
-        fused_logits.mode = 1;
-        fused_logits.n = c.vocab;
-        fused_logits.n_tiles = c.vocab / 128;
-        fused_logits.kb = d / 64;
-        fused_logits.g = ws_grid(m->device, c.vocab, d);
-        fused_logits.rows = rows;
-    }
-    for (int l = 0; l < c.n_layers && !fused; ++l) {
+    const int passes = ws ? (rows + 127) / 128 : 1;      // the tensor-core GEMM runs once per 128 rows
+    for (int l = 0; l < c.n_layers; ++l) {
         const aded_layer_weights& w = m->layers[l];
+        const void* next_gain = l + 1 < c.n_layers ? m->layers[l + 1].norm1 : m->top.final_norm;
+        auto wmap = [&](int which) { return ws ? 4 * l + which : -1; };      // TMA descriptor of a weight matrix (plain GEMM: none)
         GemmOut o;
-        { Span sp(m, PROF_GEMM, 1, st); o = launch_gemm(m, 4 * l + WS_MAP_QKV, xm, m->x, w.wqkv, m->y32, rows, 3 * d, d, st); }
+        { Span sp(m, PROF_GEMM, passes, st); o = launch_gemm(m, wmap(WS_MAP_QKV), ws ? xm : -1, m->x, w.wqkv, m->y32, rows, 3 * d, d, WS_EPI_SLOTS, TK_GEMM_QKV, st); }
         { Span sp(m, PROF_OTHER, 1, st); launch_rope_kv(m, kv, o, l, rows, st); }
         { Span sp(m, PROF_ATTN, 1, st); launch_tree_attention(m, kv, l, batch, rows, max_tree, st); }
-        { Span sp(m, PROF_GEMM, 1, st); o = launch_gemm(m, 4 * l + WS_MAP_O, xm + 1, m->attn, w.wo, m->y32, rows, d, d, st); }
+        { Span sp(m, PROF_GEMM, passes, st); o = launch_gemm(m, wmap(WS_MAP_O), ws ? xm + 1 : -1, m->attn, w.wo, m->y32, rows, d, d, WS_EPI_SLOTS, TK_GEMM_O, st); }
         { Span sp(m, PROF_OTHER, 1, st); launch_add_rmsnorm(m, &o, w.norm2, rows, st); }
-        { Span sp(m, PROF_GEMM, 1, st); o = launch_gemm(m, 4 * l + WS_MAP_GU, xm, m->x, w.wgu, m->y32, rows, 2 * F, d, st); }
+        { Span sp(m, PROF_GEMM, passes, st); o = launch_gemm(m, wmap(WS_MAP_GU), ws ? xm : -1, m->x, w.wgu, m->y32, rows, 2 * F, d, WS_EPI_SLOTS, TK_GEMM_GU, st); }
         { Span sp(m, PROF_OTHER, 1, st); launch_swiglu(m, o, rows, st); }
-        { Span sp(m, PROF_GEMM, 1, st); o = launch_gemm(m, 4 * l + WS_MAP_D, xm + 2, m->act, w.wd, m->y32, rows, d, F, st); }
-        const void* next_gain = l + 1 < c.n_layers ? m->layers[l + 1].norm1 : m->top.final_norm;
+        { Span sp(m, PROF_GEMM, passes, st); o = launch_gemm(m, wmap(WS_MAP_D), ws ? xm + 2 : -1, m->act, w.wd, m->y32, rows, d, F, WS_EPI_SLOTS, TK_GEMM_DOWN, st); }
         { Span sp(m, PROF_OTHER, 1, st); launch_add_rmsnorm(m, &o, next_gain, rows, st); }
         if (m->dbg_hidden)
             ADED_CUDA_TRY(cudaMemcpyAsync((char*)m->dbg_hidden + (size_t)(l + 1) * hid_bytes, m->h, hid_bytes,
                                           cudaMemcpyDeviceToDevice, st));
     }
     if (!chain_mode) {
-        GemmOut lg = fused_logits;
-        if (!fused) { Span sp(m, PROF_GEMM, 1, st); lg = launch_gemm(m, 4 * c.n_layers, xm, m->x, m->top.lm_head, m->logits, rows, c.vocab, d, st); }
-        Span sp(m, PROF_OTHER, 3, st);
-        if (m->samp_on) {
-            // sampling mode: the logits as a dense matrix, then one drawn token per node in place of the greedy one
-            launch_materialize(m, lg, m->logits, rows, st);
-            ADED_CUDA_TRY(launch_sample_rows(m->logits, rows, c.vocab, c.vocab, m->samp_temp, m->samp_top_p, m->samp_u, m->best,
-                                             m->status, st));
+        // The per-node logits are needed as a matrix only by the sampling mode and by a debug capture; the
+        // greedy choice works from per-tile candidates left by the LM head's tail.
+        const bool dense_logits = !ws || m->samp_on || m->dbg_logits;
+        GemmOut lg;
+        { Span sp(m, PROF_GEMM, passes, st);
+          lg = launch_gemm(m, ws ? 4 * c.n_layers : -1, ws ? xm : -1, m->x, m->top.lm_head, m->logits, rows, c.vocab, d,
+                           dense_logits ? WS_EPI_SLOTS : WS_EPI_ARGMAX, TK_GEMM_HEAD, st); }
+        if (!dense_logits) {
+            Span sp(m, PROF_OTHER, 1, st);
+            launch_pick_accept(m, kv, batch, c.vocab / 128, st);
+            if (m->dbg_best)
+                ADED_CUDA_TRY(cudaMemcpyAsync(m->dbg_best, m->best, (size_t)rows * sizeof(int32_t), cudaMemcpyDeviceToDevice, st));
         } else {
-            launch_argmax(m, lg, rows, st);
+            Span sp(m, PROF_OTHER, 3, st);
+            if (m->samp_on) {
+                // sampling mode: the logits as a dense matrix, then one drawn token per node in place of the greedy one
+                launch_materialize(m, lg, m->logits, rows, st);
+                ADED_CUDA_TRY(launch_sample_rows(m->logits, rows, c.vocab, c.vocab, m->samp_temp, m->samp_top_p, m->samp_u, m->best,
+                                                 m->status, st));
+            } else {
+                launch_argmax(m, lg, rows, st);
+            }
+            if (m->dbg_logits) launch_materialize(m, lg, m->dbg_logits, rows, st);
+            if (m->dbg_best)
+                ADED_CUDA_TRY(cudaMemcpyAsync(m->dbg_best, m->best, (size_t)rows * sizeof(int32_t),
+                                              cudaMemcpyDeviceToDevice, st));
+            launch_accept(m, kv, batch, st);
         }
-        if (m->dbg_logits) launch_materialize(m, lg, m->dbg_logits, rows, st);
-        if (m->dbg_best)
-            ADED_CUDA_TRY(cudaMemcpyAsync(m->dbg_best, m->best, (size_t)rows * sizeof(int32_t),
-                                          cudaMemcpyDeviceToDevice, st));
-        launch_accept(m, kv, batch, st);
     }
     {
         Span sp(m, PROF_OTHER, chain_mode ? 1 : 2, st);
@@ -296,35 +231,10 @@ static aded_status enqueue_pass(aded_model* m, aded_kv* kv, const int32_t* offse
     return ADED_OK;
 }
 
-// Adds the event times of the last replay of a profiling graph to the totals (synchronises).
-static void harvest_profile(aded_model* m, cudaStream_t st) {
-    if (m->prof_pending < 0) return;
-    cudaStreamSynchronize(st);
-    for (ProfSpan& sp : m->graphs[m->prof_pending].spans) {
-        float ms = 0.f;
-        if (cudaEventElapsedTime(&ms, sp.a, sp.b) == cudaSuccess) {
-            m->prof_ms[sp.group] += ms;
-            m->prof_n[sp.group] += sp.launches;
-        } else {
-            cudaGetLastError();
-        }
-    }
-    m->prof_pending = -1;
-}
-
-static void drop_graph(aded_model::GraphEntry& e) {
-    for (ProfSpan& sp : e.spans) { cudaEventDestroy(sp.a); cudaEventDestroy(sp.b); }
-    e.spans.clear();
-    if (e.exec) cudaGraphExecDestroy(e.exec);
-    if (e.offsets_pin) cudaFreeHost(e.offsets_pin);
-    e.exec = nullptr;
-    e.offsets_pin = nullptr;
-}
-
-// One verify / append call: publish the caller's array pointers, then run the pass.
-// With ADED_GRAPH set in the environment when the model is created: a CUDA graph captured per call
-// shape (mode, cache handle, row offsets) and replayed; otherwise, and while a debug capture is
-// armed, the kernels are launched one by one.
+// One verify / append call: publish the caller's array pointers, then run the pass, kernel by kernel
+// (every launch carries the programmatic-dependent-launch attribute).  Replaying a captured graph of the
+// pass was measured slower for a caller that waits for each step (one graph launch of some 300 kernel
+// nodes costs 2-4 ms of host time) and equal back to back, so there is no graph path.
 static aded_status forward(aded_model* m, aded_kv* kv, const int32_t* tokens, const int32_t* parents,
                            const int32_t* offsets_host, int batch, int chain_mode, int32_t* out_tokens,
                            int out_stride, int32_t* out_len, cudaStream_t st) {
@@ -340,69 +250,11 @@ static aded_status forward(aded_model* m, aded_kv* kv, const int32_t* tokens, co
     cp.out_stride = out_stride;
     // pageable source: the runtime stages the bytes before returning, so the stack object may go
     ADED_CUDA_TRY(cudaMemcpyAsync(m->call_dev, &cp, sizeof cp, cudaMemcpyHostToDevice, st));
-
-    cudaStreamCaptureStatus cap_state = cudaStreamCaptureStatusNone;
-    cudaStreamIsCapturing(st, &cap_state);
-    const bool direct = !m->graphs_on || m->samp_on || m->dbg_logits || m->dbg_best || m->dbg_hidden || cap_state != cudaStreamCaptureStatusNone;
-    if (direct) {
-        aded_status s = enqueue_pass(m, kv, offsets_host, batch, rows, max_tree, chain_mode, st);
-        m->dbg_logits = nullptr;
-        m->dbg_best = nullptr;
-        m->dbg_hidden = nullptr;
-        return s;
-    }
-    std::vector<int64_t> key;
-    key.push_back(chain_mode + (m->prof_on ? 2 : 0));   // the profiling variant carries event nodes
-    key.push_back((int64_t)(uintptr_t)kv);
-    if (m->prof_on) harvest_profile(m, st);
-    for (int b = 0; b <= batch; ++b) key.push_back(offsets_host[b]);
-    aded_model::GraphEntry* hit = nullptr;
-    for (auto& e : m->graphs)
-        if (e.key == key) { hit = &e; break; }
-    if (!hit) {
-        if (m->graphs.size() >= 24) {          // forget the least recently used shape
-            size_t old = 0;
-            for (size_t i = 1; i < m->graphs.size(); ++i)
-                if (m->graphs[i].last_use < m->graphs[old].last_use) old = i;
-            harvest_profile(m, st);
-            drop_graph(m->graphs[old]);
-            m->graphs.erase(m->graphs.begin() + old);
-        }
-        aded_model::GraphEntry e;
-        e.key = key;
-        e.exec = nullptr;
-        e.offsets_pin = nullptr;
-        e.last_use = 0;
-        if (cudaMallocHost((void**)&e.offsets_pin, (batch + 1) * sizeof(int32_t)) != cudaSuccess) {
-            cudaGetLastError();
-            return enqueue_pass(m, kv, offsets_host, batch, rows, max_tree, chain_mode, st);
-        }
-        memcpy(e.offsets_pin, offsets_host, (batch + 1) * sizeof(int32_t));
-        cudaGraph_t graph = nullptr;
-        bool ok = cudaStreamBeginCapture(st, cudaStreamCaptureModeThreadLocal) == cudaSuccess;
-        if (ok) {
-            const uint64_t before = aded_launch_count();
-            m->capture_spans = &e.spans;
-            const aded_status s = enqueue_pass(m, kv, e.offsets_pin, batch, rows, max_tree, chain_mode, st);
-            m->capture_spans = nullptr;
-            note_launch(-(int)(aded_launch_count() - before));   // captured, not launched
-            ok = cudaStreamEndCapture(st, &graph) == cudaSuccess && s == ADED_OK && graph != nullptr;
-        }
-        if (ok) ok = cudaGraphInstantiate(&e.exec, graph, 0) == cudaSuccess;
-        if (graph) cudaGraphDestroy(graph);
-        if (!ok) {
-            cudaGetLastError();
-            drop_graph(e);
-            return enqueue_pass(m, kv, offsets_host, batch, rows, max_tree, chain_mode, st);
-        }
-        m->graphs.push_back(e);
-        hit = &m->graphs.back();
-    }
-    hit->last_use = ++m->graph_clock;
-    ADED_CUDA_TRY(cudaGraphLaunch(hit->exec, st));
-    if (m->prof_on) m->prof_pending = (int)(hit - m->graphs.data());
-    note_launch(pass_launches(m, rows, chain_mode));
-    return ADED_OK;
+    const aded_status s = enqueue_pass(m, kv, offsets_host, batch, rows, max_tree, chain_mode, st);
+    m->dbg_logits = nullptr;
+    m->dbg_best = nullptr;
+    m->dbg_hidden = nullptr;
+    return s;
 }
 
 }  // namespace aded
@@ -444,13 +296,6 @@ aded_status aded_model_create(const aded_model_config* cfg, const aded_weights* 
     m->samp_top_p = 1.f;
     m->samp_u = nullptr;
     m->prof_on = false;
-    m->capture_spans = nullptr;
-    m->prof_pending = -1;
-    // Replaying a captured pass is opt-in: with some 330 kernel nodes per pass the host time of one
-    // graph launch was measured at 2-4 ms against 0.7 ms for launching the kernels one by one, so a
-    // caller that waits for every step's result is faster with plain launches.
-    m->graphs_on = getenv("ADED_GRAPH") != nullptr;
-    m->graph_clock = 0;
     m->call_dev = nullptr;
     m->ws_ready = false;
     m->ws_slots = nullptr;
@@ -470,7 +315,6 @@ aded_status aded_model_create(const aded_model_config* cfg, const aded_weights* 
 aded_status aded_model_destroy(aded_model* m) {
     if (!m) return ADED_ERR_INVALID_ARG;
     for (void* p : m->owned) cudaFree(p);
-    for (auto& e : m->graphs) drop_graph(e);
     for (ProfSpan& sp : m->prof_spans) { cudaEventDestroy(sp.a); cudaEventDestroy(sp.b); }
     for (cudaEvent_t e : m->prof_pool) cudaEventDestroy(e);
     delete m;
@@ -509,7 +353,7 @@ aded_status aded_kv_create(const aded_model* m, int32_t batch, const int32_t* ca
         // kernel's last key block and must hold finite values.
         if (cudaMemset(p, 0, bytes) != cudaSuccess) s = ADED_ERR_CUDA;
     }
-    if (s == ADED_OK && m->att_tc) {
+    if (s == ADED_OK && m->att_tc_ok) {
         std::vector<CUtensorMap> maps(batch);
         for (int b = 0; b < batch && s == ADED_OK; ++b)
             if (!aded::attn_tc_make_kv_map(&maps[b], kv->base[b], (uint64_t)kv->cap[b], (uint64_t)c.n_layers * 2 * c.n_heads)) s = ADED_ERR_CUDA;
@@ -693,7 +537,7 @@ aded_status aded_debug_gemm(aded_model* m, int32_t layer, int32_t which, const v
     float* ybuf = which == 4 ? m->logits : m->y32;
     ADED_CUDA_TRY(cudaMemcpyAsync(xbuf, x_dev, (size_t)rows * k * m->elem, cudaMemcpyDeviceToDevice, st));
     note_launch();
-    const GemmOut o = launch_gemm(m, w_map, x_map, xbuf, w, ybuf, rows, n, k, st);
+    const GemmOut o = launch_gemm(m, m->ws_ready ? w_map : -1, m->ws_ready ? x_map : -1, xbuf, w, ybuf, rows, n, k, WS_EPI_SLOTS, TK_OTHER, st);
     launch_materialize(m, o, y_dev, rows, st);
     ADED_CUDA_TRY(cudaGetLastError());
     return ADED_OK;
@@ -725,7 +569,6 @@ aded_status aded_profile_begin(aded_model* m) {
     if (!m) return ADED_ERR_INVALID_ARG;
     for (ProfSpan& sp : m->prof_spans) { m->prof_pool.push_back(sp.a); m->prof_pool.push_back(sp.b); }
     m->prof_spans.clear();
-    m->prof_pending = -1;
     for (int g = 0; g < PROF_GROUPS; ++g) { m->prof_ms[g] = 0.f; m->prof_n[g] = 0; }
     m->prof_on = true;
     return ADED_OK;
@@ -735,7 +578,6 @@ aded_status aded_profile_end(aded_model* m, float* out_ms_host, int32_t* out_lau
     if (!m || !out_ms_host || !out_launches_host) return ADED_ERR_INVALID_ARG;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     m->prof_on = false;
-    harvest_profile(m, st);
     ADED_CUDA_TRY(cudaStreamSynchronize(st));
     for (ProfSpan& sp : m->prof_spans) {
         float ms = 0.f;
@@ -750,6 +592,58 @@ aded_status aded_profile_end(aded_model* m, float* out_ms_host, int32_t* out_lau
     return ADED_OK;
 }
 
+aded_status aded_trace_begin(aded_model* m, void* stream) {
+    if (!m) return ADED_ERR_INVALID_ARG;
+    const int32_t on_and_count[2] = {1, 0};
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    ADED_CUDA_TRY(cudaMemcpyAsync(m->status + 1, on_and_count, sizeof on_and_count, cudaMemcpyHostToDevice, st));
+    ADED_CUDA_TRY(cudaStreamSynchronize(st));     // the two words are a stack variable
+    return ADED_OK;
+}
+
+aded_status aded_trace_end(aded_model* m, uint64_t* out_ns_host, int32_t* out_kind_host, int32_t max_marks,
+                           int32_t* out_n_host, void* stream) {
+    if (!m || !out_ns_host || !out_kind_host || !out_n_host || max_marks < 1) return ADED_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    int32_t words[2] = {0, 0};
+    ADED_CUDA_TRY(cudaMemcpyAsync(words, m->status + 1, sizeof words, cudaMemcpyDeviceToHost, st));
+    ADED_CUDA_TRY(cudaStreamSynchronize(st));
+    const int32_t off = 0;
+    ADED_CUDA_TRY(cudaMemcpyAsync(m->status + 1, &off, sizeof off, cudaMemcpyHostToDevice, st));
+    const long long taken = words[1];
+    long long n = taken < TRACE_CAP ? taken : TRACE_CAP;      // the ring keeps the last TRACE_CAP marks
+    if (n > max_marks) n = max_marks;
+    std::vector<uint64_t> ts(TRACE_CAP);
+    std::vector<int32_t> kind(TRACE_CAP);
+    ADED_CUDA_TRY(cudaMemcpyAsync(ts.data(), m->status + 4, TRACE_CAP * sizeof(uint64_t), cudaMemcpyDeviceToHost, st));
+    ADED_CUDA_TRY(cudaMemcpyAsync(kind.data(), m->status + 4 + 2 * TRACE_CAP, TRACE_CAP * sizeof(int32_t), cudaMemcpyDeviceToHost, st));
+    ADED_CUDA_TRY(cudaStreamSynchronize(st));
+    for (long long i = 0; i < n; ++i) {                       // the last n marks, oldest first
+        const long long src = (taken - n + i) & (TRACE_CAP - 1);
+        out_ns_host[i] = ts[src];
+        out_kind_host[i] = kind[src];
+    }
+    *out_n_host = (int32_t)n;
+    return ADED_OK;
+}
+
+aded_status aded_debug_wait_timeout(aded_model* m, int32_t which, uint64_t limit_cycles, void* stream) {
+    if (!m || which < 0 || which > 1 || limit_cycles < 1 || limit_cycles > (1ull << 32)) return ADED_ERR_INVALID_ARG;
+    // the counter the probe polls: a word of the trace area that only ever holds a small count
+    const uint32_t* quiet = reinterpret_cast<const uint32_t*>(m->status + 3);
+    note_launch();
+    ADED_CUDA_TRY(ws_wait_probe(which, (long long)limit_cycles, quiet, m->status, static_cast<cudaStream_t>(stream)));
+    return ADED_OK;
+}
+
+aded_status aded_debug_attention_kernel(aded_model* m, int32_t which) {
+    if (!m || which < 0 || which > 1) return ADED_ERR_INVALID_ARG;
+    if (which == 0) { m->att_tc = m->att_tc_ok; return ADED_OK; }
+    if (!m->att_mma) return ADED_ERR_UNSUPPORTED;
+    m->att_tc = false;
+    return ADED_OK;
+}
+
 uint64_t aded_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 
 aded_status aded_model_poll_status(aded_model* m, aded_status* out_host, void* stream) {
@@ -760,6 +654,11 @@ aded_status aded_model_poll_status(aded_model* m, aded_status* out_host, void* s
     ADED_CUDA_TRY(cudaStreamSynchronize(st));
     if (v != 0) {
         ADED_CUDA_TRY(cudaMemsetAsync(m->status, 0, sizeof v, st));
+        // a pass that gave up in the middle of a projection's tail may have left its meeting counters mid-count
+        if (m->ws_ready) {
+            ADED_CUDA_TRY(cudaMemsetAsync(m->ws_counters, 0, (size_t)(m->cfg.vocab / 128) * sizeof(uint32_t), st));
+            m->ws_epoch = 0;
+        }
         ADED_CUDA_TRY(cudaStreamSynchronize(st));
     }
     *out_host = static_cast<aded_status>(v);

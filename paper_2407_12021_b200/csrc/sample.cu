@@ -54,6 +54,7 @@ __global__ void __launch_bounds__(SM_THREADS)
 k_sample_rows(const float* __restrict__ logits, int vocab, int ld, float temperature, float top_p,
               const float* __restrict__ u, int32_t* __restrict__ out, const int32_t* status) {
     pdl_enter();
+    if (status && first_thread_of_grid()) trace_mark(status, TK_PICK);
     if (status && *status != 0) return;
     __shared__ unsigned long long s_mass[2048];
     __shared__ unsigned int s_cnt[2048];

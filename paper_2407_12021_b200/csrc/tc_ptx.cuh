@@ -7,7 +7,7 @@
 
 namespace aded {
 
-constexpr long long TC_WAIT_CYCLES = 4000000000ll;   // about two seconds of SM clock
+constexpr long long TC_WAIT_CYCLES = 400000000ll;    // default limit of a device-side wait: about 0.2 s of SM clock
 
 // ---- PTX wrappers -------------------------------------------------------------------------
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -21,8 +21,8 @@ __device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
 __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
-// Bounded wait for the phase with the given parity; false when the limit ran out.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
+// Bounded wait for the phase with the given parity; false when the limit (SM clock cycles) ran out.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, long long limit = TC_WAIT_CYCLES) {
     const uint32_t addr = smem_u32(bar);
     const long long t0 = clock64();
     for (uint32_t spin = 0;; ++spin) {
@@ -33,7 +33,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
             "selp.u32 %0, 1, 0, p;\n\t}"
             : "=r"(done) : "r"(addr), "r"(parity) : "memory");
         if (done) return true;
-        if ((spin & 1023) == 1023 && clock64() - t0 > TC_WAIT_CYCLES) return false;
+        if ((spin & 1023) == 1023 && clock64() - t0 > limit) return false;
     }
 }
 __device__ __forceinline__ void tma_load_2d(const CUtensorMap* map, uint64_t* bar, void* dst, int c0, int c1) {

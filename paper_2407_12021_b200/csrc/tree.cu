@@ -13,6 +13,7 @@ __global__ void k_tree_prologue(const CallPtrs* __restrict__ call,
                                 const int32_t* __restrict__ cap, int vocab, int chain_mode,
                                 RowMeta rows, int32_t* status) {
     pdl_enter();
+    if (first_thread_of_grid()) trace_mark(status, TK_OTHER);
     const int32_t* __restrict__ tokens = call->tokens;
     const int32_t* __restrict__ parents = call->parents;
     const int b = blockIdx.x;
@@ -66,6 +67,7 @@ __global__ void k_accept(const CallPtrs* __restrict__ call,
                          int32_t* __restrict__ path, int32_t* __restrict__ new_len,
                          const int32_t* status, int batch) {
     pdl_enter();
+    if (first_thread_of_grid()) trace_mark(status, TK_PICK);
     const int32_t* __restrict__ tokens = call->tokens;
     const int32_t* __restrict__ parents = call->parents;
     int32_t* __restrict__ out_tokens = call->out_tokens;
@@ -86,31 +88,8 @@ __global__ void k_accept(const CallPtrs* __restrict__ call,
     }
     __syncthreads();
     if (threadIdx.x != 0) return;
-    if (pass_status != 0) {
-        out_len[b] = 0;
-        new_len[b] = len[b];
-        return;
-    }
-    uint64_t ok_lo = 1ull, ok_hi = 0ull;   // approved set; the root always is
-    int deepest = 0, deepest_depth = 0;
-    for (int i = 1; i < T; ++i) {
-        const int p = s_par[i];
-        const bool p_ok = p < 64 ? (ok_lo >> p) & 1 : (ok_hi >> (p - 64)) & 1;
-        if (p_ok && s_tok[i] == s_best[p]) {
-            if (i < 64) ok_lo |= 1ull << i; else ok_hi |= 1ull << (i - 64);
-            const int d = s_dep[i];
-            if (d > deepest_depth) { deepest_depth = d; deepest = i; }
-        }
-    }
-    // path[j] for j = depth .. 0 by climbing; the node at depth j is path element j
-    int cur = deepest;
-    for (int j = deepest_depth; j >= 0; --j) {
-        path[b * ADED_MAX_NODES + j] = cur;
-        out_tokens[(size_t)b * out_stride + j] = s_best[cur];
-        cur = s_par[cur];
-    }
-    out_len[b] = deepest_depth + 1;
-    new_len[b] = len[b] + deepest_depth + 1;
+    approval_walk(s_par, s_tok, s_best, s_dep, T, pass_status, len[b], out_tokens + (size_t)b * out_stride, out_len + b,
+                  path + b * ADED_MAX_NODES, new_len + b);
 }
 
 // Compaction: the tree's K/V were written at slots L + node index; the accepted path p_0 = 0 <
@@ -122,6 +101,7 @@ __global__ void k_compact(char* const* __restrict__ base, const int32_t* __restr
                           const int32_t* __restrict__ len, const int32_t* __restrict__ new_len,
                           const int32_t* __restrict__ path, int hd, const int32_t* status) {
     pdl_enter();
+    if (first_thread_of_grid()) trace_mark(status, TK_OTHER);
     if (*status != 0) return;
     const int b = blockIdx.y;
     const int n_acc = new_len[b] - len[b];
@@ -139,6 +119,7 @@ __global__ void k_compact(char* const* __restrict__ base, const int32_t* __restr
 __global__ void k_commit(int32_t* len, const int32_t* __restrict__ new_len, const int32_t* __restrict__ row_off,
                          int chain_mode, const int32_t* status, int batch) {
     pdl_enter();
+    if (first_thread_of_grid()) trace_mark(status, TK_STEP_END);
     const int b = blockIdx.x * blockDim.x + threadIdx.x;
     if (b >= batch || *status != 0) return;
     len[b] = chain_mode ? len[b] + (row_off[b + 1] - row_off[b]) : new_len[b];

@@ -30,6 +30,7 @@ __global__ void __launch_bounds__(128) k_tree_attn_plain(
         const int32_t* __restrict__ cap, const int32_t* __restrict__ len, const int32_t* __restrict__ row_seq,
         const uint64_t* __restrict__ anc, int layer, int H, int rows, float scale, const int32_t* status) {
     pdl_enter();
+    if (first_thread_of_grid()) trace_mark(status, TK_ATTN);
     if (*status != 0) return;
     constexpr int PER = HD / 32;
     const int warp = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
@@ -185,6 +186,7 @@ __global__ void __launch_bounds__(NW * 32) k_tree_attn_mma(AttnArgs a) {
         }
     }
     pdl_wait();
+    if (first_thread_of_grid()) trace_mark(a.status, TK_ATTN);
     // The status word is fetched along with the rest of the call's metadata and acted on before the
     // first store, so that it does not cost a memory round trip of its own.  Until then nothing is
     // written, and every load below stays inside the cache block and the row arrays whatever a failed
@@ -468,11 +470,9 @@ static void launch_mma_nw(aded_model* m, AttnArgs& a, int batch, int splits, cud
         attr[n].val.clusterDim.z = 1;
         ++n;
     }
-    if (pdl_enabled()) {
-        attr[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-        attr[n].val.programmaticStreamSerializationAllowed = 1;
-        ++n;
-    }
+    attr[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[n].val.programmaticStreamSerializationAllowed = 1;
+    ++n;
     cfg.attrs = attr;
     cfg.numAttrs = n;
     cudaLaunchKernelEx(&cfg, k_tree_attn_mma<HD, NW>, a);

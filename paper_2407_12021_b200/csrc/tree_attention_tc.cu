@@ -220,6 +220,7 @@ k_tree_attn_tc(const __grid_constant__ CUtensorMap map_q, AttnTcArgs a) {
         }
     }
     pdl_wait();
+    if (first_thread_of_grid()) trace_mark(a.status, TK_ATTN);
     const int pass_status = *a.status;
 
     const int hh = blockIdx.x, split = blockIdx.y, b = blockIdx.z / a.row_blocks;
@@ -592,11 +593,9 @@ void launch_tree_attention_tc(aded_model* m, aded_kv* kv, int layer, int batch, 
         attr[n].val.clusterDim.z = 1;
         ++n;
     }
-    if (pdl_enabled()) {
-        attr[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-        attr[n].val.programmaticStreamSerializationAllowed = 1;
-        ++n;
-    }
+    attr[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[n].val.programmaticStreamSerializationAllowed = 1;
+    ++n;
     cfg.attrs = attr;
     cfg.numAttrs = n;
     cudaLaunchKernelEx(&cfg, k_tree_attn_tc, m->att_q_map, a);

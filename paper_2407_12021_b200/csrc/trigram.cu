@@ -95,8 +95,22 @@ __device__ __forceinline__ void tg_add(const TgView& t, int a, int b, int c, uin
             int32_t have = *reinterpret_cast<volatile int32_t*>(&bk->e[e].tok);
             if (have == -1) have = atomicCAS(&bk->e[e].tok, -1, c) == -1 ? c : *reinterpret_cast<volatile int32_t*>(&bk->e[e].tok);
             if (have == c) {
-                const uint32_t old = atomicAdd(&bk->e[e].cnt, inc);
-                if (old > t.cap - inc) atomicMin(&bk->e[e].cnt, t.cap);   // inc <= cap (callers clamp)
+                if (inc == 1) {
+                    // the per-step update: cap <= 2^31 - 1 and at most 2^31 threads add 1 before the minimum below
+                    // takes effect, so the 32-bit count cannot wrap
+                    const uint32_t old = atomicAdd(&bk->e[e].cnt, 1u);
+                    if (old >= t.cap) atomicMin(&bk->e[e].cnt, t.cap);
+                } else {
+                    // imports add arbitrary counts: saturate in one step, so that two large additions to one
+                    // tri-gram cannot carry the count past 2^32 between an add and a later minimum
+                    uint32_t seen = *reinterpret_cast<volatile uint32_t*>(&bk->e[e].cnt);
+                    for (;;) {
+                        const uint32_t want = seen >= t.cap || inc > t.cap - seen ? t.cap : seen + inc;
+                        const uint32_t prev = atomicCAS(&bk->e[e].cnt, seen, want);
+                        if (prev == seen) break;
+                        seen = prev;      // (another thread moved the count; every retry follows a change made by someone else)
+                    }
+                }
                 return;
             }
         }
@@ -739,6 +753,7 @@ aded_status aded_trigram_create(const aded_trigram_config* cfg, aded_trigram** o
     *out = nullptr;
     if (cfg->vocab < 1 || cfg->log2_buckets < 4 || cfg->log2_buckets > 28 || cfg->overflow_buckets < 0)
         return ADED_ERR_INVALID_ARG;
+    if (cfg->cap > 0x7fffffffu) return ADED_ERR_INVALID_ARG;     // counts are kept below 2^31 so that concurrent adds cannot wrap
     aded_trigram* t = new (std::nothrow) aded_trigram();
     if (!t) return ADED_ERR_OOM;
     t->cfg = *cfg;

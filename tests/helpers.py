@@ -65,9 +65,19 @@ class GpuSession:
         return k.cpu().double().numpy(), v.cpu().double().numpy()
 
 
-def compare_step(shape, gpu: Dict, cpu: Dict, tokens, parents, where: str = "") -> Dict[str, float]:
-    """Element-wise comparison of one verification step.  Returns the worst errors seen."""
-    tol = LOGIT_TOL[shape.dtype]
+def compare_step(shape, gpu: Dict, cpu: Dict, tokens, parents, where: str = "", beyond_allowance: int = 0,
+                 logit_tol: Optional[float] = None) -> Dict[str, float]:
+    """Element-wise comparison of one verification step.  Returns the worst errors seen.
+
+    Logits: per row max |gpu - cpu| / max |cpu| within `logit_tol` (default: the dtype's tolerance).
+    Greedy tokens: equal, except at near-ties.  The asserted bar is the fixed one: a differing token is
+    exempt only where the checker's top-2 margin is below MARGIN_EXEMPT (1e-2).  `beyond_allowance` is the
+    number of differing tokens with a larger margin a test tolerates; it is 0 unless the test states, beside
+    the call, why more are expected (an end-to-end run through several layers of a random-init bf16 network,
+    whose logits legitimately differ by up to the logit tolerance).  Even an allowed one must be explained by
+    the measured deviation of its own row (margin < 2 x that row's max |gpu - cpu|: two logits can each move
+    by that much), and every one is printed."""
+    tol = LOGIT_TOL[shape.dtype] if logit_tol is None else logit_tol
     lg, lc = gpu["logits"], cpu["logits"]
     assert lg.shape == lc.shape
     rel = np.max(np.abs(lg - lc), axis=1) / np.max(np.abs(lc), axis=1)
@@ -75,13 +85,17 @@ def compare_step(shape, gpu: Dict, cpu: Dict, tokens, parents, where: str = "") 
     margin = ov.top2_margin(lc)
     delta = np.max(np.abs(lg - lc), axis=1)            # measured logit deviation of every row
     diff = np.nonzero(gpu["best"] != cpu["best"])[0]
+    beyond = []
     for i in diff:
-        # A different greedy token is acceptable only at a near-tie: the checker's margin is below the
-        # fixed threshold, or below what this row's measured logit deviation (itself inside the logit
-        # tolerance, checked above) can explain -- two logits can each move by delta.
-        assert margin[i] < max(MARGIN_EXEMPT, 2 * delta[i]), (
-            f"{where}: greedy token of node {i} differs ({gpu['best'][i]} vs {cpu['best'][i]}) with top-2 margin "
-            f"{margin[i]:.3e}, logit deviation {delta[i]:.3e}")
+        if margin[i] < MARGIN_EXEMPT:
+            continue
+        beyond.append(int(i))
+        print(f"{where}: greedy token of node {i} differs ({gpu['best'][i]} vs {cpu['best'][i]}) beyond the 1e-2 margin: "
+              f"top-2 margin {margin[i]:.3e}, logit deviation of the row {delta[i]:.3e}")
+        assert margin[i] < 2 * delta[i], f"{where}: node {i}: margin {margin[i]:.3e} is not explained by the row's deviation {delta[i]:.3e}"
+    assert len(beyond) <= beyond_allowance, (
+        f"{where}: {len(beyond)} greedy tokens differ where the checker's top-2 margin is >= {MARGIN_EXEMPT} "
+        f"(nodes {beyond}); allowed here: {beyond_allowance}")
     # the accepted sequence must equal the checker's walk over the GPU's own per-node choices;
     # when no node differed that is the checker's answer itself
     path, out = ov.accept_walk(tokens, parents, gpu["best"])
@@ -89,9 +103,42 @@ def compare_step(shape, gpu: Dict, cpu: Dict, tokens, parents, where: str = "") 
     assert gpu["accept_len"] == len(out)
     if len(diff) == 0:
         assert gpu["out_tokens"] == cpu["out_tokens"] and gpu["accept_len"] == cpu["accept_len"]
-    beyond = int(sum(margin[i] >= MARGIN_EXEMPT for i in diff))
-    return {"logit_rel": float(rel.max()), "flipped": int(len(diff)), "flipped_beyond_1e-2": beyond,
+    return {"logit_rel": float(rel.max()), "flipped": int(len(diff)), "flipped_beyond_1e-2": len(beyond),
             "min_margin": float(margin.min())}
+
+
+def layerwise_check(arch, ow, tokens, parents, L: int, hidden: np.ndarray, cache_before: Dict[int, tuple],
+                    gpu: Dict, where: str, shape, max_tol: float = 2e-2, rms_tol: float = 1e-2) -> Dict[str, float]:
+    """Teacher-forced, layer-by-layer comparison of a verification step at the model's full depth.
+
+    `hidden` [n_layers + 1][T][d] is the device's residual stream before layer 0 and after every layer,
+    `cache_before[l]` = (K, V) [H, L, hd] the committed cache of layer l the step started from, for the
+    layers to check.  Each such layer is re-run by the checker from the device's own input and cache and
+    must give the device's output within max_tol (max) / rms_tol (rms) of the output's scale; the LM
+    head and the greedy choice are re-run from the device's final hidden states and held to the fixed
+    token rule (no differing token where the checker's top-2 margin is >= 1e-2).  Returns the worst
+    figures and, per checked layer, the keys/values the checker computed for the tree nodes."""
+    paths, depth = ov.paths_and_depths(parents)
+    pos = L + np.asarray(depth)
+    assert np.array_equal(hidden[0], ow.embed_rows(tokens)), f"{where}: embedding rows are copies"
+    worst_max, worst_rms, kv_new = 0.0, 0.0, {}
+    for l in sorted(cache_before):
+        kc, vc = cache_before[l]
+        h_out, k, v = ov.decoder_layer(arch, ow.layer(l), kc, vc, hidden[l], paths, pos)
+        err = np.abs(h_out - hidden[l + 1])
+        rel_max = err.max() / np.abs(h_out).max()
+        rel_rms = float(np.sqrt((err ** 2).mean() / (h_out ** 2).mean()))
+        print(f"{where} layer {l}: max {rel_max:.3e} rms {rel_rms:.3e} differing {np.mean(err > 0):.3f}")
+        assert rel_max <= max_tol and rel_rms <= rms_tol, (where, l, rel_max, rel_rms)
+        worst_max, worst_rms = max(worst_max, float(rel_max)), max(worst_rms, rel_rms)
+        kv_new[l] = (k, v)
+    lc = ov.lm_head(arch, ow, hidden[arch.n_layers])
+    step_cpu = {"logits": lc, "best": ov.greedy(lc)}
+    step_cpu["out_tokens"] = ov.accept_walk(tokens, parents, step_cpu["best"])[1]
+    step_cpu["accept_len"] = len(step_cpu["out_tokens"])
+    head = compare_step(shape, gpu, step_cpu, tokens, parents, f"{where} LM head", beyond_allowance=0, logit_tol=2e-3)
+    print(f"{where} LM head from the device's hidden states:", head)
+    return {"layer_max": worst_max, "layer_rms": worst_rms, "head": head, "kv_new": kv_new, "cpu": step_cpu}
 
 
 def compare_cache(shape, sess: GpuSession, cache: ov.Cache, pos0: int, n: int, layers: Sequence[int], where=""):

@@ -186,3 +186,36 @@ def test_export_prune_save_load(cuda_device, tmp_path):
     B.aded_trigram_clear(t)
     assert _entries_gpu(B, t) == {} and B.aded_trigram_stats(t) == (0, 0)
     assert B.aded_trigram_poll_status(t) == 0 and B.aded_trigram_poll_status(t2) == 0
+
+
+def test_import_of_duplicate_entries_with_large_counts_saturates(cuda_device):
+    """Imported counts may be large and one tri-gram may appear several times in an import: the stored count
+    is min(sum, cap) as in the checker's merge, never a wrapped 32-bit sum.  The default cap is 2^31 - 1;
+    a cap above it is refused."""
+    from paper_2407_12021_b200 import binding as B
+    big = 2 ** 31 - 2
+    keys, counts, entries = [], [], []
+    for i in range(64):                       # 64 tri-grams, each four times in one import, counts near 2^31
+        for rep in range(4):
+            keys.append([i % 7, i % 5, i])
+            counts.append(big - rep)
+            entries.append(((i % 7, i % 5, i), big - rep))
+    for cap in (0, 1000, 2 ** 31 - 1):
+        t = B.aded_trigram_create(100, log2_buckets=8, overflow_buckets=64, cap=cap)
+        st = TrigramStore(cap=cap if cap else 2 ** 31 - 1)
+        st.update([1, 2, 3, 1, 2, 3])          # an entry that is there before the import
+        B.aded_trigram_update(t, torch.tensor([1, 2, 3, 1, 2, 3], dtype=torch.int32, device=cuda_device))
+        kt = torch.tensor(keys + [[1, 2, 3]], dtype=torch.int32, device=cuda_device)
+        ct = torch.tensor([c - 2 ** 32 if c >= 2 ** 31 else c for c in counts + [big]], dtype=torch.int32, device=cuda_device)
+        B.aded_trigram_import(t, kt, ct)
+        for key, n in entries + [((1, 2, 3), big)]:
+            st.merge({key: n})
+        torch.cuda.synchronize()
+        assert B.aded_trigram_poll_status(t) == 0
+        for i in range(64):
+            assert B.aded_trigram_get(t, i % 7, i % 5, i) == st.count(i % 7, i % 5, i) == st.cap
+        assert B.aded_trigram_get(t, 1, 2, 3) == st.count(1, 2, 3) == st.cap
+        assert B.aded_trigram_get(t, 2, 3, 1) == st.count(2, 3, 1) == 1
+    with pytest.raises(B.AdedError) as err:
+        B.aded_trigram_create(100, log2_buckets=8, overflow_buckets=64, cap=2 ** 31)
+    assert err.value.status == 1

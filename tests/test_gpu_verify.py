@@ -159,67 +159,6 @@ def test_verify_host_entry_point(cuda_device):
     assert int(n[0]) == cpu["accept_len"] and out[:int(n[0])].tolist() == cpu["out_tokens"]
 
 
-def test_graph_replay_gives_the_same_steps(cuda_device, monkeypatch):
-    """A model created with ADED_GRAPH set captures the pass once per call shape and replays it; the
-    decoded steps must equal those of the checker, replay after replay."""
-    monkeypatch.setenv("ADED_GRAPH", "1")
-    shape, arch, ow, cache, sess, prompt = _c1_setup(cuda_device, seed=23)
-    monkeypatch.delenv("ADED_GRAPH")
-    root = prompt[-1]
-    for step in range(4):      # the same tree shape every step: one capture, three replays
-        tokens, parents = gen.make_tree(16, 4, 4, shape.vocab, 40 + step, root_token=root)
-        cpu = ov.verify(arch, ow, cache, tokens, parents)
-        gpu = sess.verify(tokens, parents, capture=False)
-        assert gpu["status"] == 0
-        assert gpu["accept_len"] == cpu["accept_len"] and gpu["out_tokens"] == cpu["out_tokens"], f"step {step}"
-        assert sess.length() == cache.length
-        root = cpu["out_tokens"][-1]
-
-
-@pytest.mark.parametrize("heads,hd,layers,ffn", [(4, 64, 2, 384), (8, 128, 3, 2048)])
-def test_persistent_projection_kernel_matches_separate_kernels(cuda_device, monkeypatch, heads, hd, layers, ffn):
-    """A model created with ADED_FUSED set runs the projections of a layer and the steps between them in
-    one persistent kernel with grid barriers.  Same arithmetic and the same order of the partial
-    sums of every projection; only the RMSNorm's sum of squares is added up in another order (128
-    threads per row instead of 1024), so activations and cache rows of the first layer may differ in the last bf16 bit, later ones by what
-    that grows to.
-    Also covers projections with fewer work units than CTAs."""
-    from paper_2407_12021_b200 import binding as B
-    shape = gen.ModelShape(f"bf16-{heads}x{hd}", layers, heads * hd, heads, hd, ffn, 1024, "bf16")
-    w = H.weights_to(gen.model_weights(shape, 77), cuda_device)
-    prompt = gen.zipf_tokens(91, shape.vocab, 77, 50).to(torch.int32).cuda()
-    tokens, parents = gen.make_tree(48, 5, 4, shape.vocab, 78, root_token=int(prompt[-1]))
-    results = []
-    for fused in (False, True):
-        if fused:
-            monkeypatch.setenv("ADED_FUSED", "1")
-        else:
-            monkeypatch.delenv("ADED_FUSED", raising=False)
-        m = B.aded_model_create(shape, w, max_rows=128, max_batch=1)
-        kv = B.aded_kv_create(m, [512])
-        n0 = B.aded_launch_count()
-        B.aded_append(m, kv, prompt[:-1].contiguous())
-        launches = B.aded_launch_count() - n0
-        out = torch.full((48,), -7, dtype=torch.int32, device="cuda")
-        alen = torch.full((1,), -7, dtype=torch.int32, device="cuda")
-        B.aded_verify(m, kv, H.i32(tokens), H.i32(parents), out, alen)
-        torch.cuda.synchronize()
-        assert B.aded_model_poll_status(m) == 0
-        bufs = [B.aded_debug_read_buffer(m, i, 48).clone() for i in range(5)]
-        n = B.aded_kv_len(kv, 0)
-        rows = [t.clone() for l in range(layers) for t in B.aded_kv_read(kv, 0, l, 0, n)]
-        torch.cuda.synchronize()
-        results.append((launches, out.tolist(), int(alen[0]), n, bufs, rows))
-    monkeypatch.delenv("ADED_FUSED", raising=False)
-    (l0, out0, a0, n0_, b0, r0), (l1, out1, a1, n1, b1, r1) = results
-    assert l1 < l0, "the persistent kernel was not used"
-    assert (out0, a0, n0_) == (out1, a1, n1)
-    for x, y in zip(b0 + r0, b1 + r1):
-        x, y = x.float(), y.float()
-        # a last-bit difference after one layer grows through the next ones (a random-init network amplifies one-ulp differences)
-        assert (x - y).abs().max() <= 2e-2 * x.abs().max()
-
-
 def test_c2_one_7b_layer_bf16(cuda_device):
     """Workload 2: one Llama-2-7B-shaped layer + LM head in bf16, cache pre-filled with 1024 N(0,1)
     positions, 64-node depth-6 tree with branching <= 4."""
@@ -255,21 +194,18 @@ def test_c2_one_7b_layer_bf16(cuda_device):
 
 
 @pytest.mark.parametrize("nodes,ctx,depth", [(100, 300, 6), (64, 2047, 6), (5, 1, 2)])
-def test_attention_kernels_agree(cuda_device, monkeypatch, nodes, ctx, depth):
-    """head_dim 128 has two attention kernels: tcgen05 (the default) and mma.sync (ADED_ATTN_MMA set when the
-    model is created).  Same rounding points (integer reference in the log2 domain, numerators rounded to
-    bf16, unrounded row sums); the fp32 sums run in another order, so outputs agree to a few bf16 ulps."""
+def test_attention_kernels_agree(cuda_device, nodes, ctx, depth):
+    """head_dim 128 has two attention kernels: tcgen05 (the default) and mma.sync (selected with
+    aded_debug_attention_kernel).  Same rounding points (integer reference in the log2 domain, numerators
+    rounded to bf16, unrounded row sums); the fp32 sums run in another order, so outputs agree to a few bf16 ulps."""
     from paper_2407_12021_b200 import binding as B
     shape = gen.ModelShape("bf16-4x128", 2, 512, 4, 128, 1024, 1024, "bf16")
     w = H.weights_to(gen.model_weights(shape, 31), cuda_device)
     tokens, parents = gen.make_tree(nodes, depth, 4, shape.vocab, 32)
     results = []
     for mma in (False, True):
-        if mma:
-            monkeypatch.setenv("ADED_ATTN_MMA", "1")
-        else:
-            monkeypatch.delenv("ADED_ATTN_MMA", raising=False)
         m = B.aded_model_create(shape, w, max_rows=128, max_batch=1)
+        B.aded_debug_attention_kernel(m, 1 if mma else 0)
         kv = B.aded_kv_create(m, [ctx + 256])
         for l in range(shape.n_layers):
             k, v = gen.kv_normal(shape, ctx, 33, l, device=cuda_device)
@@ -280,7 +216,6 @@ def test_attention_kernels_agree(cuda_device, monkeypatch, nodes, ctx, depth):
         torch.cuda.synchronize()
         assert B.aded_model_poll_status(m) == 0
         results.append((B.aded_debug_read_buffer(m, 3, nodes).float().clone(), B.aded_debug_read_buffer(m, 0, nodes).float().clone()))
-    monkeypatch.delenv("ADED_ATTN_MMA", raising=False)
     (att0, h0), (att1, h1) = results
     assert (att0 - att1).abs().max() <= 2e-2 * att0.abs().max()
     assert (h0 - h1).abs().max() <= 2e-2 * h0.abs().max()
@@ -322,3 +257,31 @@ def test_bf16_small_models_tree_shapes(cuda_device, heads, hd, nodes, depth, ctx
         assert sess.length() == cache.length
         H.compare_cache(shape, sess, cache, ctx, cache.length - ctx, range(shape.n_layers), f"cache step {step}")
         root = gpu["out_tokens"][-1]
+
+
+@pytest.mark.parametrize("which", [0, 1])
+def test_bounded_wait_runs_out_and_the_handle_recovers(cuda_device, which):
+    """Every device-side wait of the library is bounded and ends in a status code, not a hang.  The probe makes
+    one such wait run out for real -- an mbarrier nobody arrives at (which = 0), an arrival counter nobody
+    raises (1) -- with a limit of about a millisecond.  Expected: the kernel returns, the model reports
+    ADED_ERR_TIMEOUT, a step submitted while the error is pending does nothing (accept length 0, cache
+    untouched), and after the status has been read the handle works as before."""
+    import time
+    shape = gen.ModelShape("bf16-4x128", 2, 512, 4, 128, 1024, 1024, "bf16")
+    w = H.weights_to(gen.model_weights(shape, 91), cuda_device)
+    sess = H.GpuSession(shape, w, capacity=512)
+    prompt = gen.zipf_tokens(70, shape.vocab, 91, 50).tolist()
+    sess.append(prompt[:-1])
+    tokens, parents = gen.make_tree(24, 4, 4, shape.vocab, 92, root_token=prompt[-1])
+    good = sess.verify(tokens, parents, capture=False)
+    assert good["status"] == 0 and good["accept_len"] >= 1
+    sess.B.aded_kv_set_len(sess.kv, 0, 69)
+    t0 = time.perf_counter()
+    sess.B.aded_debug_wait_timeout(sess.model, which, 2_000_000)
+    torch.cuda.synchronize()
+    assert time.perf_counter() - t0 < 1.0, "the wait did not end at its limit"
+    pending = sess.verify(tokens, parents, capture=False)          # reads (and clears) the status after the call
+    assert pending["status"] == 8 and pending["accept_len"] == 0 and sess.length() == 69
+    assert sess.B.aded_model_poll_status(sess.model) == 0
+    again = sess.verify(tokens, parents, capture=False)
+    assert again["status"] == 0 and again["out_tokens"] == good["out_tokens"] and sess.length() == 69 + good["accept_len"]

@@ -1,5 +1,5 @@
 """aded_greedy_noalloc -- the allocation-free greedy token choice -- against the library's own
-per-node greedy choice.
+per-node greedy choice and the CPU checker's.
 
 Some users of the library cannot allocate device memory while decoding: the device heap belongs to
 another component of their process (a framework's memory pool), or their latency budget forbids
@@ -56,6 +56,10 @@ def test_noalloc_greedy_matches_verify_twice_in_a_row(cuda_device):
     # integer results: the bar is exact equality, as for every index the library produces
     assert torch.equal(got_a, best_a)
     assert torch.equal(got_b, best_b)
+    # and equal to the CPU checker's greedy choice on the very same logits (largest value, lowest id among equals)
+    from oracle import verify as ov
+    assert got_a.cpu().tolist() == ov.greedy(logits_a.cpu().double().numpy()).tolist()
+    assert got_b.cpu().tolist() == ov.greedy(logits_b.cpu().double().numpy()).tolist()
     # and once more on the first input: still the same after the array held other rows
     again = torch.full((128,), -1, dtype=torch.int32, device=cuda_device)
     B.aded_greedy_noalloc(logits_a, again)
@@ -74,7 +78,32 @@ def test_noalloc_greedy_tie_rule_and_limits(cuda_device):
     B.aded_greedy_noalloc(x, got)
     torch.cuda.synchronize()
     assert got.tolist() == [17, 4000, 0]
+    # a row without any finite candidate (all -inf) yields token 0, as the verification step's choice does
+    y = torch.full((2, 300), float("-inf"), dtype=torch.float32, device=cuda_device)
+    y[1, 299] = -3.0e38
+    got2 = torch.full((2,), -1, dtype=torch.int32, device=cuda_device)
+    B.aded_greedy_noalloc(y, got2)
+    torch.cuda.synchronize()
+    assert got2.tolist() == [0, 299]
     too_many = torch.zeros((B.ADED_NOALLOC_MAX_ROWS + 1, 8), dtype=torch.float32, device=cuda_device)
     with pytest.raises(B.AdedError) as err:
         B.aded_greedy_noalloc(too_many, torch.empty(B.ADED_NOALLOC_MAX_ROWS + 1, dtype=torch.int32, device=cuda_device))
     assert err.value.status == 1
+
+
+def test_noalloc_greedy_leaves_device_memory_as_it_found_it(cuda_device):
+    """What the entry point promises the callers it exists for: after its first call on the device (which looks
+    up the scratch array's address), a call neither takes nor returns device memory.  Free device memory, as
+    the driver reports it, is the same before and after a warm call; torch's own pool is not touched either."""
+    from paper_2407_12021_b200 import binding as B
+    x = torch.randn((64, 4096), dtype=torch.float32, device=cuda_device)
+    got = torch.empty(64, dtype=torch.int32, device=cuda_device)
+    B.aded_greedy_noalloc(x, got)              # first call on this device: address look-up
+    torch.cuda.synchronize()
+    free0, _ = torch.cuda.mem_get_info(cuda_device)
+    reserved0 = torch.cuda.memory_reserved(cuda_device)
+    B.aded_greedy_noalloc(x, got)
+    torch.cuda.synchronize()
+    free1, _ = torch.cuda.mem_get_info(cuda_device)
+    assert free1 == free0 and torch.cuda.memory_reserved(cuda_device) == reserved0
+    assert got.cpu().tolist() == x.cpu().argmax(dim=1).tolist()
