@@ -254,69 +254,73 @@ def run_ours(args, rank, world):
     return result
 
 
-PLANT_KEEP = 0.6        # share of the model's own tri-grams the planted table knows
-PLANT_COUNT = 1 << 20   # their count: above anything the prompt put into the table
+PLANT_KEEP = 0.6        # chance that the table already knows the next tri-gram of the model's text
 
 
 def planted_arm(B, model, kv, fresh_table, ctx, ctx0, base_len, fill_d, wl, shape, steps, warm, dev, world, rank):
     """A second timed decode in which drafts are approved.  With random-init weights the model's greedy text is
-    unrelated to the Zipf prompt, so a table built from the prompt alone never predicts it (accept length 1).  Here
-    the table is told, before decoding starts, a seeded PLANT_KEEP share of the tri-grams of the model's OWN
-    greedy continuation (recorded first, by ordinary decode steps from the same prompt) -- the state the paper's
-    adaptive table reaches on text it has seen before.  Draft trees then come from top-k lists that hold the
-    model's path, accept lengths spread over 1 .. depth + 1 (mean about 1 / (1 - keep)), and the approved K/V rows
-    are compacted inside the timed region.  Same model, cache, prompt and filler as the main arm."""
+    unrelated to the Zipf prompt, so a table built from the prompt never predicts it (accept length 1 in the main
+    arm).  Here the table is taught, step by step, part of what the model is about to say -- the state the paper's
+    adaptive table reaches on text it has seen before.  Every step has a seeded target accept length a (geometric:
+    one more token with probability PLANT_KEEP, at most depth + 1; mean about 2.4, the range of the paper's
+    Table 1).  Before the timed call, a - 1 untimed rehearsal calls of the same step run on the same cache state:
+    each emits one token more than the one before and the step's own table update learns its tri-grams; cache
+    length and context are rolled back after each.  The timed call then finds the model's path in the top-k
+    trees, approves about a tokens and compacts their K/V rows.  (A recorded text cannot be planted instead:
+    in a random-init bf16 network a token's logits move by a few percent with its slot in the tree, so a
+    replay drifts off any recording within some tens of tokens; rehearsing on the spot keeps the numerics of
+    the timed call identical to the last rehearsal's.)  Steps are timed one by one with CUDA events, the
+    device idle before each; same model, prompt, cache and filler as the main arm."""
     n, total = wl.tree_nodes, steps + warm
-    n_rec = int(total / (1.0 - PLANT_KEEP)) + 32                 # decode steps to record: one token each
-    rec_out = torch.zeros((n_rec, n), dtype=torch.int32, device=dev)
-    rec_len = torch.zeros((n_rec, 1), dtype=torch.int32, device=dev)
+    u = gen.uniform01(total * 8, SEED + rank, 7777).tolist()
+    targets = []
+    for s in range(total):
+        a = 1
+        while a < wl.tree_depth + 1 and u[s * 8 + a] < PLANT_KEEP:
+            a += 1
+        targets.append(a)
     B.aded_kv_set_len(kv, 0, base_len)
     table = fresh_table()
     ctx.copy_(ctx0)
-    for s in range(n_rec):
-        B.aded_decode_step(model, kv, table, ctx, n, wl.tree_depth, wl.topk, fill_d[s % total], rec_out[s], rec_len[s], None)
-    torch.cuda.synchronize()
-    lens = rec_len[:, 0].tolist()
-    text = ctx0.tolist() + [t for s in range(n_rec) for t in rec_out[s, :lens[s]].tolist()]
-    keep = (gen.uniform01(len(text) - 2, SEED + rank, 7777) < PLANT_KEEP).tolist()
-    keys = [text[i:i + 3] for i in range(len(text) - 2) if keep[i]]
-    table = fresh_table()
-    B.aded_trigram_import(table, torch.tensor(keys, dtype=torch.int32, device=dev).contiguous(),
-                          torch.full((len(keys),), PLANT_COUNT, dtype=torch.int32, device=dev))
-    B.aded_kv_set_len(kv, 0, base_len)
-    ctx.copy_(ctx0)
+    s_out = torch.zeros(n, dtype=torch.int32, device=dev)
+    s_len = torch.zeros(1, dtype=torch.int32, device=dev)
     p_out = torch.zeros((total, n), dtype=torch.int32, device=dev)
     p_len = torch.zeros((total, 1), dtype=torch.int32, device=dev)
     p_real = torch.zeros((total, 1), dtype=torch.int32, device=dev)
-    ev = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
-    torch.cuda.synchronize()
+    length, times = base_len, []
+    if world > 1:
+        torch.distributed.barrier()
     for step in range(total):
-        if step == warm:
-            if world > 1:
-                torch.distributed.barrier()
-            torch.cuda.synchronize()
-            ev[0].record()
+        saved = ctx.clone()
+        for _ in range(targets[step] - 1):                        # rehearsals (untimed)
+            B.aded_decode_step(model, kv, table, ctx, n, wl.tree_depth, wl.topk, fill_d[step], s_out, s_len, None)
+            B.aded_kv_set_len(kv, 0, length)                      # (synchronises)
+            ctx.copy_(saved)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
         B.aded_decode_step(model, kv, table, ctx, n, wl.tree_depth, wl.topk, fill_d[step], p_out[step], p_len[step], p_real[step])
-    ev[1].record()
-    torch.cuda.synchronize()
+        e1.record()
+        torch.cuda.synchronize()
+        a = int(p_len[step])
+        assert a >= 1, (B.aded_model_poll_status(model), B.aded_trigram_poll_status(table))
+        length += a
+        times.append(e0.elapsed_time(e1))
     assert B.aded_model_poll_status(model) == 0 and B.aded_trigram_poll_status(table) == 0
-    ms = ev[0].elapsed_time(ev[1])
+    assert B.aded_kv_len(kv, 0) == length
     plens = p_len[:, 0].tolist()
-    emitted = [t for s in range(total) for t in p_out[s, :plens[s]].tolist()]
     accepted = sum(plens[warm:])
+    ms = sum(times[warm:])
     hist = {}
     for a in plens[warm:]:
         hist[a] = hist.get(a, 0) + 1
-    # verification equals plain decoding: the text must be the recorded one (a near-tie may legitimately move a token)
-    m = min(len(emitted), len(text) - 2)
-    same = emitted[:m] == text[2:2 + m]
-    first_diff = next((i for i in range(m) if emitted[i] != text[2 + i]), None)
     return {"ms": ms, "accepted": accepted, "ms_per_step": ms / steps, "accept_len_mean": accepted / steps,
+            "accept_len_target_mean": sum(targets[warm:]) / steps,
+            "steps_reaching_their_target": sum(1 for s in range(warm, total) if plens[s] >= targets[s]),
             "accept_len_histogram": {str(k): hist[k] for k in sorted(hist)},
             "tree_nodes_from_table_mean": float(p_real[warm:].float().mean()),
-            "table": f"prompt tri-grams + a seeded {PLANT_KEEP:.0%} of the tri-grams of the model's own greedy continuation "
-                     f"({len(keys)} of {len(text) - 2}, count {PLANT_COUNT})",
-            "text_equals_recorded_decode": same, "first_difference_at_token": first_diff, "tokens_compared": m}
+            "timing": "sum of per-step CUDA-event times, device idle before each step (untimed rehearsal calls in between)",
+            "table": f"prompt tri-grams, then taught on the spot: target accept length per step geometric with p = {PLANT_KEEP}"}
 
 
 def stage_times(marks, n_layers):
@@ -488,11 +492,13 @@ def run_c5(args, rank, world):
                 times.append(e0.elapsed_time(e1))
         assert B.aded_model_poll_status(model) == 0
         B.aded_trace_begin(model)
-        for b in range(batch):
-            B.aded_kv_set_len(kv, b, ctx_len[b])
-        B.aded_verify_batch(model, kv, offsets, tok, par, out, out_len)
-        B.aded_verify_batch(model, kv, offsets, tok, par, out, out_len)      # (a second pass so that the trace holds a whole one)
+        for _ in range(2):                                         # (two passes so that the trace holds a whole one)
+            for b in range(batch):
+                B.aded_kv_set_len(kv, b, ctx_len[b])
+            B.aded_verify_batch(model, kv, offsets, tok, par, out, out_len)
         ts, kinds = B.aded_trace_end(model)
+        torch.cuda.synchronize()
+        assert B.aded_model_poll_status(model) == 0
         ends = [i for i, kd in enumerate(kinds) if kd == 11]
         gemm_us = attn_us = 0.0
         if len(ends) >= 2:
@@ -502,6 +508,7 @@ def run_c5(args, rank, world):
                     gemm_us += dt
                 elif kinds[i] == 6:
                     attn_us += dt
+        gemm_us, attn_us = max(gemm_us, 1e-3), max(attn_us, 1e-3)
         ms = statistics.median(times)
         kv_bytes = shape.kv_bytes_per_position() * sum(ctx_len)
         flops = 2.0 * (shape.weight_bytes_per_step / 2) * rows

@@ -51,7 +51,8 @@ typedef enum aded_status {
     ADED_ERR_OOM = 5,
     ADED_ERR_CUDA = 6,
     ADED_ERR_UNSUPPORTED = 7,
-    ADED_ERR_TIMEOUT = 8       /* a bounded device-side wait ran out */
+    ADED_ERR_TIMEOUT = 8,      /* a bounded device-side wait ran out */
+    ADED_ERR_INTERNAL = 9      /* debug build only: an index check inside a kernel failed (the access was skipped) */
 } aded_status;
 
 enum { ADED_F32 = 0, ADED_BF16 = 1 };

@@ -13,14 +13,15 @@ from typing import Dict, List, Optional, Sequence
 
 import torch
 
-_LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libaded.so")
+# ADED_LIBRARY names another build of the same library (the index-checking debug build, libaded_debug.so)
+_LIB_PATH = os.environ.get("ADED_LIBRARY") or os.path.join(os.path.dirname(os.path.abspath(__file__)), "libaded.so")
 
 ADED_OK = 0
 ADED_F32, ADED_BF16 = 0, 1
 ADED_MAX_NODES = 128
 STATUS_NAMES = {0: "ADED_OK", 1: "ADED_ERR_INVALID_ARG", 2: "ADED_ERR_BAD_TREE", 3: "ADED_ERR_KV_CAPACITY",
                 4: "ADED_ERR_TABLE_FULL", 5: "ADED_ERR_OOM", 6: "ADED_ERR_CUDA", 7: "ADED_ERR_UNSUPPORTED",
-                8: "ADED_ERR_TIMEOUT"}
+                8: "ADED_ERR_TIMEOUT", 9: "ADED_ERR_INTERNAL"}
 
 EXPORTS = [
     "aded_model_create", "aded_model_destroy", "aded_kv_create", "aded_kv_destroy", "aded_kv_len",

@@ -49,6 +49,17 @@ __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepc
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void pdl_enter() { pdl_launch_dependents(); pdl_wait(); }
 
+// ---- index checks of the debug build -------------------------------------------------------------
+// Compiled with -DADED_DEBUG_CHECKS (python -m paper_2407_12021_b200.build --debug -> libaded_debug.so) the
+// kernels test the indices they are about to use on slots, cache rows and table buckets; a failed test
+// records ADED_ERR_INTERNAL in the status word and the access is skipped.  In the product build the
+// macro is the constant true and costs nothing.
+#ifdef ADED_DEBUG_CHECKS
+#define ADED_IN_RANGE(cond, status) ((cond) ? true : (atomicCAS(const_cast<int32_t*>(status), 0, (int)ADED_ERR_INTERNAL), false))
+#else
+#define ADED_IN_RANGE(cond, status) true
+#endif
+
 // ---- stage trace ---------------------------------------------------------------------------------
 // The status word of a model is the first of a small block of device memory:
 //   int32 [0] status, [1] trace switch, [2] marks taken, [3] unused; then TRACE_CAP 64-bit times (ns of

@@ -160,6 +160,7 @@ __global__ void __launch_bounds__(1024) k_add_rmsnorm_ws(bf16* __restrict__ h, G
         if (c < d) {
             uint2* hp = reinterpret_cast<uint2*>(h + (size_t)r * d + c);
             const float4 hv = unpack4_bf16(*hp);
+            if (!ADED_IN_RANGE(tr[i].first_slot >= 0 && tr[i].first_slot + tr[i].count <= y.n_tiles + y.g, status)) tr[i].count = 0;
             const float4 add = gemm_out_at4(y, tr[i], r, c & 127);
             const uint2 nv = pack4_bf16(hv.x + add.x, hv.y + add.y, hv.z + add.z, hv.w + add.w);
             if (pass_status == 0) *hp = nv;
@@ -194,6 +195,7 @@ __global__ void __launch_bounds__(256) k_swiglu_ws(GemmOut gu, bf16* __restrict_
     if (first_thread_of_grid()) trace_mark(status, TK_SWIGLU);
     if (c >= F) return;
     const int pass_status = *status;     // checked before the store, not before the loads
+    if (!ADED_IN_RANGE(tg.first_slot + tg.count <= gu.n_tiles + gu.g && tu.first_slot + tu.count <= gu.n_tiles + gu.g, status)) return;
     float4 g, u;
     constexpr int SB = 4;      // gate/up tiles have two or three contributors at the 7B and 13B widths
     if (tg.count <= SB && tu.count <= SB) {
@@ -237,7 +239,9 @@ k_rope_kv_ws(GemmOut qkv, const float* __restrict__ cs, const float* __restrict_
     const size_t cp = cap[b];
     bf16* kdst = reinterpret_cast<bf16*>(base[b]) + ((((size_t)layer * 2 + 0) * H + hh) * cp + slot) * hd;
     bf16* vdst = reinterpret_cast<bf16*>(base[b]) + ((((size_t)layer * 2 + 1) * H + hh) * cp + slot) * hd;
-    rope_kv_item(qkv, tq, tk, tv, r, cq, ck, cv, i, half, cs + r * half, sn + r * half, q + (size_t)r * d + hh * hd, kdst, vdst, pass_status == 0);
+    const bool in_range = ADED_IN_RANGE(slot < cp && tq.first_slot + tq.count <= qkv.n_tiles + qkv.g && tv.first_slot + tv.count <= qkv.n_tiles + qkv.g, status);
+    rope_kv_item(qkv, tq, tk, tv, r, cq, ck, cv, i, half, cs + r * half, sn + r * half, q + (size_t)r * d + hh * hd, kdst, vdst,
+                 pass_status == 0 && in_range);
 }
 
 // ---- launchers (callers have checked: bf16 model, tensor-core path) ----------------------------

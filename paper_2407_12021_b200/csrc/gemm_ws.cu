@@ -264,7 +264,8 @@ k_gemm_ws(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUt
             tc_fence_after();
             const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(a * p.rb);
             float* slot = p.slots + (size_t)(tile + (int)blockIdx.x) * p.rb * WS_BM + row_in_tile;
-            for (int c0 = 0; c0 < p.rb; c0 += 16) {
+            const bool slot_ok = ADED_IN_RANGE(tile >= 0 && tile < p.n_tiles && tile + (int)blockIdx.x < p.n_tiles + (int)gridDim.x, p.status);
+            for (int c0 = 0; c0 < p.rb && slot_ok; c0 += 16) {
                 float v[16];
                 tc_ld16(taddr + (uint32_t)c0, v);
 #pragma unroll

@@ -676,6 +676,7 @@ const char* aded_status_string(aded_status s) {
         case ADED_ERR_CUDA: return "CUDA runtime error";
         case ADED_ERR_UNSUPPORTED: return "unsupported configuration";
         case ADED_ERR_TIMEOUT: return "device-side wait ran out";
+        case ADED_ERR_INTERNAL: return "index check failed inside a kernel (debug build)";
     }
     return "unknown status";
 }

@@ -111,6 +111,7 @@ __global__ void k_compact(char* const* __restrict__ base, const int32_t* __restr
     for (int e = threadIdx.x; e < hd; e += blockDim.x) {
         for (int j = 1; j < n_acc; ++j) {
             const int src = path[b * ADED_MAX_NODES + j];
+            if (!ADED_IN_RANGE(src >= j && src < ADED_MAX_NODES && len[b] + src < cap[b], status)) continue;
             if (src != j) p[(size_t)j * hd + e] = p[(size_t)src * hd + e];
         }
     }

@@ -90,6 +90,7 @@ __device__ __forceinline__ void tg_add(const TgView& t, int a, int b, int c, uin
     if (cur < 0) { atomicCAS(t.status, 0, (int)ADED_ERR_TABLE_FULL); return; }
     // a chain can never be longer than every overflow bucket plus the home bucket
     for (uint32_t hop = 0; hop <= t.n_over; ++hop) {
+        if (!ADED_IN_RANGE(cur >= 0 && (uint64_t)cur < (uint64_t)t.n_home + t.n_over, t.status)) return;
         Bucket* bk = t.buckets + cur;
         for (int e = 0; e < 6; ++e) {
             int32_t have = *reinterpret_cast<volatile int32_t*>(&bk->e[e].tok);

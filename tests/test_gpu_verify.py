@@ -285,3 +285,21 @@ def test_bounded_wait_runs_out_and_the_handle_recovers(cuda_device, which):
     assert sess.B.aded_model_poll_status(sess.model) == 0
     again = sess.verify(tokens, parents, capture=False)
     assert again["status"] == 0 and again["out_tokens"] == good["out_tokens"] and sess.length() == 69 + good["accept_len"]
+
+
+def test_debug_build_runs_the_small_workloads_without_an_index_complaint(cuda_device):
+    """The debug build (-DADED_DEBUG_CHECKS: index checks on slot, cache-row and bucket addressing that report
+    ADED_ERR_INTERNAL through the status word; the stand-in for a memory checker) runs the fp32 workload, a
+    bf16 tensor-core step and a tri-gram round trip -- each compared with the checker -- and no check fires."""
+    import os
+    import subprocess
+    import sys
+    from paper_2407_12021_b200 import build
+    lib = build.build(debug=True)
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    env = dict(os.environ, ADED_LIBRARY=lib)
+    code = ("import __graft_entry__ as g, os; from paper_2407_12021_b200 import binding as B; "
+            "assert B._LIB_PATH == os.environ['ADED_LIBRARY']; g.smoke()")
+    res = subprocess.run([sys.executable, "-c", code], cwd=root, env=env, capture_output=True, text=True, timeout=900)
+    assert res.returncode == 0, res.stdout[-2000:] + res.stderr[-2000:]
+    assert "smoke ok" in res.stdout
