@@ -231,9 +231,65 @@ __device__ __forceinline__ unsigned long long tg_select_round(const TgView& t, i
     return best;
 }
 
-// One warp per query.  k selection rounds over the context's chain; a round picks the largest
-// packed (count, ~token) strictly below the previous pick, which yields count descending, token
-// ascending among equals, without storing the list.
+// The k <= TG_LIST largest packed (count, ~token) keys of the chain that starts at `home`, in descending order
+// (count descending, token ascending among equals), in ONE walk over the chain: lanes 0..5 each keep the best
+// TG_LIST keys of their entry slot of every bucket in registers (sorted insertion); afterwards the six lists
+// are merged by k warp-wide maxima, the lane that held a maximum dropping it.  Keys are distinct (a context
+// holds a token once).  Every lane returns the same list in `out` (0 = nothing left); `total` = sum of the counts.
+constexpr int TG_LIST = 8;
+static_assert(TG_LIST >= ADED_DRAFT_MAX_K, "the draft tree takes its lists in one walk");
+__device__ __forceinline__ void tg_select_list(const TgView& t, int64_t home, int k, int lane,
+                                               unsigned long long (&out)[TG_LIST], uint32_t* total_out) {
+    unsigned long long loc[TG_LIST];
+#pragma unroll
+    for (int i = 0; i < TG_LIST; ++i) loc[i] = 0;
+    uint32_t total = 0;
+    int64_t cur = home;
+    for (uint32_t hop = 0; cur >= 0 && hop <= t.n_over; ++hop) {
+        const Bucket* bk = t.buckets + cur;
+        if (lane < 6) {
+            const int32_t tk = bk->e[lane].tok;
+            const uint32_t cn = bk->e[lane].cnt;
+            if (tk >= 0) {
+                total += cn;
+                unsigned long long key = ((unsigned long long)cn << 32) | (0xFFFFFFFFu - (uint32_t)tk);
+                if (cn >= t.min_count && cn > 0 && key > loc[TG_LIST - 1]) {
+#pragma unroll
+                    for (int i = 0; i < TG_LIST; ++i) {       // sorted insertion: the key sinks to its place
+                        if (key > loc[i]) { const unsigned long long tmp = loc[i]; loc[i] = key; key = tmp; }
+                    }
+                }
+            }
+        }
+        const uint32_t nxt = bk->next;
+        cur = nxt == 0 ? -1 : (int64_t)nxt;
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) total += __shfl_xor_sync(0xffffffffu, total, o);
+    if (total_out) *total_out = total;
+#pragma unroll
+    for (int r = 0; r < TG_LIST; ++r) {
+        unsigned long long best = 0;
+        if (r < k) {
+            best = loc[0];
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) {
+                const unsigned long long ob = __shfl_xor_sync(0xffffffffu, best, o);
+                if (ob > best) best = ob;
+            }
+            if (best != 0 && loc[0] == best) {                // this lane held it: drop it
+#pragma unroll
+                for (int i = 0; i + 1 < TG_LIST; ++i) loc[i] = loc[i + 1];
+                loc[TG_LIST - 1] = 0;
+            }
+        }
+        out[r] = best;
+    }
+}
+
+// One warp per query.  Up to TG_LIST continuations: one walk over the context's chain (tg_select_list).  Longer
+// lists: k selection rounds, a round picking the largest packed (count, ~token) strictly below the previous
+// pick, which yields count descending, token ascending among equals, without storing the list.
 __global__ void k_tg_topk(TgView t, const int32_t* __restrict__ ctx, int q, int k, int32_t* __restrict__ out_tok,
                           uint32_t* __restrict__ out_cnt, uint32_t* __restrict__ out_total) {
     const int w = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
@@ -242,6 +298,22 @@ __global__ void k_tg_topk(TgView t, const int32_t* __restrict__ ctx, int q, int 
     const int a = ctx[2 * w], b = ctx[2 * w + 1];
     int64_t home = -1;
     if (a >= 0 && b >= 0 && a < t.vocab && b < t.vocab) home = tg_find_home(t, tg_key(a, b), false);
+    if (k <= TG_LIST) {
+        unsigned long long list[TG_LIST];
+        uint32_t total;
+        tg_select_list(t, home, k, lane, list, &total);
+        if (lane == 0) {
+#pragma unroll
+            for (int r = 0; r < TG_LIST; ++r) {
+                if (r < k) {
+                    out_tok[(size_t)w * k + r] = list[r] ? (int32_t)(0xFFFFFFFFu - (uint32_t)list[r]) : -1;
+                    out_cnt[(size_t)w * k + r] = (uint32_t)(list[r] >> 32);
+                }
+            }
+            if (out_total) out_total[w] = total;
+        }
+        return;
+    }
     unsigned long long prev = ~0ull;
     for (int round = 0; round < k; ++round) {
         uint32_t total;
@@ -327,11 +399,12 @@ k_draft_tree(TgView t, const int32_t* __restrict__ ctx, int n_nodes, int max_dep
             const int u = node == 0 ? prev_token : s_tok[s_par[node]], w = s_tok[node];
             int64_t home = -1;
             if (u >= 0 && w >= 0 && u < t.vocab && w < t.vocab) home = tg_find_home(t, tg_key(u, w), false);
-            unsigned long long prev = ~0ull;
-            for (int round = 0; round < k; ++round) {
-                const unsigned long long best = tg_select_round(t, home, prev, lane, nullptr);
-                if (lane == 0) s_cand[node * ADED_DRAFT_MAX_K + round] = best ? (int32_t)(0xFFFFFFFFu - (uint32_t)best) : -1;
-                prev = best ? best : 0;
+            unsigned long long list[TG_LIST];          // (k <= ADED_DRAFT_MAX_K = TG_LIST: one walk over the chain)
+            tg_select_list(t, home, k, lane, list, nullptr);
+            if (lane == 0) {
+#pragma unroll
+                for (int r = 0; r < TG_LIST; ++r)
+                    if (r < k) s_cand[node * ADED_DRAFT_MAX_K + r] = list[r] ? (int32_t)(0xFFFFFFFFu - (uint32_t)list[r]) : -1;
             }
         }
         __syncthreads();
