@@ -297,7 +297,7 @@ bool attn_prepare();
 int ws_grid_limit(int device);
 int ws_grid(int device, int n, int k);
 size_t ws_slot_floats(int device, int max_n, int max_rows);
-cudaError_t ws_launch(const CUtensorMap& map_w, const CUtensorMap& map_x, int rows, int row0, int n, int k,
+cudaError_t ws_launch(const CUtensorMap& map_w, const CUtensorMap& map_x, int rows, int row0, int blk, int n, int k,
                       float* slots, int32_t* status, const WsEpilogue& epi, int trace_kind, int device, cudaStream_t st);
 enum { WS_MAP_QKV = 0, WS_MAP_O = 1, WS_MAP_GU = 2, WS_MAP_D = 3 };   // per-layer map order
 cudaError_t ws_wait_probe(int which, long long limit_cycles, const uint32_t* never_raised, int32_t* status, cudaStream_t st);

@@ -319,7 +319,7 @@ GemmOut launch_gemm(aded_model* m, int w_map, int x_map, const void* x, const vo
     out.n = n;
     out.rows = rows;
     if (m->ws_ready && w_map >= 0 && x_map >= 0 && ws_supported(n, k)) {
-        // tensor-core path, 128 rows of x per pass over the weights; the result stays in slots
+        // tensor-core path, up to 128 (or 256) rows of x per pass over the weights; the result stays in slots
         const int table = w_map < 4 * m->cfg.n_layers ? w_map % 4 : 4;
         WsEpilogue e = {};
         e.mode = epi_mode;
@@ -327,11 +327,14 @@ GemmOut launch_gemm(aded_model* m, int w_map, int x_map, const void* x, const vo
         e.counters = m->ws_counters;
         e.cand_val = m->cand_val;
         e.cand_idx = m->cand_idx;
-        for (int row0 = 0; row0 < rows; row0 += 128) {
-            const int part = rows - row0 < 128 ? rows - row0 : 128;
+        // a pass takes 128 rows; calls with more rows (ragged batches) use 256-row passes: half as many trips over W
+        const int blk = rows > 128 ? 256 : 128;
+        for (int row0 = 0; row0 < rows; row0 += blk) {
+            const int part = rows - row0 < blk ? rows - row0 : blk;
             if (epi_mode != WS_EPI_SLOTS) e.epoch = ++m->ws_epoch;
-            ws_launch(m->ws_maps[w_map], m->ws_maps[x_map], part, row0, n, k, m->ws_slots, m->status, e, trace_kind, m->device, st);
+            ws_launch(m->ws_maps[w_map], m->ws_maps[x_map], part, row0, blk, n, k, m->ws_slots, m->status, e, trace_kind, m->device, st);
         }
+        out.blk_shift = blk == 256 ? 8 : 7;
         out.mode = 1;
         out.slots = m->ws_slots;
         out.n_tiles = n / 128;

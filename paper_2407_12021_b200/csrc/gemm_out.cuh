@@ -10,8 +10,9 @@
 //
 // Slot numbering: the segment of tile t computed by CTA c goes to slot t + c.  Walking the units
 // in order, (t, c) never decreases and one of them grows at every segment boundary, so the sums
-// are distinct.  A slot holds [rb][128] floats (rb = rows of the pass padded to 16).  Passes over
-// more than 128 rows use one slot region per 128-row block.
+// are distinct.  A slot holds [rb][128] floats (rb = rows of the pass padded to 16).  A pass takes up to 128
+// rows, or up to 256 when the call has more than 128 (half as many passes over the weights); a call with more
+// rows than one pass takes uses one slot region per pass.
 #pragma once
 
 #include <cuda_bf16.h>
@@ -32,7 +33,8 @@ struct GemmOut {
     int mode;
     int n;                // result columns
     int n_tiles, kb, g;   // mode 1: 128-column tiles, k blocks per tile, CTAs of the GEMM launch
-    int rows;             // rows of the whole result (all row blocks)
+    int rows;             // rows of the whole result (all passes)
+    int blk_shift;        // mode 1: log2 of the rows a pass takes (7 or 8)
 };
 
 // First work unit of CTA c when `units` units are split over `g` CTAs.
@@ -59,18 +61,22 @@ __host__ __device__ __forceinline__ TileRef gemm_tile_ref(int n_tiles, int kb, i
     return t;
 }
 
-// Rows padded to 16 of the 128-row block that holds row r.
+// Rows padded to 16 of the pass that holds row r, and where that pass's slot region starts.
 __device__ __forceinline__ int gemm_block_rb(const GemmOut& o, int r) {
-    const int left = o.rows - (r & ~127);
-    const int in_blk = left < 128 ? left : 128;
+    const int blk = 1 << o.blk_shift;
+    const int left = o.rows - ((r >> o.blk_shift) << o.blk_shift);
+    const int in_blk = left < blk ? left : blk;
     return (in_blk + 15) & ~15;
+}
+__device__ __forceinline__ const float* gemm_slot_row(const GemmOut& o, const TileRef& t, int r, int rb) {
+    const size_t region = (size_t)(r >> o.blk_shift) * (size_t)(o.n_tiles + o.g) * ((size_t)128 << o.blk_shift);
+    return o.slots + region + ((size_t)t.first_slot * rb + (r & ((1 << o.blk_shift) - 1))) * 128;
 }
 
 // Value of result element (r, tile * 128 + col) given the tile's contributors.
 __device__ __forceinline__ float gemm_out_at(const GemmOut& o, const TileRef& t, int r, int col) {
     const int rb = gemm_block_rb(o, r);
-    const size_t region = (size_t)(r >> 7) * (size_t)(o.n_tiles + o.g) * 128 * 128;
-    const float* p = o.slots + region + ((size_t)t.first_slot * rb + (r & 127)) * 128 + col;
+    const float* p = gemm_slot_row(o, t, r, rb) + col;
     const size_t stride = (size_t)rb * 128;
     float sum = 0.f;
 #pragma unroll 4
@@ -90,8 +96,7 @@ __device__ __forceinline__ float4 f4_add(float4 a, float4 b) { return make_float
 // Columns col .. col+3 (col % 4 == 0) of tile t, row r: slots added in CTA order.
 __device__ __forceinline__ float4 gemm_out_at4(const GemmOut& o, const TileRef& t, int r, int col) {
     const int rb = gemm_block_rb(o, r);
-    const size_t region = (size_t)(r >> 7) * (size_t)(o.n_tiles + o.g) * 128 * 128;
-    const float* p = o.slots + region + ((size_t)t.first_slot * rb + (r & 127)) * 128 + col;
+    const float* p = gemm_slot_row(o, t, r, rb) + col;
     const size_t stride = (size_t)rb * 128;
     float4 sum = make_float4(0.f, 0.f, 0.f, 0.f);
     // Up to GO_BATCH contributors are fetched at once (predicated loads, no branch between them) and
@@ -118,8 +123,7 @@ __device__ __forceinline__ float4 gemm_out_at4(const GemmOut& o, const TileRef& 
 template <int B>
 __device__ __forceinline__ void gemm_out_fetch4(const GemmOut& o, const TileRef& t, int r, int col, float4 (&v)[B]) {
     const int rb = gemm_block_rb(o, r);
-    const size_t region = (size_t)(r >> 7) * (size_t)(o.n_tiles + o.g) * 128 * 128;
-    const float* p = o.slots + region + ((size_t)t.first_slot * rb + (r & 127)) * 128 + col;
+    const float* p = gemm_slot_row(o, t, r, rb) + col;
     const size_t stride = (size_t)rb * 128;
 #pragma unroll
     for (int j = 0; j < B; ++j)

@@ -2,7 +2,7 @@
 // tensor cores (tcgen05, accumulators in TMEM, operands staged by TMA), with the step that consumes
 // each projection folded into the kernel's tail.
 //
-//   y[r, n] = sum_k x[r, k] * w[n, k]        r < rows <= 128,  w row-major [N, K], x row-major [R, K]
+//   y[r, n] = sum_k x[r, k] * w[n, k]        r < rows <= 256,  w row-major [N, K], x row-major [R, K]
 //
 // A verification step multiplies at most 128 tree nodes with every weight matrix, so the kernel is
 // bound by reading W once from HBM.  Mapping:
@@ -56,7 +56,8 @@ struct WsParams {
     int n, k;            // W is [n, k]
     int n_tiles, kb;     // tiles of 128 W rows, k blocks per tile
     int stages;
-    int tmem_cols;       // power of two >= 2 * rb
+    int tmem_cols;       // power of two >= n_acc * rb
+    int n_acc;           // TMEM accumulators: two (the next segment's MMAs run under the drain) up to 128 rows, one beyond
     int trace_kind;
     int narrow;          // units * (CTAs + 1) < 2^31: the work split can be computed in 32-bit arithmetic
     float* slots;        // this row block's slot region: [n_tiles + gridDim.x][rb][128] fp32
@@ -223,8 +224,8 @@ k_gemm_ws(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUt
                 const int kb0 = (int)(u % p.kb);
                 long long ue = u + (p.kb - kb0);
                 if (ue > u1) ue = u1;
-                const int a = seg & 1;
-                const uint32_t aph = (uint32_t)(seg >> 1) & 1;
+                const int a = seg % p.n_acc;
+                const uint32_t aph = (uint32_t)(seg / p.n_acc) & 1;
                 if (!__all_sync(0xffffffffu, mbar_wait(&acc_empty[a], aph ^ 1))) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(a * p.rb);
@@ -258,8 +259,8 @@ k_gemm_ws(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUt
             const int tile = (int)(u / p.kb), kb0 = (int)(u % p.kb);
             long long ue = u + (p.kb - kb0);
             if (ue > u1) ue = u1;
-            const int a = seg & 1;
-            const uint32_t aph = (uint32_t)(seg >> 1) & 1;
+            const int a = seg % p.n_acc;
+            const uint32_t aph = (uint32_t)(seg / p.n_acc) & 1;
             if (!mbar_wait(&acc_full[a], aph)) { s_flag[0] = 1; atomicCAS(p.status, 0, (int)ADED_ERR_TIMEOUT); break; }
             tc_fence_after();
             const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(a * p.rb);
@@ -422,8 +423,8 @@ int ws_grid(int device, int n, int k) {
 
 // Floats of slot storage for results of up to max_n columns and max_rows rows.
 size_t ws_slot_floats(int device, int max_n, int max_rows) {
-    const size_t blocks = ((size_t)max_rows + 127) / 128;
-    return blocks * ((size_t)max_n / WS_BM + ws_grid_limit(device)) * 128 * WS_BM;
+    const size_t passes = ((size_t)max_rows + 255) / 256;          // (regions of 256 rows also hold two regions of 128)
+    return passes * ((size_t)max_n / WS_BM + ws_grid_limit(device)) * 256 * WS_BM;
 }
 
 // Raises the kernel's dynamic shared-memory limit; once per process, before any launch or capture.
@@ -435,9 +436,9 @@ bool ws_prepare() {
 // Shapes the tensor-core path takes.
 bool ws_supported(int n, int k) { return n % WS_BM == 0 && k % WS_BK == 0 && k >= WS_BK; }
 
-// One pass: rows [row0, row0 + rows) of x (rows <= 128) against all of W.  Partial tiles go to the
-// slot region of row block row0 / 128; `epi` says whether the kernel's tail reduces them to greedy candidates.
-cudaError_t ws_launch(const CUtensorMap& map_w, const CUtensorMap& map_x, int rows, int row0, int n, int k,
+// One pass: rows [row0, row0 + rows) of x (rows <= blk = 128 or 256) against all of W.  Partial tiles go to the
+// slot region of pass row0 / blk; `epi` says whether the kernel's tail reduces them to greedy candidates.
+cudaError_t ws_launch(const CUtensorMap& map_w, const CUtensorMap& map_x, int rows, int row0, int blk, int n, int k,
                       float* slots, int32_t* status, const WsEpilogue& epi, int trace_kind, int device, cudaStream_t st) {
     WsParams p;
     p.rows = rows;
@@ -452,12 +453,13 @@ cudaError_t ws_launch(const CUtensorMap& map_w, const CUtensorMap& map_x, int ro
     // (a smaller footprint lets the scheduler stack three on some SMs and leave others empty).
     p.stages = (int)((100 * 1024) / stage_bytes);
     if (p.stages > 8) p.stages = 8;
+    p.n_acc = p.rb > 128 ? 1 : 2;          // two CTAs per SM share 512 TMEM columns
     p.tmem_cols = 32;
-    while (p.tmem_cols < 2 * p.rb) p.tmem_cols *= 2;
+    while (p.tmem_cols < p.n_acc * p.rb) p.tmem_cols *= 2;
     p.trace_kind = trace_kind;
     const int grid = ws_grid(device, n, k);
     p.narrow = (long long)p.n_tiles * p.kb * (grid + 1) < (1ll << 31);
-    p.slots = slots + (size_t)(row0 / 128) * (size_t)(p.n_tiles + grid) * 128 * WS_BM;
+    p.slots = slots + (size_t)(row0 / blk) * (size_t)(p.n_tiles + grid) * blk * WS_BM;
     p.status = status;
     p.epi = epi;
     const size_t smem = (size_t)p.stages * stage_bytes + 1024 + 256;

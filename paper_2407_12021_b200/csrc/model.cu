@@ -174,7 +174,7 @@ static aded_status enqueue_pass(aded_model* m, aded_kv* kv, const int32_t* offse
     }
     const size_t hid_bytes = (size_t)rows * d * m->elem;
     if (m->dbg_hidden) ADED_CUDA_TRY(cudaMemcpyAsync(m->dbg_hidden, m->h, hid_bytes, cudaMemcpyDeviceToDevice, st));
-    const int passes = ws ? (rows + 127) / 128 : 1;      // the tensor-core GEMM runs once per 128 rows
+    const int passes = !ws ? 1 : rows > 128 ? (rows + 255) / 256 : 1;      // the tensor-core GEMM runs once per 128 rows (256 in calls with more)
     for (int l = 0; l < c.n_layers; ++l) {
         const aded_layer_weights& w = m->layers[l];
         const void* next_gain = l + 1 < c.n_layers ? m->layers[l + 1].norm1 : m->top.final_norm;

@@ -52,8 +52,17 @@ def test_7b_shapes(cuda_device, rows):
 
 
 def test_more_rows_than_one_pass(cuda_device):
-    """Batches beyond 128 rows run as several passes over the weights."""
-    B, w, model = _model(SMALL16, cuda_device, 43, max_rows=300)
+    """Calls with more than 128 rows run as passes of up to 256 rows over the weights (one accumulator of 256
+    tensor-memory columns): a single wide pass with a ragged tail (129, 256), two passes (300), five (1228)."""
+    B, w, model = _model(SMALL16, cuda_device, 43, max_rows=1228)
     for which in (0, 3):
         _check(B, model, w, which, 300, 43)
         _check(B, model, w, which, 129, 44)
+        _check(B, model, w, which, 256, 45)
+    _check(B, model, w, 4, 1228, 46)
+
+
+def test_7b_shape_wide_pass(cuda_device):
+    B, w, model = _model(gen.LLAMA7B_1L, cuda_device, 47, max_rows=416)
+    for which in (0, 1, 2, 3):
+        _check(B, model, w, which, 416, 47)
