@@ -39,3 +39,26 @@ def test_two_replicas_aggregate_max_time_and_summed_tokens():
 def test_single_rank_passes_through():
     import bench
     assert bench.aggregate_over_ranks(3.0, 4.0, 5, 1, torch.device("cpu")) == (3.0, 4.0, 5)
+
+
+def test_stage_times_from_a_synthetic_trace():
+    """bench.stage_times: marks are (time in ns, kind) at the end of every kernel's dependency wait; the gap to the
+    next mark belongs to the earlier kernel; whole passes are delimited by the commit mark (kind 11)."""
+    import bench
+    layers = 2
+    # one pass: prologue-ish (0) 1 us, then per layer qkv (1) 10, rotary (8) 2, attention (6) 5, o (2) 4, norm (7) 1,
+    # gate/up (3) 20, swiglu (9) 2, down (4) 8, norm (7) 1; LM head (5) 30, pick (10) 3, commit (11) 7 (until the next pass)
+    per_layer = [(1, 10), (8, 2), (6, 5), (2, 4), (7, 1), (3, 20), (9, 2), (4, 8), (7, 1)]
+    one_pass = [(0, 1)] + per_layer * layers + [(5, 30), (10, 3), (11, 7)]
+    ts, kinds, t = [], [], 1000
+    for kind, us in [(11, 7)] + one_pass * 3:          # starts in the middle of a pass: only whole passes count
+        ts.append(t)
+        kinds.append(kind)
+        t += us * 1000
+    got = bench.stage_times((ts, kinds), layers)
+    assert got["steps_traced"] == 3
+    assert got["us_per_layer"] == {"gemm_qkv": 10.0, "attention": 5.0, "gemm_o": 4.0, "rmsnorm": 2.0, "gemm_gate_up": 20.0,
+                                   "gemm_down": 8.0, "rotary_kv": 2.0, "swiglu": 2.0}
+    assert got["us_per_step"] == {"gemm_lm_head": 30.0, "pick_accept": 3.0, "other": 1.0, "between_passes": 7.0}
+    assert got["us_per_layer_projections"] == 42.0 and got["us_per_layer_total"] == 53.0
+    assert bench.stage_times(([1, 2], [0, 11]), layers) is None       # no whole pass in the trace
