@@ -193,7 +193,7 @@ def test_c2_one_7b_layer_bf16(cuda_device):
     assert cpu2["accept_len"] >= 2
 
 
-@pytest.mark.parametrize("nodes,ctx,depth", [(100, 300, 6), (64, 2047, 6), (5, 1, 2)])
+@pytest.mark.parametrize("nodes,ctx,depth", [(100, 300, 6), (64, 2047, 6), (5, 1, 2), (128, 1000, 8), (65, 31, 7), (97, 4100, 5)])
 def test_attention_kernels_agree(cuda_device, nodes, ctx, depth):
     """head_dim 128 has two attention kernels: tcgen05 (the default) and mma.sync (selected with
     aded_debug_attention_kernel).  Same rounding points (integer reference in the log2 domain, numerators
