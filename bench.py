@@ -236,6 +236,11 @@ def run_ours(args, rank, world):
     kv_bytes_step = shape.kv_bytes_per_position() * (base_len + final_len) / 2
     step_bytes = gemm_bytes_step + kv_bytes_step
     whole = step_bytes / (dev_ms / steps * 1e-3) / 1e9
+    if in_step:     # the same kernel inside the timed, overlapped pass: weight bytes over the GEMM stages' own time
+        gemm_us_step = in_step["us_per_layer_projections"] * shape.n_layers + in_step["us_per_step"].get("gemm_lm_head", 0.0)
+        if gemm_us_step > 0:
+            in_step["gemm_gbs"] = round(gemm_bytes_step / (gemm_us_step * 1e-6) / 1e9, 1)
+            in_step["gemm_frac_of_peak"] = round(in_step["gemm_gbs"] / pk["hbm_gbs"], 4)
     result = {
         "ms": dev_ms, "e2e_ms": e2e_ms, "accepted": accepted, "per_step": per_step, "clocks": clocks,
         "launches": launches, "h2d": h2d, "d2h": d2h, "setup_s": setup_s,
