@@ -9,16 +9,17 @@
 //     shared memory exactly as in the mma.sync kernel;
 //   * warp 0 streams 64-key blocks of K and V with TMA (two boxes of 64 x 64 per block, 128-byte
 //     swizzle) into two stages each; warp 1 issues tcgen05.mma; warps 2..5 run the softmax;
-//   * S = Q K^T: M = 64 (query rows), K = 128.  An M = 64 accumulator occupies 16 lanes of each of the
-//     four TMEM lane quarters, so two of them interleave: the scores of keys 0..31 of the block go to
-//     lanes 0..15 of every quarter and those of keys 32..63 to lanes 16..31.  A softmax warp therefore
-//     reads, with one 32-lane load, 32 scores per thread: thread (lane & 15) + 16 * quarter is the
-//     query row, lane >> 4 the key half.  A row's two threads sit in the same warp and share the
-//     row maximum with one shuffle; nothing else crosses threads;
-//   * O += P V: P (bf16) is written by the softmax warps into a K-major swizzled tile, V is used as
-//     stored (keys x head_dim, i.e. MN-major B operand); the two 64-column halves of O interleave in
-//     TMEM the same way, so each thread owns half a row of O.  O stays in TMEM over all blocks; when a
-//     row's reference moves (rare: it is an integer) its owner rescales its part in place;
+//   * S = Q K^T: M = 64 (query rows), N = 64 (the block's keys), K = 128: 8 instructions.  An M = 64
+//     accumulator occupies lanes 0..15 of each of the four TMEM lane quarters.  A softmax warp reads
+//     it with the 16-lane load whose second half-warp takes the same lanes 32 columns further
+//     (16x32bx2): thread (lane & 15) + 16 * quarter is the query row, lane >> 4 the key half, 32 scores
+//     per thread.  A row's two threads sit in the same warp and share the row maximum with one
+//     shuffle; nothing else crosses threads;
+//   * O += P V: M = 64, N = 128 (head_dim), K = 64 keys: 4 instructions.  P (bf16) is written by the
+//     softmax warps into a K-major swizzled tile, V is used as stored (keys x head_dim, i.e. MN-major
+//     B operand whose two 64-element halves are one sub-tile apart); a thread owns half a row of O
+//     (the same split load, 64 columns apart).  O stays in TMEM over all blocks; when a row's
+//     reference moves (rare: it is an integer) its owner rescales its part in place;
 //   * all S/P/O hand-overs go through mbarriers (tcgen05.commit on the MMA side); every wait is
 //     bounded and a wait that runs out raises ADED_ERR_TIMEOUT, after which the CTA still takes part
 //     in the cluster's barriers and frees its TMEM.
@@ -37,8 +38,8 @@ constexpr int AT_ROWS = 64;       // query rows per CTA
 constexpr int AT_HD = 128;
 constexpr int AT_STAGES = 2;      // K and V blocks in flight
 constexpr int AT_THREADS = 192;
-constexpr int AT_TMEM_COLS = 128; // S: 2 x 32, O: 64
-constexpr uint32_t AT_S_COL = 0, AT_O_COL = 64;
+constexpr int AT_TMEM_COLS = 256; // S: 2 x 64, O: 128 (lanes 0..15 of every lane quarter)
+constexpr uint32_t AT_S_COL = 0, AT_O_COL = 128;
 constexpr float AT_SLACK = 8.f;   // how far a row's maximum may exceed its reference (log2 domain) before O is rescaled
 constexpr uint32_t AT_SUB = 64 * 128;            // bytes of a 64-row x 128-byte sub-tile
 // shared-memory map (from a 1024-byte aligned base)
@@ -107,6 +108,33 @@ __device__ __forceinline__ uint64_t smem_desc_mn_sw128(uint32_t addr, uint32_t l
     d |= (uint64_t)1 << 46;
     d |= (uint64_t)2 << 61;
     return d;
+}
+
+// 32 fp32 columns of lanes 0..15 of this warp's TMEM lane quarter: threads 0..15 get columns c .. c + 31 of
+// lane `thread`, threads 16..31 the columns SPLIT further of lane `thread - 16`.
+template <int SPLIT>
+__device__ __forceinline__ void tc_ld32_split(uint32_t taddr, uint32_t* r) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.16x32bx2.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32], %33;"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr), "n"(SPLIT) : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+template <int SPLIT>
+__device__ __forceinline__ void tc_st32_split(uint32_t taddr, const uint32_t* r) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.16x32bx2.x32.b32 [%32], %33, {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31};"
+        ::"r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+          "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]),
+          "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]),
+          "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31]),
+          "r"(taddr), "n"(SPLIT) : "memory");
+    asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
 }
 
 // Bounded wait that also gives up when another thread of the CTA has raised the abort flag.
@@ -287,17 +315,15 @@ k_tree_attn_tc(const __grid_constant__ CUtensorMap map_q, AttnTcArgs a) {
     } else if (warp == 1) {
         // ---------------- MMA issuer (the whole warp runs this; one elected lane issues) ----------------
         if (nblk > 0) {
-            // fp32 accumulate, bf16 operands; S: M 64 x N 32, both operands K-major; O: M 64 x N 64, B MN-major
-            const uint32_t idesc_s = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(32 >> 3) << 17) | ((uint32_t)(64 >> 4) << 24);
-            const uint32_t idesc_o = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((uint32_t)(64 >> 3) << 17) | ((uint32_t)(64 >> 4) << 24);
+            // fp32 accumulate, bf16 operands; S: M 64 x N 64, both operands K-major; O: M 64 x N 128, B MN-major
+            const uint32_t idesc_s = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(64 >> 3) << 17) | ((uint32_t)(64 >> 4) << 24);
+            const uint32_t idesc_o = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((uint32_t)(128 >> 3) << 17) | ((uint32_t)(64 >> 4) << 24);
             const uint64_t q_desc = smem_desc_sw128(smem_u32(base + AT_OFF_Q)), k_desc = smem_desc_sw128(smem_u32(base + AT_OFF_K));
             const uint64_t p_desc = smem_desc_sw128(smem_u32(base + AT_OFF_P)), v_desc = smem_desc_mn_sw128(smem_u32(base + AT_OFF_V), AT_SUB);
             bool ok = at_wait(q_full, 0, s_flag);
             __syncwarp();
             const uint32_t off0 = (uint32_t)s_off[0], off1 = (uint32_t)s_off[1];    // published by the producer before q
-            // Scores of block j: key half kh goes to lanes 16 * kh .. 16 * kh + 15 of every lane quarter.  The
-            // two halves accumulate into different lanes and alternate, so that consecutive instructions do
-            // not depend on each other.  (Descriptor addresses are in 16-byte units.)
+            // (Descriptor addresses are in 16-byte units.)
             auto issue_s = [&](int j) -> bool {
                 const int s = j & 1;
                 bool w = at_wait(&k_full[s], ((uint32_t)(j >> 1) + (s ? off1 : off0)) & 1, s_flag);
@@ -305,17 +331,13 @@ k_tree_attn_tc(const __grid_constant__ CUtensorMap map_q, AttnTcArgs a) {
                 if (!__all_sync(0xffffffffu, w)) return false;
                 tc_fence_after();
                 const uint64_t kd = k_desc + (uint64_t)((uint32_t)s * 2 * AT_SUB >> 4);
+                const uint32_t d = tmem_base + AT_S_COL + (uint32_t)s * 64;
 #pragma unroll
                 for (int h = 0; h < 2; ++h) {
 #pragma unroll
-                    for (int kk = 0; kk < 4; ++kk) {
-#pragma unroll
-                        for (int kh = 0; kh < 2; ++kh) {
-                            const uint32_t d = tmem_base + ((uint32_t)(kh * 16) << 16) + AT_S_COL + (uint32_t)s * 32;
-                            tc_mma_bf16_elect(d, q_desc + (uint64_t)((h * AT_SUB + kk * 32) >> 4),
-                                              kd + (uint64_t)((h * AT_SUB + kh * 4096 + kk * 32) >> 4), idesc_s, (h | kk) ? 1u : 0u);
-                        }
-                    }
+                    for (int kk = 0; kk < 4; ++kk)
+                        tc_mma_bf16_elect(d, q_desc + (uint64_t)((h * AT_SUB + kk * 32) >> 4), kd + (uint64_t)((h * AT_SUB + kk * 32) >> 4), idesc_s,
+                                          (h | kk) ? 1u : 0u);
                 }
                 tc_commit_elect(&k_empty[s]);
                 tc_commit_elect(&s_full[s]);
@@ -329,13 +351,8 @@ k_tree_attn_tc(const __grid_constant__ CUtensorMap map_q, AttnTcArgs a) {
                 tc_fence_after();
                 const uint64_t pd = p_desc + (uint64_t)((uint32_t)s * AT_SUB >> 4), vd = v_desc + (uint64_t)((uint32_t)s * 2 * AT_SUB >> 4);
 #pragma unroll
-                for (int kk = 0; kk < 4; ++kk) {
-#pragma unroll
-                    for (int h = 0; h < 2; ++h) {
-                        const uint32_t d = tmem_base + ((uint32_t)(h * 16) << 16) + AT_O_COL;
-                        tc_mma_bf16_elect(d, pd + (uint64_t)((kk * 32) >> 4), vd + (uint64_t)((h * AT_SUB + kk * 2048) >> 4), idesc_o, (j | kk) ? 1u : 0u);
-                    }
-                }
+                for (int kk = 0; kk < 4; ++kk)
+                    tc_mma_bf16_elect(tmem_base + AT_O_COL, pd + (uint64_t)((kk * 32) >> 4), vd + (uint64_t)((kk * 2048) >> 4), idesc_o, (j | kk) ? 1u : 0u);
                 tc_commit_elect(&v_empty[s]);
                 tc_commit_elect(&p_empty[s]);
                 return true;
@@ -365,7 +382,7 @@ k_tree_attn_tc(const __grid_constant__ CUtensorMap map_q, AttnTcArgs a) {
             if (!__all_sync(0xffffffffu, at_wait(&s_full[s], (uint32_t)(j >> 1) & 1, s_flag))) { ok = false; break; }
             tc_fence_after();
             uint32_t sr[32];
-            tc_ld32(lane_addr + AT_S_COL + (uint32_t)s * 32, sr);
+            tc_ld32_split<32>(lane_addr + AT_S_COL + (uint32_t)s * 64, sr);
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(&s_empty[s]);
@@ -401,10 +418,10 @@ k_tree_attn_tc(const __grid_constant__ CUtensorMap map_q, AttnTcArgs a) {
 #pragma unroll
                 for (int part = 0; part < 2; ++part) {
                     uint32_t o[32];
-                    tc_ld32(lane_addr + AT_O_COL + (uint32_t)part * 32, o);
+                    tc_ld32_split<64>(lane_addr + AT_O_COL + (uint32_t)part * 32, o);
 #pragma unroll
                     for (int c = 0; c < 32; ++c) o[c] = __float_as_uint(__uint_as_float(o[c]) * corr);
-                    tc_st32(lane_addr + AT_O_COL + (uint32_t)part * 32, o);
+                    tc_st32_split<64>(lane_addr + AT_O_COL + (uint32_t)part * 32, o);
                 }
                 tc_fence_before();
                 lsum *= corr;
@@ -441,7 +458,7 @@ k_tree_attn_tc(const __grid_constant__ CUtensorMap map_q, AttnTcArgs a) {
 #pragma unroll
             for (int part = 0; part < 2; ++part) {
                 uint32_t o[32];
-                tc_ld32(lane_addr + AT_O_COL + (uint32_t)part * 32, o);
+                tc_ld32_split<64>(lane_addr + AT_O_COL + (uint32_t)part * 32, o);
 #pragma unroll
                 for (int c4 = 0; c4 < 8; ++c4) {
                     const int idx = half * 16 + part * 8 + c4;

@@ -254,6 +254,45 @@ def test_attention_kernels_agree(cuda_device, nodes, ctx, depth):
     assert att0.abs().max() > 0
 
 
+@pytest.mark.parametrize("nodes", [40, 100])
+def test_attention_reference_moves_within_a_split(cuda_device, nodes):
+    """Keys whose magnitude grows with the position: every 64-key block's largest score exceeds the previous
+    block's by far more than the slack the tensor-core kernel allows its integer reference, so the rare path that
+    rescales the running output in tensor memory runs in every block.  Same answer as the checker (whose reference
+    is the row's overall maximum: scaling by a power of two commutes with the bf16 rounding of the numerators)."""
+    shape = gen.ModelShape("bf16-4x128", 1, 512, 4, 128, 3 * 128, 1024, "bf16")      # one layer: q is the same on both sides
+    w = gen.model_weights(shape, 77)
+    for p in w["layers"]:
+        for k in ("wqkv", "wo", "wgu", "wd"):
+            p[k] = (p[k].float() * 3).to(torch.bfloat16)
+    ctx = 2000
+    sess = H.GpuSession(shape, H.weights_to(w, cuda_device), capacity=ctx + 256)
+    arch = ov.arch_from_shape(shape)
+    ow = ov.Weights(w, keep=True)
+    cache = ov.Cache(arch)
+    ramp = (1.0 + torch.arange(ctx, dtype=torch.float32) / 20.0).view(1, ctx, 1)
+    for l in range(shape.n_layers):
+        k, v = gen.kv_normal(shape, ctx, 78, l)
+        k = (k.float() * ramp).to(torch.bfloat16)
+        sess.B.aded_kv_load(sess.kv, 0, l, k.to(cuda_device), v.to(cuda_device))
+        cache.load(l, k, v)
+    tokens, parents = gen.make_tree(nodes, 6, 4, shape.vocab, 79)
+    # the scores do climb: per head, the best key of the last quarter beats the best of the first by more than 2^8
+    trace = {}
+    ov.forward_tree(arch, ow, cache, tokens, parents, want_logits=False, trace=trace)
+    q = np.asarray(trace["q"]).reshape(nodes, shape.n_heads, shape.head_dim)
+    kl = np.asarray(cache.k[shape.n_layers - 1], dtype=np.float64)          # [H, L, hd]
+    sc = np.einsum("thd,hld->thl", q, kl[:, :ctx]) * (1.4426950408889634 / np.sqrt(shape.head_dim))
+    assert np.all(sc[:, :, 3 * ctx // 4:].max(axis=2) - sc[:, :, :ctx // 4].max(axis=2) > 8.0)
+    cpu = ov.verify(arch, ow, cache, tokens, parents)
+    gpu = sess.verify(tokens, parents)
+    assert gpu["status"] == 0
+    H.compare_step(shape, gpu, cpu, tokens, parents, f"climbing keys, {nodes} nodes")
+    att = sess.B.aded_debug_read_buffer(sess.model, 3, nodes).double().cpu().numpy()
+    ref = np.asarray(trace["attn"], dtype=np.float64).reshape(att.shape)
+    assert np.abs(att - ref).max() <= 2e-2 * np.abs(ref).max()
+
+
 @pytest.mark.parametrize("heads,hd,nodes,depth,ctx", [(4, 64, 128, 8, 100), (2, 128, 37, 5, 191), (2, 128, 128, 8, 70),
                                                      (4, 64, 16, 3, 64), (2, 128, 1, 0, 129)])
 def test_bf16_small_models_tree_shapes(cuda_device, heads, hd, nodes, depth, ctx):
