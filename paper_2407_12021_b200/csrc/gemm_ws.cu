@@ -1,6 +1,6 @@
 // Weight-streaming bf16 GEMM for the decoder's projections, FFN and LM head on the 5th-generation
-// tensor cores (tcgen05, accumulators in TMEM, operands staged by TMA), with the step that consumes
-// each projection folded into the kernel's tail.
+// tensor cores (tcgen05, accumulators in TMEM, operands staged by TMA); the LM head's variant also
+// reduces its result to per-tile greedy candidates in the kernel's tail.
 //
 //   y[r, n] = sum_k x[r, k] * w[n, k]        r < rows <= 256,  w row-major [N, K], x row-major [R, K]
 //
