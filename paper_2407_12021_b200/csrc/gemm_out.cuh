@@ -3,10 +3,10 @@
 // The plain GEMM writes y[r, n] directly.  The tensor-core weight-streaming GEMM splits its
 // (W tile, k block) work units evenly over its CTAs, so a 128-column tile of the result is
 // generally the sum of several CTAs' partial tiles.  Every CTA stores its partial tile to a slot, and
-// whoever consumes the result -- the tail of the GEMM kernel itself (rotary/K-V write, residual add,
-// SwiGLU, greedy candidates; gemm_ws.cu) or a later kernel (a captured logits matrix, sampling) --
-// adds a tile's slots while it reads, always in ascending CTA order, so the sum is the same on
-// every run.
+// whoever consumes the result -- the next kernel (rotary/K-V write, residual add + RMSNorm, SwiGLU,
+// a captured logits matrix, sampling; dense_ws.cu, dense.cu) or, for the LM head's greedy candidates,
+// the tail of the GEMM kernel itself (gemm_ws.cu) -- adds a tile's slots while it reads, always in
+// ascending CTA order, so the sum is the same on every run.
 //
 // Slot numbering: the segment of tile t computed by CTA c goes to slot t + c.  Walking the units
 // in order, (t, c) never decreases and one of them grows at every segment boundary, so the sums
