@@ -72,7 +72,9 @@ typedef struct aded_model_config {
 } aded_model_config;
 
 /* Device pointers to row-major weights, output feature major ([out, in]); BORROWED: they must
- * outlive the model.  wqkv [3d, d] holds the query rows, then key rows, then value rows, head h
+ * outlive the model.  (bf16 models also keep a re-tiled private copy of the matrices, made in
+ * aded_model_create: see aded_debug_weight_layout.  Changing the caller's matrices afterwards is
+ * not supported.)  wqkv [3d, d] holds the query rows, then key rows, then value rows, head h
  * owning rows h*head_dim .. (h+1)*head_dim - 1 of each block; wgu [2F, d] holds the gate rows
  * then the up rows; rotary pairs are (i, i + head_dim/2) within a head. */
 typedef struct aded_layer_weights {
@@ -242,6 +244,14 @@ aded_status aded_debug_wait_timeout(aded_model* m, int32_t which, uint64_t limit
  * always uses).  Selects the one later calls on this model use, so that a test can compare them.
  * ADED_ERR_UNSUPPORTED for models without a tensor-core attention kernel (fp32). */
 aded_status aded_debug_attention_kernel(aded_model* m, int32_t which);
+
+/* bf16 models on the tensor-core path keep a private copy of every projection, FFN and LM-head matrix, re-tiled so
+ * that each block of the GEMM kernel reads one contiguous run of memory (as many bytes again as those matrices;
+ * made once in aded_model_create; when the device has no room for it, the GEMMs read the caller's row-major
+ * matrices instead, which is slower).  which = 0: use the copies (the default when they exist;
+ * ADED_ERR_UNSUPPORTED when they do not), 1: read the caller's matrices.  Results are identical bit for bit; the
+ * switch exists so that a test can say so.  ADED_ERR_UNSUPPORTED for models without the tensor-core GEMM. */
+aded_status aded_debug_weight_layout(aded_model* m, int32_t which);
 
 /* Copy out one of the model's activation buffers as the last verify/append call left it (after
  * its last layer): which = 0 residual stream h [rows, d], 1 normalised input x [rows, d], 2 rotated

@@ -26,7 +26,7 @@ STATUS_NAMES = {0: "ADED_OK", 1: "ADED_ERR_INVALID_ARG", 2: "ADED_ERR_BAD_TREE",
 EXPORTS = [
     "aded_model_create", "aded_model_destroy", "aded_kv_create", "aded_kv_destroy", "aded_kv_len",
     "aded_kv_load", "aded_kv_set_len", "aded_kv_read", "aded_append", "aded_verify", "aded_verify_batch", "aded_verify_host",
-    "aded_debug_capture", "aded_debug_capture_hidden", "aded_debug_gemm", "aded_debug_read_buffer", "aded_greedy_noalloc", "aded_profile_begin", "aded_profile_end", "aded_trace_begin", "aded_trace_end", "aded_debug_attention_kernel", "aded_debug_wait_timeout", "aded_launch_count", "aded_model_poll_status", "aded_trigram_create", "aded_trigram_destroy",
+    "aded_debug_capture", "aded_debug_capture_hidden", "aded_debug_gemm", "aded_debug_read_buffer", "aded_greedy_noalloc", "aded_profile_begin", "aded_profile_end", "aded_trace_begin", "aded_trace_end", "aded_debug_attention_kernel", "aded_debug_weight_layout", "aded_debug_wait_timeout", "aded_launch_count", "aded_model_poll_status", "aded_trigram_create", "aded_trigram_destroy",
     "aded_trigram_update", "aded_trigram_update_host", "aded_trigram_topk", "aded_trigram_topk_host",
     "aded_trigram_get", "aded_trigram_stats", "aded_trigram_poll_status", "aded_draft_tree", "aded_decode_step",
     "aded_decode_step_host", "aded_verify_sampled", "aded_sample_tokens", "aded_trigram_export",
@@ -329,6 +329,10 @@ def aded_debug_wait_timeout(model: Model, which: int, limit_cycles: int) -> None
 
 def aded_debug_attention_kernel(model: Model, which: int) -> None:
     _check(_lib.aded_debug_attention_kernel(model.handle, c_int32(which)), "aded_debug_attention_kernel")
+
+
+def aded_debug_weight_layout(model: Model, which: int) -> None:
+    _check(_lib.aded_debug_weight_layout(model.handle, c_int32(which)), "aded_debug_weight_layout")
 
 
 def aded_launch_count() -> int:

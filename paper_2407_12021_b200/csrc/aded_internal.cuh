@@ -236,6 +236,8 @@ struct aded_model {
     // tensor-core GEMM path (bf16 models): TMA descriptors and split-tile scratch
     bool ws_ready;
     std::vector<CUtensorMap> ws_maps;   // per layer: wqkv, wo, wgu, wd; then lm_head; then x, attn, act
+    std::vector<void*> ws_tiled;        // the weight matrices re-tiled for the tensor-core GEMM (same indices as ws_maps), model-owned
+    bool ws_use_tiled;                  // GEMMs read the re-tiled copies (else the caller's matrices through ws_maps)
     float* ws_slots;                    // partial result tiles (see gemm_out.cuh)
     aded::TileRef* ws_tiles[5];         // contributor tables of the wqkv, wo, wgu, wd and LM-head results
     uint32_t* ws_counters;              // arrival counters of the LM head's tail, one per tile
@@ -297,7 +299,8 @@ bool attn_prepare();
 int ws_grid_limit(int device);
 int ws_grid(int device, int n, int k);
 size_t ws_slot_floats(int device, int max_n, int max_rows);
-cudaError_t ws_launch(const CUtensorMap& map_w, const CUtensorMap& map_x, int rows, int row0, int blk, int n, int k,
+cudaError_t ws_retile(const void* w, void* out, int n, int k, cudaStream_t st);
+cudaError_t ws_launch(const CUtensorMap& map_w, const void* w_tiled, const CUtensorMap& map_x, int rows, int row0, int blk, int n, int k,
                       float* slots, int32_t* status, const WsEpilogue& epi, int trace_kind, int device, cudaStream_t st);
 enum { WS_MAP_QKV = 0, WS_MAP_O = 1, WS_MAP_GU = 2, WS_MAP_D = 3 };   // per-layer map order
 cudaError_t ws_wait_probe(int which, long long limit_cycles, const uint32_t* never_raised, int32_t* status, cudaStream_t st);

@@ -61,9 +61,18 @@ struct WsParams {
     int trace_kind;
     int narrow;          // units * (CTAs + 1) < 2^31: the work split can be computed in 32-bit arithmetic
     float* slots;        // this row block's slot region: [n_tiles + gridDim.x][rb][128] fp32
+    const uint8_t* w_tiled;  // W re-tiled (ws_retile): unit (tile, k block) is 16 KB at (tile * kb + k block) * 16 KB, swizzled as staged
     int32_t* status;
     WsEpilogue epi;
 };
+
+// One contiguous copy of `bytes` (a multiple of 16, both addresses 16-byte aligned) from global to shared memory,
+// completing on an mbarrier like a tensor-map copy.
+__device__ __forceinline__ void bulk_load_hint(void* dst, const void* src, uint32_t bytes, uint64_t* bar, uint64_t policy) {
+    asm volatile(
+        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
+        ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)), "l"(policy) : "memory");
+}
 
 // Waits until the counter has reached `target` (arrivals are counted modulo 2^32 and never reset).
 __device__ __forceinline__ bool ws_poll(const uint32_t* counter, uint32_t target, long long limit = WS_MEET_CYCLES) {
@@ -184,7 +193,8 @@ k_gemm_ws(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUt
                 const long long u = u0 + i;
                 const int tile = (int)(u / p.kb), kb = (int)(u % p.kb);
                 mbar_expect_tx(&full[i], stage_bytes);
-                tma_load_2d_hint(&map_w, &full[i], base + (size_t)i * stage_bytes, kb * WS_BK, tile * WS_BM, pol_stream);
+                if (p.w_tiled) bulk_load_hint(base + (size_t)i * stage_bytes, p.w_tiled + (size_t)u * a_bytes, a_bytes, &full[i], pol_stream);
+                else tma_load_2d_hint(&map_w, &full[i], base + (size_t)i * stage_bytes, kb * WS_BK, tile * WS_BM, pol_stream);
             }
             pdl_wait();
             if (blockIdx.x == 0) trace_mark(p.status, p.trace_kind);
@@ -201,7 +211,8 @@ k_gemm_ws(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUt
                 uint8_t* sa = base + (size_t)s * stage_bytes;
                 uint8_t* sb = sa + a_bytes;
                 mbar_expect_tx(&full[s], stage_bytes);
-                tma_load_2d_hint(&map_w, &full[s], sa, kb * WS_BK, tile * WS_BM, pol_stream);
+                if (p.w_tiled) bulk_load_hint(sa, p.w_tiled + (size_t)u * a_bytes, a_bytes, &full[s], pol_stream);
+                else tma_load_2d_hint(&map_w, &full[s], sa, kb * WS_BK, tile * WS_BM, pol_stream);
                 for (int r = 0; r < p.rb; r += 16) tma_load_2d(&map_x, &full[s], sb + r * 128, kb * WS_BK, p.row0 + r);
                 if (++s == p.stages) { s = 0; ph ^= 1; }
             }
@@ -373,6 +384,25 @@ cudaError_t ws_wait_probe(int which, long long limit_cycles, const uint32_t* nev
     return cudaGetLastError();
 }
 
+// W [n, k] row-major -> units of 128 rows x 64 columns, unit (tile, k block) at (tile * (k / 64) + k block) * 16 KB, each
+// stored as the kernel stages it: row r at byte r * 128, its 16-byte chunk c at position c ^ (r & 7) (128-byte swizzle).
+// A CTA's consecutive units are then one contiguous run of HBM.  One thread per 16-byte chunk.
+__global__ void k_ws_retile(const uint4* __restrict__ w, uint4* __restrict__ out, int n, int k) {
+    const size_t chunks = (size_t)n * k / 8;
+    const int kb_n = k / WS_BK;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < chunks; i += (size_t)gridDim.x * blockDim.x) {
+        const size_t row = i / (k / 8);
+        const int cc = (int)(i % (k / 8));                  // chunk within the row
+        const int tile = (int)(row / WS_BM), r = (int)(row % WS_BM), kb = cc / 8, c = cc % 8;
+        out[((size_t)tile * kb_n + kb) * (WS_BM * 8) + (size_t)r * 8 + (c ^ (r & 7))] = w[i];
+    }
+}
+
+cudaError_t ws_retile(const void* w, void* out, int n, int k, cudaStream_t st) {
+    k_ws_retile<<<2048, 256, 0, st>>>(static_cast<const uint4*>(w), static_cast<uint4*>(out), n, k);
+    return cudaGetLastError();
+}
+
 // ---- host side --------------------------------------------------------------------------------
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -438,9 +468,10 @@ bool ws_supported(int n, int k) { return n % WS_BM == 0 && k % WS_BK == 0 && k >
 
 // One pass: rows [row0, row0 + rows) of x (rows <= blk = 128 or 256) against all of W.  Partial tiles go to the
 // slot region of pass row0 / blk; `epi` says whether the kernel's tail reduces them to greedy candidates.
-cudaError_t ws_launch(const CUtensorMap& map_w, const CUtensorMap& map_x, int rows, int row0, int blk, int n, int k,
+cudaError_t ws_launch(const CUtensorMap& map_w, const void* w_tiled, const CUtensorMap& map_x, int rows, int row0, int blk, int n, int k,
                       float* slots, int32_t* status, const WsEpilogue& epi, int trace_kind, int device, cudaStream_t st) {
     WsParams p;
+    p.w_tiled = static_cast<const uint8_t*>(w_tiled);
     p.rows = rows;
     p.rb = (rows + 15) / 16 * 16;
     p.row0 = row0;

@@ -125,6 +125,38 @@ static aded_status alloc_model(aded_model* m) {
              ws_make_map(&m->ws_maps[4 * L + 1], m->x, R, d, 16) && ws_make_map(&m->ws_maps[4 * L + 2], m->attn, R, d, 16) &&
              ws_make_map(&m->ws_maps[4 * L + 3], m->act, R, F, 16);
         if (ok) {
+            // Private re-tiled copies of the weight matrices (as many bytes again as the matrices): each GEMM CTA
+            // then reads one contiguous run of HBM instead of 128 strided lines per tile.  One allocation; when
+            // the device has no room for it the GEMMs read the caller's row-major matrices through tensor maps.
+            m->ws_tiled.assign(4 * L + 1, nullptr);
+            m->ws_use_tiled = false;
+            auto matrix = [&](int i, const void** src, size_t* nn, size_t* kk) {
+                const int l = i / 4, kind = i % 4;
+                if (i == 4 * L) { *src = m->top.lm_head; *nn = V; *kk = d; return; }
+                const aded_layer_weights& w = m->layers[l];
+                *src = kind == WS_MAP_QKV ? w.wqkv : kind == WS_MAP_O ? w.wo : kind == WS_MAP_GU ? w.wgu : w.wd;
+                *nn = kind == WS_MAP_QKV ? 3 * d : kind == WS_MAP_O ? d : kind == WS_MAP_GU ? 2 * F : d;
+                *kk = kind == WS_MAP_D ? F : d;
+            };
+            size_t total = 0;
+            for (int i = 0; i < 4 * L + 1; ++i) {
+                const void* src; size_t nn, kk;
+                matrix(i, &src, &nn, &kk);
+                total += nn * kk * 2;
+            }
+            uint8_t* pool = nullptr;
+            if (dev_alloc(m, &pool, total) == ADED_OK) {
+                size_t at = 0;
+                for (int i = 0; i < 4 * L + 1; ++i) {
+                    const void* src; size_t nn, kk;
+                    matrix(i, &src, &nn, &kk);
+                    ADED_CUDA_TRY(ws_retile(src, pool + at, (int)nn, (int)kk, nullptr));
+                    m->ws_tiled[i] = pool + at;
+                    at += nn * kk * 2;
+                }
+                ADED_CUDA_TRY(cudaDeviceSynchronize());
+                m->ws_use_tiled = true;
+            }
             size_t widest = 3 * d;
             if (2 * F > widest) widest = 2 * F;
             if (V > widest) widest = V;
@@ -641,6 +673,18 @@ aded_status aded_debug_attention_kernel(aded_model* m, int32_t which) {
     if (which == 0) { m->att_tc = m->att_tc_ok; return ADED_OK; }
     if (!m->att_mma) return ADED_ERR_UNSUPPORTED;
     m->att_tc = false;
+    return ADED_OK;
+}
+
+aded_status aded_debug_weight_layout(aded_model* m, int32_t which) {
+    if (!m || which < 0 || which > 1) return ADED_ERR_INVALID_ARG;
+    if (!m->ws_ready) return ADED_ERR_UNSUPPORTED;
+    if (which == 0) {
+        if (m->ws_tiled.empty() || !m->ws_tiled[0]) return ADED_ERR_UNSUPPORTED;
+        m->ws_use_tiled = true;
+        return ADED_OK;
+    }
+    m->ws_use_tiled = false;
     return ADED_OK;
 }
 

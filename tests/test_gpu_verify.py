@@ -254,6 +254,35 @@ def test_attention_kernels_agree(cuda_device, nodes, ctx, depth):
     assert att0.abs().max() > 0
 
 
+def test_weight_layouts_agree_bit_for_bit(cuda_device):
+    """The tensor-core GEMM reads the model's re-tiled private copies of the weight matrices by default and the
+    caller's row-major matrices on request (aded_debug_weight_layout): the same sums in the same order, so logits,
+    tokens and cache rows are identical; both against the checker once."""
+    from paper_2407_12021_b200 import binding as B
+    shape = gen.ModelShape("bf16-4x128", 2, 512, 4, 128, 1408, 1024, "bf16")
+    w = gen.model_weights(shape, 91)
+    arch = ov.arch_from_shape(shape)
+    ow = ov.Weights(w, keep=True)
+    tokens, parents = gen.make_tree(100, 7, 4, shape.vocab, 92)
+    prompt = gen.zipf_tokens(150, shape.vocab, 93, 50).tolist()
+    results = []
+    for which in (0, 1):
+        sess = H.GpuSession(shape, H.weights_to(w, cuda_device), capacity=512)
+        B.aded_debug_weight_layout(sess.model, which)
+        sess.append(prompt)
+        gpu = sess.verify(tokens, parents)
+        assert gpu["status"] == 0
+        k, v = sess.read_kv(1, 0, sess.length())
+        results.append((gpu, k, v))
+    (g0, k0, v0), (g1, k1, v1) = results
+    assert np.array_equal(g0["logits"], g1["logits"]) and g0["out_tokens"] == g1["out_tokens"]
+    assert np.array_equal(k0, k1) and np.array_equal(v0, v1)
+    cache = ov.Cache(arch)
+    ov.append(arch, ow, cache, prompt)
+    cpu = ov.verify(arch, ow, cache, tokens, parents)
+    H.compare_step(shape, g0, cpu, tokens, parents, "re-tiled weights")
+
+
 @pytest.mark.parametrize("nodes", [40, 100])
 def test_attention_reference_moves_within_a_split(cuda_device, nodes):
     """Keys whose magnitude grows with the position: every 64-key block's largest score exceeds the previous
