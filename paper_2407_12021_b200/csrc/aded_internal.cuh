@@ -235,7 +235,7 @@ struct aded_model {
 
     // tensor-core GEMM path (bf16 models): TMA descriptors and split-tile scratch
     bool ws_ready;
-    std::vector<CUtensorMap> ws_maps;   // per layer: wqkv, wo, wgu, wd; then lm_head; then x, attn, act
+    std::vector<CUtensorMap> ws_maps;   // per layer: wqkv, wo, wgu, wd; then lm_head; then x, attn, act (boxes of 16 rows); then the same three with boxes of 64 rows
     std::vector<void*> ws_tiled;        // the weight matrices re-tiled for the tensor-core GEMM (same indices as ws_maps), model-owned
     bool ws_use_tiled;                  // GEMMs read the re-tiled copies (else the caller's matrices through ws_maps)
     float* ws_slots;                    // partial result tiles (see gemm_out.cuh)
@@ -300,7 +300,8 @@ int ws_grid_limit(int device);
 int ws_grid(int device, int n, int k);
 size_t ws_slot_floats(int device, int max_n, int max_rows);
 cudaError_t ws_retile(const void* w, void* out, int n, int k, cudaStream_t st);
-cudaError_t ws_launch(const CUtensorMap& map_w, const void* w_tiled, const CUtensorMap& map_x, int rows, int row0, int blk, int n, int k,
+cudaError_t ws_launch(const CUtensorMap& map_w, const void* w_tiled, const CUtensorMap& map_x, const CUtensorMap& map_x64, int rows, int row0, int blk,
+                      int n, int k,
                       float* slots, int32_t* status, const WsEpilogue& epi, int trace_kind, int device, cudaStream_t st);
 enum { WS_MAP_QKV = 0, WS_MAP_O = 1, WS_MAP_GU = 2, WS_MAP_D = 3 };   // per-layer map order
 cudaError_t ws_wait_probe(int which, long long limit_cycles, const uint32_t* never_raised, int32_t* status, cudaStream_t st);

@@ -332,7 +332,7 @@ GemmOut launch_gemm(aded_model* m, int w_map, int x_map, const void* x, const vo
         for (int row0 = 0; row0 < rows; row0 += blk) {
             const int part = rows - row0 < blk ? rows - row0 : blk;
             if (epi_mode != WS_EPI_SLOTS) e.epoch = ++m->ws_epoch;
-            ws_launch(m->ws_maps[w_map], m->ws_use_tiled ? m->ws_tiled[w_map] : nullptr, m->ws_maps[x_map], part, row0, blk, n, k, m->ws_slots, m->status, e, trace_kind, m->device, st);
+            ws_launch(m->ws_maps[w_map], m->ws_use_tiled ? m->ws_tiled[w_map] : nullptr, m->ws_maps[x_map], m->ws_maps[x_map + 3], part, row0, blk, n, k, m->ws_slots, m->status, e, trace_kind, m->device, st);
         }
         out.blk_shift = blk == 256 ? 8 : 7;
         out.mode = 1;

@@ -139,7 +139,8 @@ __device__ __forceinline__ void ws_row_argmax(const WsParams& p, const TileRef& 
 
 template <bool TAIL>
 __global__ void __launch_bounds__(WS_THREADS, 2)
-k_gemm_ws(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_x, const __grid_constant__ WsParams p) {
+k_gemm_ws(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_x64,
+          const __grid_constant__ WsParams p) {
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     // carve: stages x (W tile 16 KB | x tile rb*128 B), then barriers
     uint8_t* base = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
@@ -183,37 +184,50 @@ k_gemm_ws(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUt
         if (lane == 0 && live) {
             asm volatile("prefetch.tensormap [%0];" ::"l"(&map_w) : "memory");
             asm volatile("prefetch.tensormap [%0];" ::"l"(&map_x) : "memory");
+            asm volatile("prefetch.tensormap [%0];" ::"l"(&map_x64) : "memory");
             uint64_t pol_stream;
             asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol_stream));
             // Weights do not depend on the previous kernel: fill the pipeline with W tiles first, then
             // wait for the previous kernel (which produces x) and add the x tiles of those stages.
-            const long long n_units = u1 - u0;
-            const int ahead = (int)(n_units < p.stages ? n_units : p.stages);
+            // This one thread feeds the whole pipeline, so its per-unit work is kept small: (tile, k block) advance
+            // by increments (no 64-bit divisions), x comes in boxes of 64 rows where the pass has that many (one
+            // request instead of four), and W is one bulk copy.
+            const int n_units = (int)(u1 - u0);
+            const int ahead = n_units < p.stages ? n_units : p.stages;
+            const int tile0 = (int)(u0 / p.kb), kb0 = (int)(u0 % p.kb);
+            auto load_x = [&](uint64_t* bar, uint8_t* sb, int kb) {
+                int r = 0;
+                for (; r + 64 <= p.rb; r += 64) tma_load_2d(&map_x64, bar, sb + r * 128, kb * WS_BK, p.row0 + r);
+                for (; r < p.rb; r += 16) tma_load_2d(&map_x, bar, sb + r * 128, kb * WS_BK, p.row0 + r);
+            };
+            int tile = tile0, kb = kb0;
             for (int i = 0; i < ahead; ++i) {
-                const long long u = u0 + i;
-                const int tile = (int)(u / p.kb), kb = (int)(u % p.kb);
                 mbar_expect_tx(&full[i], stage_bytes);
-                if (p.w_tiled) bulk_load_hint(base + (size_t)i * stage_bytes, p.w_tiled + (size_t)u * a_bytes, a_bytes, &full[i], pol_stream);
+                if (p.w_tiled) bulk_load_hint(base + (size_t)i * stage_bytes, p.w_tiled + (size_t)(u0 + i) * a_bytes, a_bytes, &full[i], pol_stream);
                 else tma_load_2d_hint(&map_w, &full[i], base + (size_t)i * stage_bytes, kb * WS_BK, tile * WS_BM, pol_stream);
+                if (++kb == p.kb) { kb = 0; ++tile; }
             }
             pdl_wait();
             if (blockIdx.x == 0) trace_mark(p.status, p.trace_kind);
-            for (int i = 0; i < ahead; ++i) {
-                const int kb = (int)((u0 + i) % p.kb);
-                uint8_t* sb = base + (size_t)i * stage_bytes + a_bytes;
-                for (int r = 0; r < p.rb; r += 16) tma_load_2d(&map_x, &full[i], sb + r * 128, kb * WS_BK, p.row0 + r);
+            {
+                int kbx = kb0;
+                for (int i = 0; i < ahead; ++i) {
+                    load_x(&full[i], base + (size_t)i * stage_bytes + a_bytes, kbx);
+                    if (++kbx == p.kb) kbx = 0;
+                }
             }
             int s = ahead == p.stages ? 0 : ahead;
             uint32_t ph = ahead == p.stages ? 1 : 0;
-            for (long long u = u0 + ahead; u < u1 && !s_flag[0]; ++u) {
-                const int tile = (int)(u / p.kb), kb = (int)(u % p.kb);
+            const uint8_t* wsrc = p.w_tiled + (size_t)(u0 + ahead) * a_bytes;
+            for (int i = ahead; i < n_units && !s_flag[0]; ++i) {
                 if (!mbar_wait(&empty[s], ph ^ 1)) { s_flag[0] = 1; atomicCAS(p.status, 0, (int)ADED_ERR_TIMEOUT); break; }
                 uint8_t* sa = base + (size_t)s * stage_bytes;
-                uint8_t* sb = sa + a_bytes;
                 mbar_expect_tx(&full[s], stage_bytes);
-                if (p.w_tiled) bulk_load_hint(sa, p.w_tiled + (size_t)u * a_bytes, a_bytes, &full[s], pol_stream);
+                if (p.w_tiled) bulk_load_hint(sa, wsrc, a_bytes, &full[s], pol_stream);
                 else tma_load_2d_hint(&map_w, &full[s], sa, kb * WS_BK, tile * WS_BM, pol_stream);
-                for (int r = 0; r < p.rb; r += 16) tma_load_2d(&map_x, &full[s], sb + r * 128, kb * WS_BK, p.row0 + r);
+                load_x(&full[s], sa + a_bytes, kb);
+                wsrc += a_bytes;
+                if (++kb == p.kb) { kb = 0; ++tile; }
                 if (++s == p.stages) { s = 0; ph ^= 1; }
             }
         }
@@ -468,7 +482,8 @@ bool ws_supported(int n, int k) { return n % WS_BM == 0 && k % WS_BK == 0 && k >
 
 // One pass: rows [row0, row0 + rows) of x (rows <= blk = 128 or 256) against all of W.  Partial tiles go to the
 // slot region of pass row0 / blk; `epi` says whether the kernel's tail reduces them to greedy candidates.
-cudaError_t ws_launch(const CUtensorMap& map_w, const void* w_tiled, const CUtensorMap& map_x, int rows, int row0, int blk, int n, int k,
+cudaError_t ws_launch(const CUtensorMap& map_w, const void* w_tiled, const CUtensorMap& map_x, const CUtensorMap& map_x64, int rows, int row0, int blk,
+                      int n, int k,
                       float* slots, int32_t* status, const WsEpilogue& epi, int trace_kind, int device, cudaStream_t st) {
     WsParams p;
     p.w_tiled = static_cast<const uint8_t*>(w_tiled);
@@ -494,8 +509,8 @@ cudaError_t ws_launch(const CUtensorMap& map_w, const void* w_tiled, const CUten
     p.status = status;
     p.epi = epi;
     const size_t smem = (size_t)p.stages * stage_bytes + 1024 + 256;
-    if (epi.mode == WS_EPI_ARGMAX) return launch_k(k_gemm_ws<true>, dim3(grid), dim3(WS_THREADS), smem, st, map_w, map_x, p);
-    return launch_k(k_gemm_ws<false>, dim3(grid), dim3(WS_THREADS), smem, st, map_w, map_x, p);
+    if (epi.mode == WS_EPI_ARGMAX) return launch_k(k_gemm_ws<true>, dim3(grid), dim3(WS_THREADS), smem, st, map_w, map_x, map_x64, p);
+    return launch_k(k_gemm_ws<false>, dim3(grid), dim3(WS_THREADS), smem, st, map_w, map_x, map_x64, p);
 }
 
 }  // namespace aded

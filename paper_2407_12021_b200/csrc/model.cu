@@ -112,7 +112,7 @@ static aded_status alloc_model(aded_model* m) {
     if (c.dtype == ADED_BF16 && ws_supported(3 * (int)d, (int)d) && ws_supported((int)d, (int)d) && ws_supported(2 * (int)F, (int)d) &&
         ws_supported((int)d, (int)F) && ws_supported((int)V, (int)d)) {
         const int L = c.n_layers;
-        m->ws_maps.resize(4 * L + 4);
+        m->ws_maps.resize(4 * L + 7);
         bool ok = ws_prepare();
         for (int l = 0; l < L && ok; ++l) {
             const aded_layer_weights& w = m->layers[l];
@@ -123,7 +123,9 @@ static aded_status alloc_model(aded_model* m) {
         }
         ok = ok && ws_make_map(&m->ws_maps[4 * L], m->top.lm_head, V, d, 128) &&
              ws_make_map(&m->ws_maps[4 * L + 1], m->x, R, d, 16) && ws_make_map(&m->ws_maps[4 * L + 2], m->attn, R, d, 16) &&
-             ws_make_map(&m->ws_maps[4 * L + 3], m->act, R, F, 16);
+             ws_make_map(&m->ws_maps[4 * L + 3], m->act, R, F, 16) &&
+             ws_make_map(&m->ws_maps[4 * L + 4], m->x, R, d, 64) && ws_make_map(&m->ws_maps[4 * L + 5], m->attn, R, d, 64) &&
+             ws_make_map(&m->ws_maps[4 * L + 6], m->act, R, F, 64);
         if (ok) {
             // Private re-tiled copies of the weight matrices (as many bytes again as the matrices): each GEMM CTA
             // then reads one contiguous run of HBM instead of 128 strided lines per tile.  One allocation; when
