@@ -240,6 +240,7 @@ struct aded_model {
     bool ws_use_tiled;                  // GEMMs read the re-tiled copies (else the caller's matrices through ws_maps)
     float* ws_slots;                    // partial result tiles (see gemm_out.cuh)
     aded::TileRef* ws_tiles[5];         // contributor tables of the wqkv, wo, wgu, wd and LM-head results
+    bool ws_one_per_sm[5];              // which of those five GEMMs launch one CTA per SM instead of two
     uint32_t* ws_counters;              // arrival counters of the LM head's tail, one per tile
     uint32_t ws_epoch;                  // LM-head launches with a tail so far (host side of the counters)
     float* cand_val;                    // [R][vocab / 128] per-tile greedy candidates of the LM head
@@ -297,12 +298,12 @@ bool ws_supported(int n, int k);
 bool ws_prepare();
 bool attn_prepare();
 int ws_grid_limit(int device);
-int ws_grid(int device, int n, int k);
+int ws_grid(int device, int n, int k, bool one_per_sm);
 size_t ws_slot_floats(int device, int max_n, int max_rows);
 cudaError_t ws_retile(const void* w, void* out, int n, int k, cudaStream_t st);
 cudaError_t ws_launch(const CUtensorMap& map_w, const void* w_tiled, const CUtensorMap& map_x, const CUtensorMap& map_x64, int rows, int row0, int blk,
                       int n, int k,
-                      float* slots, int32_t* status, const WsEpilogue& epi, int trace_kind, int device, cudaStream_t st);
+                      float* slots, int32_t* status, const WsEpilogue& epi, int trace_kind, int device, bool one_per_sm, cudaStream_t st);
 enum { WS_MAP_QKV = 0, WS_MAP_O = 1, WS_MAP_GU = 2, WS_MAP_D = 3 };   // per-layer map order
 cudaError_t ws_wait_probe(int which, long long limit_cycles, const uint32_t* never_raised, int32_t* status, cudaStream_t st);
 

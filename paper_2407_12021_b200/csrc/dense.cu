@@ -332,14 +332,14 @@ GemmOut launch_gemm(aded_model* m, int w_map, int x_map, const void* x, const vo
         for (int row0 = 0; row0 < rows; row0 += blk) {
             const int part = rows - row0 < blk ? rows - row0 : blk;
             if (epi_mode != WS_EPI_SLOTS) e.epoch = ++m->ws_epoch;
-            ws_launch(m->ws_maps[w_map], m->ws_use_tiled ? m->ws_tiled[w_map] : nullptr, m->ws_maps[x_map], m->ws_maps[x_map + 3], part, row0, blk, n, k, m->ws_slots, m->status, e, trace_kind, m->device, st);
+            ws_launch(m->ws_maps[w_map], m->ws_use_tiled ? m->ws_tiled[w_map] : nullptr, m->ws_maps[x_map], m->ws_maps[x_map + 3], part, row0, blk, n, k, m->ws_slots, m->status, e, trace_kind, m->device, m->ws_one_per_sm[table], st);
         }
         out.blk_shift = blk == 256 ? 8 : 7;
         out.mode = 1;
         out.slots = m->ws_slots;
         out.n_tiles = n / 128;
         out.kb = k / 64;
-        out.g = ws_grid(m->device, n, k);
+        out.g = ws_grid(m->device, n, k, m->ws_one_per_sm[table]);
         out.tiles = m->ws_tiles[table];
         return out;
     }

@@ -458,10 +458,12 @@ int ws_grid_limit(int device) {
     return cached;
 }
 
-// CTAs a launch over n_tiles x kb units uses.
-int ws_grid(int device, int n, int k) {
+// CTAs a launch over n_tiles x kb units uses: two per SM, or one per SM (with twice the stages, so the same bytes
+// in flight).  With one per SM a tile has half as many contributors, so the kernel that gathers the slots reads half
+// as much; used where that kernel is the next thing on the critical path (see ws_one_per_sm in model.cu).
+int ws_grid(int device, int n, int k, bool one_per_sm) {
     const long long units = (long long)(n / WS_BM) * (k / WS_BK);
-    const int g = ws_grid_limit(device);
+    const int g = ws_grid_limit(device) / (one_per_sm ? 2 : 1);
     return units < g ? (int)units : g;
 }
 
@@ -473,7 +475,7 @@ size_t ws_slot_floats(int device, int max_n, int max_rows) {
 
 // Raises the kernel's dynamic shared-memory limit; once per process, before any launch or capture.
 bool ws_prepare() {
-    return cudaFuncSetAttribute(k_gemm_ws<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 112 * 1024) == cudaSuccess &&
+    return cudaFuncSetAttribute(k_gemm_ws<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024) == cudaSuccess &&
            cudaFuncSetAttribute(k_gemm_ws<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 112 * 1024) == cudaSuccess;
 }
 
@@ -484,7 +486,7 @@ bool ws_supported(int n, int k) { return n % WS_BM == 0 && k % WS_BK == 0 && k >
 // slot region of pass row0 / blk; `epi` says whether the kernel's tail reduces them to greedy candidates.
 cudaError_t ws_launch(const CUtensorMap& map_w, const void* w_tiled, const CUtensorMap& map_x, const CUtensorMap& map_x64, int rows, int row0, int blk,
                       int n, int k,
-                      float* slots, int32_t* status, const WsEpilogue& epi, int trace_kind, int device, cudaStream_t st) {
+                      float* slots, int32_t* status, const WsEpilogue& epi, int trace_kind, int device, bool one_per_sm, cudaStream_t st) {
     WsParams p;
     p.w_tiled = static_cast<const uint8_t*>(w_tiled);
     p.rows = rows;
@@ -496,14 +498,15 @@ cudaError_t ws_launch(const CUtensorMap& map_w, const void* w_tiled, const CUten
     p.kb = k / WS_BK;
     const uint32_t stage_bytes = WS_BM * 128 + p.rb * 128;
     // About 100 KB per CTA: exactly two CTAs fit on an SM, so a launch of 2 x SMs CTAs is spread evenly
-    // (a smaller footprint lets the scheduler stack three on some SMs and leave others empty).
-    p.stages = (int)((100 * 1024) / stage_bytes);
+    // (a smaller footprint lets the scheduler stack three on some SMs and leave others empty); about 200 KB
+    // for a launch of one CTA per SM.
+    p.stages = (int)(((one_per_sm ? 200 : 100) * 1024) / stage_bytes);
     if (p.stages > 8) p.stages = 8;
     p.n_acc = p.rb > 128 ? 1 : 2;          // two CTAs per SM share 512 TMEM columns
     p.tmem_cols = 32;
     while (p.tmem_cols < p.n_acc * p.rb) p.tmem_cols *= 2;
     p.trace_kind = trace_kind;
-    const int grid = ws_grid(device, n, k);
+    const int grid = ws_grid(device, n, k, one_per_sm);
     p.narrow = (long long)p.n_tiles * p.kb * (grid + 1) < (1ll << 31);
     p.slots = slots + (size_t)(row0 / blk) * (size_t)(p.n_tiles + grid) * blk * WS_BM;
     p.status = status;

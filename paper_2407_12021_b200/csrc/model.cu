@@ -166,7 +166,13 @@ static aded_status alloc_model(aded_model* m) {
             // which slots make up each 128-column tile of each projection's result
             const int shapes[5][2] = {{3 * (int)d, (int)d}, {(int)d, (int)d}, {2 * (int)F, (int)d}, {(int)d, (int)F}, {(int)V, (int)d}};
             for (int i = 0; i < 5; ++i) {
-                const int nt = shapes[i][0] / 128, kb = shapes[i][1] / 64, g = ws_grid(m->device, shapes[i][0], shapes[i][1]);
+                // O, gate/up and down launch one CTA per SM: their tiles then have half as many contributors and the
+                // kernel that gathers them (residual + norm, SwiGLU), which is next on the critical path, reads half as
+                // much (measured: two norms 12.8 -> 9.2 us per layer, the O and down GEMMs themselves unchanged).  QKV
+                // keeps two (with one, the rotary step gains 0.8 us and the attention behind it loses 1.6), and so
+                // does the LM head (its tail: 52.7 -> 58.8 us with one).
+                m->ws_one_per_sm[i] = i == WS_MAP_O || i == WS_MAP_GU || i == WS_MAP_D;
+                const int nt = shapes[i][0] / 128, kb = shapes[i][1] / 64, g = ws_grid(m->device, shapes[i][0], shapes[i][1], m->ws_one_per_sm[i]);
                 std::vector<TileRef> table(nt);
                 for (int t = 0; t < nt; ++t) table[t] = gemm_tile_ref(nt, kb, g, t);
                 TRY(dev_alloc(m, &m->ws_tiles[i], (size_t)nt));
